@@ -1,0 +1,312 @@
+// TEST INFRASTRUCTURE ONLY -- plain, slow, single-threaded CPU statement of the routing
+// simulator.  Nothing in the product path may link, import or call this file; it shares no
+// code, header, table or helper with the CUDA library.  It exists so that tests (and the
+// timed CPU baseline of the benchmark) have an independent definition to compare against.
+//
+// What it computes, per cost-model candidate, for each request of a Mooncake-style trace in
+// trace order (paper Section 2.2, Eq. 1-3, and Section 2.3):
+//   * the longest cached prefix (in 512-token blocks) of the request on every replica
+//     (Section 1: prefix caching removes the prefill of earlier turns; Section 4 "prefix-cache"
+//     baseline: proxy-side index of dispatched requests),
+//   * the proxy-recorded queue signal: total input tokens of requests dispatched to a replica
+//     that have no completion event yet (text below Eq. 1),
+//   * the weighted score of Eq. 3 with explicit weights (w_net, w_prefill, w_queue) and the
+//     argmin replica,
+//   * an LRU block cache and a slot/queue service model per replica (the paper calls for
+//     "a sufficiently accurate simulator of cache and continuous-batching dynamics",
+//     Section 2.1, without giving one; the model here is this project's explicit statement),
+//   * TTFT = network + queue wait + prefill of the uncached tokens (Eq. 1) and E2E latency,
+//     reduced to their p95 (Section 4: the tuning objective is p95 TTFT).
+//
+// Pinned by tests/test_oracle_*.py: hand-worked traces, brute-force prefix matching, an
+// independently written list-based LRU, Lindley's recursion, closed forms and invariants.
+// Parity unpinned: the absolute TTFT/E2E values against the paper's tables (they need the
+// paper's engines, model and trace).
+//
+// Build: g++ -O2 -std=c++17 -ffp-contract=off -shared -fPIC gorgo_oracle.cpp -o libgorgo_oracle.so
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <map>
+#include <set>
+#include <unordered_map>
+#include <utility>
+#include <vector>
+
+namespace {
+
+// Recency key of a cached block: request index of its last touch and its position in that
+// request.  Eviction order: smaller seq first; inside one request the DEEPEST block first, so
+// a cache filled by prefix-sharing requests stays prefix-closed.
+struct Key {
+    uint64_t seq;
+    uint32_t pos;
+};
+struct KeyEvictsBefore {
+    bool operator()(const Key& a, const Key& b) const {
+        if (a.seq != b.seq) return a.seq < b.seq;
+        return a.pos > b.pos;
+    }
+};
+
+struct Replica {
+    std::unordered_map<uint64_t, Key> cache;              // block id -> recency key
+    std::map<Key, uint64_t, KeyEvictsBefore> order;       // recency key -> block id
+    std::vector<double> free_at;                          // per slot: time it becomes free
+    std::multiset<std::pair<double, uint64_t>> inflight;  // (finish time, input tokens)
+    int64_t load = 0;                                     // sum of in-flight input tokens
+};
+
+uint64_t mix64(uint64_t z) {  // splitmix64 finaliser (Steele, Lea, Flood 2014)
+    z ^= z >> 30;
+    z *= 0xbf58476d1ce4e5b9ULL;
+    z ^= z >> 27;
+    z *= 0x94d049bb133111ebULL;
+    z ^= z >> 31;
+    return z;
+}
+
+struct Oracle {
+    uint32_t R, G, S, B, K;
+    uint64_t C;
+    double prefill_ms, tpot_ms;
+    std::vector<double> rtt;  // [G][R]
+    uint64_t N;
+    std::vector<double> ts;
+    std::vector<uint32_t> in_tok, out_tok;
+    std::vector<uint16_t> origin;
+    std::vector<uint64_t> off, ids;
+    std::vector<Replica> rep;
+    uint64_t next = 0;        // next request to process
+    uint64_t stats[4] = {0, 0, 0, 0};  // sum_i min(h_i+1,n), sum h*, sum n, sum evicted
+};
+
+}  // namespace
+
+extern "C" {
+
+struct gorgo_oracle_config {
+    uint32_t n_replicas, n_regions, slots_per_replica, block_tokens;
+    uint64_t cache_blocks;
+    uint32_t n_params;
+    uint32_t _pad;
+    double prefill_ms_per_token, tpot_ms;
+};
+
+// Copies everything; returns NULL on a malformed configuration.
+void* gorgo_oracle_create(const gorgo_oracle_config* cfg, const double* rtt_ms,
+                          uint64_t n_requests, const double* ts_ms, const uint32_t* input_tokens,
+                          const uint32_t* output_tokens, const uint16_t* origin,
+                          const uint64_t* hash_off, const uint64_t* hash_ids) {
+    if (!cfg || !rtt_ms || cfg->n_replicas == 0 || cfg->n_regions == 0 ||
+        cfg->slots_per_replica == 0 || cfg->block_tokens == 0)
+        return nullptr;
+    if (cfg->n_params != 3 && cfg->n_params != 3 + cfg->n_replicas) return nullptr;
+    Oracle* o = new Oracle();
+    o->R = cfg->n_replicas; o->G = cfg->n_regions; o->S = cfg->slots_per_replica;
+    o->B = cfg->block_tokens; o->K = cfg->n_params; o->C = cfg->cache_blocks;
+    o->prefill_ms = cfg->prefill_ms_per_token; o->tpot_ms = cfg->tpot_ms;
+    o->rtt.assign(rtt_ms, rtt_ms + (size_t)o->G * o->R);
+    o->N = n_requests;
+    o->ts.assign(ts_ms, ts_ms + n_requests);
+    o->in_tok.assign(input_tokens, input_tokens + n_requests);
+    o->out_tok.assign(output_tokens, output_tokens + n_requests);
+    if (origin) o->origin.assign(origin, origin + n_requests);
+    else o->origin.assign(n_requests, 0);
+    o->off.assign(hash_off, hash_off + n_requests + 1);
+    o->ids.assign(hash_ids, hash_ids + hash_off[n_requests]);
+    o->rep.resize(o->R);
+    for (auto& rp : o->rep) rp.free_at.assign(o->S, 0.0);
+    return o;
+}
+
+void gorgo_oracle_destroy(void* h) { delete static_cast<Oracle*>(h); }
+
+// Back to the empty state (no cached blocks, all slots free at time 0, nothing in flight).
+void gorgo_oracle_reset(void* h) {
+    Oracle* o = static_cast<Oracle*>(h);
+    for (auto& rp : o->rep) {
+        rp.cache.clear(); rp.order.clear(); rp.inflight.clear();
+        rp.free_at.assign(o->S, 0.0); rp.load = 0;
+    }
+    o->next = 0;
+    std::memset(o->stats, 0, sizeof(o->stats));
+}
+
+// Routes the next `count` requests with cost-model parameters w[0..K) and timestamp scale
+// `scale`, committing cache and queue state.  All outputs are optional (NULL) and indexed from
+// the first request of this call.  Returns the number of requests processed.
+//   route[j], hit[j]        chosen replica and its prefix-hit length in blocks
+//   ttft[j], e2e[j]         simulated latencies in ms
+//   hit_all[j*R+i]          prefix-hit length on every replica (before the commit)
+//   load_all[j*R+i]         in-flight input tokens on every replica as seen by the score
+//   cost_all[j*R+i]         the score of Eq. 3
+//   evicted[j]              blocks evicted from the chosen replica by this request
+//   occ_after[j]            occupancy of the chosen replica after the commit
+uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count,
+                          uint8_t* route, uint16_t* hit, double* ttft, double* e2e,
+                          uint16_t* hit_all, int64_t* load_all, double* cost_all,
+                          uint32_t* evicted, uint64_t* occ_after) {
+    Oracle* o = static_cast<Oracle*>(h);
+    const uint32_t R = o->R;
+    std::vector<uint64_t> hits(R), unc(R);
+    std::vector<double> cost(R);
+    uint64_t done = 0;
+    for (; done < count && o->next < o->N; ++done, ++o->next) {
+        const uint64_t r = o->next;
+        const double t = scale * o->ts[r];                 // scaled arrival time at the proxy
+        const uint32_t g = o->origin[r];
+        const uint64_t n = o->off[r + 1] - o->off[r];
+        const uint64_t* id = o->ids.data() + o->off[r];
+        const uint64_t in = o->in_tok[r];
+
+        for (uint32_t i = 0; i < R; ++i) {
+            Replica& rp = o->rep[i];
+            // completion events seen by the proxy: finish <= t is no longer in flight
+            while (!rp.inflight.empty() && rp.inflight.begin()->first <= t) {
+                rp.load -= (int64_t)rp.inflight.begin()->second;
+                rp.inflight.erase(rp.inflight.begin());
+            }
+            // longest cached prefix, stop at the first missing block
+            uint64_t hh = 0;
+            while (hh < n && rp.cache.count(id[hh])) ++hh;
+            hits[i] = hh;
+            unc[i] = in - std::min<uint64_t>(hh * o->B, in);
+            double q = (double)rp.load;
+            if (o->K != 3) q = q * w[3 + i];               // per-replica queue-load normaliser
+            // Eq. 3 with explicit weights: three products, two sums, in this order
+            const double a = w[0] * o->rtt[(size_t)g * R + i];
+            const double b = w[1] * (double)unc[i];
+            const double c = w[2] * q;
+            cost[i] = (a + b) + c;
+            if (hit_all) hit_all[done * R + i] = (uint16_t)hh;
+            if (load_all) load_all[done * R + i] = rp.load;
+            if (cost_all) cost_all[done * R + i] = cost[i];
+            o->stats[0] += std::min<uint64_t>(hh + 1, n);
+        }
+        uint32_t best = 0;                                 // lowest index wins ties
+        for (uint32_t i = 1; i < R; ++i)
+            if (cost[i] < cost[best]) best = i;
+
+        // ---- cache commit on the chosen replica (set semantics) ----
+        Replica& rp = o->rep[best];
+        std::vector<char> present(n, 0);
+        uint64_t missing = 0;
+        for (uint64_t k = 0; k < n; ++k) {
+            auto it = rp.cache.find(id[k]);
+            if (it != rp.cache.end()) {
+                present[k] = 1;
+                rp.order.erase(it->second);
+                it->second = Key{r, (uint32_t)k};
+                rp.order.emplace(it->second, id[k]);
+            } else {
+                ++missing;
+            }
+        }
+        uint64_t occ = rp.cache.size();
+        uint64_t E = (occ + missing > o->C) ? (occ + missing - o->C) : 0;
+        uint32_t ev = 0;
+        while (E > 0) {
+            auto victim = rp.order.begin();                // smallest key; never of this request
+            if (victim == rp.order.end() || victim->first.seq == r) break;
+            rp.cache.erase(victim->second);
+            rp.order.erase(victim);
+            --E; ++ev;
+        }
+        for (uint64_t k = 0; k < n; ++k) {
+            if (!present[k]) {
+                Key key{r, (uint32_t)k};
+                rp.cache.emplace(id[k], key);
+                rp.order.emplace(key, id[k]);
+            }
+        }
+
+        // ---- service commit on the chosen replica ----
+        const double arrive = t + o->rtt[(size_t)g * R + best];
+        uint32_t slot = 0;
+        for (uint32_t s = 1; s < o->S; ++s)
+            if (rp.free_at[s] < rp.free_at[slot]) slot = s;
+        const double start = std::max(arrive, rp.free_at[slot]);
+        const double prefill = o->prefill_ms * (double)unc[best];
+        const double first = start + prefill;
+        const uint32_t out = o->out_tok[r];
+        const double decode = o->tpot_ms * (double)(out > 0 ? out - 1 : 0);
+        const double finish = first + decode;
+        rp.free_at[slot] = finish;
+        rp.inflight.emplace(finish, in);
+        rp.load += (int64_t)in;
+
+        if (route) route[done] = (uint8_t)best;
+        if (hit) hit[done] = (uint16_t)hits[best];
+        if (ttft) ttft[done] = first - t;
+        if (e2e) e2e[done] = finish - t;
+        if (evicted) evicted[done] = ev;
+        if (occ_after) occ_after[done] = rp.cache.size();
+        o->stats[1] += hits[best];
+        o->stats[2] += n;
+        o->stats[3] += ev;
+    }
+    return done;
+}
+
+// Nearest-rank percentile: the k-th smallest with k = ceil(0.95 n) in integers.
+double gorgo_oracle_p95(const double* v, uint64_t n) {
+    if (n == 0) return 0.0;
+    std::vector<double> s(v, v + n);
+    std::sort(s.begin(), s.end());
+    const uint64_t k = (95 * n + 99) / 100;
+    return s[k - 1];
+}
+
+// out[2*i] = occupancy of replica i, out[2*i+1] = order-independent sum (mod 2^64) over its
+// cached blocks of mix64(id ^ mix64(seq*65536 + pos)).
+void gorgo_oracle_digest(void* h, uint64_t* out) {
+    Oracle* o = static_cast<Oracle*>(h);
+    for (uint32_t i = 0; i < o->R; ++i) {
+        uint64_t sum = 0;
+        for (const auto& kv : o->rep[i].cache)
+            sum += mix64(kv.first ^ mix64(kv.second.seq * 65536ULL + kv.second.pos));
+        out[2 * i] = o->rep[i].cache.size();
+        out[2 * i + 1] = sum;
+    }
+}
+
+// Cached blocks of one replica in eviction order (first = next victim).  Returns the
+// occupancy; writes at most `cap` entries.
+uint64_t gorgo_oracle_dump(void* h, uint32_t replica, uint64_t cap, uint64_t* ids,
+                           uint64_t* seq, uint32_t* pos) {
+    Oracle* o = static_cast<Oracle*>(h);
+    uint64_t j = 0;
+    for (const auto& kv : o->rep[replica].order) {
+        if (j < cap) {
+            if (ids) ids[j] = kv.second;
+            if (seq) seq[j] = kv.first.seq;
+            if (pos) pos[j] = kv.first.pos;
+        }
+        ++j;
+    }
+    return j;
+}
+
+// loads[i] = in-flight input tokens, inflight[i] = number of in-flight requests (as of the
+// last processed request), free_at[i*S+s] = slot release times.
+void gorgo_oracle_queues(void* h, int64_t* loads, uint64_t* inflight, double* free_at) {
+    Oracle* o = static_cast<Oracle*>(h);
+    for (uint32_t i = 0; i < o->R; ++i) {
+        if (loads) loads[i] = o->rep[i].load;
+        if (inflight) inflight[i] = o->rep[i].inflight.size();
+        if (free_at)
+            for (uint32_t s = 0; s < o->S; ++s) free_at[(size_t)i * o->S + s] = o->rep[i].free_at[s];
+    }
+}
+
+void gorgo_oracle_stats(void* h, uint64_t* out4) {
+    Oracle* o = static_cast<Oracle*>(h);
+    std::memcpy(out4, o->stats, sizeof(o->stats));
+}
+
+uint64_t gorgo_oracle_position(void* h) { return static_cast<Oracle*>(h)->next; }
+
+}  // extern "C"
