@@ -1,0 +1,166 @@
+/* gorgo.h -- C ABI of libgorgo_b200: batched replay of a population of GORGO routing
+ * cost-model parameter vectors over one request trace on one NVIDIA B200 (sm_100a).
+ *
+ * The operation (paper Section 2.2, Eq. 1-3; Section 2.3): for every candidate parameter
+ * vector and every request of the trace, in trace order, compute on every replica the
+ * longest cached prefix of the request's 512-token blocks, the score
+ *     cost_i = ((w_net * RTT[origin][i]) + (w_prefill * uncached_tokens_i)) + (w_queue * q_i)
+ * with q_i the proxy-recorded in-flight input tokens of replica i (optionally times a
+ * per-replica normaliser), route to the lowest-index argmin, update that replica's LRU block
+ * cache and its slot/queue state under the deterministic service model below, and record
+ * TTFT = network + queue wait + prefill of the uncached tokens (Eq. 1) and the end-to-end
+ * latency.  Each candidate's latencies are reduced to their 95th percentile (nearest rank),
+ * the objective the paper tunes (Section 4).
+ *
+ * Service model (the paper names the need for one in Section 2.1 but gives none): S slots per
+ * replica; a request arrives at the engine RTT after its scaled timestamp, takes the slot that
+ * frees first, prefills `prefill_ms_per_token` x uncached tokens, then decodes
+ * `tpot_ms` x max(output_tokens-1, 0); it counts as in flight at the proxy until it finishes.
+ * The cache learns a request at dispatch; eviction is LRU by (request index, block position),
+ * deepest block of the oldest request first.  All cost and time arithmetic is IEEE fp64,
+ * round-to-nearest, no fused multiply-add, in the order written above.
+ *
+ * Conventions: every function returns GORGO_OK (0) or a negative gorgo_status.  No function
+ * throws, aborts or prints.  Pointers are HOST pointers unless the comment says DEVICE.  The
+ * library never allocates or frees device memory: the caller supplies every device buffer
+ * (256-byte aligned) and keeps it alive while the handle uses it.  `cuda_stream` is a
+ * cudaStream_t passed as void* (NULL = the default stream); work is enqueued on it and, unless
+ * stated otherwise, the call does not wait for it.  A handle may be used by one host thread at
+ * a time; distinct handles are independent.
+ */
+#ifndef GORGO_H_
+#define GORGO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gorgo_sim gorgo_sim_t;
+
+typedef enum gorgo_status {
+  GORGO_OK = 0,
+  GORGO_ERR_INVALID_ARG = -1,         /* NULL pointer, zero size, value out of the stated range   */
+  GORGO_ERR_BAD_TRACE = -2,           /* trace violates a precondition listed at gorgo_trace_upload */
+  GORGO_ERR_NONFINITE_PARAM = -3,     /* NaN/Inf among the cost-model parameters or the time scale */
+  GORGO_ERR_WORKSPACE_TOO_SMALL = -4, /* a caller-supplied device buffer is smaller than required  */
+  GORGO_ERR_CUDA = -5,                /* a CUDA runtime call failed                                */
+  GORGO_ERR_DEVICE_LIMIT = -6,        /* a bounded device loop hit its limit (internal invariant)  */
+  GORGO_ERR_NO_TRACE = -7,            /* the call needs an uploaded trace                          */
+  GORGO_ERR_OUT_OF_ORDER = -8         /* gorgo_route_batch: `first` is not the next request        */
+} gorgo_status;
+
+/* Simulator configuration; copied by gorgo_sim_create (rtt_ms included). */
+typedef struct gorgo_config {
+  uint32_t n_replicas;          /* R, 1..64                                                      */
+  uint32_t n_regions;           /* G >= 1, origin regions of requests; G*R <= 4096               */
+  uint32_t slots_per_replica;   /* S, 1..65535 (paper: max_concurrent_requests = 64, Section 4)   */
+  uint32_t block_tokens;        /* B >= 1 tokens per cache block (512)                            */
+  uint64_t cache_blocks;        /* C >= 1 blocks per replica                                      */
+  uint32_t n_params;            /* K: 3 = (w_net, w_prefill, w_queue), or 3 + R with per-replica  */
+                                /* queue-load normalisers appended                                */
+  uint32_t reserved;            /* must be 0                                                      */
+  double prefill_ms_per_token;  /* finite, >= 0                                                   */
+  double tpot_ms;               /* finite, >= 0: time per output token after the first            */
+  const double *rtt_ms;         /* G*R row-major [origin][replica], finite, >= 0                  */
+  int32_t device;               /* CUDA device ordinal                                            */
+} gorgo_config_t;
+
+/* Section 2.2 (signals of Eq. 2): creates a simulator for one replica fleet. */
+int gorgo_sim_create(const gorgo_config_t *cfg, gorgo_sim_t **out);
+int gorgo_sim_destroy(gorgo_sim_t *sim);
+
+/* Upper bound of the device bytes gorgo_trace_upload needs for a trace of `n_requests`
+ * requests with `n_block_ids` block ids in total. */
+int gorgo_trace_bytes(uint64_t n_requests, uint64_t n_block_ids, uint64_t *bytes_out);
+
+/* Section 3 (Mooncake-format trace: timestamps plus request metadata).  Validates the host
+ * arrays, renumbers block ids to dense 32-bit numbers (only equality of ids matters), builds
+ * the per-occurrence "next occurrence of the same block" links used by the LRU, and copies
+ * everything into `dev_trace_buf` (DEVICE, caller-owned, must stay alive and untouched while the
+ * trace is in use).  Waits for the copy, so the host arrays may be freed on return.
+ * Preconditions (else GORGO_ERR_BAD_TRACE): 1 <= n_requests < 2^32-1; ts_ms finite, >= 0 and
+ * non-decreasing; hash_off[0] = 0, non-decreasing, hash_off[n] < 2^32-1;
+ * blocks of request r = hash_off[r+1]-hash_off[r] = ceil(input_tokens[r]/B) <= min(C, 65535);
+ * no id twice inside one request; origin[r] < G (origin may be NULL = all 0). */
+int gorgo_trace_upload(gorgo_sim_t *sim, uint64_t n_requests, const double *ts_ms,
+                       const uint32_t *input_tokens, const uint32_t *output_tokens,
+                       const uint16_t *origin, const uint64_t *hash_off,
+                       const uint64_t *hash_ids, void *dev_trace_buf, uint64_t dev_trace_bytes,
+                       void *cuda_stream);
+
+/* Facts about the uploaded trace: requests, block ids in total, distinct block ids. */
+int gorgo_trace_info(const gorgo_sim_t *sim, uint64_t *n_requests, uint64_t *n_block_ids,
+                     uint64_t *n_distinct);
+
+/* Device bytes gorgo_eval_population needs to keep `resident_candidates` replays in flight at
+ * once (a population larger than that is evaluated in waves).  Needs an uploaded trace. */
+int gorgo_workspace_bytes(const gorgo_sim_t *sim, uint32_t resident_candidates,
+                          uint64_t *bytes_out);
+
+/* Section 2.3 (evaluating candidate weights; objective p95 TTFT, Section 4).  Replays the whole
+ * uploaded trace once per candidate from the empty state, timestamps multiplied by `time_scale`
+ * (Section 3), and reduces each candidate's TTFT and E2E to p95.
+ *   params        P*K doubles row-major, HOST or DEVICE (detected); all finite (host copies are
+ *                 checked: GORGO_ERR_NONFINITE_PARAM)
+ *   workspace     DEVICE scratch of workspace_bytes >= gorgo_workspace_bytes(sim, 1)
+ *   p95_ttft_ms,  DEVICE, P doubles each
+ *   p95_e2e_ms
+ *   route         DEVICE P*N bytes or NULL: chosen replica per candidate and request
+ *   hit_blocks    DEVICE P*N uint16 or NULL: prefix-hit length on the chosen replica
+ *   state_digest  DEVICE P*R*2 uint64 or NULL: per replica (occupancy, sum over cached blocks of
+ *                 mix64(id ^ mix64(seq*65536+pos)) mod 2^64), mix64 = splitmix64 finaliser,
+ *                 id = the caller's 64-bit block id, (seq, pos) = request and position of the
+ *                 block's last touch
+ *   stats         DEVICE P*4 uint64 or NULL: per candidate the sums over requests of
+ *                 sum_i min(h_i+1, n), h on the chosen replica, n, evicted blocks
+ *   cand_status   DEVICE P int32 or NULL: 0, or nonzero if a bounded loop hit its limit
+ * Outputs are valid once `cuda_stream` has been synchronised. */
+int gorgo_eval_population(gorgo_sim_t *sim, uint32_t n_candidates, const double *params,
+                          double time_scale, void *workspace, uint64_t workspace_bytes,
+                          void *cuda_stream, double *p95_ttft_ms, double *p95_e2e_ms,
+                          uint8_t *route, uint16_t *hit_blocks, uint64_t *state_digest,
+                          uint64_t *stats, int32_t *cand_status);
+
+/* Same evaluation with HOST inputs and outputs: copies `params` (HOST, P*K) to the device,
+ * runs, copies p95_ttft_ms / p95_e2e_ms (HOST, P doubles each; pinned memory makes the copies
+ * asynchronous) back and waits for the stream.  Returns GORGO_ERR_DEVICE_LIMIT if any candidate
+ * reported a nonzero status. */
+int gorgo_eval_population_host(gorgo_sim_t *sim, uint32_t n_candidates, const double *params,
+                               double time_scale, void *workspace, uint64_t workspace_bytes,
+                               void *cuda_stream, double *p95_ttft_ms, double *p95_e2e_ms);
+
+/* Online use (Section 2.3, the proxy routing live requests): one persistent simulator state in
+ * caller memory.  gorgo_state_bytes gives its size; gorgo_sim_reset empties it. */
+int gorgo_state_bytes(const gorgo_sim_t *sim, uint64_t *bytes_out);
+int gorgo_sim_reset(gorgo_sim_t *sim, void *state_workspace, uint64_t state_bytes,
+                    void *cuda_stream);
+
+/* Routes requests [first, first+count) of the uploaded trace, in order, with one parameter
+ * vector (HOST, K doubles), commits cache and queue state into `state_workspace` (DEVICE) and
+ * returns the decisions.  `first` must equal the number of requests the state has already seen
+ * (else the state is left untouched and gorgo_state_status reports GORGO_ERR_OUT_OF_ORDER).
+ *   route (DEVICE, count bytes), hit_blocks (DEVICE, count uint16, or NULL),
+ *   ttft_ms / e2e_ms (DEVICE, count doubles, or NULL). */
+int gorgo_route_batch(gorgo_sim_t *sim, const double *params, double time_scale, uint64_t first,
+                      uint64_t count, void *state_workspace, uint64_t state_bytes,
+                      void *cuda_stream, uint8_t *route, uint16_t *hit_blocks, double *ttft_ms,
+                      double *e2e_ms);
+
+/* Digest of the caches held in a persistent state (same definition as state_digest above):
+ * `digest` DEVICE R*2 uint64. */
+int gorgo_state_digest(gorgo_sim_t *sim, void *state_workspace, uint64_t state_bytes,
+                       void *cuda_stream, uint64_t *digest);
+
+/* Waits for `cuda_stream`, then reports how many requests the state has seen and whether a
+ * device-side limit or an out-of-order batch was recorded (return value). */
+int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_bytes,
+                       void *cuda_stream, uint64_t *requests_seen);
+
+const char *gorgo_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GORGO_H_ */

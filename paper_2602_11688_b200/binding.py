@@ -1,0 +1,276 @@
+"""ctypes binding of ``libgorgo_b200.so``: the functions of ``include/gorgo.h`` under the same
+names (argument marshalling only), plus ``GorgoSim``, a small holder of the torch tensors that
+serve as device buffers.  Every step of the simulation runs in the CUDA library; if the library
+is missing this module raises instead of computing anything on the CPU.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgorgo_b200.so")
+
+GORGO_OK = 0
+GORGO_ERR_INVALID_ARG = -1
+GORGO_ERR_BAD_TRACE = -2
+GORGO_ERR_NONFINITE_PARAM = -3
+GORGO_ERR_WORKSPACE_TOO_SMALL = -4
+GORGO_ERR_CUDA = -5
+GORGO_ERR_DEVICE_LIMIT = -6
+GORGO_ERR_NO_TRACE = -7
+GORGO_ERR_OUT_OF_ORDER = -8
+
+EXPORTS = [
+    "gorgo_sim_create", "gorgo_sim_destroy", "gorgo_trace_bytes", "gorgo_trace_upload",
+    "gorgo_trace_info", "gorgo_workspace_bytes", "gorgo_eval_population",
+    "gorgo_eval_population_host", "gorgo_state_bytes", "gorgo_sim_reset", "gorgo_route_batch",
+    "gorgo_state_digest", "gorgo_state_status", "gorgo_strerror",
+]
+
+
+class gorgo_config_t(C.Structure):
+    _fields_ = [("n_replicas", C.c_uint32), ("n_regions", C.c_uint32),
+                ("slots_per_replica", C.c_uint32), ("block_tokens", C.c_uint32),
+                ("cache_blocks", C.c_uint64), ("n_params", C.c_uint32), ("reserved", C.c_uint32),
+                ("prefill_ms_per_token", C.c_double), ("tpot_ms", C.c_double),
+                ("rtt_ms", C.c_void_p), ("device", C.c_int32)]
+
+
+class GorgoError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {gorgo_strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def load():
+    """Load the shared library (built by ``paper_2602_11688_b200.build``); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2602_11688_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, u32, u64, dbl, i32 = C.c_void_p, C.c_uint32, C.c_uint64, C.c_double, C.c_int
+    pu64 = C.POINTER(C.c_uint64)
+    sig = {
+        "gorgo_sim_create": [C.POINTER(gorgo_config_t), C.POINTER(vp)],
+        "gorgo_sim_destroy": [vp],
+        "gorgo_trace_bytes": [u64, u64, pu64],
+        "gorgo_trace_upload": [vp, u64, vp, vp, vp, vp, vp, vp, vp, u64, vp],
+        "gorgo_trace_info": [vp, pu64, pu64, pu64],
+        "gorgo_workspace_bytes": [vp, u32, pu64],
+        "gorgo_eval_population": [vp, u32, vp, dbl, vp, u64, vp, vp, vp, vp, vp, vp, vp, vp],
+        "gorgo_eval_population_host": [vp, u32, vp, dbl, vp, u64, vp, vp, vp],
+        "gorgo_state_bytes": [vp, pu64],
+        "gorgo_sim_reset": [vp, vp, u64, vp],
+        "gorgo_route_batch": [vp, vp, dbl, u64, u64, vp, u64, vp, vp, vp, vp, vp],
+        "gorgo_state_digest": [vp, vp, u64, vp, vp],
+        "gorgo_state_status": [vp, vp, u64, vp, pu64],
+    }
+    for name, argtypes in sig.items():
+        fn = getattr(lib, name)
+        fn.argtypes = argtypes
+        fn.restype = i32
+    lib.gorgo_strerror.argtypes = [i32]
+    lib.gorgo_strerror.restype = C.c_char_p
+    _lib = lib
+    return lib
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _dev_ptr(t) -> Optional[int]:
+    """Raw device address of a torch tensor (None passes NULL)."""
+    return None if t is None else int(t.data_ptr())
+
+
+# ------------------------------------------------------------------ same-name entry points
+def gorgo_strerror(code: int) -> str:
+    return load().gorgo_strerror(int(code)).decode()
+
+
+def gorgo_sim_create(*, n_replicas, n_regions, slots_per_replica, block_tokens, cache_blocks,
+                     n_params, prefill_ms_per_token, tpot_ms, rtt_ms, device=0):
+    """Returns (status, handle)."""
+    rtt = np.ascontiguousarray(rtt_ms, dtype=np.float64)
+    cfg = gorgo_config_t(int(n_replicas), int(n_regions), int(slots_per_replica),
+                         int(block_tokens), int(cache_blocks), int(n_params), 0,
+                         float(prefill_ms_per_token), float(tpot_ms),
+                         rtt.ctypes.data, int(device))
+    h = C.c_void_p()
+    rc = load().gorgo_sim_create(C.byref(cfg), C.byref(h))
+    return rc, h
+
+
+def gorgo_sim_destroy(sim) -> int:
+    return load().gorgo_sim_destroy(sim)
+
+
+def gorgo_trace_bytes(n_requests: int, n_block_ids: int):
+    out = C.c_uint64()
+    rc = load().gorgo_trace_bytes(int(n_requests), int(n_block_ids), C.byref(out))
+    return rc, out.value
+
+
+def gorgo_trace_upload(sim, ts_ms, input_tokens, output_tokens, origin, hash_off, hash_ids,
+                       dev_trace_buf, stream: int = 0) -> int:
+    ts = np.ascontiguousarray(ts_ms, dtype=np.float64)
+    it = np.ascontiguousarray(input_tokens, dtype=np.uint32)
+    ot = np.ascontiguousarray(output_tokens, dtype=np.uint32)
+    org = None if origin is None else np.ascontiguousarray(origin, dtype=np.uint16)
+    off = np.ascontiguousarray(hash_off, dtype=np.uint64)
+    ids = np.ascontiguousarray(hash_ids, dtype=np.uint64)
+    return load().gorgo_trace_upload(sim, ts.shape[0], _np_ptr(ts), _np_ptr(it), _np_ptr(ot),
+                                     _np_ptr(org), _np_ptr(off), _np_ptr(ids),
+                                     _dev_ptr(dev_trace_buf), dev_trace_buf.numel(), stream)
+
+
+def gorgo_trace_info(sim):
+    a, b, c = C.c_uint64(), C.c_uint64(), C.c_uint64()
+    rc = load().gorgo_trace_info(sim, C.byref(a), C.byref(b), C.byref(c))
+    return rc, a.value, b.value, c.value
+
+
+def gorgo_workspace_bytes(sim, resident_candidates: int):
+    out = C.c_uint64()
+    rc = load().gorgo_workspace_bytes(sim, int(resident_candidates), C.byref(out))
+    return rc, out.value
+
+
+def gorgo_eval_population(sim, n_candidates, params, time_scale, workspace, stream,
+                          p95_ttft_ms, p95_e2e_ms, route=None, hit_blocks=None,
+                          state_digest=None, stats=None, cand_status=None) -> int:
+    """``params`` is a contiguous float64 numpy array (host) or torch CUDA tensor (device);
+    every other array argument is a torch CUDA tensor or None."""
+    pp = _np_ptr(params) if isinstance(params, np.ndarray) else _dev_ptr(params)
+    return load().gorgo_eval_population(
+        sim, int(n_candidates), pp, float(time_scale), _dev_ptr(workspace), workspace.numel(),
+        stream, _dev_ptr(p95_ttft_ms), _dev_ptr(p95_e2e_ms), _dev_ptr(route),
+        _dev_ptr(hit_blocks), _dev_ptr(state_digest), _dev_ptr(stats), _dev_ptr(cand_status))
+
+
+def gorgo_eval_population_host(sim, n_candidates, params, time_scale, workspace, stream,
+                               p95_ttft_ms, p95_e2e_ms) -> int:
+    """``params`` / ``p95_*`` are host buffers: numpy arrays or (pinned) CPU torch tensors."""
+    def host_ptr(x):
+        return _np_ptr(x) if isinstance(x, np.ndarray) else int(x.data_ptr())
+    return load().gorgo_eval_population_host(
+        sim, int(n_candidates), host_ptr(params), float(time_scale), _dev_ptr(workspace),
+        workspace.numel(), stream, host_ptr(p95_ttft_ms), host_ptr(p95_e2e_ms))
+
+
+def gorgo_state_bytes(sim):
+    out = C.c_uint64()
+    rc = load().gorgo_state_bytes(sim, C.byref(out))
+    return rc, out.value
+
+
+def gorgo_sim_reset(sim, state_workspace, stream: int = 0) -> int:
+    return load().gorgo_sim_reset(sim, _dev_ptr(state_workspace), state_workspace.numel(), stream)
+
+
+def gorgo_route_batch(sim, params, time_scale, first, count, state_workspace, stream, route,
+                      hit_blocks=None, ttft_ms=None, e2e_ms=None) -> int:
+    w = np.ascontiguousarray(params, dtype=np.float64)
+    return load().gorgo_route_batch(sim, _np_ptr(w), float(time_scale), int(first), int(count),
+                                    _dev_ptr(state_workspace), state_workspace.numel(), stream,
+                                    _dev_ptr(route), _dev_ptr(hit_blocks), _dev_ptr(ttft_ms),
+                                    _dev_ptr(e2e_ms))
+
+
+def gorgo_state_digest(sim, state_workspace, stream, digest) -> int:
+    return load().gorgo_state_digest(sim, _dev_ptr(state_workspace), state_workspace.numel(),
+                                     stream, _dev_ptr(digest))
+
+
+def gorgo_state_status(sim, state_workspace, stream: int = 0):
+    seen = C.c_uint64()
+    rc = load().gorgo_state_status(sim, _dev_ptr(state_workspace), state_workspace.numel(),
+                                   stream, C.byref(seen))
+    return rc, seen.value
+
+
+# ------------------------------------------------------------------------ buffer holder
+class GorgoSim:
+    """Owns the handle and the torch tensors used as device buffers (plumbing only)."""
+
+    def __init__(self, workload, device: int = 0):
+        import torch
+        self.torch = torch
+        self.device = torch.device("cuda", device)
+        self.w = workload
+        rc, self.h = gorgo_sim_create(rtt_ms=workload.rtt_ms, device=device,
+                                      **workload.config_dict())
+        if rc != GORGO_OK:
+            raise GorgoError(rc, "gorgo_sim_create")
+        self.R = workload.spec.n_replicas
+        self.K = workload.n_params
+        self.N = workload.n_requests
+        rc, nbytes = gorgo_trace_bytes(self.N, int(workload.hash_off[-1]))
+        self.trace_buf = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        rc = gorgo_trace_upload(self.h, workload.ts_ms, workload.input_tokens,
+                                workload.output_tokens, workload.origin, workload.hash_off,
+                                workload.hash_ids, self.trace_buf, self.stream)
+        if rc != GORGO_OK:
+            raise GorgoError(rc, "gorgo_trace_upload")
+        self.workspace = None
+
+    @property
+    def stream(self) -> int:
+        return int(self.torch.cuda.current_stream(self.device).cuda_stream)
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.torch.cuda.synchronize(self.device)
+            gorgo_sim_destroy(self.h)
+            self.h = None
+        self.trace_buf = None
+        self.workspace = None
+
+    def ensure_workspace(self, resident: int, max_bytes: Optional[int] = None) -> int:
+        """Allocate a workspace for up to ``resident`` candidates in flight (fewer if
+        ``max_bytes`` does not allow it).  Returns the resident count actually provided."""
+        torch = self.torch
+        while True:
+            rc, nbytes = gorgo_workspace_bytes(self.h, resident)
+            if rc != GORGO_OK:
+                raise GorgoError(rc, "gorgo_workspace_bytes")
+            if max_bytes is None or nbytes <= max_bytes or resident == 1:
+                break
+            resident = max(1, min(resident - 1, int(resident * max_bytes / nbytes)))
+        if self.workspace is None or self.workspace.numel() < nbytes:
+            self.workspace = None
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        return resident
+
+    def eval_population(self, params, time_scale=1.0, *, want_route=False, want_hit=False,
+                        want_digest=False, want_stats=False, resident=None, max_bytes=None):
+        """Device-output evaluation; returns a dict of torch CUDA tensors."""
+        torch = self.torch
+        params = np.ascontiguousarray(params, dtype=np.float64)
+        P = params.shape[0]
+        self.ensure_workspace(P if resident is None else resident, max_bytes)
+        dev = self.device
+        out = dict(p95_ttft=torch.empty(P, dtype=torch.float64, device=dev),
+                   p95_e2e=torch.empty(P, dtype=torch.float64, device=dev),
+                   status=torch.zeros(P, dtype=torch.int32, device=dev))
+        out["route"] = torch.empty((P, self.N), dtype=torch.uint8, device=dev) if want_route else None
+        out["hit"] = torch.empty((P, self.N), dtype=torch.uint16, device=dev) if want_hit else None
+        out["digest"] = torch.empty((P, self.R, 2), dtype=torch.uint64, device=dev) if want_digest else None
+        out["stats"] = torch.empty((P, 4), dtype=torch.uint64, device=dev) if want_stats else None
+        rc = gorgo_eval_population(self.h, P, params, time_scale, self.workspace, self.stream,
+                                   out["p95_ttft"], out["p95_e2e"], out["route"], out["hit"],
+                                   out["digest"], out["stats"], out["status"])
+        if rc != GORGO_OK:
+            raise GorgoError(rc, "gorgo_eval_population")
+        return out

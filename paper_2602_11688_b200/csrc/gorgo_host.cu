@@ -1,0 +1,532 @@
+// Host shell of libgorgo_b200: the C ABI declared in include/gorgo.h.  Argument checks, trace
+// preparation (validation, dense renumbering of block ids, next-occurrence links), workspace
+// layout, wave scheduling and kernel launches.  No step of the simulation runs on the host.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/gorgo.h"
+#include "gorgo_internal.h"
+
+using namespace gorgo;
+
+struct gorgo_sim {
+  Model m;
+  std::vector<double> rtt;
+  int device = 0;
+  bool has_trace = false;
+  TraceView tr = {};
+};
+
+namespace {
+
+constexpr uint64_t kAlign = 256;
+inline uint64_t align_up(uint64_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// 64-bit id -> dense number, open addressing, grows by doubling.
+struct IdMap {
+  std::vector<uint64_t> keys;
+  std::vector<uint32_t> vals;  // 0 = empty, else dense + 1
+  uint64_t mask = 0, used = 0;
+  static uint64_t hash(uint64_t z) {
+    z ^= z >> 33; z *= 0xff51afd7ed558ccdULL; z ^= z >> 33; z *= 0xc4ceb9fe1a85ec53ULL;
+    return z ^ (z >> 33);
+  }
+  explicit IdMap(uint64_t cap_pow2) : keys(cap_pow2), vals(cap_pow2, 0), mask(cap_pow2 - 1) {}
+  void grow() {
+    IdMap bigger((mask + 1) * 2);
+    for (uint64_t i = 0; i <= mask; ++i)
+      if (vals[i]) bigger.put(keys[i], vals[i]);
+    keys.swap(bigger.keys); vals.swap(bigger.vals); mask = bigger.mask;
+  }
+  void put(uint64_t k, uint32_t v) {
+    uint64_t i = hash(k) & mask;
+    while (vals[i]) i = (i + 1) & mask;
+    keys[i] = k; vals[i] = v; ++used;
+  }
+  // returns dense number, assigning `next` if the id is new
+  uint32_t get_or_add(uint64_t k, uint32_t& next) {
+    uint64_t i = hash(k) & mask;
+    while (vals[i]) {
+      if (keys[i] == k) return vals[i] - 1;
+      i = (i + 1) & mask;
+    }
+    if ((used + 1) * 2 > mask + 1) { grow(); return get_or_add(k, next); }
+    keys[i] = k; vals[i] = next + 1; ++used;
+    return next++;
+  }
+};
+
+StateLayout make_layout(const Model& m) {
+  StateLayout l;
+  uint64_t o = sizeof(CandHeader);
+  l.rep_off = o; o += (uint64_t)m.R * sizeof(RepState);
+  const uint64_t rs = (uint64_t)m.R * m.S;
+  l.free_at_off = o; o += rs * 8;
+  l.head_fin_off = o; o += rs * 8;
+  l.head_off = o; o += rs * 4;
+  l.tail_off = o; o += rs * 4;
+  l.bytes = align_up(o);
+  return l;
+}
+
+// Byte offsets of the regions of a workspace for `res` resident candidates.
+struct WsLayout {
+  uint64_t params, rtt, status, p95, masks, states, fin, slot_next, lru_next, route_log, ttft,
+      e2e, total;
+  uint64_t mask_stride;
+  StateLayout st;
+};
+
+WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
+  WsLayout w;
+  const Model& m = s->m;
+  const uint64_t N = s->tr.n_req;
+  w.st = make_layout(m);
+  w.mask_stride = align_up((uint64_t)s->tr.n_distinct * mask_bytes_for(m.R));
+  uint64_t o = 0;
+  w.params = o; o = align_up(o + res * m.K * 8);
+  w.rtt = o; o = align_up(o + (uint64_t)m.G * m.R * 8);
+  w.status = o; o = align_up(o + res * 4);
+  w.p95 = o; o = align_up(o + res * 16);
+  w.masks = o; o = align_up(o + res * w.mask_stride);
+  w.states = o; o = align_up(o + res * w.st.bytes);
+  w.fin = o; o = align_up(o + res * N * 8);
+  w.slot_next = o; o = align_up(o + res * N * 4);
+  w.lru_next = o; o = align_up(o + res * N * 4);
+  w.route_log = o; o = align_up(o + res * N);
+  w.ttft = o; if (with_latency) o = align_up(o + res * N * 8);
+  w.e2e = o; if (with_latency) o = align_up(o + res * N * 8);
+  w.total = o;
+  return w;
+}
+
+bool is_device_pointer(const void* p) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return false; }
+  return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged;
+}
+
+bool all_finite(const double* v, uint64_t n) {
+  for (uint64_t i = 0; i < n; ++i)
+    if (!std::isfinite(v[i])) return false;
+  return true;
+}
+
+bool finite_nonneg(double v) { return std::isfinite(v) && v >= 0.0; }
+
+int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, void* workspace,
+              uint64_t workspace_bytes, cudaStream_t st, double* p95_ttft, double* p95_e2e,
+              uint8_t* route, uint16_t* hit, uint64_t* digest, uint64_t* stats, int32_t* cand_status,
+              bool host_io) {
+  if (!sim || !params || !workspace || P == 0) return GORGO_ERR_INVALID_ARG;
+  if (!p95_ttft || !p95_e2e) return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  if (!finite_nonneg(scale)) return GORGO_ERR_NONFINITE_PARAM;
+  if ((uintptr_t)workspace % kAlign) return GORGO_ERR_INVALID_ARG;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  const Model& m = sim->m;
+  const uint64_t N = sim->tr.n_req;
+  const bool params_on_device = !host_io && is_device_pointer(params);
+  if (!params_on_device && !all_finite(params, (uint64_t)P * m.K)) return GORGO_ERR_NONFINITE_PARAM;
+
+  // largest number of resident candidates the workspace can hold
+  uint64_t lo = 0, hi = P;
+  while (lo < hi) {
+    const uint64_t mid = (lo + hi + 1) / 2;
+    if (make_ws(sim, mid, true).total <= workspace_bytes) lo = mid; else hi = mid - 1;
+  }
+  if (lo == 0) return GORGO_ERR_WORKSPACE_TOO_SMALL;
+  const uint32_t res = (uint32_t)lo;
+  const WsLayout w = make_ws(sim, res, true);
+  unsigned char* base = static_cast<unsigned char*>(workspace);
+  double* d_params = reinterpret_cast<double*>(base + w.params);
+  double* d_rtt = reinterpret_cast<double*>(base + w.rtt);
+  int32_t* d_status = reinterpret_cast<int32_t*>(base + w.status);
+  double* d_p95 = reinterpret_cast<double*>(base + w.p95);
+
+  if (cudaMemcpyAsync(d_rtt, sim->rtt.data(), sim->rtt.size() * 8, cudaMemcpyHostToDevice, st) !=
+      cudaSuccess)
+    return GORGO_ERR_CUDA;
+  std::vector<int32_t> h_status;
+  if (host_io) h_status.assign(P, 0);
+
+  for (uint32_t p0 = 0; p0 < P; p0 += res) {
+    const uint32_t pw = (P - p0 < res) ? (P - p0) : res;
+    const double* wave_params;
+    if (params_on_device) {
+      wave_params = params + (size_t)p0 * m.K;
+    } else {
+      if (cudaMemcpyAsync(d_params, params + (size_t)p0 * m.K, (size_t)pw * m.K * 8,
+                          cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return GORGO_ERR_CUDA;
+      wave_params = d_params;
+    }
+    if (launch_reset(base + w.masks, (uint64_t)pw * w.mask_stride, base + w.states, w.st, m, pw,
+                     st) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+    if (stats && cudaMemsetAsync(stats + (size_t)p0 * 4, 0, (size_t)pw * 32, st) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+
+    ReplayArgs a = {};
+    a.m = m; a.tr = sim->tr; a.scale = scale;
+    a.first = 0; a.count = (uint32_t)N; a.check_order = 0;
+    a.rtt = d_rtt; a.params = wave_params;
+    a.masks = base + w.masks; a.mask_stride = w.mask_stride;
+    a.states = base + w.states; a.lay = w.st;
+    a.fin = reinterpret_cast<double*>(base + w.fin);
+    a.slot_next = reinterpret_cast<uint32_t*>(base + w.slot_next);
+    a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
+    a.route_log = route ? route + (size_t)p0 * N : base + w.route_log;
+    a.route_log_stride = N;
+    a.route_out = nullptr;
+    a.hit_out = hit ? hit + (size_t)p0 * N : nullptr;
+    a.ttft_out = reinterpret_cast<double*>(base + w.ttft);
+    a.e2e_out = reinterpret_cast<double*>(base + w.e2e);
+    a.out_stride = N;
+    a.stats = stats ? stats + (size_t)p0 * 4 : nullptr;
+    a.status_out = cand_status ? cand_status + p0 : d_status;
+    if (launch_replay(a, pw, st) != cudaSuccess) return GORGO_ERR_CUDA;
+
+    SelectArgs s = {};
+    s.ttft = a.ttft_out; s.e2e = a.e2e_out; s.stride = N; s.n = (uint32_t)N;
+    s.p95_ttft = host_io ? d_p95 : p95_ttft + p0;
+    s.p95_e2e = host_io ? d_p95 + res : p95_e2e + p0;
+    if (launch_select(s, pw, st) != cudaSuccess) return GORGO_ERR_CUDA;
+
+    if (digest) {
+      DigestArgs d = {};
+      d.m = m; d.tr = sim->tr; d.states = base + w.states; d.lay = w.st;
+      d.route_log = a.route_log; d.route_log_stride = N;
+      d.digest = digest + (size_t)p0 * m.R * 2;
+      if (launch_digest(d, pw, st) != cudaSuccess) return GORGO_ERR_CUDA;
+    }
+    if (host_io) {
+      if (cudaMemcpyAsync(p95_ttft + p0, d_p95, (size_t)pw * 8, cudaMemcpyDeviceToHost, st) !=
+              cudaSuccess ||
+          cudaMemcpyAsync(p95_e2e + p0, d_p95 + res, (size_t)pw * 8, cudaMemcpyDeviceToHost, st) !=
+              cudaSuccess ||
+          cudaMemcpyAsync(h_status.data() + p0, d_status, (size_t)pw * 4, cudaMemcpyDeviceToHost,
+                          st) != cudaSuccess)
+        return GORGO_ERR_CUDA;
+    }
+  }
+  if (host_io) {
+    if (cudaStreamSynchronize(st) != cudaSuccess) return GORGO_ERR_CUDA;
+    for (uint32_t p = 0; p < P; ++p)
+      if (h_status[p] != 0) return GORGO_ERR_DEVICE_LIMIT;
+  }
+  return GORGO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gorgo_sim_create(const gorgo_config_t* cfg, gorgo_sim_t** out) {
+  if (!cfg || !out || !cfg->rtt_ms) return GORGO_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->n_replicas < 1 || cfg->n_replicas > 64 || cfg->n_regions < 1 ||
+      (uint64_t)cfg->n_regions * cfg->n_replicas > 4096 || cfg->slots_per_replica < 1 ||
+      cfg->slots_per_replica > 65535 || cfg->block_tokens < 1 || cfg->cache_blocks < 1 ||
+      cfg->cache_blocks > 0xFFFFFFF0ull || cfg->reserved != 0)
+    return GORGO_ERR_INVALID_ARG;
+  if (cfg->n_params != 3 && cfg->n_params != 3 + cfg->n_replicas) return GORGO_ERR_INVALID_ARG;
+  if (!finite_nonneg(cfg->prefill_ms_per_token) || !finite_nonneg(cfg->tpot_ms))
+    return GORGO_ERR_INVALID_ARG;
+  const uint64_t gr = (uint64_t)cfg->n_regions * cfg->n_replicas;
+  for (uint64_t i = 0; i < gr; ++i)
+    if (!finite_nonneg(cfg->rtt_ms[i])) return GORGO_ERR_INVALID_ARG;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess) { cudaGetLastError(); return GORGO_ERR_CUDA; }
+  if (cfg->device < 0 || cfg->device >= n_dev) return GORGO_ERR_INVALID_ARG;
+  gorgo_sim* s = new (std::nothrow) gorgo_sim();
+  if (!s) return GORGO_ERR_INVALID_ARG;
+  s->m.R = cfg->n_replicas; s->m.G = cfg->n_regions; s->m.S = cfg->slots_per_replica;
+  s->m.B = cfg->block_tokens; s->m.K = cfg->n_params; s->m.C = cfg->cache_blocks;
+  s->m.prefill_ms = cfg->prefill_ms_per_token; s->m.tpot_ms = cfg->tpot_ms;
+  s->rtt.assign(cfg->rtt_ms, cfg->rtt_ms + gr);
+  s->device = cfg->device;
+  *out = s;
+  return GORGO_OK;
+}
+
+int gorgo_sim_destroy(gorgo_sim_t* sim) {
+  if (!sim) return GORGO_ERR_INVALID_ARG;
+  delete sim;
+  return GORGO_OK;
+}
+
+int gorgo_trace_bytes(uint64_t n_requests, uint64_t n_block_ids, uint64_t* bytes_out) {
+  if (!bytes_out) return GORGO_ERR_INVALID_ARG;
+  *bytes_out = align_up(n_requests * sizeof(ReqRec)) + align_up(n_block_ids * 4) +
+               align_up(n_block_ids * 8) + align_up(n_block_ids * 8) + kAlign;
+  return GORGO_OK;
+}
+
+int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_ms,
+                       const uint32_t* input_tokens, const uint32_t* output_tokens,
+                       const uint16_t* origin, const uint64_t* hash_off, const uint64_t* hash_ids,
+                       void* dev_trace_buf, uint64_t dev_trace_bytes, void* cuda_stream) {
+  if (!sim || !ts_ms || !input_tokens || !output_tokens || !hash_off || !dev_trace_buf)
+    return GORGO_ERR_INVALID_ARG;
+  if ((uintptr_t)dev_trace_buf % kAlign) return GORGO_ERR_INVALID_ARG;
+  const Model& m = sim->m;
+  const uint64_t N = n_requests;
+  if (N < 1 || N >= 0xFFFFFFFFull) return GORGO_ERR_BAD_TRACE;
+  if (hash_off[0] != 0) return GORGO_ERR_BAD_TRACE;
+  for (uint64_t r = 0; r < N; ++r)
+    if (hash_off[r + 1] < hash_off[r]) return GORGO_ERR_BAD_TRACE;
+  const uint64_t T = hash_off[N];
+  if (T >= 0xFFFFFFFFull) return GORGO_ERR_BAD_TRACE;
+  if (T > 0 && !hash_ids) return GORGO_ERR_INVALID_ARG;
+  uint64_t need = 0;
+  gorgo_trace_bytes(N, T, &need);
+  if (dev_trace_bytes < need) return GORGO_ERR_WORKSPACE_TOO_SMALL;
+  const uint64_t nmax = m.C < 65535 ? m.C : 65535;
+
+  std::vector<ReqRec> req(N);
+  double prev_t = 0.0;
+  for (uint64_t r = 0; r < N; ++r) {
+    const double t = ts_ms[r];
+    if (!finite_nonneg(t) || t < prev_t) return GORGO_ERR_BAD_TRACE;
+    prev_t = t;
+    const uint64_t n = hash_off[r + 1] - hash_off[r];
+    const uint64_t want = ((uint64_t)input_tokens[r] + m.B - 1) / m.B;
+    if (n != want || n > nmax) return GORGO_ERR_BAD_TRACE;
+    const uint16_t g = origin ? origin[r] : (uint16_t)0;
+    if (g >= m.G) return GORGO_ERR_BAD_TRACE;
+    ReqRec& q = req[r];
+    q.ts_ms = t; q.off = (uint32_t)hash_off[r]; q.in_tok = input_tokens[r];
+    q.out_tok = output_tokens[r]; q.nblk = (uint16_t)n; q.origin = g; q.pad[0] = q.pad[1] = 0;
+  }
+
+  // dense renumbering in order of first appearance; an id twice in one request is an error
+  std::vector<uint32_t> ids(T);
+  std::vector<uint64_t> raw;
+  {
+    IdMap map(1ull << 16);
+    std::vector<uint32_t> seen_in;  // request (+1) that last contained the dense id
+    uint32_t next = 0;
+    for (uint64_t r = 0; r < N; ++r) {
+      for (uint64_t g = hash_off[r]; g < hash_off[r + 1]; ++g) {
+        const uint32_t before = next;
+        const uint32_t d = map.get_or_add(hash_ids[g], next);
+        if (next != before) { raw.push_back(hash_ids[g]); seen_in.push_back(0); }
+        if (seen_in[d] == (uint32_t)r + 1) return GORGO_ERR_BAD_TRACE;
+        seen_in[d] = (uint32_t)r + 1;
+        ids[g] = d;
+      }
+    }
+  }
+  const uint64_t D = raw.size();
+
+  // next occurrence of the same block, and the request it belongs to
+  std::vector<uint2> occ(T);
+  {
+    std::vector<uint32_t> last_g(D, kNone), last_r(D, kNone);
+    for (uint64_t r = N; r-- > 0;) {
+      for (uint64_t g = hash_off[r + 1]; g-- > hash_off[r];) {
+        const uint32_t d = ids[g];
+        occ[g] = make_uint2(last_g[d], last_r[d]);
+        last_g[d] = (uint32_t)g;
+        last_r[d] = (uint32_t)r;
+      }
+    }
+  }
+
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* base = static_cast<unsigned char*>(dev_trace_buf);
+  uint64_t o = 0;
+  unsigned char* d_req = base + o; o += align_up(N * sizeof(ReqRec));
+  unsigned char* d_ids = base + o; o += align_up(T * 4);
+  unsigned char* d_occ = base + o; o += align_up(T * 8);
+  unsigned char* d_raw = base + o; o += align_up(D * 8);
+  bool ok = cudaMemcpyAsync(d_req, req.data(), N * sizeof(ReqRec), cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (T > 0) {
+    ok = ok && cudaMemcpyAsync(d_ids, ids.data(), T * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d_occ, occ.data(), T * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d_raw, raw.data(), D * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); sim->has_trace = false; return GORGO_ERR_CUDA; }
+  sim->tr.req = reinterpret_cast<const ReqRec*>(d_req);
+  sim->tr.ids = reinterpret_cast<const uint32_t*>(d_ids);
+  sim->tr.occ_next = reinterpret_cast<const uint2*>(d_occ);
+  sim->tr.raw_id = reinterpret_cast<const uint64_t*>(d_raw);
+  sim->tr.n_req = (uint32_t)N; sim->tr.n_ids = (uint32_t)T; sim->tr.n_distinct = (uint32_t)D;
+  sim->has_trace = true;
+  return GORGO_OK;
+}
+
+int gorgo_trace_info(const gorgo_sim_t* sim, uint64_t* n_requests, uint64_t* n_block_ids,
+                     uint64_t* n_distinct) {
+  if (!sim) return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  if (n_requests) *n_requests = sim->tr.n_req;
+  if (n_block_ids) *n_block_ids = sim->tr.n_ids;
+  if (n_distinct) *n_distinct = sim->tr.n_distinct;
+  return GORGO_OK;
+}
+
+int gorgo_workspace_bytes(const gorgo_sim_t* sim, uint32_t resident_candidates,
+                          uint64_t* bytes_out) {
+  if (!sim || !bytes_out || resident_candidates == 0) return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  *bytes_out = make_ws(sim, resident_candidates, true).total;
+  return GORGO_OK;
+}
+
+int gorgo_eval_population(gorgo_sim_t* sim, uint32_t n_candidates, const double* params,
+                          double time_scale, void* workspace, uint64_t workspace_bytes,
+                          void* cuda_stream, double* p95_ttft_ms, double* p95_e2e_ms,
+                          uint8_t* route, uint16_t* hit_blocks, uint64_t* state_digest,
+                          uint64_t* stats, int32_t* cand_status) {
+  return eval_impl(sim, n_candidates, params, time_scale, workspace, workspace_bytes,
+                   static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, route,
+                   hit_blocks, state_digest, stats, cand_status, false);
+}
+
+int gorgo_eval_population_host(gorgo_sim_t* sim, uint32_t n_candidates, const double* params,
+                               double time_scale, void* workspace, uint64_t workspace_bytes,
+                               void* cuda_stream, double* p95_ttft_ms, double* p95_e2e_ms) {
+  return eval_impl(sim, n_candidates, params, time_scale, workspace, workspace_bytes,
+                   static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, nullptr,
+                   nullptr, nullptr, nullptr, nullptr, true);
+}
+
+int gorgo_state_bytes(const gorgo_sim_t* sim, uint64_t* bytes_out) {
+  if (!sim || !bytes_out) return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  *bytes_out = make_ws(sim, 1, false).total;
+  return GORGO_OK;
+}
+
+static int state_check(gorgo_sim_t* sim, void* ws, uint64_t bytes, WsLayout* w) {
+  if (!sim || !ws) return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  if ((uintptr_t)ws % kAlign) return GORGO_ERR_INVALID_ARG;
+  *w = make_ws(sim, 1, false);
+  if (bytes < w->total) return GORGO_ERR_WORKSPACE_TOO_SMALL;
+  return GORGO_OK;
+}
+
+int gorgo_sim_reset(gorgo_sim_t* sim, void* state_workspace, uint64_t state_bytes,
+                    void* cuda_stream) {
+  WsLayout w;
+  const int rc = state_check(sim, state_workspace, state_bytes, &w);
+  if (rc != GORGO_OK) return rc;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  unsigned char* base = static_cast<unsigned char*>(state_workspace);
+  if (launch_reset(base + w.masks, w.mask_stride, base + w.states, w.st, sim->m, 1,
+                   static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return GORGO_ERR_CUDA;
+  return GORGO_OK;
+}
+
+int gorgo_route_batch(gorgo_sim_t* sim, const double* params, double time_scale, uint64_t first,
+                      uint64_t count, void* state_workspace, uint64_t state_bytes,
+                      void* cuda_stream, uint8_t* route, uint16_t* hit_blocks, double* ttft_ms,
+                      double* e2e_ms) {
+  WsLayout w;
+  const int rc = state_check(sim, state_workspace, state_bytes, &w);
+  if (rc != GORGO_OK) return rc;
+  if (!params || !route) return GORGO_ERR_INVALID_ARG;
+  const uint64_t N = sim->tr.n_req;
+  if (first > N || count > N - first) return GORGO_ERR_INVALID_ARG;
+  if (!finite_nonneg(time_scale) || !all_finite(params, sim->m.K)) return GORGO_ERR_NONFINITE_PARAM;
+  if (count == 0) return GORGO_OK;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* base = static_cast<unsigned char*>(state_workspace);
+  double* d_params = reinterpret_cast<double*>(base + w.params);
+  double* d_rtt = reinterpret_cast<double*>(base + w.rtt);
+  if (cudaMemcpyAsync(d_rtt, sim->rtt.data(), sim->rtt.size() * 8, cudaMemcpyHostToDevice, st) !=
+          cudaSuccess ||
+      cudaMemcpyAsync(d_params, params, (size_t)sim->m.K * 8, cudaMemcpyHostToDevice, st) !=
+          cudaSuccess)
+    return GORGO_ERR_CUDA;
+  ReplayArgs a = {};
+  a.m = sim->m; a.tr = sim->tr; a.scale = time_scale;
+  a.first = (uint32_t)first; a.count = (uint32_t)count; a.check_order = 1;
+  a.rtt = d_rtt; a.params = d_params;
+  a.masks = base + w.masks; a.mask_stride = w.mask_stride;
+  a.states = base + w.states; a.lay = w.st;
+  a.fin = reinterpret_cast<double*>(base + w.fin);
+  a.slot_next = reinterpret_cast<uint32_t*>(base + w.slot_next);
+  a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
+  a.route_log = base + w.route_log; a.route_log_stride = N;
+  a.route_out = route; a.hit_out = hit_blocks; a.ttft_out = ttft_ms; a.e2e_out = e2e_ms;
+  a.out_stride = count;
+  a.stats = nullptr; a.status_out = nullptr;
+  if (launch_replay(a, 1, st) != cudaSuccess) return GORGO_ERR_CUDA;
+  return GORGO_OK;
+}
+
+int gorgo_state_digest(gorgo_sim_t* sim, void* state_workspace, uint64_t state_bytes,
+                       void* cuda_stream, uint64_t* digest) {
+  WsLayout w;
+  const int rc = state_check(sim, state_workspace, state_bytes, &w);
+  if (rc != GORGO_OK) return rc;
+  if (!digest) return GORGO_ERR_INVALID_ARG;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  unsigned char* base = static_cast<unsigned char*>(state_workspace);
+  DigestArgs d = {};
+  d.m = sim->m; d.tr = sim->tr; d.states = base + w.states; d.lay = w.st;
+  d.route_log = base + w.route_log; d.route_log_stride = sim->tr.n_req;
+  d.digest = digest;
+  if (launch_digest(d, 1, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return GORGO_ERR_CUDA;
+  return GORGO_OK;
+}
+
+int gorgo_state_status(gorgo_sim_t* sim, void* state_workspace, uint64_t state_bytes,
+                       void* cuda_stream, uint64_t* requests_seen) {
+  WsLayout w;
+  const int rc = state_check(sim, state_workspace, state_bytes, &w);
+  if (rc != GORGO_OK) return rc;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CandHeader h;
+  if (cudaMemcpyAsync(&h, static_cast<unsigned char*>(state_workspace) + w.states, sizeof(h),
+                      cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return GORGO_ERR_CUDA;
+  if (requests_seen) *requests_seen = h.processed;
+  return h.status;
+}
+
+const char* gorgo_strerror(int code) {
+  switch (code) {
+    case GORGO_OK: return "ok";
+    case GORGO_ERR_INVALID_ARG: return "invalid argument";
+    case GORGO_ERR_BAD_TRACE: return "trace violates a precondition";
+    case GORGO_ERR_NONFINITE_PARAM: return "non-finite parameter or time scale";
+    case GORGO_ERR_WORKSPACE_TOO_SMALL: return "device buffer too small";
+    case GORGO_ERR_CUDA: return "CUDA runtime error";
+    case GORGO_ERR_DEVICE_LIMIT: return "device-side loop limit reached";
+    case GORGO_ERR_NO_TRACE: return "no trace uploaded";
+    case GORGO_ERR_OUT_OF_ORDER: return "request batch out of order";
+    default: return "unknown gorgo status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,124 @@
+// Internal declarations shared by the host shell and the kernels of libgorgo_b200.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace gorgo {
+
+constexpr uint32_t kNone = 0xFFFFFFFFu;
+
+// One request of the trace as the kernels read it: exactly one 32-byte sector.
+struct __align__(32) ReqRec {
+  double ts_ms;       // arrival at the proxy (unscaled)
+  uint32_t off;       // first block id of the request in the flat id array
+  uint32_t in_tok;    // input tokens
+  uint32_t out_tok;   // output tokens
+  uint16_t nblk;      // number of blocks
+  uint16_t origin;    // origin region
+  uint32_t pad[2];
+};
+static_assert(sizeof(ReqRec) == 32, "ReqRec must be one sector");
+
+// Per-(candidate, replica) scalars kept in global memory between launches.
+struct __align__(32) RepState {
+  long long load;     // in-flight input tokens
+  double min_fin;     // earliest finish among in-flight requests (+inf if none)
+  uint32_t occ;       // cached blocks
+  uint32_t cur_req;   // eviction cursor: request whose touches are examined next (kNone: none yet)
+  int32_t cur_pos;    //   next position of that request to examine (counts down; <0: exhausted)
+  uint32_t lru_tail;  // last request routed to this replica (kNone: none yet)
+};
+static_assert(sizeof(RepState) == 32, "RepState layout");
+
+// Header of one candidate's state block.
+struct __align__(32) CandHeader {
+  uint32_t processed;  // requests replayed so far
+  int32_t status;      // 0, or a gorgo_status recorded by a kernel
+  uint32_t pad[6];
+};
+
+// Device-resident trace (pointers into the caller's trace buffer).
+struct TraceView {
+  const ReqRec* req;       // [N]
+  const uint32_t* ids;     // [T] dense block ids, request after request
+  const uint2* occ_next;   // [T] (.x = flat index of the next occurrence of the same block or
+                           //      kNone, .y = request of that occurrence)
+  const uint64_t* raw_id;  // [D] caller's 64-bit id of each dense id
+  uint32_t n_req, n_ids, n_distinct;
+};
+
+// Model constants.
+struct Model {
+  uint32_t R, G, S, B, K;
+  uint64_t C;
+  double prefill_ms, tpot_ms;
+};
+
+// Layout of one candidate's state block (bytes from its start); the mask array of the
+// candidate lives in a separate region.
+struct StateLayout {
+  uint64_t rep_off;        // RepState[R]
+  uint64_t free_at_off;    // double[R*S]   time each slot frees
+  uint64_t head_fin_off;   // double[R*S]   finish of the oldest in-flight request of the slot
+  uint64_t head_off;       // uint32[R*S]   that request (kNone: slot has nothing in flight)
+  uint64_t tail_off;       // uint32[R*S]   newest request queued on the slot
+  uint64_t bytes;          // size of the block (multiple of 256)
+};
+
+// Everything one replay launch needs.  Candidate p of the launch uses element/byte strides.
+struct ReplayArgs {
+  Model m;
+  TraceView tr;
+  double scale;
+  uint32_t first, count;          // requests [first, first+count)
+  uint32_t check_order;           // 1: refuse (status) unless header.processed == first
+  const double* rtt;              // [G*R] device
+  const double* params;           // [P*K] device
+  unsigned char* masks;           // [P * mask_stride] bytes
+  uint64_t mask_stride;           // bytes per candidate
+  unsigned char* states;          // [P * layout.bytes]
+  StateLayout lay;
+  // per-request arrays, candidate p at + p*N elements
+  double* fin;                    // finish time of each request
+  uint32_t* slot_next;            // next request queued on the same (replica, slot)
+  uint32_t* lru_next;             // next request routed to the same replica
+  uint8_t* route_log;             // chosen replica of every request replayed so far
+  uint64_t route_log_stride;      // elements between candidates
+  // outputs, candidate p at + p*out_stride, request r at + (r-first); any may be null
+  uint8_t* route_out;
+  uint16_t* hit_out;
+  double* ttft_out;
+  double* e2e_out;
+  uint64_t out_stride;
+  uint64_t* stats;                // [P*4] or null (accumulated)
+  int32_t* status_out;            // [P] or null
+};
+
+struct SelectArgs {
+  const double* ttft;             // [P*stride]
+  const double* e2e;
+  uint64_t stride;
+  uint32_t n;                     // values per candidate
+  double* p95_ttft;               // [P]
+  double* p95_e2e;
+};
+
+struct DigestArgs {
+  Model m;
+  TraceView tr;
+  const unsigned char* states;
+  StateLayout lay;
+  const uint8_t* route_log;
+  uint64_t route_log_stride;
+  uint64_t* digest;               // [P*R*2], zeroed by the launcher
+};
+
+cudaError_t launch_reset(unsigned char* masks, uint64_t mask_bytes_total, unsigned char* states,
+                         const StateLayout& lay, const Model& m, uint32_t n_cand,
+                         cudaStream_t st);
+cudaError_t launch_replay(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st);
+cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st);
+cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st);
+uint32_t mask_bytes_for(uint32_t n_replicas);
+
+}  // namespace gorgo

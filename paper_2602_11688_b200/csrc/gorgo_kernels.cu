@@ -1,0 +1,550 @@
+// Kernels of libgorgo_b200 (sm_100a): population replay, p95 selection, state digest, reset.
+//
+// Data layout chosen for this machine rather than per-replica hash tables:
+//  * block ids are dense 32-bit numbers (renumbered at upload in order of first appearance, so
+//    the blocks of one conversation are runs of consecutive numbers);
+//  * per candidate ONE direct-indexed array `mask[id]` whose bit i says "block id is cached on
+//    replica i".  A request's prefix probe on all R replicas is one coalesced read of its n
+//    mask words, a prefix-AND across lanes and a few ballots;
+//  * exact LRU without per-block recency stamps: the recency order of replica i is the order of
+//    the requests routed to it (a linked list through `lru_next`), deepest block first inside a
+//    request.  An eviction cursor walks that order; a touch (request n, position k) is still the
+//    block's latest touch on replica i iff no later occurrence of the block (static
+//    `occ_next` links computed at upload) belongs to a request routed to i.  Live touches at
+//    the cursor are the LRU victims; stale ones are skipped for good;
+//  * in-flight accounting through per-slot FIFO chains (finish times on one slot never
+//    decrease), with the earliest finish per replica cached so the common case is one compare.
+// One warp replays one candidate; requests are strictly ordered inside a candidate, so the
+// parallelism is across candidates, across the blocks of a request and across replicas.
+#include "gorgo_internal.h"
+
+namespace gorgo {
+
+namespace {
+
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+__device__ __forceinline__ double d_inf() { return __longlong_as_double(0x7FF0000000000000LL); }
+
+template <typename T> struct MaskOps;
+template <> struct MaskOps<uint8_t>  { using Sh = uint32_t; };
+template <> struct MaskOps<uint16_t> { using Sh = uint32_t; };
+template <> struct MaskOps<uint32_t> { using Sh = uint32_t; };
+template <> struct MaskOps<uint64_t> { using Sh = uint64_t; };
+
+template <typename MaskT>
+__device__ __forceinline__ MaskT shfl_up_mask(MaskT v, int d) {
+  using Sh = typename MaskOps<MaskT>::Sh;
+  return (MaskT)__shfl_up_sync(kFull, (Sh)v, d);
+}
+template <typename MaskT>
+__device__ __forceinline__ MaskT shfl_mask(MaskT v, int src) {
+  using Sh = typename MaskOps<MaskT>::Sh;
+  return (MaskT)__shfl_sync(kFull, (Sh)v, src);
+}
+template <typename MaskT>
+__device__ __forceinline__ int first_bit(MaskT v) {  // v != 0
+  if (sizeof(MaskT) == 8) return __ffsll((long long)v) - 1;
+  return __ffs((int)(uint32_t)v) - 1;
+}
+
+__device__ __forceinline__ long long warp_sum_ll(long long v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(kFull, v, d);
+  return v;
+}
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(kFull, v, d);
+  return v;
+}
+__device__ __forceinline__ double warp_min_d(double v) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) v = fmin(v, __shfl_xor_sync(kFull, v, d));
+  return v;
+}
+// Minimum of (value, index) pairs, the lower index winning equal values.
+__device__ __forceinline__ void warp_argmin(double& v, uint32_t& i) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    const double ov = __shfl_xor_sync(kFull, v, d);
+    const uint32_t oi = __shfl_xor_sync(kFull, i, d);
+    if (ov < v || (ov == v && oi < i)) { v = ov; i = oi; }
+  }
+}
+
+// Is the touch at flat position g (a block of a request routed to replica `rep`) no longer
+// the block's latest touch there, looking at requests up to `r_now`?  `rep_now` is the route of
+// request r_now if its log entry has not been written yet (else pass the logged value).
+__device__ __forceinline__ bool touch_is_stale(const TraceView& tr, const uint8_t* route_log,
+                                               uint32_t g, uint32_t rep, uint32_t r_now,
+                                               uint32_t rep_now) {
+  uint2 nx = tr.occ_next[g];
+  while (nx.x != kNone && nx.y <= r_now) {
+    const uint32_t rt = (nx.y == r_now) ? rep_now : (uint32_t)route_log[nx.y];
+    if (rt == rep) return true;
+    nx = tr.occ_next[nx.x];
+  }
+  return false;
+}
+
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {  // splitmix64 finaliser
+  z ^= z >> 30; z *= 0xbf58476d1ce4e5b9ULL;
+  z ^= z >> 27; z *= 0x94d049bb133111ebULL;
+  z ^= z >> 31;
+  return z;
+}
+
+// ------------------------------------------------------------------------------ replay
+template <typename MaskT>
+__global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
+  const uint32_t p = blockIdx.x;
+  const uint32_t lane = threadIdx.x;
+  const uint32_t R = a.m.R, S = a.m.S, K = a.m.K, G = a.m.G;
+  const uint32_t N = a.tr.n_req;
+
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* s_rtt = reinterpret_cast<double*>(smem_raw);   // [G*R]
+  double* s_w = s_rtt + (size_t)G * R;                   // [K]
+  double* s_minfin = s_w + K;                            // [R]
+  long long* s_load = reinterpret_cast<long long*>(s_minfin + R);  // [R]
+  uint32_t* s_occ = reinterpret_cast<uint32_t*>(s_load + R);       // [R]
+  uint32_t* s_curreq = s_occ + R;
+  int32_t* s_curpos = reinterpret_cast<int32_t*>(s_curreq + R);
+  uint32_t* s_lrutail = reinterpret_cast<uint32_t*>(s_curpos + R);
+
+  unsigned char* st = a.states + (size_t)p * a.lay.bytes;
+  CandHeader* hdr = reinterpret_cast<CandHeader*>(st);
+  RepState* g_rep = reinterpret_cast<RepState*>(st + a.lay.rep_off);
+  double* free_at = reinterpret_cast<double*>(st + a.lay.free_at_off);
+  double* head_fin = reinterpret_cast<double*>(st + a.lay.head_fin_off);
+  uint32_t* head = reinterpret_cast<uint32_t*>(st + a.lay.head_off);
+  uint32_t* tail = reinterpret_cast<uint32_t*>(st + a.lay.tail_off);
+  MaskT* mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
+  double* fin = a.fin + (size_t)p * N;
+  uint32_t* slot_next = a.slot_next + (size_t)p * N;
+  uint32_t* lru_next = a.lru_next + (size_t)p * N;
+  uint8_t* route_log = a.route_log + (size_t)p * a.route_log_stride;
+  const ReqRec* req = a.tr.req;
+  const uint32_t* ids = a.tr.ids;
+
+  if (a.check_order && hdr->processed != a.first) {
+    if (lane == 0) {
+      hdr->status = -8;
+      if (a.status_out) a.status_out[p] = -8;
+    }
+    return;
+  }
+
+  for (uint32_t i = lane; i < G * R; i += 32) s_rtt[i] = a.rtt[i];
+  for (uint32_t i = lane; i < K; i += 32) s_w[i] = a.params[(size_t)p * K + i];
+  for (uint32_t i = lane; i < R; i += 32) {
+    const RepState rs = g_rep[i];
+    s_minfin[i] = rs.min_fin; s_load[i] = rs.load; s_occ[i] = rs.occ;
+    s_curreq[i] = rs.cur_req; s_curpos[i] = rs.cur_pos; s_lrutail[i] = rs.lru_tail;
+  }
+  __syncwarp();
+
+  const double w_net = s_w[0], w_pre = s_w[1], w_que = s_w[2];
+  const MaskT all_reps = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0
+                                                  : (MaskT)((((MaskT)1) << (R & 63)) - 1);
+  int32_t status = 0;
+  unsigned long long st_probe = 0, st_hit = 0, st_blk = 0, st_evict = 0;
+
+  for (uint32_t j = 0; j < a.count; ++j) {
+    const uint32_t r = a.first + j;
+    const ReqRec rec = req[r];
+    const double t = __dmul_rn(a.scale, rec.ts_ms);
+    const uint32_t n = rec.nblk, off = rec.off, in_tok = rec.in_tok;
+    const double* rtt_row = s_rtt + (size_t)rec.origin * R;
+
+    // ---- queue signal: drop requests that completed by t (finish <= t)
+    for (uint32_t i0 = 0; i0 < R; i0 += 32) {
+      const uint32_t i = i0 + lane;
+      unsigned due = __ballot_sync(kFull, i < R && s_minfin[i] <= t);
+      while (due) {
+        const uint32_t ii = i0 + (uint32_t)__ffs((int)due) - 1;
+        due &= due - 1;
+        long long tok = 0;
+        double mn = d_inf();
+        for (uint32_t s = lane; s < S; s += 32) {
+          const size_t x = (size_t)ii * S + s;
+          double hf = head_fin[x];
+          if (hf <= t) {
+            uint32_t hd = head[x];
+            uint32_t guard = 0;
+            do {
+              tok += (long long)req[hd].in_tok;
+              const uint32_t nx = slot_next[hd];
+              if (nx == kNone) { hd = kNone; hf = d_inf(); }
+              else { hd = nx; hf = fin[nx]; }
+              if (++guard > N) { status = -6; break; }
+            } while (hf <= t);
+            head[x] = hd;
+            head_fin[x] = hf;
+          }
+          mn = fmin(mn, hf);
+        }
+        tok = warp_sum_ll(tok);
+        mn = warp_min_d(mn);
+        if (lane == 0) { s_load[ii] -= tok; s_minfin[ii] = mn; }
+      }
+    }
+    __syncwarp();
+
+    // ---- prefix probe on every replica: h_i = leading blocks whose mask has bit i
+    uint32_t h0 = 0, h1 = 0;  // this lane's replicas: lane and lane+32
+    {
+      MaskT alive = all_reps;
+      for (uint32_t c = 0; c < n && alive != 0; c += 32) {
+        const uint32_t k = c + lane;
+        MaskT pm = 0;
+        if (k < n) pm = mask[ids[off + k]];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const MaskT o = shfl_up_mask<MaskT>(pm, d);
+          if ((int)lane >= d) pm &= o;
+        }
+        pm &= alive;
+        MaskT it = shfl_mask<MaskT>(pm, 0);
+        while (it != 0) {
+          const int i = first_bit<MaskT>(it);
+          it &= (MaskT)(it - 1);
+          const unsigned b = __ballot_sync(kFull, (pm >> i) & 1);
+          if ((uint32_t)(i & 31) == lane) {
+            if (i < 32) h0 += __popc(b); else h1 += __popc(b);
+          }
+        }
+        alive = shfl_mask<MaskT>(pm, 31);
+      }
+    }
+
+    // ---- score of Eq. 3 (fixed order, no FMA) and lowest-index argmin
+    double best_c = d_inf();
+    uint32_t best_i = kNone;
+    uint32_t unc0 = 0, unc1 = 0;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const uint32_t i = lane + 32u * half;
+      if (i < R) {
+        const uint32_t h = half ? h1 : h0;
+        const unsigned long long hb = (unsigned long long)h * a.m.B;
+        const uint32_t unc = in_tok - (uint32_t)(hb < in_tok ? hb : in_tok);
+        if (half) unc1 = unc; else unc0 = unc;
+        double q = (double)s_load[i];
+        if (K != 3) q = __dmul_rn(q, s_w[3 + i]);
+        double c = __dadd_rn(__dadd_rn(__dmul_rn(w_net, rtt_row[i]), __dmul_rn(w_pre, (double)unc)),
+                             __dmul_rn(w_que, q));
+        if (c != c) c = (i == 0) ? -d_inf() : d_inf();  // a NaN score wins only at index 0
+        if (c < best_c || best_i == kNone) { best_c = c; best_i = i; }
+        const uint32_t pr = h + 1 < n ? h + 1 : n;
+        st_probe += pr;
+      }
+    }
+    warp_argmin(best_c, best_i);
+    const uint32_t istar = best_i;
+    const uint32_t hstar = __shfl_sync(kFull, istar < 32 ? h0 : h1, istar & 31);
+    const uint32_t uncstar = __shfl_sync(kFull, istar < 32 ? unc0 : unc1, istar & 31);
+    const MaskT bit = (MaskT)(((MaskT)1) << istar);
+
+    // ---- cache commit: set the replica's bit on the missing blocks
+    uint32_t missing = 0;
+    for (uint32_t c = 0; c < n; c += 32) {
+      const uint32_t k = c + lane;
+      bool miss = false;
+      if (k < n) {
+        const uint32_t id = ids[off + k];
+        const MaskT mv = mask[id];
+        if (!(mv & bit)) { mask[id] = (MaskT)(mv | bit); miss = true; }
+      }
+      missing += __popc(__ballot_sync(kFull, miss));
+    }
+    uint32_t occ = s_occ[istar] + missing;
+    uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
+    uint32_t evicted = 0;
+    if (need > 0) {
+      uint32_t cr = s_curreq[istar];
+      int32_t cp = s_curpos[istar];
+      uint32_t coff = (cr != kNone) ? req[cr].off : 0u;
+      unsigned long long guard = 0;
+      const unsigned long long guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
+      while (need > 0) {
+        if (++guard > guard_max) { status = -6; break; }
+        if (cp < 0) {  // this request is used up: go to the next one routed here
+          const uint32_t nx = (cr == kNone) ? kNone : lru_next[cr];
+          if (nx == kNone) { status = -6; break; }
+          cr = nx;
+          const ReqRec cre = req[cr];
+          coff = cre.off;
+          cp = (int32_t)cre.nblk - 1;
+          continue;
+        }
+        const int32_t k = cp - (int32_t)lane;   // deepest position first
+        bool live = false;
+        uint32_t g = 0;
+        if (k >= 0) {
+          g = coff + (uint32_t)k;
+          live = !touch_is_stale(a.tr, route_log, g, istar, r, istar);
+        }
+        const unsigned lv = __ballot_sync(kFull, live);
+        const uint32_t cnt = __popc(lv);
+        unsigned take;
+        int32_t adv;
+        if (cnt <= need) { take = lv; adv = 32; }
+        else {
+          const unsigned pos = __fns(lv, 0, (int)need);
+          take = lv & ((2u << pos) - 1u);
+          adv = (int32_t)pos + 1;
+        }
+        if ((take >> lane) & 1u) {
+          const uint32_t id = ids[g];
+          mask[id] = (MaskT)(mask[id] & (MaskT)~bit);
+        }
+        const uint32_t tk = __popc(take);
+        need -= tk;
+        evicted += tk;
+        cp -= adv;
+      }
+      if (lane == 0) { s_curreq[istar] = cr; s_curpos[istar] = cp; }
+    }
+    occ -= evicted;
+
+    // ---- service commit: earliest-free slot, lowest index on ties
+    double bv = d_inf();
+    uint32_t bs = kNone;
+    for (uint32_t s = lane; s < S; s += 32) {
+      const double v = free_at[(size_t)istar * S + s];
+      if (v < bv || bs == kNone) { bv = v; bs = s; }
+    }
+    warp_argmin(bv, bs);
+    const double arrive = __dadd_rn(t, rtt_row[istar]);
+    const double start = (bv > arrive) ? bv : arrive;
+    const double first = __dadd_rn(start, __dmul_rn(a.m.prefill_ms, (double)uncstar));
+    const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
+    const double finish = __dadd_rn(first, __dmul_rn(a.m.tpot_ms, (double)dec_tok));
+
+    if (lane == 0) {
+      const size_t x = (size_t)istar * S + bs;
+      fin[r] = finish;
+      slot_next[r] = kNone;
+      if (head[x] == kNone) {
+        head[x] = r;
+        head_fin[x] = finish;
+        s_minfin[istar] = fmin(s_minfin[istar], finish);
+      } else {
+        slot_next[tail[x]] = r;
+      }
+      tail[x] = r;
+      free_at[x] = finish;
+      s_load[istar] += (long long)in_tok;
+      s_occ[istar] = occ;
+      // recency order of the replica: append this request
+      const uint32_t lt = s_lrutail[istar];
+      if (lt != kNone) lru_next[lt] = r;
+      lru_next[r] = kNone;
+      if (s_curreq[istar] == kNone) { s_curreq[istar] = r; s_curpos[istar] = (int32_t)n - 1; }
+      s_lrutail[istar] = r;
+      route_log[r] = (uint8_t)istar;
+      const size_t o = (size_t)p * a.out_stride + j;
+      if (a.route_out) a.route_out[o] = (uint8_t)istar;
+      if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
+      if (a.ttft_out) a.ttft_out[o] = __dsub_rn(first, t);
+      if (a.e2e_out) a.e2e_out[o] = __dsub_rn(finish, t);
+      st_hit += hstar; st_blk += n; st_evict += evicted;
+    }
+    __syncwarp();
+  }
+
+  // ---- write the replica scalars back
+  for (uint32_t i = lane; i < R; i += 32) {
+    RepState rs;
+    rs.min_fin = s_minfin[i]; rs.load = s_load[i]; rs.occ = s_occ[i];
+    rs.cur_req = s_curreq[i]; rs.cur_pos = s_curpos[i]; rs.lru_tail = s_lrutail[i];
+    g_rep[i] = rs;
+  }
+  st_probe = warp_sum_u64(st_probe);
+  status = __reduce_min_sync(kFull, status);
+  if (lane == 0) {
+    hdr->processed = a.first + a.count;
+    if (status != 0) hdr->status = status;
+    if (a.status_out && (status != 0 || !a.check_order)) a.status_out[p] = status;
+    if (a.stats) {
+      unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
+      s4[0] += st_probe; s4[1] += st_hit; s4[2] += st_blk; s4[3] += st_evict;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------- reset
+__global__ void reset_states_kernel(unsigned char* states, StateLayout lay, uint32_t R, uint32_t S,
+                                    uint32_t n_cand) {
+  const uint32_t p = blockIdx.x;
+  if (p >= n_cand) return;
+  unsigned char* st = states + (size_t)p * lay.bytes;
+  if (threadIdx.x == 0) {
+    CandHeader h = {};
+    *reinterpret_cast<CandHeader*>(st) = h;
+  }
+  RepState* rep = reinterpret_cast<RepState*>(st + lay.rep_off);
+  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
+    RepState rs;
+    rs.load = 0; rs.min_fin = d_inf(); rs.occ = 0; rs.cur_req = kNone; rs.cur_pos = -1;
+    rs.lru_tail = kNone;
+    rep[i] = rs;
+  }
+  double* free_at = reinterpret_cast<double*>(st + lay.free_at_off);
+  double* head_fin = reinterpret_cast<double*>(st + lay.head_fin_off);
+  uint32_t* head = reinterpret_cast<uint32_t*>(st + lay.head_off);
+  uint32_t* tail = reinterpret_cast<uint32_t*>(st + lay.tail_off);
+  for (uint32_t x = threadIdx.x; x < R * S; x += blockDim.x) {
+    free_at[x] = 0.0; head_fin[x] = d_inf(); head[x] = kNone; tail[x] = kNone;
+  }
+}
+
+// ------------------------------------------------------------------------------ select
+// Exact k-th smallest (k = ceil(0.95 n), nearest rank) of n doubles by most-significant-digit
+// radix selection on order-preserving 64-bit keys; one CTA per (candidate, metric).
+__device__ __forceinline__ uint64_t key_of(double v) {
+  const uint64_t b = (uint64_t)__double_as_longlong(v);
+  return (b >> 63) ? ~b : (b | 0x8000000000000000ULL);
+}
+__device__ __forceinline__ double value_of(uint64_t k) {
+  const uint64_t b = (k >> 63) ? (k & 0x7FFFFFFFFFFFFFFFULL) : ~k;
+  return __longlong_as_double((long long)b);
+}
+
+constexpr int kSelectThreads = 1024;
+
+__global__ void __launch_bounds__(kSelectThreads) select_p95_kernel(const SelectArgs a) {
+  const uint32_t p = blockIdx.x;
+  const double* v = (blockIdx.y == 0 ? a.ttft : a.e2e) + (size_t)p * a.stride;
+  double* out = (blockIdx.y == 0 ? a.p95_ttft : a.p95_e2e) + p;
+  const uint32_t n = a.n;
+  __shared__ uint32_t hist[256];
+  __shared__ uint64_t s_prefix;
+  __shared__ uint32_t s_rank;
+  if (n == 0) { if (threadIdx.x == 0) *out = 0.0; return; }
+  if (threadIdx.x == 0) {
+    s_prefix = 0;
+    s_rank = (uint32_t)((95ull * n + 99ull) / 100ull) - 1u;  // 0-based rank
+  }
+  uint64_t have = 0;  // mask of the key bits fixed so far
+  for (int shift = 56; shift >= 0; shift -= 8) {
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    const uint64_t prefix = s_prefix;
+    for (uint32_t base = threadIdx.x & ~31u; base < n; base += blockDim.x) {
+      const uint32_t i = base + (threadIdx.x & 31u);
+      const uint64_t k = (i < n) ? key_of(v[i]) : 0;
+      const bool in = (i < n) && (k & have) == prefix;
+      const uint32_t d = (uint32_t)(k >> shift) & 255u;
+      // one atomic per distinct digit among the matching lanes of the warp
+      const unsigned act = __ballot_sync(kFull, in);
+      if (in) {
+        const unsigned peers = __match_any_sync(act, d);
+        if ((uint32_t)(__ffs((int)peers) - 1) == (threadIdx.x & 31u)) atomicAdd(&hist[d], __popc(peers));
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t rank = s_rank, d = 0;
+      while (d < 255 && rank >= hist[d]) { rank -= hist[d]; ++d; }
+      s_rank = rank;
+      s_prefix = prefix | ((uint64_t)d << shift);
+    }
+    have |= (uint64_t)255 << shift;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = value_of(s_prefix);
+}
+
+// ------------------------------------------------------------------------------ digest
+// Per replica: occupancy and the sum over cached blocks of mix64(id ^ mix64(seq*65536+pos)).
+// A block's latest touch on its replica is cached iff it lies at or after the eviction cursor.
+__global__ void __launch_bounds__(256) digest_kernel(const DigestArgs a) {
+  const uint32_t p = blockIdx.x;
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t warp = (blockIdx.y * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t n_warps = (gridDim.y * blockDim.x) >> 5;
+  const unsigned char* st = a.states + (size_t)p * a.lay.bytes;
+  const CandHeader* hdr = reinterpret_cast<const CandHeader*>(st);
+  const RepState* rep = reinterpret_cast<const RepState*>(st + a.lay.rep_off);
+  const uint8_t* route_log = a.route_log + (size_t)p * a.route_log_stride;
+  const uint32_t done = hdr->processed;
+  if (done == 0) return;
+  unsigned long long* dg = reinterpret_cast<unsigned long long*>(a.digest) + (size_t)p * a.m.R * 2;
+  for (uint32_t n = warp; n < done; n += n_warps) {
+    const uint32_t i = route_log[n];
+    const uint32_t cr = rep[i].cur_req;
+    const int32_t cp = rep[i].cur_pos;
+    if (cr == kNone || n < cr) continue;
+    const ReqRec rec = a.tr.req[n];
+    unsigned long long sum = 0, cnt = 0;
+    for (uint32_t k = lane; k < rec.nblk; k += 32) {
+      if (n == cr && (int32_t)k > cp) continue;
+      const uint32_t g = rec.off + k;
+      if (touch_is_stale(a.tr, route_log, g, i, done - 1, route_log[done - 1])) continue;
+      const uint64_t id = a.tr.raw_id[a.tr.ids[g]];
+      sum += mix64(id ^ mix64((uint64_t)n * 65536ULL + k));
+      cnt += 1;
+    }
+    sum = warp_sum_u64(sum);
+    cnt = warp_sum_u64(cnt);
+    if (lane == 0 && cnt) {
+      atomicAdd(&dg[2 * i], cnt);
+      atomicAdd(&dg[2 * i + 1], sum);
+    }
+  }
+}
+
+template <typename MaskT>
+cudaError_t launch_replay_t(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st) {
+  const size_t smem = ((size_t)a.m.G * a.m.R + a.m.K + a.m.R) * sizeof(double) +
+                      (size_t)a.m.R * (sizeof(long long) + 4 * sizeof(uint32_t));
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  replay_kernel<MaskT><<<n_cand, 32, smem, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+uint32_t mask_bytes_for(uint32_t n_replicas) {
+  return n_replicas <= 8 ? 1u : n_replicas <= 16 ? 2u : n_replicas <= 32 ? 4u : 8u;
+}
+
+cudaError_t launch_reset(unsigned char* masks, uint64_t mask_bytes_total, unsigned char* states,
+                         const StateLayout& lay, const Model& m, uint32_t n_cand,
+                         cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(masks, 0, mask_bytes_total, st);
+  if (e != cudaSuccess) return e;
+  reset_states_kernel<<<n_cand, 128, 0, st>>>(states, lay, m.R, m.S, n_cand);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_replay(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st) {
+  switch (mask_bytes_for(a.m.R)) {
+    case 1: return launch_replay_t<uint8_t>(a, n_cand, st);
+    case 2: return launch_replay_t<uint16_t>(a, n_cand, st);
+    case 4: return launch_replay_t<uint32_t>(a, n_cand, st);
+    default: return launch_replay_t<uint64_t>(a, n_cand, st);
+  }
+}
+
+cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st) {
+  select_p95_kernel<<<dim3(n_cand, 2), kSelectThreads, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(a.digest, 0, (size_t)n_cand * a.m.R * 2 * sizeof(uint64_t), st);
+  if (e != cudaSuccess) return e;
+  const uint32_t chunks = 64;
+  digest_kernel<<<dim3(n_cand, chunks), 256, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace gorgo

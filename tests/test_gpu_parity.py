@@ -1,0 +1,286 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Routes, prefix-hit lengths, cache digests and counters must be bit-exact; p95
+TTFT/E2E within 1e-9 relative."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+from oracle import gorgo_oracle as O
+from paper_2602_11688_b200 import workloads as W
+from tests.util import check_population, gpu_eval, small_trace
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def test_w1_handworked_trace_on_gpu():
+    g = json.load(open(os.path.join(GOLDEN, "w1_handworked.json")))
+    names, reqs = {}, []
+    for q in g["requests"]:
+        ids = [names.setdefault(b, 100 + len(names)) for b in q["blocks"]]
+        reqs.append((q["t_ms"], q["input_tokens"], q["output_tokens"], ids))
+    c = g["config"]
+    w = W.handmade(c["rtt_ms"], reqs, slots=c["slots"], cache_blocks=c["cache_blocks"],
+                   params=[c["params"]])
+    res = gpu_eval(w, scale=1.0)
+    e = g["expected"]
+    assert res["route"][0].tolist() == e["route"]
+    assert res["hit"][0].tolist() == e["hit_blocks"]
+    assert res["p95_ttft"][0] == pytest.approx(e["p95_ttft_ms"], rel=1e-12)
+    assert res["p95_e2e"][0] == pytest.approx(e["p95_e2e_ms"], rel=1e-12)
+    assert res["digest"][0][:, 0].tolist() == [4, 2]
+    assert res["stats"][0][3] == 2
+
+
+@pytest.mark.parametrize("structured", [True, False])
+@pytest.mark.parametrize("R,normalised", [(1, False), (3, False), (8, True), (9, False), (16, False),
+                                          (17, True), (32, False), (33, False), (64, True)])
+def test_small_traces_all_mask_widths(R, normalised, structured):
+    rng = np.random.default_rng(R * 2 + structured)
+    reqs = small_trace(R + 7 * structured, n_req=400, structured=structured)
+    K = 3 + R if normalised else 3
+    P = 6
+    params = rng.normal(1.0, 0.3, size=(P, 3))
+    params[0] = (1.0, 0.0, 0.0)
+    params[1] = (0.0, 1.0, 0.0)
+    if normalised:
+        params = np.concatenate([params, rng.lognormal(0, 0.3, size=(P, R))], axis=1)
+    w = W.handmade(rng.uniform(5, 60, size=R), reqs, slots=2, cache_blocks=9, params=params)
+    assert w.n_params == K
+    check_population(w, scale=1.0)
+
+
+def test_multi_region_rtt_rows():
+    rng = np.random.default_rng(5)
+    reqs = small_trace(11, n_req=300)
+    G, R = 3, 5
+    org = rng.integers(0, G, size=len(reqs))
+    w = W.handmade(rng.uniform(5, 200, size=(G, R)), reqs, slots=3, cache_blocks=12,
+                   n_regions=G, origin=org, params=rng.normal(1.0, 0.3, size=(4, 3)))
+    check_population(w, scale=1.0)
+
+
+def test_edge_cases_empty_prompt_long_prompt_exact_fit_and_saturated_slot():
+    B = 512
+    reqs = [(0.0, 0, 5, []),                                    # no blocks at all
+            (1.0, 100 * B, 3, list(range(1, 101))),             # 100 blocks: several lane rounds
+            (2.0, 0, 0, []),
+            (3.0, 100 * B - 7, 1, list(range(1, 100)) + [500]),  # shares 99 blocks
+            (3.0, 70 * B, 2, list(range(200, 270))),            # same timestamp as the previous one
+            (4.0, 100 * B, 9, list(range(1, 101))),
+            (5.0, 33 * B, 9, list(range(300, 333))),
+            (6.0, 100 * B, 1, list(range(100, 0, -1)))]         # same blocks, reversed order
+    params = [(1.0, 1.0, 1.0), (0.0, 1.0, 0.0), (1.0, 0.01, 0.0), (-1.0, 0.5, 0.2)]
+    for C in (100, 101, 170, 1000):                             # 100 = exactly one request fits
+        w = W.handmade([10.0, 20.0], reqs, slots=1, cache_blocks=C, params=params)
+        check_population(w, scale=1.0)
+    # one request only
+    w = W.handmade([10.0, 20.0, 5.0], reqs[1:2], slots=2, cache_blocks=100, params=params)
+    check_population(w, scale=1.0)
+
+
+def test_huge_weights_give_infinite_and_nan_scores_like_the_scan():
+    reqs = small_trace(3, n_req=120)
+    params = [(1e308, 1e308, 1e308), (-1e308, 1e308, 1e308), (1e308, -1e308, -1e308),
+              (1e308, -1e308, 1e308), (0.0, 1e308, -1e308)]
+    w = W.handmade([10.0, 400.0, 90.0], reqs, slots=2, cache_blocks=10, params=params)
+    check_population(w, scale=1.0)
+
+
+def test_tiny_config_full():
+    w = W.make_workload("tiny")
+    check_population(w)
+    for scale in (0.25, 4.0):
+        check_population(w, scale=scale)
+
+
+def test_regions_config_full():
+    w = W.make_workload("regions")
+    check_population(w)
+
+
+def test_longctx_reduced_with_heavy_eviction():
+    w = W.make_workload("longctx", n_requests=30_000, cache_blocks=4_000, population=16)
+    gpu, refs = check_population(w)
+    assert sum(int(r[4][3]) for r in refs) > 0                  # evictions did happen
+
+
+def test_largest_reduced_with_normalisers():
+    w = W.make_workload("largest", n_requests=20_000, cache_blocks=3_000, population=12)
+    check_population(w)
+
+
+def test_sweep_reduced_all_scales():
+    w = W.make_workload("sweep", n_requests=20_000, cache_blocks=3_000, population=8)
+    for scale in w.spec.time_scales:
+        check_population(w, scale=scale)
+
+
+def test_waves_give_the_same_answer_as_one_wave():
+    from paper_2602_11688_b200 import binding as gb
+    w = W.make_workload("tiny", population=8)
+    sim = gb.GorgoSim(w)
+    rc, one = gb.gorgo_workspace_bytes(sim.h, 1)
+    rc, three = gb.gorgo_workspace_bytes(sim.h, 3)
+    full = gpu_eval(w, sim=sim)
+    sim.workspace = None
+    waves = gpu_eval(w, sim=sim, resident=3, max_bytes=three)    # 3 + 3 + 2
+    assert sim.workspace.numel() == three
+    single = gpu_eval(w, sim=sim, resident=1, max_bytes=one)
+    sim.close()
+    for k in ("route", "hit", "digest", "stats", "p95_ttft", "p95_e2e"):
+        assert (full[k] == waves[k]).all() and (full[k] == single[k]).all(), k
+
+
+def test_runs_are_deterministic():
+    w = W.make_workload("regions", n_requests=10_000, cache_blocks=2_000, population=32)
+    a = gpu_eval(w)
+    b = gpu_eval(w)
+    for k in ("route", "hit", "digest", "stats", "p95_ttft", "p95_e2e"):
+        assert (a[k] == b[k]).all(), k
+
+
+def test_host_buffer_entry_point_matches_device_one():
+    import torch
+    from paper_2602_11688_b200 import binding as gb
+    w = W.make_workload("tiny")
+    sim = gb.GorgoSim(w)
+    dev = gpu_eval(w, sim=sim)
+    P = w.params.shape[0]
+    params = torch.from_numpy(w.params.copy()).pin_memory()
+    a = torch.empty(P, dtype=torch.float64).pin_memory()
+    b = torch.empty(P, dtype=torch.float64).pin_memory()
+    rc = gb.gorgo_eval_population_host(sim.h, P, params, 1.0, sim.workspace, sim.stream, a, b)
+    assert rc == gb.GORGO_OK
+    assert (a.numpy() == dev["p95_ttft"]).all() and (b.numpy() == dev["p95_e2e"]).all()
+    # plain numpy host buffers work too
+    a2, b2 = np.zeros(P), np.zeros(P)
+    rc = gb.gorgo_eval_population_host(sim.h, P, w.params, 1.0, sim.workspace, sim.stream, a2, b2)
+    assert rc == gb.GORGO_OK and (a2 == dev["p95_ttft"]).all()
+    sim.close()
+
+
+def test_device_resident_params():
+    import torch
+    from paper_2602_11688_b200 import binding as gb
+    w = W.make_workload("tiny")
+    sim = gb.GorgoSim(w)
+    ref = gpu_eval(w, sim=sim)
+    P = w.params.shape[0]
+    dp = torch.from_numpy(w.params.copy()).cuda()
+    a = torch.empty(P, dtype=torch.float64, device="cuda")
+    b = torch.empty(P, dtype=torch.float64, device="cuda")
+    rc = gb.gorgo_eval_population(sim.h, P, dp, 1.0, sim.workspace, sim.stream, a, b)
+    torch.cuda.synchronize()
+    assert rc == gb.GORGO_OK and (a.cpu().numpy() == ref["p95_ttft"]).all()
+    sim.close()
+
+
+def test_route_batch_continues_a_persistent_state():
+    import torch
+    from paper_2602_11688_b200 import binding as gb
+    w = W.make_workload("regions", n_requests=6_000, cache_blocks=1_500)
+    par = w.params[7]
+    sim = gb.GorgoSim(w)
+    rc, nbytes = gb.gorgo_state_bytes(sim.h)
+    assert rc == gb.GORGO_OK
+    state = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    assert gb.gorgo_sim_reset(sim.h, state, sim.stream) == gb.GORGO_OK
+    o = O.Oracle.from_workload(w)
+    R = w.spec.n_replicas
+    first = 0
+    for count in (1, 999, 2500, 1, 2499):
+        route = torch.empty(count, dtype=torch.uint8, device="cuda")
+        hit = torch.empty(count, dtype=torch.uint16, device="cuda")
+        ttft = torch.empty(count, dtype=torch.float64, device="cuda")
+        e2e = torch.empty(count, dtype=torch.float64, device="cuda")
+        rc = gb.gorgo_route_batch(sim.h, par, 1.0, first, count, state, sim.stream, route, hit,
+                                  ttft, e2e)
+        assert rc == gb.GORGO_OK
+        dg = torch.empty((R, 2), dtype=torch.uint64, device="cuda")
+        assert gb.gorgo_state_digest(sim.h, state, sim.stream, dg) == gb.GORGO_OK
+        rc, seen = gb.gorgo_state_status(sim.h, state, sim.stream)
+        first += count
+        assert rc == gb.GORGO_OK and seen == first
+        ref = o.run(par, 1.0, count)
+        assert (route.cpu().numpy() == ref.route).all()
+        assert (hit.cpu().numpy() == ref.hit).all()
+        assert (ttft.cpu().numpy() == ref.ttft).all()          # same fp64 operations: identical
+        assert (e2e.cpu().numpy() == ref.e2e).all()
+        assert dg.cpu().numpy().tolist() == o.digest().tolist()
+    # a batch that is not the next one is refused and leaves the state alone
+    route = torch.empty(10, dtype=torch.uint8, device="cuda")
+    assert gb.gorgo_route_batch(sim.h, par, 1.0, 10, 10, state, sim.stream, route) == gb.GORGO_OK
+    rc, seen = gb.gorgo_state_status(sim.h, state, sim.stream)
+    assert rc == gb.GORGO_ERR_OUT_OF_ORDER and seen == first
+    # reset starts over
+    assert gb.gorgo_sim_reset(sim.h, state, sim.stream) == gb.GORGO_OK
+    rc = gb.gorgo_route_batch(sim.h, par, 1.0, 0, 10, state, sim.stream, route)
+    rc, seen = gb.gorgo_state_status(sim.h, state, sim.stream)
+    assert rc == gb.GORGO_OK and seen == 10
+    o.reset()
+    assert (route.cpu().numpy() == o.run(par, 1.0, 10).route).all()
+    sim.close()
+
+
+def test_abi_rejects_bad_input():
+    import torch
+    from paper_2602_11688_b200 import binding as gb
+    w = W.make_workload("tiny", n_requests=200)
+    kw = w.config_dict()
+    rc, h = gb.gorgo_sim_create(rtt_ms=w.rtt_ms, **{**kw, "n_replicas": 65})
+    assert rc == gb.GORGO_ERR_INVALID_ARG
+    rc, h = gb.gorgo_sim_create(rtt_ms=-w.rtt_ms, **kw)
+    assert rc == gb.GORGO_ERR_INVALID_ARG
+    rc, h = gb.gorgo_sim_create(rtt_ms=w.rtt_ms, **{**kw, "n_params": 4})
+    assert rc == gb.GORGO_ERR_INVALID_ARG
+    rc, h = gb.gorgo_sim_create(rtt_ms=w.rtt_ms, **kw)
+    assert rc == gb.GORGO_OK
+    rc, n = gb.gorgo_workspace_bytes(h, 1)
+    assert rc == gb.GORGO_ERR_NO_TRACE
+    rc, nbytes = gb.gorgo_trace_bytes(w.n_requests, int(w.hash_off[-1]))
+    buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    args = dict(ts_ms=w.ts_ms, input_tokens=w.input_tokens, output_tokens=w.output_tokens,
+                origin=w.origin, hash_off=w.hash_off, hash_ids=w.hash_ids)
+
+    def upload(**over):
+        a = {**args, **over}
+        return gb.gorgo_trace_upload(h, a["ts_ms"], a["input_tokens"], a["output_tokens"],
+                                     a["origin"], a["hash_off"], a["hash_ids"], buf, 0)
+    ts = w.ts_ms.copy(); ts[5] = ts[4] - 1.0
+    assert upload(ts_ms=ts) == gb.GORGO_ERR_BAD_TRACE            # time goes backwards
+    ts = w.ts_ms.copy(); ts[5] = np.nan
+    assert upload(ts_ms=ts) == gb.GORGO_ERR_BAD_TRACE
+    it = w.input_tokens.copy(); it[3] += 512
+    assert upload(input_tokens=it) == gb.GORGO_ERR_BAD_TRACE     # block count != ceil(in/B)
+    ids = w.hash_ids.copy()
+    r = int(np.argmax(np.diff(w.hash_off.astype(np.int64)) >= 2))
+    ids[int(w.hash_off[r]) + 1] = ids[int(w.hash_off[r])]
+    assert upload(hash_ids=ids) == gb.GORGO_ERR_BAD_TRACE        # an id twice in one request
+    org = w.origin.copy(); org[0] = 9
+    assert upload(origin=org) == gb.GORGO_ERR_BAD_TRACE
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    assert gb.gorgo_trace_upload(h, w.ts_ms, w.input_tokens, w.output_tokens, w.origin, w.hash_off,
+                                 w.hash_ids, small, 0) == gb.GORGO_ERR_WORKSPACE_TOO_SMALL
+    assert upload() == gb.GORGO_OK
+    rc, nreq, nids, ndist = gb.gorgo_trace_info(h)
+    assert (rc, nreq, nids) == (gb.GORGO_OK, w.n_requests, int(w.hash_off[-1]))
+    assert ndist == len(np.unique(w.hash_ids))
+    rc, need = gb.gorgo_workspace_bytes(h, 2)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    a = torch.empty(2, dtype=torch.float64, device="cuda")
+    b = torch.empty(2, dtype=torch.float64, device="cuda")
+    bad = w.params[:2].copy(); bad[1, 2] = np.inf
+    assert gb.gorgo_eval_population(h, 2, bad, 1.0, ws, 0, a, b) == gb.GORGO_ERR_NONFINITE_PARAM
+    assert gb.gorgo_eval_population(h, 2, w.params[:2].copy(), float("nan"), ws, 0, a, b) == \
+        gb.GORGO_ERR_NONFINITE_PARAM
+    tiny_ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    assert gb.gorgo_eval_population(h, 2, w.params[:2].copy(), 1.0, tiny_ws, 0, a, b) == \
+        gb.GORGO_ERR_WORKSPACE_TOO_SMALL
+    assert gb.gorgo_eval_population(h, 2, w.params[:2].copy(), 1.0, ws, 0, a, None) == \
+        gb.GORGO_ERR_INVALID_ARG
+    assert gb.gorgo_eval_population(h, 2, w.params[:2].copy(), 1.0, ws, 0, a, b) == gb.GORGO_OK
+    torch.cuda.synchronize()
+    assert gb.gorgo_sim_destroy(h) == gb.GORGO_OK

@@ -11,39 +11,9 @@ import pytest
 
 from oracle import gorgo_oracle as O
 from paper_2602_11688_b200 import workloads as W
+from tests.util import small_trace
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
-
-
-def small_trace(seed, n_req=300, n_sessions=12, max_blocks=7, structured=True, B=512,
-                rate_ms=40.0):
-    """Tiny random trace.  structured: sessions extend their own prefix (ids imply their
-    prefix); otherwise every request is a random subset of a small id pool in random order."""
-    rng = np.random.default_rng(seed)
-    reqs, t = [], 0.0
-    conv = {}
-    nxt = 1000
-    for _ in range(n_req):
-        t += float(rng.exponential(rate_ms))
-        if structured:
-            s = int(rng.integers(n_sessions))
-            ids = conv.get(s)
-            if ids is None or len(ids) >= max_blocks or rng.random() < 0.25:
-                k = int(rng.integers(1, 4))
-                ids = list(range(nxt, nxt + k)); nxt += k
-            else:
-                k = int(rng.integers(1, 3))
-                ids = ids + list(range(nxt, nxt + k)); nxt += k
-                ids = ids[:max_blocks]
-            conv[s] = ids
-        else:
-            k = int(rng.integers(1, max_blocks + 1))
-            ids = [int(x) for x in rng.choice(np.arange(1, 40), size=k, replace=False)]
-        n = len(ids)
-        in_tok = (n - 1) * B + int(rng.integers(1, B + 1))
-        out = int(rng.integers(0, 30))
-        reqs.append((t, in_tok, out, ids))
-    return reqs
 
 
 def recency_list_replay(requests, routes, R, C):
