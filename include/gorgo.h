@@ -158,6 +158,14 @@ int gorgo_state_digest(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
 int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_bytes,
                        void *cuda_stream, uint64_t *requests_seen);
 
+/* Measurement aid (no counterpart in the paper).  With profiling enabled, gorgo_eval_population
+ * records a CUDA event on `cuda_stream` directly before and after each launch of the replay
+ * kernel (one launch per wave, at most 32 waves are timed).  gorgo_last_replay_ms waits for those
+ * events and returns the summed device time of the replay launches of the most recent
+ * evaluation and their number. */
+int gorgo_set_profiling(gorgo_sim_t *sim, int enable);
+int gorgo_last_replay_ms(gorgo_sim_t *sim, double *replay_ms, uint32_t *launches);
+
 const char *gorgo_strerror(int code);
 
 #ifdef __cplusplus

@@ -28,7 +28,8 @@ EXPORTS = [
     "gorgo_sim_create", "gorgo_sim_destroy", "gorgo_trace_bytes", "gorgo_trace_upload",
     "gorgo_trace_info", "gorgo_workspace_bytes", "gorgo_eval_population",
     "gorgo_eval_population_host", "gorgo_state_bytes", "gorgo_sim_reset", "gorgo_route_batch",
-    "gorgo_state_digest", "gorgo_state_status", "gorgo_strerror",
+    "gorgo_state_digest", "gorgo_state_status", "gorgo_set_profiling", "gorgo_last_replay_ms",
+    "gorgo_strerror",
 ]
 
 
@@ -74,6 +75,8 @@ def load():
         "gorgo_route_batch": [vp, vp, dbl, u64, u64, vp, u64, vp, vp, vp, vp, vp],
         "gorgo_state_digest": [vp, vp, u64, vp, vp],
         "gorgo_state_status": [vp, vp, u64, vp, pu64],
+        "gorgo_set_profiling": [vp, i32],
+        "gorgo_last_replay_ms": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint32)],
     }
     for name, argtypes in sig.items():
         fn = getattr(lib, name)
@@ -198,6 +201,17 @@ def gorgo_state_status(sim, state_workspace, stream: int = 0):
     rc = load().gorgo_state_status(sim, _dev_ptr(state_workspace), state_workspace.numel(),
                                    stream, C.byref(seen))
     return rc, seen.value
+
+
+def gorgo_set_profiling(sim, enable: bool) -> int:
+    return load().gorgo_set_profiling(sim, int(bool(enable)))
+
+
+def gorgo_last_replay_ms(sim):
+    """Returns (status, summed replay-kernel milliseconds, timed launches) of the last evaluation."""
+    ms, n = C.c_double(), C.c_uint32()
+    rc = load().gorgo_last_replay_ms(sim, C.byref(ms), C.byref(n))
+    return rc, ms.value, n.value
 
 
 # ------------------------------------------------------------------------ buffer holder

@@ -17,6 +17,10 @@ struct gorgo_sim {
   int device = 0;
   bool has_trace = false;
   TraceView tr = {};
+  // optional CUDA-event timing of the replay kernel (one pair per wave of the last evaluation)
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev;
+  uint32_t ev_used = 0;
 };
 
 namespace {
@@ -162,6 +166,7 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
     return GORGO_ERR_CUDA;
   std::vector<int32_t> h_status;
   if (host_io) h_status.assign(P, 0);
+  sim->ev_used = 0;
 
   for (uint32_t p0 = 0; p0 < P; p0 += res) {
     const uint32_t pw = (P - p0 < res) ? (P - p0) : res;
@@ -198,7 +203,13 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
     a.out_stride = N;
     a.stats = stats ? stats + (size_t)p0 * 4 : nullptr;
     a.status_out = cand_status ? cand_status + p0 : d_status;
+    const bool timed = sim->profiling && sim->ev_used + 2 <= sim->ev.size();
+    if (timed && cudaEventRecord(sim->ev[sim->ev_used], st) != cudaSuccess) return GORGO_ERR_CUDA;
     if (launch_replay(a, pw, st) != cudaSuccess) return GORGO_ERR_CUDA;
+    if (timed) {
+      if (cudaEventRecord(sim->ev[sim->ev_used + 1], st) != cudaSuccess) return GORGO_ERR_CUDA;
+      sim->ev_used += 2;
+    }
 
     SelectArgs s = {};
     s.ttft = a.ttft_out; s.e2e = a.e2e_out; s.stride = N; s.n = (uint32_t)N;
@@ -265,6 +276,10 @@ int gorgo_sim_create(const gorgo_config_t* cfg, gorgo_sim_t** out) {
 
 int gorgo_sim_destroy(gorgo_sim_t* sim) {
   if (!sim) return GORGO_ERR_INVALID_ARG;
+  if (!sim->ev.empty()) {
+    DeviceGuard guard(sim->device);
+    for (cudaEvent_t e : sim->ev) cudaEventDestroy(e);
+  }
   delete sim;
   return GORGO_OK;
 }
@@ -512,6 +527,42 @@ int gorgo_state_status(gorgo_sim_t* sim, void* state_workspace, uint64_t state_b
     return GORGO_ERR_CUDA;
   if (requests_seen) *requests_seen = h.processed;
   return h.status;
+}
+
+int gorgo_set_profiling(gorgo_sim_t* sim, int enable) {
+  if (!sim) return GORGO_ERR_INVALID_ARG;
+  if (enable && sim->ev.empty()) {
+    DeviceGuard guard(sim->device);
+    if (!guard.ok) return GORGO_ERR_CUDA;
+    sim->ev.resize(64);
+    for (size_t i = 0; i < sim->ev.size(); ++i) {
+      if (cudaEventCreate(&sim->ev[i]) != cudaSuccess) {
+        for (size_t j = 0; j < i; ++j) cudaEventDestroy(sim->ev[j]);
+        sim->ev.clear();
+        return GORGO_ERR_CUDA;
+      }
+    }
+  }
+  sim->profiling = enable != 0;
+  sim->ev_used = 0;
+  return GORGO_OK;
+}
+
+int gorgo_last_replay_ms(gorgo_sim_t* sim, double* replay_ms, uint32_t* launches) {
+  if (!sim || !replay_ms) return GORGO_ERR_INVALID_ARG;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  double sum = 0.0;
+  for (uint32_t i = 0; i + 1 < sim->ev_used; i += 2) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(sim->ev[i + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, sim->ev[i], sim->ev[i + 1]) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+    sum += ms;
+  }
+  *replay_ms = sum;
+  if (launches) *launches = sim->ev_used / 2;
+  return GORGO_OK;
 }
 
 const char* gorgo_strerror(int code) {
