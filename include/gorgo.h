@@ -48,7 +48,9 @@ typedef enum gorgo_status {
   GORGO_ERR_CUDA = -5,                /* a CUDA runtime call failed                                */
   GORGO_ERR_DEVICE_LIMIT = -6,        /* a bounded device loop hit its limit (internal invariant)  */
   GORGO_ERR_NO_TRACE = -7,            /* the call needs an uploaded trace                          */
-  GORGO_ERR_OUT_OF_ORDER = -8         /* gorgo_route_batch: `first` is not the next request        */
+  GORGO_ERR_OUT_OF_ORDER = -8,        /* gorgo_route_batch: `first` is not the next request        */
+  GORGO_ERR_STATIC_LIMIT = -9         /* gorgo_eval_population_static: trace too large for the     */
+                                      /* library's built-in scratch array                          */
 } gorgo_status;
 
 /* Simulator configuration; copied by gorgo_sim_create (rtt_ms included). */
@@ -165,6 +167,34 @@ int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
  * evaluation and their number. */
 int gorgo_set_profiling(gorgo_sim_t *sim, int enable);
 int gorgo_last_replay_ms(gorgo_sim_t *sim, double *replay_ms, uint32_t *launches);
+
+/* Population evaluation for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a packaging variant of gorgo_eval_population).  Some hosts of this library
+ * own no allocator they may call at the moment they want a score: code running inside another
+ * framework's memory plan whose pool is already carved up, a plugin that was handed its input
+ * and output buffers and nothing else, a latency-critical control loop (the proxy re-tuning its
+ * weights) that must not hit cudaMalloc's implicit device synchronisation.  For them the replay
+ * scratch (cache masks, replica and slot state, per-request chains, latency arrays) lives in an
+ * array compiled into the library, GORGO_STATIC_SCRATCH_BYTES long, that every GPU which loads
+ * the library holds until the process exits.  The call allocates and frees nothing, on host
+ * paths of the CUDA runtime included: no cudaMalloc, cudaFree or allocating library routine.
+ *
+ * Arguments are those of gorgo_eval_population without the workspace, digest, counters and
+ * status: `params` HOST or DEVICE (P*K doubles), `p95_ttft_ms` / `p95_e2e_ms` DEVICE (P doubles
+ * each), `route` DEVICE P*N bytes or NULL, `hit_blocks` DEVICE P*N uint16 or NULL.
+ * Limit: the scratch of ONE candidate, gorgo_workspace_bytes(sim, 1), must not exceed
+ * GORGO_STATIC_SCRATCH_BYTES, else GORGO_ERR_STATIC_LIMIT and nothing runs; a population whose
+ * candidates do not all fit at once is evaluated in waves.  (Per candidate the scratch is about
+ * 33 bytes per request plus 1 to 8 bytes per distinct block id.)
+ * The first call on a device looks up the array's device address; make that first call outside
+ * any stream capture.  All calls in a process share the one array per GPU and it keeps what the
+ * previous call left there; each call clears what it needs to start from zero, but two calls
+ * whose GPU work overlaps (different streams, different handles, different threads) race on it:
+ * serialise them. */
+#define GORGO_STATIC_SCRATCH_BYTES (64u << 20)
+int gorgo_eval_population_static(gorgo_sim_t *sim, uint32_t n_candidates, const double *params,
+                                 double time_scale, void *cuda_stream, double *p95_ttft_ms,
+                                 double *p95_e2e_ms, uint8_t *route, uint16_t *hit_blocks);
 
 const char *gorgo_strerror(int code);
 

@@ -23,13 +23,15 @@ GORGO_ERR_CUDA = -5
 GORGO_ERR_DEVICE_LIMIT = -6
 GORGO_ERR_NO_TRACE = -7
 GORGO_ERR_OUT_OF_ORDER = -8
+GORGO_ERR_STATIC_LIMIT = -9
+GORGO_STATIC_SCRATCH_BYTES = 64 << 20
 
 EXPORTS = [
     "gorgo_sim_create", "gorgo_sim_destroy", "gorgo_trace_bytes", "gorgo_trace_upload",
     "gorgo_trace_info", "gorgo_workspace_bytes", "gorgo_eval_population",
     "gorgo_eval_population_host", "gorgo_state_bytes", "gorgo_sim_reset", "gorgo_route_batch",
     "gorgo_state_digest", "gorgo_state_status", "gorgo_set_profiling", "gorgo_last_replay_ms",
-    "gorgo_strerror",
+    "gorgo_eval_population_static", "gorgo_strerror",
 ]
 
 
@@ -75,6 +77,7 @@ def load():
         "gorgo_route_batch": [vp, vp, dbl, u64, u64, vp, u64, vp, vp, vp, vp, vp],
         "gorgo_state_digest": [vp, vp, u64, vp, vp],
         "gorgo_state_status": [vp, vp, u64, vp, pu64],
+        "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp],
         "gorgo_set_profiling": [vp, i32],
         "gorgo_last_replay_ms": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint32)],
     }
@@ -170,6 +173,18 @@ def gorgo_eval_population_host(sim, n_candidates, params, time_scale, workspace,
     return load().gorgo_eval_population_host(
         sim, int(n_candidates), host_ptr(params), float(time_scale), _dev_ptr(workspace),
         workspace.numel(), stream, host_ptr(p95_ttft_ms), host_ptr(p95_e2e_ms))
+
+
+def gorgo_eval_population_static(sim, n_candidates, params, time_scale, stream, p95_ttft_ms,
+                                 p95_e2e_ms, route=None, hit_blocks=None) -> int:
+    """Evaluation that uses the scratch array built into the library instead of a workspace, for
+    callers that may not allocate device memory.  ``params``: float64 numpy array (host) or torch
+    CUDA tensor; outputs: torch CUDA tensors.  Returns GORGO_ERR_STATIC_LIMIT when one
+    candidate's scratch exceeds GORGO_STATIC_SCRATCH_BYTES.  Calls must not overlap on the GPU."""
+    pp = _np_ptr(params) if isinstance(params, np.ndarray) else _dev_ptr(params)
+    return load().gorgo_eval_population_static(
+        sim, int(n_candidates), pp, float(time_scale), stream, _dev_ptr(p95_ttft_ms),
+        _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks))
 
 
 def gorgo_state_bytes(sim):

@@ -3,6 +3,7 @@
 // layout, wave scheduling and kernel launches.  No step of the simulation runs on the host.
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -565,6 +566,57 @@ int gorgo_last_replay_ms(gorgo_sim_t* sim, double* replay_ms, uint32_t* launches
   return GORGO_OK;
 }
 
+// ---- evaluation without any caller- or library-side allocation ---------------------------
+// Scratch that ships with the library image: every GPU that loads libgorgo_b200 reserves this
+// much global memory until the process exits.  In host code `g_static_scratch` is only a handle
+// for the runtime, not an address a kernel could use; the device address is looked up once per
+// device with cudaGetSymbolAddress (that device being current) and kept here.
+static __device__ __align__(256) unsigned char g_static_scratch[GORGO_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the built-in scratch on the CURRENT device (looked up on first use).
+int static_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return GORGO_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_ptr[device]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return GORGO_ERR_CUDA;
+    }
+    g_scratch_ptr[device] = p;
+  }
+  *out = g_scratch_ptr[device];
+  return GORGO_OK;
+}
+}  // namespace
+
+int gorgo_eval_population_static(gorgo_sim_t* sim, uint32_t n_candidates, const double* params,
+                                 double time_scale, void* cuda_stream, double* p95_ttft_ms,
+                                 double* p95_e2e_ms, uint8_t* route, uint16_t* hit_blocks) {
+  if (!sim) return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  // one candidate's replay state must fit; a larger population then runs in waves inside it
+  if (make_ws(sim, 1, true).total > (uint64_t)GORGO_STATIC_SCRATCH_BYTES)
+    return GORGO_ERR_STATIC_LIMIT;
+  void* scratch = nullptr;
+  {
+    DeviceGuard guard(sim->device);
+    if (!guard.ok) return GORGO_ERR_CUDA;
+    const int rc = static_scratch_address(sim->device, &scratch);
+    if (rc != GORGO_OK) return rc;
+  }
+  // the evaluation clears the cache masks and replica/slot state of every wave before replaying,
+  // so whatever an earlier call left in the array is never read
+  return eval_impl(sim, n_candidates, params, time_scale, scratch, GORGO_STATIC_SCRATCH_BYTES,
+                   static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, route,
+                   hit_blocks, nullptr, nullptr, nullptr, false);
+}
+
 const char* gorgo_strerror(int code) {
   switch (code) {
     case GORGO_OK: return "ok";
@@ -576,6 +628,7 @@ const char* gorgo_strerror(int code) {
     case GORGO_ERR_DEVICE_LIMIT: return "device-side loop limit reached";
     case GORGO_ERR_NO_TRACE: return "no trace uploaded";
     case GORGO_ERR_OUT_OF_ORDER: return "request batch out of order";
+    case GORGO_ERR_STATIC_LIMIT: return "problem does not fit the library's built-in scratch array";
     default: return "unknown gorgo status";
   }
 }
