@@ -82,6 +82,8 @@ StateLayout make_layout(const Model& m) {
   l.head_fin_off = o; o += rs * 8;
   l.head_off = o; o += rs * 4;
   l.tail_off = o; o += rs * 4;
+  l.head_next_off = o; o += rs * 4;
+  l.head_tok_off = o; o += rs * 4;
   l.bytes = align_up(o);
   return l;
 }

@@ -62,6 +62,8 @@ struct StateLayout {
   uint64_t head_fin_off;   // double[R*S]   finish of the oldest in-flight request of the slot
   uint64_t head_off;       // uint32[R*S]   that request (kNone: slot has nothing in flight)
   uint64_t tail_off;       // uint32[R*S]   newest request queued on the slot
+  uint64_t head_next_off;  // uint32[R*S]   request queued right behind the head (kNone: none)
+  uint64_t head_tok_off;   // uint32[R*S]   input tokens of the head request
   uint64_t bytes;          // size of the block (multiple of 256)
 };
 
@@ -72,6 +74,7 @@ struct ReplayArgs {
   double scale;
   uint32_t first, count;          // requests [first, first+count)
   uint32_t check_order;           // 1: refuse (status) unless header.processed == first
+  uint32_t slots_in_smem;         // set by the launcher: per-slot state fits in shared memory
   const double* rtt;              // [G*R] device
   const double* params;           // [P*K] device
   unsigned char* masks;           // [P * mask_stride] bytes

@@ -15,7 +15,9 @@
 //  * in-flight accounting through per-slot FIFO chains (finish times on one slot never
 //    decrease), with the earliest finish per replica cached so the common case is one compare.
 // One warp replays one candidate; requests are strictly ordered inside a candidate, so the
-// parallelism is across candidates, across the blocks of a request and across replicas.
+// parallelism is across candidates, across the blocks of a request and across replicas.  A
+// second warp of the same CTA runs ahead through the (state-independent) trace and prefetches
+// what the replay warp will touch, since the replay is bound by memory latency, not bandwidth.
 #include "gorgo_internal.h"
 
 namespace gorgo {
@@ -96,30 +98,172 @@ __device__ __forceinline__ uint64_t mix64(uint64_t z) {  // splitmix64 finaliser
 }
 
 // ------------------------------------------------------------------------------ replay
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
+// Clear `bit` of mask[id] without reading it back (a reduction performed in L2).
 template <typename MaskT>
-__global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
+__device__ __forceinline__ void mask_clear_bit(MaskT* mask, uint32_t id, MaskT bit) {
+  if (sizeof(MaskT) == 8) {
+    atomicAnd(reinterpret_cast<unsigned long long*>(mask) + id, ~(unsigned long long)bit);
+  } else {
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(mask + id);
+    const uint32_t sh = (uint32_t)(addr & 3u) * 8u;
+    atomicAnd(reinterpret_cast<unsigned int*>(addr & ~(uintptr_t)3), ~((uint32_t)bit << sh));
+  }
+}
+// Mask words are read and written around L1: they are also changed by reductions in L2.
+template <typename MaskT>
+__device__ __forceinline__ MaskT mask_load(const MaskT* mask, uint32_t id) {
+  return __ldcg(mask + id);
+}
+template <>
+__device__ __forceinline__ uint8_t mask_load<uint8_t>(const uint8_t* mask, uint32_t id) {
+  return __ldcg(reinterpret_cast<const unsigned char*>(mask) + id);
+}
+template <>
+__device__ __forceinline__ uint16_t mask_load<uint16_t>(const uint16_t* mask, uint32_t id) {
+  return __ldcg(reinterpret_cast<const unsigned short*>(mask) + id);
+}
+template <>
+__device__ __forceinline__ uint64_t mask_load<uint64_t>(const uint64_t* mask, uint32_t id) {
+  return __ldcg(reinterpret_cast<const unsigned long long*>(mask) + id);
+}
+template <typename MaskT>
+__device__ __forceinline__ void mask_store(MaskT* mask, uint32_t id, MaskT v) {
+  __stcg(mask + id, v);
+}
+template <>
+__device__ __forceinline__ void mask_store<uint8_t>(uint8_t* mask, uint32_t id, uint8_t v) {
+  __stcg(reinterpret_cast<unsigned char*>(mask) + id, (unsigned char)v);
+}
+template <>
+__device__ __forceinline__ void mask_store<uint16_t>(uint16_t* mask, uint32_t id, uint16_t v) {
+  __stcg(reinterpret_cast<unsigned short*>(mask) + id, (unsigned short)v);
+}
+template <>
+__device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id, uint64_t v) {
+  __stcg(reinterpret_cast<unsigned long long*>(mask) + id, (unsigned long long)v);
+}
+
+constexpr int kRegChunks = 8;     // request blocks held in registers: 8 x 32 = 256
+constexpr int kEvictBatches = 4;  // touches examined per lane and eviction round
+constexpr uint32_t kAhead = 48;   // how far the helper warp runs ahead of the replay (requests)
+
+// Shared-memory view of one candidate's small state.
+struct Smem {
+  double* rtt; double* w; double* minfin; long long* load;
+  uint32_t* occ; uint32_t* curreq; int32_t* curpos; uint32_t* lrutail;
+  volatile uint32_t* progress;
+};
+
+// Helper warp: runs ahead of the replay warp of the same candidate and pulls what it will touch
+// into L2 (mask words, next-occurrence links at the eviction cursors) and L1/L2 (request
+// records, block ids).  Pure prefetching: it changes no state and may stop at any time.
+template <typename MaskT>
+__device__ void helper_warp(const ReplayArgs& a, const Smem& sm, const MaskT* mask,
+                            const uint32_t* lru_next, uint32_t lane) {
+  const ReqRec* req = a.tr.req;
+  const uint32_t* ids = a.tr.ids;
+  const uint32_t end = a.first + a.count;
+  const uint32_t R = a.m.R;
+  uint32_t pos = a.first;
+  uint32_t idle = 0;
+  constexpr uint32_t kLineShift = sizeof(MaskT) == 1 ? 5 : sizeof(MaskT) == 2 ? 4
+                                  : sizeof(MaskT) == 4 ? 3 : 2;   // ids per 32-byte sector
+  while (pos < end) {
+    const uint32_t cur = *sm.progress;
+    if (cur >= end) break;
+    if (pos < cur) pos = cur;                       // fell behind: skip what is already done
+    if (pos >= cur + kAhead) {
+      if (++idle > (1u << 24)) break;               // bounded wait; prefetching is optional
+      __nanosleep(256);
+      continue;
+    }
+    // one batch of up to 16 requests: every lane fetches one record, then the warp walks them
+    const uint32_t nb = min(16u, end - pos);
+    ReqRec mine = {};
+    if (lane < nb) mine = req[pos + lane];
+    for (uint32_t j = 0; j < nb; ++j) {
+      const uint32_t off = __shfl_sync(kFull, mine.off, j);
+      const uint32_t n = __shfl_sync(kFull, (uint32_t)mine.nblk, j);
+      for (uint32_t c = 0; c < n; c += 32) {
+        const uint32_t k = c + lane;
+        const uint32_t id = (k < n) ? ids[off + k] : 0u;
+        const uint32_t prev = __shfl_up_sync(kFull, id, 1);
+        if (k < n && (lane == 0 || (prev >> kLineShift) != (id >> kLineShift)))
+          prefetch_l2(mask + id);
+      }
+    }
+    // eviction cursors: the links and ids of the next touches of every replica
+    for (uint32_t i = lane; i < R; i += 32) {
+      uint32_t cr = sm.curreq[i];
+      int32_t cp = sm.curpos[i];
+      int32_t budget = 256;
+      for (int hop = 0; hop < 4 && cr != kNone && budget > 0; ++hop) {
+        if (hop > 0 || cp < 0) {
+          cr = lru_next[cr];
+          if (cr == kNone || cr >= cur) break;
+          cp = (int32_t)req[cr].nblk - 1;
+        }
+        if (cp < 0) continue;
+        const uint32_t coff = req[cr].off;
+        const int32_t lo = cp - budget + 1 > 0 ? cp - budget + 1 : 0;
+        for (int32_t k = lo & ~15; k <= cp; k += 16) {   // 16 links = 128 bytes
+          prefetch_l2(a.tr.occ_next + coff + k);
+          if ((k & 31) == 0 || k == (lo & ~15)) prefetch_l2(ids + coff + k);
+        }
+        budget -= cp - lo + 1;
+        cp = -1;
+      }
+    }
+    pos += nb;
+    idle = 0;
+  }
+}
+
+template <typename MaskT>
+__global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
   const uint32_t p = blockIdx.x;
-  const uint32_t lane = threadIdx.x;
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t warp = threadIdx.x >> 5;
   const uint32_t R = a.m.R, S = a.m.S, K = a.m.K, G = a.m.G;
   const uint32_t N = a.tr.n_req;
-
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* s_rtt = reinterpret_cast<double*>(smem_raw);   // [G*R]
-  double* s_w = s_rtt + (size_t)G * R;                   // [K]
-  double* s_minfin = s_w + K;                            // [R]
-  long long* s_load = reinterpret_cast<long long*>(s_minfin + R);  // [R]
-  uint32_t* s_occ = reinterpret_cast<uint32_t*>(s_load + R);       // [R]
-  uint32_t* s_curreq = s_occ + R;
-  int32_t* s_curpos = reinterpret_cast<int32_t*>(s_curreq + R);
-  uint32_t* s_lrutail = reinterpret_cast<uint32_t*>(s_curpos + R);
+  const uint32_t RS = R * S;
 
   unsigned char* st = a.states + (size_t)p * a.lay.bytes;
   CandHeader* hdr = reinterpret_cast<CandHeader*>(st);
   RepState* g_rep = reinterpret_cast<RepState*>(st + a.lay.rep_off);
-  double* free_at = reinterpret_cast<double*>(st + a.lay.free_at_off);
-  double* head_fin = reinterpret_cast<double*>(st + a.lay.head_fin_off);
-  uint32_t* head = reinterpret_cast<uint32_t*>(st + a.lay.head_off);
-  uint32_t* tail = reinterpret_cast<uint32_t*>(st + a.lay.tail_off);
+  double* g_free_at = reinterpret_cast<double*>(st + a.lay.free_at_off);
+  double* g_head_fin = reinterpret_cast<double*>(st + a.lay.head_fin_off);
+  uint32_t* g_head = reinterpret_cast<uint32_t*>(st + a.lay.head_off);
+  uint32_t* g_tail = reinterpret_cast<uint32_t*>(st + a.lay.tail_off);
+  uint32_t* g_head_next = reinterpret_cast<uint32_t*>(st + a.lay.head_next_off);
+  uint32_t* g_head_tok = reinterpret_cast<uint32_t*>(st + a.lay.head_tok_off);
+
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem sm;
+  sm.rtt = reinterpret_cast<double*>(smem_raw);            // [G*R]
+  sm.w = sm.rtt + (size_t)G * R;                           // [K]
+  sm.minfin = sm.w + K;                                    // [R]
+  sm.load = reinterpret_cast<long long*>(sm.minfin + R);   // [R]
+  double* dnext = reinterpret_cast<double*>(sm.load + R);
+  // per-slot state: in shared memory when it fits, else it stays in global memory
+  double *free_at = g_free_at, *head_fin = g_head_fin;
+  if (a.slots_in_smem) { free_at = dnext; head_fin = dnext + RS; dnext += 2 * (size_t)RS; }
+  sm.occ = reinterpret_cast<uint32_t*>(dnext);             // [R]
+  sm.curreq = sm.occ + R;
+  sm.curpos = reinterpret_cast<int32_t*>(sm.curreq + R);
+  sm.lrutail = reinterpret_cast<uint32_t*>(sm.curpos + R);
+  uint32_t* unext = sm.lrutail + R;
+  uint32_t *head = g_head, *tail = g_tail, *head_next = g_head_next, *head_tok = g_head_tok;
+  if (a.slots_in_smem) {
+    head = unext; tail = unext + RS; head_next = unext + 2 * (size_t)RS;
+    head_tok = unext + 3 * (size_t)RS; unext += 4 * (size_t)RS;
+  }
+  sm.progress = unext;
+
   MaskT* mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
   double* fin = a.fin + (size_t)p * N;
   uint32_t* slot_next = a.slot_next + (size_t)p * N;
@@ -128,40 +272,69 @@ __global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
 
-  if (a.check_order && hdr->processed != a.first) {
-    if (lane == 0) {
+  if (a.check_order && hdr->processed != a.first) {   // uniform over the CTA
+    if (threadIdx.x == 0) {
       hdr->status = -8;
       if (a.status_out) a.status_out[p] = -8;
     }
     return;
   }
 
-  for (uint32_t i = lane; i < G * R; i += 32) s_rtt[i] = a.rtt[i];
-  for (uint32_t i = lane; i < K; i += 32) s_w[i] = a.params[(size_t)p * K + i];
-  for (uint32_t i = lane; i < R; i += 32) {
+  for (uint32_t i = threadIdx.x; i < G * R; i += blockDim.x) sm.rtt[i] = a.rtt[i];
+  for (uint32_t i = threadIdx.x; i < K; i += blockDim.x) sm.w[i] = a.params[(size_t)p * K + i];
+  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
     const RepState rs = g_rep[i];
-    s_minfin[i] = rs.min_fin; s_load[i] = rs.load; s_occ[i] = rs.occ;
-    s_curreq[i] = rs.cur_req; s_curpos[i] = rs.cur_pos; s_lrutail[i] = rs.lru_tail;
+    sm.minfin[i] = rs.min_fin; sm.load[i] = rs.load; sm.occ[i] = rs.occ;
+    sm.curreq[i] = rs.cur_req; sm.curpos[i] = rs.cur_pos; sm.lrutail[i] = rs.lru_tail;
   }
-  __syncwarp();
+  if (a.slots_in_smem) {
+    for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) {
+      free_at[x] = g_free_at[x]; head_fin[x] = g_head_fin[x]; head[x] = g_head[x];
+      tail[x] = g_tail[x]; head_next[x] = g_head_next[x]; head_tok[x] = g_head_tok[x];
+    }
+  }
+  if (threadIdx.x == 0) *sm.progress = a.first;
+  __syncthreads();
 
-  const double w_net = s_w[0], w_pre = s_w[1], w_que = s_w[2];
+  if (warp == 1) {
+    helper_warp<MaskT>(a, sm, mask, lru_next, lane);
+    return;
+  }
+
+  const double w_net = sm.w[0], w_pre = sm.w[1], w_que = sm.w[2];
   const MaskT all_reps = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0
                                                   : (MaskT)((((MaskT)1) << (R & 63)) - 1);
   int32_t status = 0;
   unsigned long long st_probe = 0, st_hit = 0, st_blk = 0, st_evict = 0;
+  const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
 
+  ReqRec rec_next = req[a.first];
   for (uint32_t j = 0; j < a.count; ++j) {
     const uint32_t r = a.first + j;
-    const ReqRec rec = req[r];
+    const ReqRec rec = rec_next;
+    if (j + 1 < a.count) rec_next = req[r + 1];          // in flight while this request runs
     const double t = __dmul_rn(a.scale, rec.ts_ms);
     const uint32_t n = rec.nblk, off = rec.off, in_tok = rec.in_tok;
-    const double* rtt_row = s_rtt + (size_t)rec.origin * R;
+    const double* rtt_row = sm.rtt + (size_t)rec.origin * R;
+
+    // ---- issue the probe loads first: block ids, then the mask word of every block
+    uint32_t idr[kRegChunks];
+    MaskT mr[kRegChunks];
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c) {
+      const uint32_t k = c * 32u + lane;
+      idr[c] = (k < n) ? ids[off + k] : 0u;
+    }
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c) {
+      const uint32_t k = c * 32u + lane;
+      mr[c] = (k < n) ? mask_load<MaskT>(mask, idr[c]) : (MaskT)0;
+    }
 
     // ---- queue signal: drop requests that completed by t (finish <= t)
     for (uint32_t i0 = 0; i0 < R; i0 += 32) {
       const uint32_t i = i0 + lane;
-      unsigned due = __ballot_sync(kFull, i < R && s_minfin[i] <= t);
+      unsigned due = __ballot_sync(kFull, i < R && sm.minfin[i] <= t);
       while (due) {
         const uint32_t ii = i0 + (uint32_t)__ffs((int)due) - 1;
         due &= due - 1;
@@ -171,23 +344,22 @@ __global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
           const size_t x = (size_t)ii * S + s;
           double hf = head_fin[x];
           if (hf <= t) {
-            uint32_t hd = head[x];
             uint32_t guard = 0;
+            uint32_t hd, hn = head_next[x], ht = head_tok[x];
             do {
-              tok += (long long)req[hd].in_tok;
-              const uint32_t nx = slot_next[hd];
-              if (nx == kNone) { hd = kNone; hf = d_inf(); }
-              else { hd = nx; hf = fin[nx]; }
+              tok += (long long)ht;
+              hd = hn;
+              if (hd == kNone) { hf = d_inf(); hn = kNone; ht = 0; }
+              else { hf = fin[hd]; hn = slot_next[hd]; ht = req[hd].in_tok; }
               if (++guard > N) { status = -6; break; }
             } while (hf <= t);
-            head[x] = hd;
-            head_fin[x] = hf;
+            head[x] = hd; head_fin[x] = hf; head_next[x] = hn; head_tok[x] = ht;
           }
           mn = fmin(mn, hf);
         }
         tok = warp_sum_ll(tok);
         mn = warp_min_d(mn);
-        if (lane == 0) { s_load[ii] -= tok; s_minfin[ii] = mn; }
+        if (lane == 0) { sm.load[ii] -= tok; sm.minfin[ii] = mn; }
       }
     }
     __syncwarp();
@@ -196,10 +368,32 @@ __global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
     uint32_t h0 = 0, h1 = 0;  // this lane's replicas: lane and lane+32
     {
       MaskT alive = all_reps;
-      for (uint32_t c = 0; c < n && alive != 0; c += 32) {
+#pragma unroll
+      for (int c = 0; c < kRegChunks; ++c) {
+        if (c * 32u < n && alive != 0) {
+          MaskT pm = mr[c];
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            const MaskT o = shfl_up_mask<MaskT>(pm, d);
+            if ((int)lane >= d) pm &= o;
+          }
+          pm &= alive;
+          MaskT it = shfl_mask<MaskT>(pm, 0);
+          while (it != 0) {
+            const int i = first_bit<MaskT>(it);
+            it &= (MaskT)(it - 1);
+            const unsigned b = __ballot_sync(kFull, (pm >> i) & 1);
+            if ((uint32_t)(i & 31) == lane) {
+              if (i < 32) h0 += __popc(b); else h1 += __popc(b);
+            }
+          }
+          alive = shfl_mask<MaskT>(pm, 31);
+        }
+      }
+      for (uint32_t c = kRegChunks * 32u; c < n && alive != 0; c += 32) {   // very long prompts
         const uint32_t k = c + lane;
         MaskT pm = 0;
-        if (k < n) pm = mask[ids[off + k]];
+        if (k < n) pm = mask_load<MaskT>(mask, ids[off + k]);
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
           const MaskT o = shfl_up_mask<MaskT>(pm, d);
@@ -231,8 +425,8 @@ __global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
         const unsigned long long hb = (unsigned long long)h * a.m.B;
         const uint32_t unc = in_tok - (uint32_t)(hb < in_tok ? hb : in_tok);
         if (half) unc1 = unc; else unc0 = unc;
-        double q = (double)s_load[i];
-        if (K != 3) q = __dmul_rn(q, s_w[3 + i]);
+        double q = (double)sm.load[i];
+        if (K != 3) q = __dmul_rn(q, sm.w[3 + i]);
         double c = __dadd_rn(__dadd_rn(__dmul_rn(w_net, rtt_row[i]), __dmul_rn(w_pre, (double)unc)),
                              __dmul_rn(w_que, q));
         if (c != c) c = (i == 0) ? -d_inf() : d_inf();  // a NaN score wins only at index 0
@@ -249,27 +443,35 @@ __global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
 
     // ---- cache commit: set the replica's bit on the missing blocks
     uint32_t missing = 0;
-    for (uint32_t c = 0; c < n; c += 32) {
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c) {
+      if (c * 32u < n) {
+        const uint32_t k = c * 32u + lane;
+        const bool miss = (k < n) && !(mr[c] & bit);
+        if (miss) mask_store<MaskT>(mask, idr[c], (MaskT)(mr[c] | bit));
+        missing += __popc(__ballot_sync(kFull, miss));
+      }
+    }
+    for (uint32_t c = kRegChunks * 32u; c < n; c += 32) {
       const uint32_t k = c + lane;
       bool miss = false;
       if (k < n) {
         const uint32_t id = ids[off + k];
-        const MaskT mv = mask[id];
-        if (!(mv & bit)) { mask[id] = (MaskT)(mv | bit); miss = true; }
+        const MaskT mv = mask_load<MaskT>(mask, id);
+        if (!(mv & bit)) { mask_store<MaskT>(mask, id, (MaskT)(mv | bit)); miss = true; }
       }
       missing += __popc(__ballot_sync(kFull, miss));
     }
-    uint32_t occ = s_occ[istar] + missing;
+    uint32_t occ = sm.occ[istar] + missing;
     uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
     uint32_t evicted = 0;
     if (need > 0) {
-      uint32_t cr = s_curreq[istar];
-      int32_t cp = s_curpos[istar];
+      uint32_t cr = sm.curreq[istar];
+      int32_t cp = sm.curpos[istar];
       uint32_t coff = (cr != kNone) ? req[cr].off : 0u;
       unsigned long long guard = 0;
-      const unsigned long long guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
       while (need > 0) {
-        if (++guard > guard_max) { status = -6; break; }
+        if (++guard > evict_guard_max) { status = -6; break; }
         if (cp < 0) {  // this request is used up: go to the next one routed here
           const uint32_t nx = (cr == kNone) ? kNone : lru_next[cr];
           if (nx == kNone) { status = -6; break; }
@@ -279,33 +481,64 @@ __global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
           cp = (int32_t)cre.nblk - 1;
           continue;
         }
-        const int32_t k = cp - (int32_t)lane;   // deepest position first
-        bool live = false;
-        uint32_t g = 0;
-        if (k >= 0) {
-          g = coff + (uint32_t)k;
-          live = !touch_is_stale(a.tr, route_log, g, istar, r, istar);
+        // examine up to kEvictBatches x 32 touches, deepest position first; all loads of the
+        // round are issued before any is used
+        const uint32_t nbat = min((uint32_t)kEvictBatches, (2u * need + 31u) / 32u);
+        uint2 nx[kEvictBatches];
+        uint32_t vid[kEvictBatches];
+        uint32_t rt[kEvictBatches];
+        bool valid[kEvictBatches];
+#pragma unroll
+        for (int u = 0; u < kEvictBatches; ++u) {
+          const int32_t k = cp - (int32_t)(u * 32u + lane);
+          valid[u] = (uint32_t)u < nbat && k >= 0;
+          nx[u] = make_uint2(kNone, kNone);
+          vid[u] = 0;
+          if (valid[u]) {
+            const uint32_t g = coff + (uint32_t)k;
+            nx[u] = a.tr.occ_next[g];
+            vid[u] = ids[g];
+          }
         }
-        const unsigned lv = __ballot_sync(kFull, live);
-        const uint32_t cnt = __popc(lv);
-        unsigned take;
-        int32_t adv;
-        if (cnt <= need) { take = lv; adv = 32; }
-        else {
-          const unsigned pos = __fns(lv, 0, (int)need);
-          take = lv & ((2u << pos) - 1u);
-          adv = (int32_t)pos + 1;
+#pragma unroll
+        for (int u = 0; u < kEvictBatches; ++u) {   // first hop of every touch
+          rt[u] = kNone;
+          if (valid[u] && nx[u].x != kNone && nx[u].y <= r)
+            rt[u] = (nx[u].y == r) ? istar : (uint32_t)route_log[nx[u].y];
         }
-        if ((take >> lane) & 1u) {
-          const uint32_t id = ids[g];
-          mask[id] = (MaskT)(mask[id] & (MaskT)~bit);
+        int32_t adv = 0;
+#pragma unroll
+        for (int u = 0; u < kEvictBatches; ++u) {
+          if ((uint32_t)u < nbat && need > 0) {
+            bool live = false;
+            if (valid[u]) {
+              live = true;
+              uint2 c = nx[u];
+              uint32_t rr = rt[u];
+              while (c.x != kNone && c.y <= r) {     // later occurrences of the block, up to r
+                if (rr == istar) { live = false; break; }
+                c = a.tr.occ_next[c.x];
+                if (c.x != kNone && c.y <= r) rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
+              }
+            }
+            const unsigned lv = __ballot_sync(kFull, live);
+            const uint32_t cnt = __popc(lv);
+            unsigned take;
+            if (cnt <= need) { take = lv; adv += 32; }
+            else {
+              const unsigned pos = __fns(lv, 0, (int)need);
+              take = lv & ((2u << pos) - 1u);
+              adv += (int32_t)pos + 1;
+            }
+            if ((take >> lane) & 1u) mask_clear_bit<MaskT>(mask, vid[u], bit);
+            const uint32_t tk = __popc(take);
+            need -= tk;
+            evicted += tk;
+          }
         }
-        const uint32_t tk = __popc(take);
-        need -= tk;
-        evicted += tk;
         cp -= adv;
       }
-      if (lane == 0) { s_curreq[istar] = cr; s_curpos[istar] = cp; }
+      if (lane == 0) { sm.curreq[istar] = cr; sm.curpos[istar] = cp; }
     }
     occ -= evicted;
 
@@ -328,22 +561,23 @@ __global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
       fin[r] = finish;
       slot_next[r] = kNone;
       if (head[x] == kNone) {
-        head[x] = r;
-        head_fin[x] = finish;
-        s_minfin[istar] = fmin(s_minfin[istar], finish);
+        head[x] = r; head_fin[x] = finish; head_next[x] = kNone; head_tok[x] = in_tok;
+        sm.minfin[istar] = fmin(sm.minfin[istar], finish);
       } else {
-        slot_next[tail[x]] = r;
+        const uint32_t tl = tail[x];
+        slot_next[tl] = r;
+        if (tl == head[x]) head_next[x] = r;
       }
       tail[x] = r;
       free_at[x] = finish;
-      s_load[istar] += (long long)in_tok;
-      s_occ[istar] = occ;
+      sm.load[istar] += (long long)in_tok;
+      sm.occ[istar] = occ;
       // recency order of the replica: append this request
-      const uint32_t lt = s_lrutail[istar];
+      const uint32_t lt = sm.lrutail[istar];
       if (lt != kNone) lru_next[lt] = r;
       lru_next[r] = kNone;
-      if (s_curreq[istar] == kNone) { s_curreq[istar] = r; s_curpos[istar] = (int32_t)n - 1; }
-      s_lrutail[istar] = r;
+      if (sm.curreq[istar] == kNone) { sm.curreq[istar] = r; sm.curpos[istar] = (int32_t)n - 1; }
+      sm.lrutail[istar] = r;
       route_log[r] = (uint8_t)istar;
       const size_t o = (size_t)p * a.out_stride + j;
       if (a.route_out) a.route_out[o] = (uint8_t)istar;
@@ -351,16 +585,24 @@ __global__ void __launch_bounds__(32) replay_kernel(const ReplayArgs a) {
       if (a.ttft_out) a.ttft_out[o] = __dsub_rn(first, t);
       if (a.e2e_out) a.e2e_out[o] = __dsub_rn(finish, t);
       st_hit += hstar; st_blk += n; st_evict += evicted;
+      *sm.progress = r + 1;
     }
     __syncwarp();
   }
 
-  // ---- write the replica scalars back
+  // ---- write the small state back
+  if (lane == 0) *sm.progress = a.first + a.count;
   for (uint32_t i = lane; i < R; i += 32) {
     RepState rs;
-    rs.min_fin = s_minfin[i]; rs.load = s_load[i]; rs.occ = s_occ[i];
-    rs.cur_req = s_curreq[i]; rs.cur_pos = s_curpos[i]; rs.lru_tail = s_lrutail[i];
+    rs.min_fin = sm.minfin[i]; rs.load = sm.load[i]; rs.occ = sm.occ[i];
+    rs.cur_req = sm.curreq[i]; rs.cur_pos = sm.curpos[i]; rs.lru_tail = sm.lrutail[i];
     g_rep[i] = rs;
+  }
+  if (a.slots_in_smem) {
+    for (uint32_t x = lane; x < RS; x += 32) {
+      g_free_at[x] = free_at[x]; g_head_fin[x] = head_fin[x]; g_head[x] = head[x];
+      g_tail[x] = tail[x]; g_head_next[x] = head_next[x]; g_head_tok[x] = head_tok[x];
+    }
   }
   st_probe = warp_sum_u64(st_probe);
   status = __reduce_min_sync(kFull, status);
@@ -396,8 +638,11 @@ __global__ void reset_states_kernel(unsigned char* states, StateLayout lay, uint
   double* head_fin = reinterpret_cast<double*>(st + lay.head_fin_off);
   uint32_t* head = reinterpret_cast<uint32_t*>(st + lay.head_off);
   uint32_t* tail = reinterpret_cast<uint32_t*>(st + lay.tail_off);
+  uint32_t* head_next = reinterpret_cast<uint32_t*>(st + lay.head_next_off);
+  uint32_t* head_tok = reinterpret_cast<uint32_t*>(st + lay.head_tok_off);
   for (uint32_t x = threadIdx.x; x < R * S; x += blockDim.x) {
     free_at[x] = 0.0; head_fin[x] = d_inf(); head[x] = kNone; tail[x] = kNone;
+    head_next[x] = kNone; head_tok[x] = 0;
   }
 }
 
@@ -498,15 +743,19 @@ __global__ void __launch_bounds__(256) digest_kernel(const DigestArgs a) {
 }
 
 template <typename MaskT>
-cudaError_t launch_replay_t(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st) {
-  const size_t smem = ((size_t)a.m.G * a.m.R + a.m.K + a.m.R) * sizeof(double) +
-                      (size_t)a.m.R * (sizeof(long long) + 4 * sizeof(uint32_t));
+cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
+  const size_t rs = (size_t)a.m.R * a.m.S;
+  a.slots_in_smem = rs * 32 <= 32 * 1024 ? 1u : 0u;
+  size_t smem = ((size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
+                (4 * (size_t)a.m.R + 1) * sizeof(uint32_t);
+  if (a.slots_in_smem) smem += rs * 32;
+  smem = (smem + 15) / 16 * 16;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  replay_kernel<MaskT><<<n_cand, 32, smem, st>>>(a);
+  replay_kernel<MaskT><<<n_cand, 64, smem, st>>>(a);
   return cudaGetLastError();
 }
 
