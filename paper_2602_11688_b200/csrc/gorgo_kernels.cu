@@ -50,29 +50,30 @@ __device__ __forceinline__ int first_bit(MaskT v) {  // v != 0
   return __ffs((int)(uint32_t)v) - 1;
 }
 
-__device__ __forceinline__ long long warp_sum_ll(long long v) {
-#pragma unroll
-  for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(kFull, v, d);
-  return v;
-}
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(kFull, v, d);
   return v;
 }
-__device__ __forceinline__ double warp_min_d(double v) {
-#pragma unroll
-  for (int d = 16; d > 0; d >>= 1) v = fmin(v, __shfl_xor_sync(kFull, v, d));
-  return v;
+// Order-preserving 64-bit key of a double (no NaN): -0.0 is folded onto +0.0 first so that the
+// two zeros tie, as they do under '<'.
+__device__ __forceinline__ uint64_t order_key(double v) {
+  const uint64_t b = (uint64_t)__double_as_longlong(__dadd_rn(v, 0.0));
+  return (b >> 63) ? ~b : (b | 0x8000000000000000ULL);
 }
-// Minimum of (value, index) pairs, the lower index winning equal values.
-__device__ __forceinline__ void warp_argmin(double& v, uint32_t& i) {
-#pragma unroll
-  for (int d = 16; d > 0; d >>= 1) {
-    const double ov = __shfl_xor_sync(kFull, v, d);
-    const uint32_t oi = __shfl_xor_sync(kFull, i, d);
-    if (ov < v || (ov == v && oi < i)) { v = ov; i = oi; }
-  }
+__device__ __forceinline__ double order_value(uint64_t k) {
+  const uint64_t b = (k >> 63) ? (k & 0x7FFFFFFFFFFFFFFFULL) : ~k;
+  return __longlong_as_double((long long)b);
+}
+// Warp-wide minimum of 64-bit keys with the lowest index among equal keys; lanes that do not
+// take part pass key = ~0 and idx = kNone.  Returns the winning index, the key through `key`.
+__device__ __forceinline__ uint32_t warp_argmin_key(uint64_t& key, uint32_t idx) {
+  const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+  const uint32_t mh = __reduce_min_sync(kFull, hi);
+  const uint32_t ml = __reduce_min_sync(kFull, hi == mh ? lo : 0xFFFFFFFFu);
+  const bool win = hi == mh && lo == ml;
+  key = ((uint64_t)mh << 32) | ml;
+  return __reduce_min_sync(kFull, win ? idx : kNone);
 }
 
 // Is the touch at flat position g (a block of a request routed to replica `rep`) no longer
@@ -148,12 +149,12 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
 }
 
 constexpr int kRegChunks = 8;     // request blocks held in registers: 8 x 32 = 256
-constexpr int kEvictBatches = 4;  // touches examined per lane and eviction round
+constexpr int kEvictBatches = 2;  // touches examined per lane and eviction round
 constexpr uint32_t kAhead = 48;   // how far the helper warp runs ahead of the replay (requests)
 
 // Shared-memory view of one candidate's small state.
 struct Smem {
-  double* rtt; double* w; double* minfin; long long* load;
+  double* rtt; double* wrtt; double* w; double* minfin; long long* load;
   uint32_t* occ; uint32_t* curreq; int32_t* curpos; uint32_t* lrutail;
   volatile uint32_t* progress;
 };
@@ -245,7 +246,8 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem sm;
   sm.rtt = reinterpret_cast<double*>(smem_raw);            // [G*R]
-  sm.w = sm.rtt + (size_t)G * R;                           // [K]
+  sm.wrtt = sm.rtt + (size_t)G * R;                        // [G*R]  w_net * rtt
+  sm.w = sm.wrtt + (size_t)G * R;                          // [K]
   sm.minfin = sm.w + K;                                    // [R]
   sm.load = reinterpret_cast<long long*>(sm.minfin + R);   // [R]
   double* dnext = reinterpret_cast<double*>(sm.load + R);
@@ -280,7 +282,11 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
     return;
   }
 
-  for (uint32_t i = threadIdx.x; i < G * R; i += blockDim.x) sm.rtt[i] = a.rtt[i];
+  for (uint32_t i = threadIdx.x; i < G * R; i += blockDim.x) {
+    const double v = a.rtt[i];
+    sm.rtt[i] = v;
+    sm.wrtt[i] = __dmul_rn(a.params[(size_t)p * K], v);   // first product of the score
+  }
   for (uint32_t i = threadIdx.x; i < K; i += blockDim.x) sm.w[i] = a.params[(size_t)p * K + i];
   for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
     const RepState rs = g_rep[i];
@@ -301,7 +307,7 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
     return;
   }
 
-  const double w_net = sm.w[0], w_pre = sm.w[1], w_que = sm.w[2];
+  const double w_pre = sm.w[1], w_que = sm.w[2];
   const MaskT all_reps = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0
                                                   : (MaskT)((((MaskT)1) << (R & 63)) - 1);
   int32_t status = 0;
@@ -321,14 +327,30 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
     uint32_t idr[kRegChunks];
     MaskT mr[kRegChunks];
 #pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) {
+    for (int c = 0; c < kRegChunks; ++c) { idr[c] = 0u; mr[c] = (MaskT)0; }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
       const uint32_t k = c * 32u + lane;
-      idr[c] = (k < n) ? ids[off + k] : 0u;
+      if (k < n) idr[c] = ids[off + k];
+    }
+    if (n > 64) {
+#pragma unroll
+      for (int c = 2; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        if (k < n) idr[c] = ids[off + k];
+      }
     }
 #pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) {
+    for (int c = 0; c < 2; ++c) {
       const uint32_t k = c * 32u + lane;
-      mr[c] = (k < n) ? mask_load<MaskT>(mask, idr[c]) : (MaskT)0;
+      if (k < n) mr[c] = mask_load<MaskT>(mask, idr[c]);
+    }
+    if (n > 64) {
+#pragma unroll
+      for (int c = 2; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        if (k < n) mr[c] = mask_load<MaskT>(mask, idr[c]);
+      }
     }
 
     // ---- queue signal: drop requests that completed by t (finish <= t)
@@ -357,9 +379,11 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
           }
           mn = fmin(mn, hf);
         }
-        tok = warp_sum_ll(tok);
-        mn = warp_min_d(mn);
-        if (lane == 0) { sm.load[ii] -= tok; sm.minfin[ii] = mn; }
+        if (tok != 0)
+          atomicAdd(reinterpret_cast<unsigned long long*>(sm.load + ii), (unsigned long long)(-tok));
+        uint64_t mk = order_key(mn);
+        warp_argmin_key(mk, lane);
+        if (lane == 0) sm.minfin[ii] = order_value(mk);
       }
     }
     __syncwarp();
@@ -367,56 +391,38 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
     // ---- prefix probe on every replica: h_i = leading blocks whose mask has bit i
     uint32_t h0 = 0, h1 = 0;  // this lane's replicas: lane and lane+32
     {
-      MaskT alive = all_reps;
-#pragma unroll
-      for (int c = 0; c < kRegChunks; ++c) {
-        if (c * 32u < n && alive != 0) {
-          MaskT pm = mr[c];
-#pragma unroll
-          for (int d = 1; d < 32; d <<= 1) {
-            const MaskT o = shfl_up_mask<MaskT>(pm, d);
-            if ((int)lane >= d) pm &= o;
-          }
-          pm &= alive;
-          MaskT it = shfl_mask<MaskT>(pm, 0);
-          while (it != 0) {
-            const int i = first_bit<MaskT>(it);
-            it &= (MaskT)(it - 1);
-            const unsigned b = __ballot_sync(kFull, (pm >> i) & 1);
-            if ((uint32_t)(i & 31) == lane) {
-              if (i < 32) h0 += __popc(b); else h1 += __popc(b);
-            }
-          }
-          alive = shfl_mask<MaskT>(pm, 31);
-        }
-      }
-      for (uint32_t c = kRegChunks * 32u; c < n && alive != 0; c += 32) {   // very long prompts
-        const uint32_t k = c + lane;
-        MaskT pm = 0;
-        if (k < n) pm = mask_load<MaskT>(mask, ids[off + k]);
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          const MaskT o = shfl_up_mask<MaskT>(pm, d);
-          if ((int)lane >= d) pm &= o;
-        }
-        pm &= alive;
-        MaskT it = shfl_mask<MaskT>(pm, 0);
+      MaskT alive = all_reps;   // replicas whose cached prefix covers every block seen so far
+      auto probe_chunk = [&](MaskT m) {
+        MaskT it = (MaskT)(shfl_mask<MaskT>(m, 0) & alive);
+        MaskT still = 0;
         while (it != 0) {
           const int i = first_bit<MaskT>(it);
           it &= (MaskT)(it - 1);
-          const unsigned b = __ballot_sync(kFull, (pm >> i) & 1);
+          const unsigned b = __ballot_sync(kFull, (m >> i) & 1);
+          const uint32_t run = (b == kFull) ? 32u : (uint32_t)__ffs((int)~b) - 1u;
           if ((uint32_t)(i & 31) == lane) {
-            if (i < 32) h0 += __popc(b); else h1 += __popc(b);
+            if (i < 32) h0 += run; else h1 += run;
           }
+          if (run == 32u) still |= (MaskT)(((MaskT)1) << i);
         }
-        alive = shfl_mask<MaskT>(pm, 31);
+        alive = still;
+      };
+#pragma unroll
+      for (int c = 0; c < kRegChunks; ++c)
+        if (c * 32u < n && alive != 0) probe_chunk(mr[c]);
+      for (uint32_t c = kRegChunks * 32u; c < n && alive != 0; c += 32) {   // very long prompts
+        const uint32_t k = c + lane;
+        MaskT m = 0;
+        if (k < n) m = mask_load<MaskT>(mask, ids[off + k]);
+        probe_chunk(m);
       }
     }
 
     // ---- score of Eq. 3 (fixed order, no FMA) and lowest-index argmin
-    double best_c = d_inf();
+    uint64_t best_k = ~0ull;
     uint32_t best_i = kNone;
     uint32_t unc0 = 0, unc1 = 0;
+    const double* wrtt_row = sm.wrtt + (size_t)rec.origin * R;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const uint32_t i = lane + 32u * half;
@@ -427,16 +433,16 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
         if (half) unc1 = unc; else unc0 = unc;
         double q = (double)sm.load[i];
         if (K != 3) q = __dmul_rn(q, sm.w[3 + i]);
-        double c = __dadd_rn(__dadd_rn(__dmul_rn(w_net, rtt_row[i]), __dmul_rn(w_pre, (double)unc)),
+        double c = __dadd_rn(__dadd_rn(wrtt_row[i], __dmul_rn(w_pre, (double)unc)),
                              __dmul_rn(w_que, q));
         if (c != c) c = (i == 0) ? -d_inf() : d_inf();  // a NaN score wins only at index 0
-        if (c < best_c || best_i == kNone) { best_c = c; best_i = i; }
+        const uint64_t ck = order_key(c);
+        if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i; }
         const uint32_t pr = h + 1 < n ? h + 1 : n;
         st_probe += pr;
       }
     }
-    warp_argmin(best_c, best_i);
-    const uint32_t istar = best_i;
+    const uint32_t istar = warp_argmin_key(best_k, best_i);
     const uint32_t hstar = __shfl_sync(kFull, istar < 32 ? h0 : h1, istar & 31);
     const uint32_t uncstar = __shfl_sync(kFull, istar < 32 ? unc0 : unc1, istar & 31);
     const MaskT bit = (MaskT)(((MaskT)1) << istar);
@@ -523,14 +529,11 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
             }
             const unsigned lv = __ballot_sync(kFull, live);
             const uint32_t cnt = __popc(lv);
-            unsigned take;
-            if (cnt <= need) { take = lv; adv += 32; }
-            else {
-              const unsigned pos = __fns(lv, 0, (int)need);
-              take = lv & ((2u << pos) - 1u);
-              adv += (int32_t)pos + 1;
-            }
-            if ((take >> lane) & 1u) mask_clear_bit<MaskT>(mask, vid[u], bit);
+            // the first `need` live touches in lane order are the victims
+            const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+            const unsigned take = __ballot_sync(kFull, mine);
+            adv += (cnt <= need) ? 32 : 32 - __clz((int)take);
+            if (mine) mask_clear_bit<MaskT>(mask, vid[u], bit);
             const uint32_t tk = __popc(take);
             need -= tk;
             evicted += tk;
@@ -543,13 +546,14 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
     occ -= evicted;
 
     // ---- service commit: earliest-free slot, lowest index on ties
-    double bv = d_inf();
+    uint64_t bk = ~0ull;
     uint32_t bs = kNone;
     for (uint32_t s = lane; s < S; s += 32) {
-      const double v = free_at[(size_t)istar * S + s];
-      if (v < bv || bs == kNone) { bv = v; bs = s; }
+      const uint64_t vk = order_key(free_at[(size_t)istar * S + s]);
+      if (vk < bk || bs == kNone) { bk = vk; bs = s; }
     }
-    warp_argmin(bv, bs);
+    bs = warp_argmin_key(bk, bs);
+    const double bv = free_at[(size_t)istar * S + bs];
     const double arrive = __dadd_rn(t, rtt_row[istar]);
     const double start = (bv > arrive) ? bv : arrive;
     const double first = __dadd_rn(start, __dmul_rn(a.m.prefill_ms, (double)uncstar));
@@ -746,7 +750,7 @@ template <typename MaskT>
 cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
   const size_t rs = (size_t)a.m.R * a.m.S;
   a.slots_in_smem = rs * 32 <= 32 * 1024 ? 1u : 0u;
-  size_t smem = ((size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
+  size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
                 (4 * (size_t)a.m.R + 1) * sizeof(uint32_t);
   if (a.slots_in_smem) smem += rs * 32;
   smem = (smem + 15) / 16 * 16;
