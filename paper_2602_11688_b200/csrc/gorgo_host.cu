@@ -90,8 +90,8 @@ StateLayout make_layout(const Model& m) {
 
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
-  uint64_t params, rtt, status, p95, masks, states, fin, slot_next, lru_next, route_log, ttft,
-      e2e, total;
+  uint64_t params, rtt, status, p95, masks, states, lists, fin, slot_next, lru_next, route_log,
+      ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
 };
@@ -109,6 +109,7 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.p95 = o; o = align_up(o + res * 16);
   w.masks = o; o = align_up(o + res * w.mask_stride);
   w.states = o; o = align_up(o + res * w.st.bytes);
+  w.lists = o; o = align_up(o + res * evict_list_bytes(m.R));
   w.fin = o; o = align_up(o + res * N * 8);
   w.slot_next = o; o = align_up(o + res * N * 4);
   w.lru_next = o; o = align_up(o + res * N * 4);
@@ -194,6 +195,7 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
     a.rtt = d_rtt; a.params = wave_params;
     a.masks = base + w.masks; a.mask_stride = w.mask_stride;
     a.states = base + w.states; a.lay = w.st;
+    a.evict_lists = reinterpret_cast<uint4*>(base + w.lists);
     a.fin = reinterpret_cast<double*>(base + w.fin);
     a.slot_next = reinterpret_cast<uint32_t*>(base + w.slot_next);
     a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
@@ -486,6 +488,7 @@ int gorgo_route_batch(gorgo_sim_t* sim, const double* params, double time_scale,
   a.rtt = d_rtt; a.params = d_params;
   a.masks = base + w.masks; a.mask_stride = w.mask_stride;
   a.states = base + w.states; a.lay = w.st;
+  a.evict_lists = reinterpret_cast<uint4*>(base + w.lists);
   a.fin = reinterpret_cast<double*>(base + w.fin);
   a.slot_next = reinterpret_cast<uint32_t*>(base + w.slot_next);
   a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);

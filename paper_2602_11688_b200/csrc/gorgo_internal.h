@@ -75,6 +75,8 @@ struct ReplayArgs {
   uint32_t first, count;          // requests [first, first+count)
   uint32_t check_order;           // 1: refuse (status) unless header.processed == first
   uint32_t slots_in_smem;         // set by the launcher: per-slot state fits in shared memory
+  uint32_t lists_in_smem;         // set by the launcher: eviction lists fit in shared memory
+  uint4* evict_lists;             // [P * evict_list_bytes(R)] scratch used when they do not
   const double* rtt;              // [G*R] device
   const double* params;           // [P*K] device
   unsigned char* masks;           // [P * mask_stride] bytes
@@ -123,5 +125,6 @@ cudaError_t launch_replay(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st)
 cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st);
 uint32_t mask_bytes_for(uint32_t n_replicas);
+uint64_t evict_list_bytes(uint32_t n_replicas);
 
 }  // namespace gorgo

@@ -151,12 +151,23 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
 constexpr int kRegChunks = 8;     // request blocks held in registers: 8 x 32 = 256
 constexpr int kEvictBatches = 2;  // touches examined per lane and eviction round
 constexpr uint32_t kAhead = 48;   // how far the helper warp runs ahead of the replay (requests)
+constexpr uint32_t kListCap = 128;     // pre-validated eviction victims kept per replica
+constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is this close to full
 
 // Shared-memory view of one candidate's small state.
 struct Smem {
   double* rtt; double* wrtt; double* w; double* minfin; long long* load;
   uint32_t* occ; uint32_t* curreq; int32_t* curpos; uint32_t* lrutail;
   volatile uint32_t* progress;
+  // eviction rings, one per replica: filled by the scout warp, drained by the replay warp.
+  // entry = (block id, request of the block's next occurrence after the entry was made or kNone,
+  //          position of the touch in its request, request of the touch), in eviction order
+  uint4* lst;                     // [R][kListCap]
+  volatile uint32_t* act;         // replay -> scout: the replica's cache is close to full
+  volatile uint32_t* ring_head;   // entries consumed (replay warp)
+  volatile uint32_t* ring_tail;   // entries produced (scout warp)
+  volatile uint32_t* scan_cr;     // scout's own cursor into the recency order (set at activation)
+  volatile int32_t* scan_cp;
 };
 
 // Helper warp: runs ahead of the replay warp of the same candidate and pulls what it will touch
@@ -224,8 +235,98 @@ __device__ void helper_warp(const ReplayArgs& a, const Smem& sm, const MaskT* ma
   }
 }
 
+// Scout warp: for every replica whose cache is close to full it walks the recency order ahead
+// of the eviction cursor and appends to the replica's ring the touches that are still the latest
+// touch of their block (the coming eviction victims, in order).  The replay warp evicts from the
+// ring instead of validating touches on its critical path; entries that went stale after they
+// were appended are recognised there by their next-occurrence field.
 template <typename MaskT>
-__global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
+__device__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* lru_next,
+                           const uint8_t* route_log, uint32_t lane) {
+  const ReqRec* req = a.tr.req;
+  const uint32_t* ids = a.tr.ids;
+  const uint32_t end = a.first + a.count;
+  const uint32_t R = a.m.R;
+  uint32_t idle = 0;
+  uint32_t blocked0 = kNone - 1, blocked1 = kNone - 1;  // lru tail seen when the scan ran dry
+  while (true) {
+    const uint32_t prog = *sm.progress;
+    if (prog >= end) break;
+    // the active replica with the emptiest ring that can still be extended
+    uint32_t best = kNone;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const uint32_t i = lane + 32u * half;
+      if (i < R && sm.act[i]) {
+        const uint32_t fill = sm.ring_tail[i] - sm.ring_head[i];
+        const uint32_t bl = half ? blocked1 : blocked0;
+        if (fill + 32u <= kListCap && sm.lrutail[i] != bl) best = min(best, (fill << 8) | i);
+      }
+    }
+    best = __reduce_min_sync(kFull, best);
+    if (best == kNone || prog == a.first) {
+      if (++idle > (1u << 26)) break;              // bounded wait
+      __nanosleep(64);
+      continue;
+    }
+    idle = 0;
+    const uint32_t i = best & 255u;
+    __threadfence_block();
+    const uint32_t rs = prog - 1;                  // every request <= rs is fully committed
+    uint32_t cr = sm.scan_cr[i];
+    int32_t cp = sm.scan_cp[i];
+    uint32_t coff = (cr != kNone) ? req[cr].off : 0u;
+    uint32_t tail = sm.ring_tail[i];
+    uint4* out = sm.lst + (size_t)i * kListCap;
+    bool dry = false;
+    for (uint32_t round = 0; round < 6; ++round) {
+      const uint32_t room = kListCap - (tail - sm.ring_head[i]);
+      if (room < 32u) break;
+      if (cp < 0) {
+        const uint32_t nx = (cr == kNone) ? kNone : __ldcg(lru_next + cr);
+        if (nx == kNone || nx > rs) { dry = true; break; }   // end of the order as of rs
+        cr = nx;
+        const ReqRec cre = req[cr];
+        coff = cre.off;
+        cp = (int32_t)cre.nblk - 1;
+        continue;
+      }
+      const int32_t k = cp - (int32_t)lane;         // deepest position first
+      bool live = false;
+      uint32_t id = 0, nxr = kNone;
+      if (k >= 0) {
+        const uint32_t g = coff + (uint32_t)k;
+        id = ids[g];
+        uint2 c = a.tr.occ_next[g];
+        live = true;
+        while (c.x != kNone && c.y <= rs) {         // later occurrences up to rs
+          if ((uint32_t)__ldcg(route_log + c.y) == i) { live = false; break; }
+          c = a.tr.occ_next[c.x];
+        }
+        if (live && c.x != kNone) nxr = c.y;        // first occurrence after rs
+      }
+      const unsigned lv = __ballot_sync(kFull, live);
+      const uint32_t slot = tail + (uint32_t)__popc(lv & ((1u << lane) - 1u));
+      if (live) out[slot % kListCap] = make_uint4(id, nxr, (uint32_t)k, cr);
+      tail += __popc(lv);
+      cp -= 32;
+      __threadfence_block();
+      if (lane == 0) {
+        sm.scan_cr[i] = cr;
+        sm.scan_cp[i] = cp;
+        sm.ring_tail[i] = tail;
+      }
+    }
+    if (dry) {
+      const uint32_t lt = sm.lrutail[i];
+      if ((i & 31u) == lane) { if (i < 32) blocked0 = lt; else blocked1 = lt; }
+    }
+    __syncwarp();
+  }
+}
+
+template <typename MaskT>
+__global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
   const uint32_t p = blockIdx.x;
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t warp = threadIdx.x >> 5;
@@ -265,6 +366,17 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
     head_tok = unext + 3 * (size_t)RS; unext += 4 * (size_t)RS;
   }
   sm.progress = unext;
+  sm.act = unext + 1;
+  sm.ring_head = sm.act + R;
+  sm.ring_tail = sm.ring_head + R;
+  sm.scan_cr = sm.ring_tail + R;
+  sm.scan_cp = reinterpret_cast<volatile int32_t*>(sm.scan_cr + R);
+  {
+    uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R;
+    const uintptr_t al = (reinterpret_cast<uintptr_t>(after) + 15) & ~(uintptr_t)15;
+    sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(al)
+                             : a.evict_lists + (size_t)p * R * kListCap;
+  }
 
   MaskT* mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
   double* fin = a.fin + (size_t)p * N;
@@ -299,11 +411,18 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
       tail[x] = g_tail[x]; head_next[x] = g_head_next[x]; head_tok[x] = g_head_tok[x];
     }
   }
+  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
+    sm.act[i] = 0; sm.ring_head[i] = 0; sm.ring_tail[i] = 0;
+  }
   if (threadIdx.x == 0) *sm.progress = a.first;
   __syncthreads();
 
   if (warp == 1) {
     helper_warp<MaskT>(a, sm, mask, lru_next, lane);
+    return;
+  }
+  if (warp == 2) {
+    scout_warp<MaskT>(a, sm, lru_next, route_log, lane);
     return;
   }
 
@@ -474,7 +593,53 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
     if (need > 0) {
       uint32_t cr = sm.curreq[istar];
       int32_t cp = sm.curpos[istar];
-      uint32_t coff = (cr != kNone) ? req[cr].off : 0u;
+      // fast path: victims from the ring the scout warp keeps for this replica
+      if (sm.act[istar]) {
+        const uint4* lst = sm.lst + (size_t)istar * kListCap;
+        uint32_t head = sm.ring_head[istar];
+        while (need > 0) {
+          uint32_t avail = sm.ring_tail[istar] - head;
+          for (uint32_t polls = 0; avail == 0 && polls < 64; ++polls) {
+            __nanosleep(20);
+            avail = sm.ring_tail[istar] - head;
+          }
+          if (avail == 0) break;                          // the scout is behind: walk ourselves
+          __threadfence_block();
+          const uint32_t m = min(avail, 32u);
+          bool live = false, behind = false;
+          uint4 ent = make_uint4(0, 0, 0, 0);
+          if (lane < m) {
+            const uint32_t e = (head + lane) % kListCap;
+            ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+            // entries the eviction cursor has already passed (after a walk of our own) are void
+            behind = ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
+            live = !behind;
+            if (live) {
+              if (ent.y == r) live = false;               // the block is in this very request
+              else if (ent.y < r)                         // it came back in between: look again
+                live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
+            }
+          }
+          const unsigned lv = __ballot_sync(kFull, live);
+          const uint32_t cnt = __popc(lv);
+          const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+          const unsigned take = __ballot_sync(kFull, mine);
+          if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
+          const uint32_t tk = __popc(take);
+          // entries passed: the whole round, or up to the last victim taken
+          const uint32_t passed = (cnt <= need) ? m : 32u - (uint32_t)__clz((int)take);
+          need -= tk;
+          evicted += tk;
+          const uint32_t lastl = passed - 1;
+          const bool last_behind = __shfl_sync(kFull, (int)behind, lastl) != 0;
+          const uint32_t lw = __shfl_sync(kFull, ent.w, lastl);
+          const int32_t lz = (int32_t)__shfl_sync(kFull, ent.z, lastl);
+          if (!last_behind) { cr = lw; cp = lz - 1; }
+          head += passed;
+        }
+        if (lane == 0) sm.ring_head[istar] = head;
+      }
+      uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
       unsigned long long guard = 0;
       while (need > 0) {
         if (++guard > evict_guard_max) { status = -6; break; }
@@ -583,6 +748,14 @@ __global__ void __launch_bounds__(64) replay_kernel(const ReplayArgs a) {
       if (sm.curreq[istar] == kNone) { sm.curreq[istar] = r; sm.curpos[istar] = (int32_t)n - 1; }
       sm.lrutail[istar] = r;
       route_log[r] = (uint8_t)istar;
+      // hand the replica to the scout warp once its cache is close to full (before that no
+      // eviction has happened here, so the scout starts from the eviction cursor)
+      if (!sm.act[istar] && (uint64_t)occ + kPostMargin >= a.m.C) {
+        sm.scan_cr[istar] = sm.curreq[istar];
+        sm.scan_cp[istar] = sm.curpos[istar];
+        __threadfence_block();
+        sm.act[istar] = 1;
+      }
       const size_t o = (size_t)p * a.out_stride + j;
       if (a.route_out) a.route_out[o] = (uint8_t)istar;
       if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
@@ -749,21 +922,28 @@ __global__ void __launch_bounds__(256) digest_kernel(const DigestArgs a) {
 template <typename MaskT>
 cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
   const size_t rs = (size_t)a.m.R * a.m.S;
+  const size_t list_bytes = (size_t)a.m.R * kListCap * sizeof(uint4);
   a.slots_in_smem = rs * 32 <= 32 * 1024 ? 1u : 0u;
+  a.lists_in_smem = list_bytes <= 48 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
-                (4 * (size_t)a.m.R + 1) * sizeof(uint32_t);
+                (9 * (size_t)a.m.R + 1) * sizeof(uint32_t) + 16;
   if (a.slots_in_smem) smem += rs * 32;
+  if (a.lists_in_smem) smem += list_bytes;
   smem = (smem + 15) / 16 * 16;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  replay_kernel<MaskT><<<n_cand, 64, smem, st>>>(a);
+  replay_kernel<MaskT><<<n_cand, 96, smem, st>>>(a);
   return cudaGetLastError();
 }
 
 }  // namespace
+
+uint64_t evict_list_bytes(uint32_t n_replicas) {
+  return (uint64_t)n_replicas * kListCap * sizeof(uint4);
+}
 
 uint32_t mask_bytes_for(uint32_t n_replicas) {
   return n_replicas <= 8 ? 1u : n_replicas <= 16 ? 2u : n_replicas <= 32 ? 4u : 8u;
