@@ -78,19 +78,15 @@ StateLayout make_layout(const Model& m) {
   uint64_t o = sizeof(CandHeader);
   l.rep_off = o; o += (uint64_t)m.R * sizeof(RepState);
   const uint64_t rs = (uint64_t)m.R * m.S;
-  l.free_at_off = o; o += rs * 8;
-  l.head_fin_off = o; o += rs * 8;
-  l.head_off = o; o += rs * 4;
-  l.tail_off = o; o += rs * 4;
-  l.head_next_off = o; o += rs * 4;
-  l.head_tok_off = o; o += rs * 4;
+  l.slot_d_off = o; o += rs * 24;
+  l.slot_u_off = o; o += rs * 20;
   l.bytes = align_up(o);
   return l;
 }
 
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
-  uint64_t params, rtt, status, p95, masks, states, lists, fin, slot_next, lru_next, route_log,
+  uint64_t params, rtt, status, p95, masks, states, lists, qrec, lru_next, route_log,
       ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
@@ -110,8 +106,7 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.masks = o; o = align_up(o + res * w.mask_stride);
   w.states = o; o = align_up(o + res * w.st.bytes);
   w.lists = o; o = align_up(o + res * evict_list_bytes(m.R));
-  w.fin = o; o = align_up(o + res * N * 8);
-  w.slot_next = o; o = align_up(o + res * N * 4);
+  w.qrec = o; o = align_up(o + res * N * 16);
   w.lru_next = o; o = align_up(o + res * N * 4);
   w.route_log = o; o = align_up(o + res * N);
   w.ttft = o; if (with_latency) o = align_up(o + res * N * 8);
@@ -196,8 +191,7 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
     a.masks = base + w.masks; a.mask_stride = w.mask_stride;
     a.states = base + w.states; a.lay = w.st;
     a.evict_lists = reinterpret_cast<uint4*>(base + w.lists);
-    a.fin = reinterpret_cast<double*>(base + w.fin);
-    a.slot_next = reinterpret_cast<uint32_t*>(base + w.slot_next);
+    a.qrec = reinterpret_cast<uint4*>(base + w.qrec);
     a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
     a.route_log = route ? route + (size_t)p0 * N : base + w.route_log;
     a.route_log_stride = N;
@@ -489,8 +483,7 @@ int gorgo_route_batch(gorgo_sim_t* sim, const double* params, double time_scale,
   a.masks = base + w.masks; a.mask_stride = w.mask_stride;
   a.states = base + w.states; a.lay = w.st;
   a.evict_lists = reinterpret_cast<uint4*>(base + w.lists);
-  a.fin = reinterpret_cast<double*>(base + w.fin);
-  a.slot_next = reinterpret_cast<uint32_t*>(base + w.slot_next);
+  a.qrec = reinterpret_cast<uint4*>(base + w.qrec);
   a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
   a.route_log = base + w.route_log; a.route_log_stride = N;
   a.route_out = route; a.hit_out = hit_blocks; a.ttft_out = ttft_ms; a.e2e_out = e2e_ms;

@@ -58,12 +58,10 @@ struct Model {
 // candidate lives in a separate region.
 struct StateLayout {
   uint64_t rep_off;        // RepState[R]
-  uint64_t free_at_off;    // double[R*S]   time each slot frees
-  uint64_t head_fin_off;   // double[R*S]   finish of the oldest in-flight request of the slot
-  uint64_t head_off;       // uint32[R*S]   that request (kNone: slot has nothing in flight)
-  uint64_t tail_off;       // uint32[R*S]   newest request queued on the slot
-  uint64_t head_next_off;  // uint32[R*S]   request queued right behind the head (kNone: none)
-  uint64_t head_tok_off;   // uint32[R*S]   input tokens of the head request
+  uint64_t slot_d_off;     // double[3][R*S]: slot free time, finish of its oldest and second
+                           //   oldest in-flight request
+  uint64_t slot_u_off;     // uint32[5][R*S]: tokens of the oldest and second oldest, request
+                           //   index of the third oldest, newest request, queue length
   uint64_t bytes;          // size of the block (multiple of 256)
 };
 
@@ -84,8 +82,8 @@ struct ReplayArgs {
   unsigned char* states;          // [P * layout.bytes]
   StateLayout lay;
   // per-request arrays, candidate p at + p*N elements
-  double* fin;                    // finish time of each request
-  uint32_t* slot_next;            // next request queued on the same (replica, slot)
+  uint4* qrec;                    // per request (finish lo, finish hi, next request queued on
+                                  //   the same replica slot, input tokens)
   uint32_t* lru_next;             // next request routed to the same replica
   uint8_t* route_log;             // chosen replica of every request replayed so far
   uint64_t route_log_stride;      // elements between candidates

@@ -152,6 +152,8 @@ constexpr int kRegChunks = 8;     // request blocks held in registers: 8 x 32 = 
 constexpr int kEvictBatches = 2;  // touches examined per lane and eviction round
 constexpr uint32_t kAhead = 48;   // how far the helper warp runs ahead of the replay (requests)
 constexpr uint32_t kListCap = 128;     // pre-validated eviction victims kept per replica
+constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
+constexpr int kScoutBatches = 2;       // touches examined per lane and scout round
 constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is this close to full
 
 // Shared-memory view of one candidate's small state.
@@ -242,7 +244,7 @@ __device__ void helper_warp(const ReplayArgs& a, const Smem& sm, const MaskT* ma
 // were appended are recognised there by their next-occurrence field.
 template <typename MaskT>
 __device__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* lru_next,
-                           const uint8_t* route_log, uint32_t lane) {
+                           const uint8_t* route_log, uint32_t lane, uint32_t which) {
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
   const uint32_t end = a.first + a.count;
@@ -257,10 +259,11 @@ __device__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* 
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const uint32_t i = lane + 32u * half;
-      if (i < R && sm.act[i]) {
+      if (i < R && (i % kScouts) == which && sm.act[i]) {
         const uint32_t fill = sm.ring_tail[i] - sm.ring_head[i];
         const uint32_t bl = half ? blocked1 : blocked0;
-        if (fill + 32u <= kListCap && sm.lrutail[i] != bl) best = min(best, (fill << 8) | i);
+        if (fill + 32u * kScoutBatches <= kListCap && sm.lrutail[i] != bl)
+          best = min(best, (fill << 8) | i);
       }
     }
     best = __reduce_min_sync(kFull, best);
@@ -281,7 +284,7 @@ __device__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* 
     bool dry = false;
     for (uint32_t round = 0; round < 6; ++round) {
       const uint32_t room = kListCap - (tail - sm.ring_head[i]);
-      if (room < 32u) break;
+      if (room < 32u * kScoutBatches) break;
       if (cp < 0) {
         const uint32_t nx = (cr == kNone) ? kNone : __ldcg(lru_next + cr);
         if (nx == kNone || nx > rs) { dry = true; break; }   // end of the order as of rs
@@ -291,25 +294,39 @@ __device__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* 
         cp = (int32_t)cre.nblk - 1;
         continue;
       }
-      const int32_t k = cp - (int32_t)lane;         // deepest position first
-      bool live = false;
-      uint32_t id = 0, nxr = kNone;
-      if (k >= 0) {
-        const uint32_t g = coff + (uint32_t)k;
-        id = ids[g];
-        uint2 c = a.tr.occ_next[g];
-        live = true;
-        while (c.x != kNone && c.y <= rs) {         // later occurrences up to rs
-          if ((uint32_t)__ldcg(route_log + c.y) == i) { live = false; break; }
-          c = a.tr.occ_next[c.x];
+      // kScoutBatches x 32 touches, deepest position first; issue every first load up front
+      int32_t k[kScoutBatches];
+      uint32_t id[kScoutBatches];
+      uint2 c[kScoutBatches];
+#pragma unroll
+      for (int u = 0; u < kScoutBatches; ++u) {
+        k[u] = cp - (int32_t)(u * 32u + lane);
+        id[u] = 0;
+        c[u] = make_uint2(kNone, kNone);
+        if (k[u] >= 0) {
+          const uint32_t g = coff + (uint32_t)k[u];
+          id[u] = ids[g];
+          c[u] = a.tr.occ_next[g];
         }
-        if (live && c.x != kNone) nxr = c.y;        // first occurrence after rs
       }
-      const unsigned lv = __ballot_sync(kFull, live);
-      const uint32_t slot = tail + (uint32_t)__popc(lv & ((1u << lane) - 1u));
-      if (live) out[slot % kListCap] = make_uint4(id, nxr, (uint32_t)k, cr);
-      tail += __popc(lv);
-      cp -= 32;
+#pragma unroll
+      for (int u = 0; u < kScoutBatches; ++u) {
+        bool live = k[u] >= 0;
+        uint32_t nxr = kNone;
+        if (live) {
+          uint2 cc = c[u];
+          while (cc.x != kNone && cc.y <= rs) {       // later occurrences up to rs
+            if ((uint32_t)__ldcg(route_log + cc.y) == i) { live = false; break; }
+            cc = a.tr.occ_next[cc.x];
+          }
+          if (live && cc.x != kNone) nxr = cc.y;      // first occurrence after rs
+        }
+        const unsigned lv = __ballot_sync(kFull, live);
+        const uint32_t slot = tail + (uint32_t)__popc(lv & ((1u << lane) - 1u));
+        if (live) out[slot % kListCap] = make_uint4(id[u], nxr, (uint32_t)k[u], cr);
+        tail += __popc(lv);
+      }
+      cp -= 32 * kScoutBatches;
       __threadfence_block();
       if (lane == 0) {
         sm.scan_cr[i] = cr;
@@ -326,7 +343,7 @@ __device__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* 
 }
 
 template <typename MaskT>
-__global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
+__global__ void __launch_bounds__(64 + 32 * kScouts) replay_kernel(const ReplayArgs a) {
   const uint32_t p = blockIdx.x;
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t warp = threadIdx.x >> 5;
@@ -337,12 +354,8 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
   unsigned char* st = a.states + (size_t)p * a.lay.bytes;
   CandHeader* hdr = reinterpret_cast<CandHeader*>(st);
   RepState* g_rep = reinterpret_cast<RepState*>(st + a.lay.rep_off);
-  double* g_free_at = reinterpret_cast<double*>(st + a.lay.free_at_off);
-  double* g_head_fin = reinterpret_cast<double*>(st + a.lay.head_fin_off);
-  uint32_t* g_head = reinterpret_cast<uint32_t*>(st + a.lay.head_off);
-  uint32_t* g_tail = reinterpret_cast<uint32_t*>(st + a.lay.tail_off);
-  uint32_t* g_head_next = reinterpret_cast<uint32_t*>(st + a.lay.head_next_off);
-  uint32_t* g_head_tok = reinterpret_cast<uint32_t*>(st + a.lay.head_tok_off);
+  double* g_slot_d = reinterpret_cast<double*>(st + a.lay.slot_d_off);     // 3 x [R*S] doubles
+  uint32_t* g_slot_u = reinterpret_cast<uint32_t*>(st + a.lay.slot_u_off);  // 5 x [R*S] words
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem sm;
@@ -353,18 +366,26 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
   sm.load = reinterpret_cast<long long*>(sm.minfin + R);   // [R]
   double* dnext = reinterpret_cast<double*>(sm.load + R);
   // per-slot state: in shared memory when it fits, else it stays in global memory
-  double *free_at = g_free_at, *head_fin = g_head_fin;
-  if (a.slots_in_smem) { free_at = dnext; head_fin = dnext + RS; dnext += 2 * (size_t)RS; }
+  // Per-slot state (in shared memory when it fits, else it stays in global memory).  A slot is a
+  // FIFO of in-flight requests whose finish times never decrease; its two oldest entries are
+  // kept here, the rest is reached through the per-request records in global memory.
+  double* slot_d = g_slot_d;
+  if (a.slots_in_smem) { slot_d = dnext; dnext += 3 * (size_t)RS; }
+  double* free_at = slot_d;              // time the slot frees (finish of its newest request)
+  double* q0_fin = slot_d + RS;          // finish of the oldest in-flight request (+inf: none)
+  double* q1_fin = slot_d + 2 * (size_t)RS;   // finish of the second oldest
   sm.occ = reinterpret_cast<uint32_t*>(dnext);             // [R]
   sm.curreq = sm.occ + R;
   sm.curpos = reinterpret_cast<int32_t*>(sm.curreq + R);
   sm.lrutail = reinterpret_cast<uint32_t*>(sm.curpos + R);
   uint32_t* unext = sm.lrutail + R;
-  uint32_t *head = g_head, *tail = g_tail, *head_next = g_head_next, *head_tok = g_head_tok;
-  if (a.slots_in_smem) {
-    head = unext; tail = unext + RS; head_next = unext + 2 * (size_t)RS;
-    head_tok = unext + 3 * (size_t)RS; unext += 4 * (size_t)RS;
-  }
+  uint32_t* slot_u = g_slot_u;
+  if (a.slots_in_smem) { slot_u = unext; unext += 5 * (size_t)RS; }
+  uint32_t* q0_tok = slot_u;                    // input tokens of the oldest
+  uint32_t* q1_tok = slot_u + RS;               //   and of the second oldest
+  uint32_t* q2_idx = slot_u + 2 * (size_t)RS;   // request index of the third oldest (kNone: none)
+  uint32_t* tail = slot_u + 3 * (size_t)RS;     // newest request queued on the slot
+  uint32_t* qcnt = slot_u + 4 * (size_t)RS;     // requests in flight on the slot
   sm.progress = unext;
   sm.act = unext + 1;
   sm.ring_head = sm.act + R;
@@ -379,8 +400,7 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
   }
 
   MaskT* mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
-  double* fin = a.fin + (size_t)p * N;
-  uint32_t* slot_next = a.slot_next + (size_t)p * N;
+  uint4* qrec = a.qrec + (size_t)p * N;   // per request: (finish lo, finish hi, next on slot, tokens)
   uint32_t* lru_next = a.lru_next + (size_t)p * N;
   uint8_t* route_log = a.route_log + (size_t)p * a.route_log_stride;
   const ReqRec* req = a.tr.req;
@@ -406,10 +426,8 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
     sm.curreq[i] = rs.cur_req; sm.curpos[i] = rs.cur_pos; sm.lrutail[i] = rs.lru_tail;
   }
   if (a.slots_in_smem) {
-    for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) {
-      free_at[x] = g_free_at[x]; head_fin[x] = g_head_fin[x]; head[x] = g_head[x];
-      tail[x] = g_tail[x]; head_next[x] = g_head_next[x]; head_tok[x] = g_head_tok[x];
-    }
+    for (uint32_t x = threadIdx.x; x < 3 * RS; x += blockDim.x) slot_d[x] = g_slot_d[x];
+    for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) slot_u[x] = g_slot_u[x];
   }
   for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
     sm.act[i] = 0; sm.ring_head[i] = 0; sm.ring_tail[i] = 0;
@@ -421,8 +439,8 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
     helper_warp<MaskT>(a, sm, mask, lru_next, lane);
     return;
   }
-  if (warp == 2) {
-    scout_warp<MaskT>(a, sm, lru_next, route_log, lane);
+  if (warp >= 2) {
+    scout_warp<MaskT>(a, sm, lru_next, route_log, lane, warp - 2);
     return;
   }
 
@@ -433,11 +451,33 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
   unsigned long long st_probe = 0, st_hit = 0, st_blk = 0, st_evict = 0;
   const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
 
-  ReqRec rec_next = req[a.first];
+  // The trace does not depend on the state: records are fetched two requests ahead and the
+  // first 64 block ids one request ahead, so their latency is off the serial path.
+  const uint32_t last_r = a.first + a.count - 1;
+  ReqRec rec_cur = req[a.first];
+  ReqRec rec_nxt = req[min(a.first + 1, last_r)];
+  uint32_t id_pre[2];
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    const uint32_t k = c * 32u + lane;
+    id_pre[c] = (k < rec_cur.nblk) ? ids[rec_cur.off + k] : 0u;
+  }
+  // a queue refill whose load is in flight: slot index (kNone: none) and the record read
+  uint32_t pend_x = kNone;
+  uint4 pend_rec = make_uint4(0, 0, 0, 0);
+  auto flush_pending = [&]() {
+    if (pend_x != kNone) {
+      q1_fin[pend_x] = __hiloint2double((int)pend_rec.y, (int)pend_rec.x);
+      q2_idx[pend_x] = pend_rec.z;
+      q1_tok[pend_x] = pend_rec.w;
+      pend_x = kNone;
+    }
+  };
   for (uint32_t j = 0; j < a.count; ++j) {
     const uint32_t r = a.first + j;
-    const ReqRec rec = rec_next;
-    if (j + 1 < a.count) rec_next = req[r + 1];          // in flight while this request runs
+    const ReqRec rec = rec_cur;
+    rec_cur = rec_nxt;
+    rec_nxt = req[min(r + 2, last_r)];                   // in flight while this request runs
     const double t = __dmul_rn(a.scale, rec.ts_ms);
     const uint32_t n = rec.nblk, off = rec.off, in_tok = rec.in_tok;
     const double* rtt_row = sm.rtt + (size_t)rec.origin * R;
@@ -447,10 +487,12 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
     MaskT mr[kRegChunks];
 #pragma unroll
     for (int c = 0; c < kRegChunks; ++c) { idr[c] = 0u; mr[c] = (MaskT)0; }
+    idr[0] = id_pre[0];
+    idr[1] = id_pre[1];
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
+    for (int c = 0; c < 2; ++c) {                          // ids of the next request
       const uint32_t k = c * 32u + lane;
-      if (k < n) idr[c] = ids[off + k];
+      id_pre[c] = (k < rec_cur.nblk && j + 1 < a.count) ? ids[rec_cur.off + k] : 0u;
     }
     if (n > 64) {
 #pragma unroll
@@ -482,19 +524,29 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
         long long tok = 0;
         double mn = d_inf();
         for (uint32_t s = lane; s < S; s += 32) {
-          const size_t x = (size_t)ii * S + s;
-          double hf = head_fin[x];
+          const uint32_t x = ii * S + s;
+          double hf = q0_fin[x];
           if (hf <= t) {
             uint32_t guard = 0;
-            uint32_t hd, hn = head_next[x], ht = head_tok[x];
+            uint32_t cnt = qcnt[x];
             do {
-              tok += (long long)ht;
-              hd = hn;
-              if (hd == kNone) { hf = d_inf(); hn = kNone; ht = 0; }
-              else { hf = fin[hd]; hn = slot_next[hd]; ht = req[hd].in_tok; }
+              if (pend_x == x) flush_pending();           // the second entry is still in flight
+              tok += (long long)q0_tok[x];
+              --cnt;
+              if (cnt == 0) { hf = d_inf(); }
+              else {
+                hf = q1_fin[x];                            // the second becomes the oldest
+                q0_tok[x] = q1_tok[x];
+                if (cnt >= 2) {                            // fetch the new second: consumed later
+                  flush_pending();
+                  pend_rec = qrec[q2_idx[x]];
+                  pend_x = x;
+                }
+              }
               if (++guard > N) { status = -6; break; }
             } while (hf <= t);
-            head[x] = hd; head_fin[x] = hf; head_next[x] = hn; head_tok[x] = ht;
+            q0_fin[x] = hf;
+            qcnt[x] = cnt;
           }
           mn = fmin(mn, hf);
         }
@@ -725,18 +777,22 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
     const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
     const double finish = __dadd_rn(first, __dmul_rn(a.m.tpot_ms, (double)dec_tok));
 
+    flush_pending();
+    __syncwarp();
     if (lane == 0) {
       const size_t x = (size_t)istar * S + bs;
-      fin[r] = finish;
-      slot_next[r] = kNone;
-      if (head[x] == kNone) {
-        head[x] = r; head_fin[x] = finish; head_next[x] = kNone; head_tok[x] = in_tok;
+      qrec[r] = make_uint4((uint32_t)__double2loint(finish), (uint32_t)__double2hiint(finish),
+                           kNone, in_tok);
+      const uint32_t cnt = qcnt[x];
+      if (cnt == 0) {
+        q0_fin[x] = finish; q0_tok[x] = in_tok;
         sm.minfin[istar] = fmin(sm.minfin[istar], finish);
       } else {
-        const uint32_t tl = tail[x];
-        slot_next[tl] = r;
-        if (tl == head[x]) head_next[x] = r;
+        reinterpret_cast<uint32_t*>(qrec + tail[x])[2] = r;     // link behind the newest
+        if (cnt == 1) { q1_fin[x] = finish; q1_tok[x] = in_tok; q2_idx[x] = kNone; }
+        else if (cnt == 2) q2_idx[x] = r;
       }
+      qcnt[x] = cnt + 1;
       tail[x] = r;
       free_at[x] = finish;
       sm.load[istar] += (long long)in_tok;
@@ -768,6 +824,8 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
   }
 
   // ---- write the small state back
+  flush_pending();
+  __syncwarp();
   if (lane == 0) *sm.progress = a.first + a.count;
   for (uint32_t i = lane; i < R; i += 32) {
     RepState rs;
@@ -776,10 +834,8 @@ __global__ void __launch_bounds__(96) replay_kernel(const ReplayArgs a) {
     g_rep[i] = rs;
   }
   if (a.slots_in_smem) {
-    for (uint32_t x = lane; x < RS; x += 32) {
-      g_free_at[x] = free_at[x]; g_head_fin[x] = head_fin[x]; g_head[x] = head[x];
-      g_tail[x] = tail[x]; g_head_next[x] = head_next[x]; g_head_tok[x] = head_tok[x];
-    }
+    for (uint32_t x = lane; x < 3 * RS; x += 32) g_slot_d[x] = slot_d[x];
+    for (uint32_t x = lane; x < 5 * RS; x += 32) g_slot_u[x] = slot_u[x];
   }
   st_probe = warp_sum_u64(st_probe);
   status = __reduce_min_sync(kFull, status);
@@ -811,15 +867,17 @@ __global__ void reset_states_kernel(unsigned char* states, StateLayout lay, uint
     rs.lru_tail = kNone;
     rep[i] = rs;
   }
-  double* free_at = reinterpret_cast<double*>(st + lay.free_at_off);
-  double* head_fin = reinterpret_cast<double*>(st + lay.head_fin_off);
-  uint32_t* head = reinterpret_cast<uint32_t*>(st + lay.head_off);
-  uint32_t* tail = reinterpret_cast<uint32_t*>(st + lay.tail_off);
-  uint32_t* head_next = reinterpret_cast<uint32_t*>(st + lay.head_next_off);
-  uint32_t* head_tok = reinterpret_cast<uint32_t*>(st + lay.head_tok_off);
-  for (uint32_t x = threadIdx.x; x < R * S; x += blockDim.x) {
-    free_at[x] = 0.0; head_fin[x] = d_inf(); head[x] = kNone; tail[x] = kNone;
-    head_next[x] = kNone; head_tok[x] = 0;
+  double* slot_d = reinterpret_cast<double*>(st + lay.slot_d_off);
+  uint32_t* slot_u = reinterpret_cast<uint32_t*>(st + lay.slot_u_off);
+  const uint32_t RS = R * S;
+  for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) {
+    slot_d[x] = 0.0;                    // free_at
+    slot_d[RS + x] = d_inf();           // q0_fin
+    slot_d[2 * (size_t)RS + x] = d_inf();   // q1_fin
+    slot_u[x] = 0; slot_u[RS + x] = 0;  // q0_tok, q1_tok
+    slot_u[2 * (size_t)RS + x] = kNone; // q2_idx
+    slot_u[3 * (size_t)RS + x] = kNone; // tail
+    slot_u[4 * (size_t)RS + x] = 0;     // qcnt
   }
 }
 
@@ -923,11 +981,11 @@ template <typename MaskT>
 cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
   const size_t rs = (size_t)a.m.R * a.m.S;
   const size_t list_bytes = (size_t)a.m.R * kListCap * sizeof(uint4);
-  a.slots_in_smem = rs * 32 <= 32 * 1024 ? 1u : 0u;
+  a.slots_in_smem = rs * 44 <= 44 * 1024 ? 1u : 0u;
   a.lists_in_smem = list_bytes <= 48 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
                 (9 * (size_t)a.m.R + 1) * sizeof(uint32_t) + 16;
-  if (a.slots_in_smem) smem += rs * 32;
+  if (a.slots_in_smem) smem += rs * 44;
   if (a.lists_in_smem) smem += list_bytes;
   smem = (smem + 15) / 16 * 16;
   if (smem > 48 * 1024) {
@@ -935,7 +993,7 @@ cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  replay_kernel<MaskT><<<n_cand, 96, smem, st>>>(a);
+  replay_kernel<MaskT><<<n_cand, 64 + 32 * kScouts, smem, st>>>(a);
   return cudaGetLastError();
 }
 
