@@ -151,7 +151,7 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
 constexpr int kRegChunks = 8;     // request blocks held in registers: 8 x 32 = 256
 constexpr int kEvictBatches = 2;  // touches examined per lane and eviction round
 constexpr uint32_t kAhead = 48;   // how far the helper warp runs ahead of the replay (requests)
-constexpr uint32_t kListCap = 128;     // pre-validated eviction victims kept per replica
+constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
 constexpr int kScoutBatches = 2;       // touches examined per lane and scout round
 constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is this close to full
@@ -176,7 +176,7 @@ struct Smem {
 // into L2 (mask words, next-occurrence links at the eviction cursors) and L1/L2 (request
 // records, block ids).  Pure prefetching: it changes no state and may stop at any time.
 template <typename MaskT>
-__device__ void helper_warp(const ReplayArgs& a, const Smem& sm, const MaskT* mask,
+__device__ __forceinline__ void helper_warp(const ReplayArgs& a, const Smem& sm, const MaskT* mask,
                             const uint32_t* lru_next, uint32_t lane) {
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
@@ -243,7 +243,7 @@ __device__ void helper_warp(const ReplayArgs& a, const Smem& sm, const MaskT* ma
 // ring instead of validating touches on its critical path; entries that went stale after they
 // were appended are recognised there by their next-occurrence field.
 template <typename MaskT>
-__device__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* lru_next,
+__device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* lru_next,
                            const uint8_t* route_log, uint32_t lane, uint32_t which) {
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
@@ -342,126 +342,52 @@ __device__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* 
   }
 }
 
+// Named CTA barriers pairing the decide warp and the cache warp (32 + 32 threads each).
+__device__ __forceinline__ void bar_arrive(int id) {
+  __threadfence_block();
+  asm volatile("bar.arrive %0, 64;" ::"r"(id) : "memory");
+}
+__device__ __forceinline__ void bar_wait(int id) {
+  asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
+}
+constexpr int kBarHits = 1;    // cache warp -> decide warp: prefix hits of the request are posted
+constexpr int kBarRoute = 2;   // decide warp -> cache warp: the chosen replica is posted
+
+// Everything the warps of one candidate share.
 template <typename MaskT>
-__global__ void __launch_bounds__(64 + 32 * kScouts) replay_kernel(const ReplayArgs a) {
-  const uint32_t p = blockIdx.x;
-  const uint32_t lane = threadIdx.x & 31u;
-  const uint32_t warp = threadIdx.x >> 5;
-  const uint32_t R = a.m.R, S = a.m.S, K = a.m.K, G = a.m.G;
-  const uint32_t N = a.tr.n_req;
-  const uint32_t RS = R * S;
-
-  unsigned char* st = a.states + (size_t)p * a.lay.bytes;
-  CandHeader* hdr = reinterpret_cast<CandHeader*>(st);
-  RepState* g_rep = reinterpret_cast<RepState*>(st + a.lay.rep_off);
-  double* g_slot_d = reinterpret_cast<double*>(st + a.lay.slot_d_off);     // 3 x [R*S] doubles
-  uint32_t* g_slot_u = reinterpret_cast<uint32_t*>(st + a.lay.slot_u_off);  // 5 x [R*S] words
-
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+struct Ctx {
   Smem sm;
-  sm.rtt = reinterpret_cast<double*>(smem_raw);            // [G*R]
-  sm.wrtt = sm.rtt + (size_t)G * R;                        // [G*R]  w_net * rtt
-  sm.w = sm.wrtt + (size_t)G * R;                          // [K]
-  sm.minfin = sm.w + K;                                    // [R]
-  sm.load = reinterpret_cast<long long*>(sm.minfin + R);   // [R]
-  double* dnext = reinterpret_cast<double*>(sm.load + R);
-  // per-slot state: in shared memory when it fits, else it stays in global memory
-  // Per-slot state (in shared memory when it fits, else it stays in global memory).  A slot is a
-  // FIFO of in-flight requests whose finish times never decrease; its two oldest entries are
-  // kept here, the rest is reached through the per-request records in global memory.
-  double* slot_d = g_slot_d;
-  if (a.slots_in_smem) { slot_d = dnext; dnext += 3 * (size_t)RS; }
-  double* free_at = slot_d;              // time the slot frees (finish of its newest request)
-  double* q0_fin = slot_d + RS;          // finish of the oldest in-flight request (+inf: none)
-  double* q1_fin = slot_d + 2 * (size_t)RS;   // finish of the second oldest
-  sm.occ = reinterpret_cast<uint32_t*>(dnext);             // [R]
-  sm.curreq = sm.occ + R;
-  sm.curpos = reinterpret_cast<int32_t*>(sm.curreq + R);
-  sm.lrutail = reinterpret_cast<uint32_t*>(sm.curpos + R);
-  uint32_t* unext = sm.lrutail + R;
-  uint32_t* slot_u = g_slot_u;
-  if (a.slots_in_smem) { slot_u = unext; unext += 5 * (size_t)RS; }
-  uint32_t* q0_tok = slot_u;                    // input tokens of the oldest
-  uint32_t* q1_tok = slot_u + RS;               //   and of the second oldest
-  uint32_t* q2_idx = slot_u + 2 * (size_t)RS;   // request index of the third oldest (kNone: none)
-  uint32_t* tail = slot_u + 3 * (size_t)RS;     // newest request queued on the slot
-  uint32_t* qcnt = slot_u + 4 * (size_t)RS;     // requests in flight on the slot
-  sm.progress = unext;
-  sm.act = unext + 1;
-  sm.ring_head = sm.act + R;
-  sm.ring_tail = sm.ring_head + R;
-  sm.scan_cr = sm.ring_tail + R;
-  sm.scan_cp = reinterpret_cast<volatile int32_t*>(sm.scan_cr + R);
-  {
-    uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R;
-    const uintptr_t al = (reinterpret_cast<uintptr_t>(after) + 15) & ~(uintptr_t)15;
-    sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(al)
-                             : a.evict_lists + (size_t)p * R * kListCap;
-  }
+  MaskT* mask;
+  uint4* qrec;
+  uint32_t* lru_next;
+  uint8_t* route_log;
+  // per-slot state (shared or global memory)
+  double *free_at, *q0_fin, *q1_fin;
+  uint32_t *q0_tok, *q1_tok, *q2_idx, *tail, *qcnt;
+  volatile uint32_t* hits;     // [R]  prefix hit per replica of the current request
+  volatile uint32_t* route;    // chosen replica of the current request
+  volatile int32_t* status;    // first device-side limit hit by any warp
+};
 
-  MaskT* mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
-  uint4* qrec = a.qrec + (size_t)p * N;   // per request: (finish lo, finish hi, next on slot, tokens)
-  uint32_t* lru_next = a.lru_next + (size_t)p * N;
-  uint8_t* route_log = a.route_log + (size_t)p * a.route_log_stride;
+// Decide warp: queue signal, score, argmin, service model (paper Eq. 1-3).  Waits for the cache
+// warp's prefix hits of request r, publishes the route, then books the request on a slot.
+template <typename MaskT>
+__device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
+  const Smem& sm = cx.sm;
+  const uint32_t R = a.m.R, S = a.m.S, K = a.m.K;
+  const uint32_t N = a.tr.n_req;
   const ReqRec* req = a.tr.req;
-  const uint32_t* ids = a.tr.ids;
-
-  if (a.check_order && hdr->processed != a.first) {   // uniform over the CTA
-    if (threadIdx.x == 0) {
-      hdr->status = -8;
-      if (a.status_out) a.status_out[p] = -8;
-    }
-    return;
-  }
-
-  for (uint32_t i = threadIdx.x; i < G * R; i += blockDim.x) {
-    const double v = a.rtt[i];
-    sm.rtt[i] = v;
-    sm.wrtt[i] = __dmul_rn(a.params[(size_t)p * K], v);   // first product of the score
-  }
-  for (uint32_t i = threadIdx.x; i < K; i += blockDim.x) sm.w[i] = a.params[(size_t)p * K + i];
-  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
-    const RepState rs = g_rep[i];
-    sm.minfin[i] = rs.min_fin; sm.load[i] = rs.load; sm.occ[i] = rs.occ;
-    sm.curreq[i] = rs.cur_req; sm.curpos[i] = rs.cur_pos; sm.lrutail[i] = rs.lru_tail;
-  }
-  if (a.slots_in_smem) {
-    for (uint32_t x = threadIdx.x; x < 3 * RS; x += blockDim.x) slot_d[x] = g_slot_d[x];
-    for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) slot_u[x] = g_slot_u[x];
-  }
-  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
-    sm.act[i] = 0; sm.ring_head[i] = 0; sm.ring_tail[i] = 0;
-  }
-  if (threadIdx.x == 0) *sm.progress = a.first;
-  __syncthreads();
-
-  if (warp == 1) {
-    helper_warp<MaskT>(a, sm, mask, lru_next, lane);
-    return;
-  }
-  if (warp >= 2) {
-    scout_warp<MaskT>(a, sm, lru_next, route_log, lane, warp - 2);
-    return;
-  }
-
+  double *free_at = cx.free_at, *q0_fin = cx.q0_fin, *q1_fin = cx.q1_fin;
+  uint32_t *q0_tok = cx.q0_tok, *q1_tok = cx.q1_tok, *q2_idx = cx.q2_idx, *tail = cx.tail,
+           *qcnt = cx.qcnt;
+  uint4* qrec = cx.qrec;
   const double w_pre = sm.w[1], w_que = sm.w[2];
-  const MaskT all_reps = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0
-                                                  : (MaskT)((((MaskT)1) << (R & 63)) - 1);
   int32_t status = 0;
-  unsigned long long st_probe = 0, st_hit = 0, st_blk = 0, st_evict = 0;
-  const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
+  unsigned long long st_hit = 0, st_blk = 0;
 
-  // The trace does not depend on the state: records are fetched two requests ahead and the
-  // first 64 block ids one request ahead, so their latency is off the serial path.
   const uint32_t last_r = a.first + a.count - 1;
   ReqRec rec_cur = req[a.first];
   ReqRec rec_nxt = req[min(a.first + 1, last_r)];
-  uint32_t id_pre[2];
-#pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    const uint32_t k = c * 32u + lane;
-    id_pre[c] = (k < rec_cur.nblk) ? ids[rec_cur.off + k] : 0u;
-  }
   // a queue refill whose load is in flight: slot index (kNone: none) and the record read
   uint32_t pend_x = kNone;
   uint4 pend_rec = make_uint4(0, 0, 0, 0);
@@ -473,46 +399,16 @@ __global__ void __launch_bounds__(64 + 32 * kScouts) replay_kernel(const ReplayA
       pend_x = kNone;
     }
   };
+
   for (uint32_t j = 0; j < a.count; ++j) {
     const uint32_t r = a.first + j;
     const ReqRec rec = rec_cur;
     rec_cur = rec_nxt;
     rec_nxt = req[min(r + 2, last_r)];                   // in flight while this request runs
     const double t = __dmul_rn(a.scale, rec.ts_ms);
-    const uint32_t n = rec.nblk, off = rec.off, in_tok = rec.in_tok;
+    const uint32_t n = rec.nblk, in_tok = rec.in_tok;
     const double* rtt_row = sm.rtt + (size_t)rec.origin * R;
-
-    // ---- issue the probe loads first: block ids, then the mask word of every block
-    uint32_t idr[kRegChunks];
-    MaskT mr[kRegChunks];
-#pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) { idr[c] = 0u; mr[c] = (MaskT)0; }
-    idr[0] = id_pre[0];
-    idr[1] = id_pre[1];
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {                          // ids of the next request
-      const uint32_t k = c * 32u + lane;
-      id_pre[c] = (k < rec_cur.nblk && j + 1 < a.count) ? ids[rec_cur.off + k] : 0u;
-    }
-    if (n > 64) {
-#pragma unroll
-      for (int c = 2; c < kRegChunks; ++c) {
-        const uint32_t k = c * 32u + lane;
-        if (k < n) idr[c] = ids[off + k];
-      }
-    }
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      const uint32_t k = c * 32u + lane;
-      if (k < n) mr[c] = mask_load<MaskT>(mask, idr[c]);
-    }
-    if (n > 64) {
-#pragma unroll
-      for (int c = 2; c < kRegChunks; ++c) {
-        const uint32_t k = c * 32u + lane;
-        if (k < n) mr[c] = mask_load<MaskT>(mask, idr[c]);
-      }
-    }
+    const double* wrtt_row = sm.wrtt + (size_t)rec.origin * R;
 
     // ---- queue signal: drop requests that completed by t (finish <= t)
     for (uint32_t i0 = 0; i0 < R; i0 += 32) {
@@ -559,6 +455,175 @@ __global__ void __launch_bounds__(64 + 32 * kScouts) replay_kernel(const ReplayA
     }
     __syncwarp();
 
+    // ---- the queue part of the score does not need the prefix hits
+    double cq0 = 0.0, cq1 = 0.0;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const uint32_t i = lane + 32u * half;
+      if (i < R) {
+        double q = (double)sm.load[i];
+        if (K != 3) q = __dmul_rn(q, sm.w[3 + i]);
+        const double c = __dmul_rn(w_que, q);
+        if (half) cq1 = c; else cq0 = c;
+      }
+    }
+
+    bar_wait(kBarHits);                                   // prefix hits of request r are posted
+
+    // ---- score of Eq. 3 (fixed order, no FMA) and lowest-index argmin
+    uint64_t best_k = ~0ull;
+    uint32_t best_i = kNone;
+    uint32_t unc0 = 0, unc1 = 0, h0 = 0, h1 = 0;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const uint32_t i = lane + 32u * half;
+      if (i < R) {
+        const uint32_t h = cx.hits[i];
+        if (half) h1 = h; else h0 = h;
+        const unsigned long long hb = (unsigned long long)h * a.m.B;
+        const uint32_t unc = in_tok - (uint32_t)(hb < in_tok ? hb : in_tok);
+        if (half) unc1 = unc; else unc0 = unc;
+        double c = __dadd_rn(__dadd_rn(wrtt_row[i], __dmul_rn(w_pre, (double)unc)),
+                             half ? cq1 : cq0);
+        if (c != c) c = (i == 0) ? -d_inf() : d_inf();  // a NaN score wins only at index 0
+        const uint64_t ck = order_key(c);
+        if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i; }
+      }
+    }
+    const uint32_t istar = warp_argmin_key(best_k, best_i);
+    if (lane == 0) {
+      *cx.route = istar;
+      cx.route_log[r] = (uint8_t)istar;
+    }
+    bar_arrive(kBarRoute);                                // the cache warp may commit request r
+
+    const uint32_t hstar = __shfl_sync(kFull, istar < 32 ? h0 : h1, istar & 31);
+    const uint32_t uncstar = __shfl_sync(kFull, istar < 32 ? unc0 : unc1, istar & 31);
+
+    // ---- service commit: earliest-free slot, lowest index on ties
+    uint64_t bk = ~0ull;
+    uint32_t bs = kNone;
+    for (uint32_t s = lane; s < S; s += 32) {
+      const uint64_t vk = order_key(free_at[(size_t)istar * S + s]);
+      if (vk < bk || bs == kNone) { bk = vk; bs = s; }
+    }
+    bs = warp_argmin_key(bk, bs);
+    const double bv = free_at[(size_t)istar * S + bs];
+    const double arrive = __dadd_rn(t, rtt_row[istar]);
+    const double start = (bv > arrive) ? bv : arrive;
+    const double first = __dadd_rn(start, __dmul_rn(a.m.prefill_ms, (double)uncstar));
+    const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
+    const double finish = __dadd_rn(first, __dmul_rn(a.m.tpot_ms, (double)dec_tok));
+
+    flush_pending();
+    __syncwarp();
+    if (lane == 0) {
+      const size_t x = (size_t)istar * S + bs;
+      qrec[r] = make_uint4((uint32_t)__double2loint(finish), (uint32_t)__double2hiint(finish),
+                           kNone, in_tok);
+      const uint32_t cnt = qcnt[x];
+      if (cnt == 0) {
+        q0_fin[x] = finish; q0_tok[x] = in_tok;
+        sm.minfin[istar] = fmin(sm.minfin[istar], finish);
+      } else {
+        reinterpret_cast<uint32_t*>(qrec + tail[x])[2] = r;     // link behind the newest
+        if (cnt == 1) { q1_fin[x] = finish; q1_tok[x] = in_tok; q2_idx[x] = kNone; }
+        else if (cnt == 2) q2_idx[x] = r;
+      }
+      qcnt[x] = cnt + 1;
+      tail[x] = r;
+      free_at[x] = finish;
+      sm.load[istar] += (long long)in_tok;
+      const size_t o = (size_t)p * a.out_stride + j;
+      if (a.route_out) a.route_out[o] = (uint8_t)istar;
+      if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
+      if (a.ttft_out) a.ttft_out[o] = __dsub_rn(first, t);
+      if (a.e2e_out) a.e2e_out[o] = __dsub_rn(finish, t);
+      st_hit += hstar; st_blk += n;
+    }
+    __syncwarp();
+  }
+  flush_pending();
+  status = __reduce_min_sync(kFull, status);
+  if (lane == 0) {
+    if (status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
+    if (a.stats) {
+      unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
+      atomicAdd(s4 + 1, st_hit);
+      atomicAdd(s4 + 2, st_blk);
+    }
+  }
+}
+
+// Cache warp: prefix probe of every replica's block cache, then, once the route is known, the
+// LRU commit on the chosen replica (set its bit on the missing blocks, evict down to capacity).
+template <typename MaskT>
+__device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
+  const Smem& sm = cx.sm;
+  const uint32_t R = a.m.R;
+  const uint32_t N = a.tr.n_req;
+  const ReqRec* req = a.tr.req;
+  const uint32_t* ids = a.tr.ids;
+  MaskT* mask = cx.mask;
+  uint32_t* lru_next = cx.lru_next;
+  const uint8_t* route_log = cx.route_log;
+  const MaskT all_reps = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0
+                                                  : (MaskT)((((MaskT)1) << (R & 63)) - 1);
+  int32_t status = 0;
+  unsigned long long st_probe = 0, st_evict = 0;
+  const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
+
+  // The trace does not depend on the state: records are fetched two requests ahead and the
+  // first 64 block ids one request ahead, so their latency is off the serial path.
+  const uint32_t last_r = a.first + a.count - 1;
+  ReqRec rec_cur = req[a.first];
+  ReqRec rec_nxt = req[min(a.first + 1, last_r)];
+  uint32_t id_pre[2];
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    const uint32_t k = c * 32u + lane;
+    id_pre[c] = (k < rec_cur.nblk) ? ids[rec_cur.off + k] : 0u;
+  }
+
+  for (uint32_t j = 0; j < a.count; ++j) {
+    const uint32_t r = a.first + j;
+    const ReqRec rec = rec_cur;
+    rec_cur = rec_nxt;
+    rec_nxt = req[min(r + 2, last_r)];
+    const uint32_t n = rec.nblk, off = rec.off;
+
+    // ---- probe loads: block ids, then the mask word of every block
+    uint32_t idr[kRegChunks];
+    MaskT mr[kRegChunks];
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c) { idr[c] = 0u; mr[c] = (MaskT)0; }
+    idr[0] = id_pre[0];
+    idr[1] = id_pre[1];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {                          // ids of the next request
+      const uint32_t k = c * 32u + lane;
+      id_pre[c] = (k < rec_cur.nblk && j + 1 < a.count) ? ids[rec_cur.off + k] : 0u;
+    }
+    if (n > 64) {
+#pragma unroll
+      for (int c = 2; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        if (k < n) idr[c] = ids[off + k];
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const uint32_t k = c * 32u + lane;
+      if (k < n) mr[c] = mask_load<MaskT>(mask, idr[c]);
+    }
+    if (n > 64) {
+#pragma unroll
+      for (int c = 2; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        if (k < n) mr[c] = mask_load<MaskT>(mask, idr[c]);
+      }
+    }
+
     // ---- prefix probe on every replica: h_i = leading blocks whose mask has bit i
     uint32_t h0 = 0, h1 = 0;  // this lane's replicas: lane and lane+32
     {
@@ -588,34 +653,13 @@ __global__ void __launch_bounds__(64 + 32 * kScouts) replay_kernel(const ReplayA
         probe_chunk(m);
       }
     }
-
-    // ---- score of Eq. 3 (fixed order, no FMA) and lowest-index argmin
-    uint64_t best_k = ~0ull;
-    uint32_t best_i = kNone;
-    uint32_t unc0 = 0, unc1 = 0;
-    const double* wrtt_row = sm.wrtt + (size_t)rec.origin * R;
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const uint32_t i = lane + 32u * half;
-      if (i < R) {
-        const uint32_t h = half ? h1 : h0;
-        const unsigned long long hb = (unsigned long long)h * a.m.B;
-        const uint32_t unc = in_tok - (uint32_t)(hb < in_tok ? hb : in_tok);
-        if (half) unc1 = unc; else unc0 = unc;
-        double q = (double)sm.load[i];
-        if (K != 3) q = __dmul_rn(q, sm.w[3 + i]);
-        double c = __dadd_rn(__dadd_rn(wrtt_row[i], __dmul_rn(w_pre, (double)unc)),
-                             __dmul_rn(w_que, q));
-        if (c != c) c = (i == 0) ? -d_inf() : d_inf();  // a NaN score wins only at index 0
-        const uint64_t ck = order_key(c);
-        if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i; }
-        const uint32_t pr = h + 1 < n ? h + 1 : n;
-        st_probe += pr;
-      }
-    }
-    const uint32_t istar = warp_argmin_key(best_k, best_i);
-    const uint32_t hstar = __shfl_sync(kFull, istar < 32 ? h0 : h1, istar & 31);
-    const uint32_t uncstar = __shfl_sync(kFull, istar < 32 ? unc0 : unc1, istar & 31);
+    if (lane < R) cx.hits[lane] = h0;
+    if (lane + 32u < R) cx.hits[lane + 32u] = h1;
+    if (lane < R) st_probe += (h0 + 1 < n ? h0 + 1 : n);
+    if (lane + 32u < R) st_probe += (h1 + 1 < n ? h1 + 1 : n);
+    bar_arrive(kBarHits);                                 // the decide warp may score request r
+    bar_wait(kBarRoute);                                  // ... and has chosen the replica
+    const uint32_t istar = *cx.route;
     const MaskT bit = (MaskT)(((MaskT)1) << istar);
 
     // ---- cache commit: set the replica's bit on the missing blocks
@@ -761,41 +805,9 @@ __global__ void __launch_bounds__(64 + 32 * kScouts) replay_kernel(const ReplayA
       if (lane == 0) { sm.curreq[istar] = cr; sm.curpos[istar] = cp; }
     }
     occ -= evicted;
+    st_evict += evicted;
 
-    // ---- service commit: earliest-free slot, lowest index on ties
-    uint64_t bk = ~0ull;
-    uint32_t bs = kNone;
-    for (uint32_t s = lane; s < S; s += 32) {
-      const uint64_t vk = order_key(free_at[(size_t)istar * S + s]);
-      if (vk < bk || bs == kNone) { bk = vk; bs = s; }
-    }
-    bs = warp_argmin_key(bk, bs);
-    const double bv = free_at[(size_t)istar * S + bs];
-    const double arrive = __dadd_rn(t, rtt_row[istar]);
-    const double start = (bv > arrive) ? bv : arrive;
-    const double first = __dadd_rn(start, __dmul_rn(a.m.prefill_ms, (double)uncstar));
-    const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
-    const double finish = __dadd_rn(first, __dmul_rn(a.m.tpot_ms, (double)dec_tok));
-
-    flush_pending();
-    __syncwarp();
     if (lane == 0) {
-      const size_t x = (size_t)istar * S + bs;
-      qrec[r] = make_uint4((uint32_t)__double2loint(finish), (uint32_t)__double2hiint(finish),
-                           kNone, in_tok);
-      const uint32_t cnt = qcnt[x];
-      if (cnt == 0) {
-        q0_fin[x] = finish; q0_tok[x] = in_tok;
-        sm.minfin[istar] = fmin(sm.minfin[istar], finish);
-      } else {
-        reinterpret_cast<uint32_t*>(qrec + tail[x])[2] = r;     // link behind the newest
-        if (cnt == 1) { q1_fin[x] = finish; q1_tok[x] = in_tok; q2_idx[x] = kNone; }
-        else if (cnt == 2) q2_idx[x] = r;
-      }
-      qcnt[x] = cnt + 1;
-      tail[x] = r;
-      free_at[x] = finish;
-      sm.load[istar] += (long long)in_tok;
       sm.occ[istar] = occ;
       // recency order of the replica: append this request
       const uint32_t lt = sm.lrutail[istar];
@@ -803,7 +815,6 @@ __global__ void __launch_bounds__(64 + 32 * kScouts) replay_kernel(const ReplayA
       lru_next[r] = kNone;
       if (sm.curreq[istar] == kNone) { sm.curreq[istar] = r; sm.curpos[istar] = (int32_t)n - 1; }
       sm.lrutail[istar] = r;
-      route_log[r] = (uint8_t)istar;
       // hand the replica to the scout warp once its cache is close to full (before that no
       // eviction has happened here, so the scout starts from the eviction cursor)
       if (!sm.act[istar] && (uint64_t)occ + kPostMargin >= a.m.C) {
@@ -812,41 +823,139 @@ __global__ void __launch_bounds__(64 + 32 * kScouts) replay_kernel(const ReplayA
         __threadfence_block();
         sm.act[istar] = 1;
       }
-      const size_t o = (size_t)p * a.out_stride + j;
-      if (a.route_out) a.route_out[o] = (uint8_t)istar;
-      if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
-      if (a.ttft_out) a.ttft_out[o] = __dsub_rn(first, t);
-      if (a.e2e_out) a.e2e_out[o] = __dsub_rn(finish, t);
-      st_hit += hstar; st_blk += n; st_evict += evicted;
-      *sm.progress = r + 1;
+      __threadfence_block();
+      *sm.progress = r + 1;                               // request r is fully committed
     }
     __syncwarp();
   }
+  st_probe = warp_sum_u64(st_probe);
+  status = __reduce_min_sync(kFull, status);
+  if (lane == 0) {
+    if (status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
+    if (a.stats) {
+      unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
+      atomicAdd(s4 + 0, st_probe);
+      atomicAdd(s4 + 3, st_evict);
+    }
+  }
+}
+
+constexpr uint32_t kWarpDecide = 0, kWarpCache = 1, kWarpHelper = 2, kWarpScout0 = 3;
+constexpr uint32_t kReplayThreads = 32 * (3 + kScouts);
+
+template <typename MaskT>
+__global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayArgs a) {
+  const uint32_t p = blockIdx.x;
+  const uint32_t lane = threadIdx.x & 31u;
+  const uint32_t warp = threadIdx.x >> 5;
+  const uint32_t R = a.m.R, S = a.m.S, K = a.m.K, G = a.m.G;
+  const uint32_t N = a.tr.n_req;
+  const uint32_t RS = R * S;
+
+  unsigned char* st = a.states + (size_t)p * a.lay.bytes;
+  CandHeader* hdr = reinterpret_cast<CandHeader*>(st);
+  RepState* g_rep = reinterpret_cast<RepState*>(st + a.lay.rep_off);
+  double* g_slot_d = reinterpret_cast<double*>(st + a.lay.slot_d_off);     // 3 x [R*S] doubles
+  uint32_t* g_slot_u = reinterpret_cast<uint32_t*>(st + a.lay.slot_u_off);  // 5 x [R*S] words
+
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Ctx<MaskT> cx;
+  Smem& sm = cx.sm;
+  sm.rtt = reinterpret_cast<double*>(smem_raw);            // [G*R]
+  sm.wrtt = sm.rtt + (size_t)G * R;                        // [G*R]  w_net * rtt
+  sm.w = sm.wrtt + (size_t)G * R;                          // [K]
+  sm.minfin = sm.w + K;                                    // [R]
+  sm.load = reinterpret_cast<long long*>(sm.minfin + R);   // [R]
+  double* dnext = reinterpret_cast<double*>(sm.load + R);
+  // Per-slot state (in shared memory when it fits, else it stays in global memory).  A slot is a
+  // FIFO of in-flight requests whose finish times never decrease; its two oldest entries are
+  // kept here, the rest is reached through the per-request records in global memory.
+  double* slot_d = g_slot_d;
+  if (a.slots_in_smem) { slot_d = dnext; dnext += 3 * (size_t)RS; }
+  cx.free_at = slot_d;                   // time the slot frees (finish of its newest request)
+  cx.q0_fin = slot_d + RS;               // finish of the oldest in-flight request (+inf: none)
+  cx.q1_fin = slot_d + 2 * (size_t)RS;   // finish of the second oldest
+  sm.occ = reinterpret_cast<uint32_t*>(dnext);             // [R]
+  sm.curreq = sm.occ + R;
+  sm.curpos = reinterpret_cast<int32_t*>(sm.curreq + R);
+  sm.lrutail = reinterpret_cast<uint32_t*>(sm.curpos + R);
+  uint32_t* unext = sm.lrutail + R;
+  uint32_t* slot_u = g_slot_u;
+  if (a.slots_in_smem) { slot_u = unext; unext += 5 * (size_t)RS; }
+  cx.q0_tok = slot_u;                    // input tokens of the oldest
+  cx.q1_tok = slot_u + RS;               //   and of the second oldest
+  cx.q2_idx = slot_u + 2 * (size_t)RS;   // request index of the third oldest (kNone: none)
+  cx.tail = slot_u + 3 * (size_t)RS;     // newest request queued on the slot
+  cx.qcnt = slot_u + 4 * (size_t)RS;     // requests in flight on the slot
+  sm.progress = unext;
+  cx.route = unext + 1;
+  cx.status = reinterpret_cast<volatile int32_t*>(unext + 2);
+  cx.hits = unext + 3;                   // [R]
+  sm.act = unext + 3 + R;
+  sm.ring_head = sm.act + R;
+  sm.ring_tail = sm.ring_head + R;
+  sm.scan_cr = sm.ring_tail + R;
+  sm.scan_cp = reinterpret_cast<volatile int32_t*>(sm.scan_cr + R);
+  {
+    uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R;
+    const uintptr_t al = (reinterpret_cast<uintptr_t>(after) + 15) & ~(uintptr_t)15;
+    sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(al)
+                             : a.evict_lists + (size_t)p * R * kListCap;
+  }
+  cx.mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
+  cx.qrec = a.qrec + (size_t)p * N;   // per request: (finish lo, finish hi, next on slot, tokens)
+  cx.lru_next = a.lru_next + (size_t)p * N;
+  cx.route_log = a.route_log + (size_t)p * a.route_log_stride;
+
+  if (a.check_order && hdr->processed != a.first) {   // uniform over the CTA
+    if (threadIdx.x == 0) {
+      hdr->status = -8;
+      if (a.status_out) a.status_out[p] = -8;
+    }
+    return;
+  }
+
+  for (uint32_t i = threadIdx.x; i < G * R; i += blockDim.x) {
+    const double v = a.rtt[i];
+    sm.rtt[i] = v;
+    sm.wrtt[i] = __dmul_rn(a.params[(size_t)p * K], v);   // first product of the score
+  }
+  for (uint32_t i = threadIdx.x; i < K; i += blockDim.x) sm.w[i] = a.params[(size_t)p * K + i];
+  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
+    const RepState rs = g_rep[i];
+    sm.minfin[i] = rs.min_fin; sm.load[i] = rs.load; sm.occ[i] = rs.occ;
+    sm.curreq[i] = rs.cur_req; sm.curpos[i] = rs.cur_pos; sm.lrutail[i] = rs.lru_tail;
+    sm.act[i] = 0; sm.ring_head[i] = 0; sm.ring_tail[i] = 0;
+  }
+  if (a.slots_in_smem) {
+    for (uint32_t x = threadIdx.x; x < 3 * RS; x += blockDim.x) slot_d[x] = g_slot_d[x];
+    for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) slot_u[x] = g_slot_u[x];
+  }
+  if (threadIdx.x == 0) { *sm.progress = a.first; *cx.status = 0; }
+  __syncthreads();
+
+  if (warp == kWarpDecide) decide_warp<MaskT>(a, cx, p, lane);
+  else if (warp == kWarpCache) cache_warp<MaskT>(a, cx, p, lane);
+  else if (warp == kWarpHelper) helper_warp<MaskT>(a, sm, cx.mask, cx.lru_next, lane);
+  else scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, warp - kWarpScout0);
+  __syncthreads();
 
   // ---- write the small state back
-  flush_pending();
-  __syncwarp();
-  if (lane == 0) *sm.progress = a.first + a.count;
-  for (uint32_t i = lane; i < R; i += 32) {
+  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
     RepState rs;
     rs.min_fin = sm.minfin[i]; rs.load = sm.load[i]; rs.occ = sm.occ[i];
     rs.cur_req = sm.curreq[i]; rs.cur_pos = sm.curpos[i]; rs.lru_tail = sm.lrutail[i];
     g_rep[i] = rs;
   }
   if (a.slots_in_smem) {
-    for (uint32_t x = lane; x < 3 * RS; x += 32) g_slot_d[x] = slot_d[x];
-    for (uint32_t x = lane; x < 5 * RS; x += 32) g_slot_u[x] = slot_u[x];
+    for (uint32_t x = threadIdx.x; x < 3 * RS; x += blockDim.x) g_slot_d[x] = slot_d[x];
+    for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) g_slot_u[x] = slot_u[x];
   }
-  st_probe = warp_sum_u64(st_probe);
-  status = __reduce_min_sync(kFull, status);
-  if (lane == 0) {
+  if (threadIdx.x == 0) {
+    const int32_t status = *cx.status;
     hdr->processed = a.first + a.count;
     if (status != 0) hdr->status = status;
     if (a.status_out && (status != 0 || !a.check_order)) a.status_out[p] = status;
-    if (a.stats) {
-      unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
-      s4[0] += st_probe; s4[1] += st_hit; s4[2] += st_blk; s4[3] += st_evict;
-    }
   }
 }
 
@@ -982,9 +1091,9 @@ cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
   const size_t rs = (size_t)a.m.R * a.m.S;
   const size_t list_bytes = (size_t)a.m.R * kListCap * sizeof(uint4);
   a.slots_in_smem = rs * 44 <= 44 * 1024 ? 1u : 0u;
-  a.lists_in_smem = list_bytes <= 48 * 1024 ? 1u : 0u;
+  a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
-                (9 * (size_t)a.m.R + 1) * sizeof(uint32_t) + 16;
+                (10 * (size_t)a.m.R + 3) * sizeof(uint32_t) + 16;
   if (a.slots_in_smem) smem += rs * 44;
   if (a.lists_in_smem) smem += list_bytes;
   smem = (smem + 15) / 16 * 16;
@@ -993,7 +1102,7 @@ cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  replay_kernel<MaskT><<<n_cand, 64 + 32 * kScouts, smem, st>>>(a);
+  replay_kernel<MaskT><<<n_cand, kReplayThreads, smem, st>>>(a);
   return cudaGetLastError();
 }
 
