@@ -324,7 +324,7 @@ int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_m
     if (g >= m.G) return GORGO_ERR_BAD_TRACE;
     ReqRec& q = req[r];
     q.ts_ms = t; q.off = (uint32_t)hash_off[r]; q.in_tok = input_tokens[r];
-    q.out_tok = output_tokens[r]; q.nblk = (uint16_t)n; q.origin = g; q.pad[0] = q.pad[1] = 0;
+    q.out_tok = output_tokens[r]; q.nblk = (uint16_t)n; q.origin = g; q.prev_share = kNone; q.pad = 0;
   }
 
   // dense renumbering in order of first appearance; an id twice in one request is an error
@@ -335,14 +335,17 @@ int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_m
     std::vector<uint32_t> seen_in;  // request (+1) that last contained the dense id
     uint32_t next = 0;
     for (uint64_t r = 0; r < N; ++r) {
+      uint32_t latest = 0;  // latest earlier request (+1) that contains one of this one's blocks
       for (uint64_t g = hash_off[r]; g < hash_off[r + 1]; ++g) {
         const uint32_t before = next;
         const uint32_t d = map.get_or_add(hash_ids[g], next);
         if (next != before) { raw.push_back(hash_ids[g]); seen_in.push_back(0); }
         if (seen_in[d] == (uint32_t)r + 1) return GORGO_ERR_BAD_TRACE;
+        if (seen_in[d] > latest) latest = seen_in[d];
         seen_in[d] = (uint32_t)r + 1;
         ids[g] = d;
       }
+      req[r].prev_share = latest ? latest - 1 : kNone;
     }
   }
   const uint64_t D = raw.size();

@@ -15,7 +15,8 @@ struct __align__(32) ReqRec {
   uint32_t out_tok;   // output tokens
   uint16_t nblk;      // number of blocks
   uint16_t origin;    // origin region
-  uint32_t pad[2];
+  uint32_t prev_share;  // latest earlier request that shares a block with this one (kNone: none)
+  uint32_t pad;
 };
 static_assert(sizeof(ReqRec) == 32, "ReqRec must be one sector");
 

@@ -148,8 +148,7 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
   __stcg(reinterpret_cast<unsigned long long*>(mask) + id, (unsigned long long)v);
 }
 
-constexpr int kRegChunks = 8;     // request blocks held in registers: 8 x 32 = 256
-constexpr int kEvictBatches = 2;  // touches examined per lane and eviction round
+constexpr int kRegChunks = 4;     // request blocks held in registers: 4 x 32 = 128
 constexpr uint32_t kAhead = 48;   // how far the helper warp runs ahead of the replay (requests)
 constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
@@ -557,8 +556,12 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
 
 // Cache warp: prefix probe of every replica's block cache, then, once the route is known, the
 // LRU commit on the chosen replica (set its bit on the missing blocks, evict down to capacity).
+// The mask words of request r+1 are read while request r is still being committed; that early
+// read is thrown away and repeated when request r can have changed one of those words (the two
+// requests share a block, or a victim evicted for r occurs in r+1).
 template <typename MaskT>
-__device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
+__device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
+                                           uint32_t lane) {
   const Smem& sm = cx.sm;
   const uint32_t R = a.m.R;
   const uint32_t N = a.tr.n_req;
@@ -573,56 +576,30 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   unsigned long long st_probe = 0, st_evict = 0;
   const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
 
-  // The trace does not depend on the state: records are fetched two requests ahead and the
-  // first 64 block ids one request ahead, so their latency is off the serial path.
+  // The trace does not depend on the state: records run three requests ahead, the first
+  // kRegChunks*32 block ids two ahead, their mask words (state!) one ahead.
   const uint32_t last_r = a.first + a.count - 1;
   ReqRec rec_cur = req[a.first];
   ReqRec rec_nxt = req[min(a.first + 1, last_r)];
-  uint32_t id_pre[2];
+  ReqRec rec_nn = req[min(a.first + 2, last_r)];
+  uint32_t id_cur[kRegChunks], id_nxt[kRegChunks];
+  MaskT m_cur[kRegChunks];
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
+  for (int c = 0; c < kRegChunks; ++c) {
     const uint32_t k = c * 32u + lane;
-    id_pre[c] = (k < rec_cur.nblk) ? ids[rec_cur.off + k] : 0u;
+    id_cur[c] = (k < rec_cur.nblk) ? ids[rec_cur.off + k] : 0u;
+    id_nxt[c] = (k < rec_nxt.nblk) ? ids[rec_nxt.off + k] : 0u;
+  }
+#pragma unroll
+  for (int c = 0; c < kRegChunks; ++c) {
+    const uint32_t k = c * 32u + lane;
+    m_cur[c] = (k < rec_cur.nblk) ? mask_load<MaskT>(mask, id_cur[c]) : (MaskT)0;
   }
 
   for (uint32_t j = 0; j < a.count; ++j) {
     const uint32_t r = a.first + j;
     const ReqRec rec = rec_cur;
-    rec_cur = rec_nxt;
-    rec_nxt = req[min(r + 2, last_r)];
     const uint32_t n = rec.nblk, off = rec.off;
-
-    // ---- probe loads: block ids, then the mask word of every block
-    uint32_t idr[kRegChunks];
-    MaskT mr[kRegChunks];
-#pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) { idr[c] = 0u; mr[c] = (MaskT)0; }
-    idr[0] = id_pre[0];
-    idr[1] = id_pre[1];
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {                          // ids of the next request
-      const uint32_t k = c * 32u + lane;
-      id_pre[c] = (k < rec_cur.nblk && j + 1 < a.count) ? ids[rec_cur.off + k] : 0u;
-    }
-    if (n > 64) {
-#pragma unroll
-      for (int c = 2; c < kRegChunks; ++c) {
-        const uint32_t k = c * 32u + lane;
-        if (k < n) idr[c] = ids[off + k];
-      }
-    }
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      const uint32_t k = c * 32u + lane;
-      if (k < n) mr[c] = mask_load<MaskT>(mask, idr[c]);
-    }
-    if (n > 64) {
-#pragma unroll
-      for (int c = 2; c < kRegChunks; ++c) {
-        const uint32_t k = c * 32u + lane;
-        if (k < n) mr[c] = mask_load<MaskT>(mask, idr[c]);
-      }
-    }
 
     // ---- prefix probe on every replica: h_i = leading blocks whose mask has bit i
     uint32_t h0 = 0, h1 = 0;  // this lane's replicas: lane and lane+32
@@ -645,7 +622,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       };
 #pragma unroll
       for (int c = 0; c < kRegChunks; ++c)
-        if (c * 32u < n && alive != 0) probe_chunk(mr[c]);
+        if (c * 32u < n && alive != 0) probe_chunk(m_cur[c]);
       for (uint32_t c = kRegChunks * 32u; c < n && alive != 0; c += 32) {   // very long prompts
         const uint32_t k = c + lane;
         MaskT m = 0;
@@ -655,12 +632,28 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     }
     if (lane < R) cx.hits[lane] = h0;
     if (lane + 32u < R) cx.hits[lane + 32u] = h1;
+    bar_arrive(kBarHits);                                 // the decide warp may score request r
     if (lane < R) st_probe += (h0 + 1 < n ? h0 + 1 : n);
     if (lane + 32u < R) st_probe += (h1 + 1 < n ? h1 + 1 : n);
-    bar_arrive(kBarHits);                                 // the decide warp may score request r
-    bar_wait(kBarRoute);                                  // ... and has chosen the replica
+
+    // ---- while the decide warp works: early read of the mask words of request r+1, block ids
+    //      of request r+2, record of request r+3
+    const bool more = j + 1 < a.count;
+    MaskT m_nxt[kRegChunks];
+    uint32_t id_nn[kRegChunks];
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c) {
+      const uint32_t k = c * 32u + lane;
+      m_nxt[c] = (more && k < rec_nxt.nblk) ? mask_load<MaskT>(mask, id_nxt[c]) : (MaskT)0;
+      id_nn[c] = (j + 2 < a.count && k < rec_nn.nblk) ? ids[rec_nn.off + k] : 0u;
+    }
+    const ReqRec rec_n3 = req[min(r + 3, last_r)];
+
+    bar_wait(kBarRoute);                                  // the replica has been chosen
     const uint32_t istar = *cx.route;
     const MaskT bit = (MaskT)(((MaskT)1) << istar);
+    // request r+1 shares a block with r: its early mask read may miss the bits set below
+    bool redo = more && rec_nxt.prev_share == r;
 
     // ---- cache commit: set the replica's bit on the missing blocks
     uint32_t missing = 0;
@@ -668,8 +661,8 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     for (int c = 0; c < kRegChunks; ++c) {
       if (c * 32u < n) {
         const uint32_t k = c * 32u + lane;
-        const bool miss = (k < n) && !(mr[c] & bit);
-        if (miss) mask_store<MaskT>(mask, idr[c], (MaskT)(mr[c] | bit));
+        const bool miss = (k < n) && !(m_cur[c] & bit);
+        if (miss) mask_store<MaskT>(mask, id_cur[c], (MaskT)(m_cur[c] | bit));
         missing += __popc(__ballot_sync(kFull, miss));
       }
     }
@@ -689,6 +682,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     if (need > 0) {
       uint32_t cr = sm.curreq[istar];
       int32_t cp = sm.curpos[istar];
+      unsigned hit_next = 0;     // a victim's block occurs again in request r+1
       // fast path: victims from the ring the scout warp keeps for this replica
       if (sm.act[istar]) {
         const uint4* lst = sm.lst + (size_t)istar * kListCap;
@@ -705,15 +699,17 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
           bool live = false, behind = false;
           uint4 ent = make_uint4(0, 0, 0, 0);
           if (lane < m) {
-            const uint32_t e = (head + lane) % kListCap;
+            const uint32_t e = (head + lane) & (kListCap - 1);
             ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
             // entries the eviction cursor has already passed (after a walk of our own) are void
             behind = ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
             live = !behind;
             if (live) {
               if (ent.y == r) live = false;               // the block is in this very request
-              else if (ent.y < r)                         // it came back in between: look again
+              else if (ent.y < r) {                       // it came back in between: look again
                 live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
+                ent.y = r + 1;                            // where it goes next is unknown: assume r+1
+              }
             }
           }
           const unsigned lv = __ballot_sync(kFull, live);
@@ -721,6 +717,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
           const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
           const unsigned take = __ballot_sync(kFull, mine);
           if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
+          hit_next |= __ballot_sync(kFull, mine && ent.y == r + 1);
           const uint32_t tk = __popc(take);
           // entries passed: the whole round, or up to the last victim taken
           const uint32_t passed = (cnt <= need) ? m : 32u - (uint32_t)__clz((int)take);
@@ -748,61 +745,36 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
           cp = (int32_t)cre.nblk - 1;
           continue;
         }
-        // examine up to kEvictBatches x 32 touches, deepest position first; all loads of the
-        // round are issued before any is used
-        const uint32_t nbat = min((uint32_t)kEvictBatches, (2u * need + 31u) / 32u);
-        uint2 nx[kEvictBatches];
-        uint32_t vid[kEvictBatches];
-        uint32_t rt[kEvictBatches];
-        bool valid[kEvictBatches];
-#pragma unroll
-        for (int u = 0; u < kEvictBatches; ++u) {
-          const int32_t k = cp - (int32_t)(u * 32u + lane);
-          valid[u] = (uint32_t)u < nbat && k >= 0;
-          nx[u] = make_uint2(kNone, kNone);
-          vid[u] = 0;
-          if (valid[u]) {
-            const uint32_t g = coff + (uint32_t)k;
-            nx[u] = a.tr.occ_next[g];
-            vid[u] = ids[g];
+        // examine 32 touches, deepest position first
+        const int32_t k = cp - (int32_t)lane;
+        bool live = false;
+        uint32_t vid = 0, nxr = kNone;
+        if (k >= 0) {
+          const uint32_t g = coff + (uint32_t)k;
+          vid = ids[g];
+          uint2 c = a.tr.occ_next[g];
+          live = true;
+          while (c.x != kNone && c.y <= r) {       // later occurrences of the block, up to r
+            const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
+            if (rr == istar) { live = false; break; }
+            c = a.tr.occ_next[c.x];
           }
+          if (live && c.x != kNone) nxr = c.y;     // its next occurrence after r
         }
-#pragma unroll
-        for (int u = 0; u < kEvictBatches; ++u) {   // first hop of every touch
-          rt[u] = kNone;
-          if (valid[u] && nx[u].x != kNone && nx[u].y <= r)
-            rt[u] = (nx[u].y == r) ? istar : (uint32_t)route_log[nx[u].y];
-        }
-        int32_t adv = 0;
-#pragma unroll
-        for (int u = 0; u < kEvictBatches; ++u) {
-          if ((uint32_t)u < nbat && need > 0) {
-            bool live = false;
-            if (valid[u]) {
-              live = true;
-              uint2 c = nx[u];
-              uint32_t rr = rt[u];
-              while (c.x != kNone && c.y <= r) {     // later occurrences of the block, up to r
-                if (rr == istar) { live = false; break; }
-                c = a.tr.occ_next[c.x];
-                if (c.x != kNone && c.y <= r) rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
-              }
-            }
-            const unsigned lv = __ballot_sync(kFull, live);
-            const uint32_t cnt = __popc(lv);
-            // the first `need` live touches in lane order are the victims
-            const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
-            const unsigned take = __ballot_sync(kFull, mine);
-            adv += (cnt <= need) ? 32 : 32 - __clz((int)take);
-            if (mine) mask_clear_bit<MaskT>(mask, vid[u], bit);
-            const uint32_t tk = __popc(take);
-            need -= tk;
-            evicted += tk;
-          }
-        }
-        cp -= adv;
+        const unsigned lv = __ballot_sync(kFull, live);
+        const uint32_t cnt = __popc(lv);
+        // the first `need` live touches in lane order are the victims
+        const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+        const unsigned take = __ballot_sync(kFull, mine);
+        if (mine) mask_clear_bit<MaskT>(mask, vid, bit);
+        hit_next |= __ballot_sync(kFull, mine && nxr == r + 1);
+        cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
+        const uint32_t tk = __popc(take);
+        need -= tk;
+        evicted += tk;
       }
       if (lane == 0) { sm.curreq[istar] = cr; sm.curpos[istar] = cp; }
+      redo = redo || (hit_next != 0);
     }
     occ -= evicted;
     st_evict += evicted;
@@ -827,6 +799,22 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       *sm.progress = r + 1;                               // request r is fully committed
     }
     __syncwarp();
+
+    // ---- move on: request r+1 becomes current (repeat its mask read if r may have changed it)
+    rec_cur = rec_nxt; rec_nxt = rec_nn; rec_nn = rec_n3;
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c) {
+      id_cur[c] = id_nxt[c];
+      id_nxt[c] = id_nn[c];
+      m_cur[c] = m_nxt[c];
+    }
+    if (redo) {
+#pragma unroll
+      for (int c = 0; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        m_cur[c] = (k < rec_cur.nblk) ? mask_load<MaskT>(mask, id_cur[c]) : (MaskT)0;
+      }
+    }
   }
   st_probe = warp_sum_u64(st_probe);
   status = __reduce_min_sync(kFull, status);
