@@ -596,40 +596,49 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     m_cur[c] = (k < rec_cur.nblk) ? mask_load<MaskT>(mask, id_cur[c]) : (MaskT)0;
   }
 
+  // Prefix probe on every replica: h_i = leading blocks whose mask has bit i.  The first
+  // kRegChunks*32 mask words come in `mr`; longer prompts read the rest from memory.
+  auto probe = [&](const ReqRec& q, const MaskT (&mr)[kRegChunks], uint32_t& h0, uint32_t& h1) {
+    h0 = 0; h1 = 0;   // this lane's replicas: lane and lane+32
+    const uint32_t n = q.nblk;
+    MaskT alive = all_reps;   // replicas whose cached prefix covers every block seen so far
+    auto probe_chunk = [&](MaskT m) {
+      MaskT it = (MaskT)(shfl_mask<MaskT>(m, 0) & alive);
+      MaskT still = 0;
+      while (it != 0) {
+        const int i = first_bit<MaskT>(it);
+        it &= (MaskT)(it - 1);
+        const unsigned b = __ballot_sync(kFull, (m >> i) & 1);
+        const uint32_t run = (b == kFull) ? 32u : (uint32_t)__ffs((int)~b) - 1u;
+        if ((uint32_t)(i & 31) == lane) {
+          if (i < 32) h0 += run; else h1 += run;
+        }
+        if (run == 32u) still |= (MaskT)(((MaskT)1) << i);
+      }
+      alive = still;
+    };
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c)
+      if (c * 32u < n && alive != 0) probe_chunk(mr[c]);
+    for (uint32_t c = kRegChunks * 32u; c < n && alive != 0; c += 32) {   // very long prompts
+      const uint32_t k = c + lane;
+      MaskT m = 0;
+      if (k < n) m = mask_load<MaskT>(mask, ids[q.off + k]);
+      probe_chunk(m);
+    }
+  };
+  uint32_t hn0 = 0, hn1 = 0;   // prefix hits of the coming request, probed ahead
+  bool reprobe = true;         // ... which must be probed again (always true for the first)
+
   for (uint32_t j = 0; j < a.count; ++j) {
     const uint32_t r = a.first + j;
     const ReqRec rec = rec_cur;
     const uint32_t n = rec.nblk, off = rec.off;
 
-    // ---- prefix probe on every replica: h_i = leading blocks whose mask has bit i
-    uint32_t h0 = 0, h1 = 0;  // this lane's replicas: lane and lane+32
-    {
-      MaskT alive = all_reps;   // replicas whose cached prefix covers every block seen so far
-      auto probe_chunk = [&](MaskT m) {
-        MaskT it = (MaskT)(shfl_mask<MaskT>(m, 0) & alive);
-        MaskT still = 0;
-        while (it != 0) {
-          const int i = first_bit<MaskT>(it);
-          it &= (MaskT)(it - 1);
-          const unsigned b = __ballot_sync(kFull, (m >> i) & 1);
-          const uint32_t run = (b == kFull) ? 32u : (uint32_t)__ffs((int)~b) - 1u;
-          if ((uint32_t)(i & 31) == lane) {
-            if (i < 32) h0 += run; else h1 += run;
-          }
-          if (run == 32u) still |= (MaskT)(((MaskT)1) << i);
-        }
-        alive = still;
-      };
-#pragma unroll
-      for (int c = 0; c < kRegChunks; ++c)
-        if (c * 32u < n && alive != 0) probe_chunk(m_cur[c]);
-      for (uint32_t c = kRegChunks * 32u; c < n && alive != 0; c += 32) {   // very long prompts
-        const uint32_t k = c + lane;
-        MaskT m = 0;
-        if (k < n) m = mask_load<MaskT>(mask, ids[off + k]);
-        probe_chunk(m);
-      }
-    }
+    // ---- prefix hits of request r: computed while request r-1 was being decided (h_nxt), or
+    //      again now if r-1 may have changed a mask word of r
+    uint32_t h0 = hn0, h1 = hn1;
+    if (reprobe) probe(rec, m_cur, h0, h1);
     if (lane < R) cx.hits[lane] = h0;
     if (lane + 32u < R) cx.hits[lane + 32u] = h1;
     bar_arrive(kBarHits);                                 // the decide warp may score request r
@@ -648,6 +657,10 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       id_nn[c] = (j + 2 < a.count && k < rec_nn.nblk) ? ids[rec_nn.off + k] : 0u;
     }
     const ReqRec rec_n3 = req[min(r + 3, last_r)];
+    // probe request r+1 on those early words; valid unless request r changes one of them, and
+    // not attempted for prompts beyond the register window (their tail is read from memory)
+    const bool ahead = more && rec_nxt.nblk <= kRegChunks * 32u;
+    if (ahead) probe(rec_nxt, m_nxt, hn0, hn1);
 
     bar_wait(kBarRoute);                                  // the replica has been chosen
     const uint32_t istar = *cx.route;
@@ -695,40 +708,46 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
           }
           if (avail == 0) break;                          // the scout is behind: walk ourselves
           __threadfence_block();
-          const uint32_t m = min(avail, 32u);
-          bool live = false, behind = false;
-          uint4 ent = make_uint4(0, 0, 0, 0);
-          if (lane < m) {
-            const uint32_t e = (head + lane) & (kListCap - 1);
-            ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
-            // entries the eviction cursor has already passed (after a walk of our own) are void
-            behind = ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
-            live = !behind;
-            if (live) {
-              if (ent.y == r) live = false;               // the block is in this very request
-              else if (ent.y < r) {                       // it came back in between: look again
-                live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
-                ent.y = r + 1;                            // where it goes next is unknown: assume r+1
+          // up to 64 entries per round, two per lane, in ring order
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            if (need == 0 || avail <= 32u * u) break;
+            const uint32_t m = min(avail - 32u * u, 32u);
+            bool live = false, behind = false;
+            uint4 ent = make_uint4(0, 0, 0, 0);
+            if (lane < m) {
+              const uint32_t e = (head + lane) & (kListCap - 1);
+              ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+              // entries the eviction cursor has already passed (after a walk of our own) are void
+              behind = ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
+              live = !behind;
+              if (live) {
+                if (ent.y == r) live = false;             // the block is in this very request
+                else if (ent.y < r) {                     // it came back in between: look again
+                  live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
+                  ent.y = r + 1;                          // where it goes next is unknown: assume r+1
+                }
               }
             }
+            const unsigned lv = __ballot_sync(kFull, live);
+            const uint32_t cnt = __popc(lv);
+            const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+            const unsigned take = __ballot_sync(kFull, mine);
+            if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
+            hit_next |= __ballot_sync(kFull, mine && ent.y == r + 1);
+            const uint32_t tk = __popc(take);
+            // entries passed: the whole batch, or up to the last victim taken
+            const uint32_t passed = (cnt <= need) ? m : 32u - (uint32_t)__clz((int)take);
+            need -= tk;
+            evicted += tk;
+            const uint32_t lastl = passed - 1;
+            const bool last_behind = __shfl_sync(kFull, (int)behind, lastl) != 0;
+            const uint32_t lw = __shfl_sync(kFull, ent.w, lastl);
+            const int32_t lz = (int32_t)__shfl_sync(kFull, ent.z, lastl);
+            if (!last_behind) { cr = lw; cp = lz - 1; }
+            head += passed;
+            if (passed < m) break;                        // stopped inside the batch
           }
-          const unsigned lv = __ballot_sync(kFull, live);
-          const uint32_t cnt = __popc(lv);
-          const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
-          const unsigned take = __ballot_sync(kFull, mine);
-          if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
-          hit_next |= __ballot_sync(kFull, mine && ent.y == r + 1);
-          const uint32_t tk = __popc(take);
-          // entries passed: the whole round, or up to the last victim taken
-          const uint32_t passed = (cnt <= need) ? m : 32u - (uint32_t)__clz((int)take);
-          need -= tk;
-          evicted += tk;
-          const uint32_t lastl = passed - 1;
-          const bool last_behind = __shfl_sync(kFull, (int)behind, lastl) != 0;
-          const uint32_t lw = __shfl_sync(kFull, ent.w, lastl);
-          const int32_t lz = (int32_t)__shfl_sync(kFull, ent.z, lastl);
-          if (!last_behind) { cr = lw; cp = lz - 1; }
-          head += passed;
         }
         if (lane == 0) sm.ring_head[istar] = head;
       }
@@ -815,6 +834,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         m_cur[c] = (k < rec_cur.nblk) ? mask_load<MaskT>(mask, id_cur[c]) : (MaskT)0;
       }
     }
+    reprobe = redo || !ahead;
   }
   st_probe = warp_sum_u64(st_probe);
   status = __reduce_min_sync(kFull, status);
