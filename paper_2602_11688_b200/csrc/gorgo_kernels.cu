@@ -556,9 +556,9 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
 
 // Cache warp: prefix probe of every replica's block cache, then, once the route is known, the
 // LRU commit on the chosen replica (set its bit on the missing blocks, evict down to capacity).
-// The mask words of request r+1 are read while request r is still being committed; that early
-// read is thrown away and repeated when request r can have changed one of those words (the two
-// requests share a block, or a victim evicted for r occurs in r+1).
+// Mask words are read two requests ahead and probed one request ahead; such an early read is
+// repeated when a request committed in between can have changed one of the words (it shares a
+// block with the later request, or a victim evicted for it occurs in the later request).
 template <typename MaskT>
 __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
                                            uint32_t lane) {
@@ -575,30 +575,32 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   int32_t status = 0;
   unsigned long long st_probe = 0, st_evict = 0;
   const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
+  const uint32_t end = a.first + a.count;
 
-  // The trace does not depend on the state: records run three requests ahead, the first
-  // kRegChunks*32 block ids two ahead, their mask words (state!) one ahead.
-  const uint32_t last_r = a.first + a.count - 1;
-  ReqRec rec_cur = req[a.first];
-  ReqRec rec_nxt = req[min(a.first + 1, last_r)];
-  ReqRec rec_nn = req[min(a.first + 2, last_r)];
-  uint32_t id_cur[kRegChunks], id_nxt[kRegChunks];
-  MaskT m_cur[kRegChunks];
+  // What the warp needs to know of a request ahead of time.
+  struct Ahead { uint32_t off, nblk, prev_share; };
+  auto fetch = [&](uint32_t q) {
+    Ahead h = {0u, 0u, kNone};
+    if (q < end) { const ReqRec x = req[q]; h.off = x.off; h.nblk = x.nblk; h.prev_share = x.prev_share; }
+    return h;
+  };
+  auto load_ids = [&](const Ahead& q, uint32_t (&dst)[kRegChunks]) {
 #pragma unroll
-  for (int c = 0; c < kRegChunks; ++c) {
-    const uint32_t k = c * 32u + lane;
-    id_cur[c] = (k < rec_cur.nblk) ? ids[rec_cur.off + k] : 0u;
-    id_nxt[c] = (k < rec_nxt.nblk) ? ids[rec_nxt.off + k] : 0u;
-  }
+    for (int c = 0; c < kRegChunks; ++c) {
+      const uint32_t k = c * 32u + lane;
+      dst[c] = (k < q.nblk) ? ids[q.off + k] : 0u;
+    }
+  };
+  auto load_masks = [&](const Ahead& q, const uint32_t (&id)[kRegChunks], MaskT (&dst)[kRegChunks]) {
 #pragma unroll
-  for (int c = 0; c < kRegChunks; ++c) {
-    const uint32_t k = c * 32u + lane;
-    m_cur[c] = (k < rec_cur.nblk) ? mask_load<MaskT>(mask, id_cur[c]) : (MaskT)0;
-  }
-
+    for (int c = 0; c < kRegChunks; ++c) {
+      const uint32_t k = c * 32u + lane;
+      dst[c] = (k < q.nblk) ? mask_load<MaskT>(mask, id[c]) : (MaskT)0;
+    }
+  };
   // Prefix probe on every replica: h_i = leading blocks whose mask has bit i.  The first
   // kRegChunks*32 mask words come in `mr`; longer prompts read the rest from memory.
-  auto probe = [&](const ReqRec& q, const MaskT (&mr)[kRegChunks], uint32_t& h0, uint32_t& h1) {
+  auto probe = [&](const Ahead& q, const MaskT (&mr)[kRegChunks], uint32_t& h0, uint32_t& h1) {
     h0 = 0; h1 = 0;   // this lane's replicas: lane and lane+32
     const uint32_t n = q.nblk;
     MaskT alive = all_reps;   // replicas whose cached prefix covers every block seen so far
@@ -627,46 +629,46 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       probe_chunk(m);
     }
   };
+
+  // Pipeline registers: request r (cur), r+1 (nxt), r+2 (nn), r+3 (n3).  The trace does not
+  // depend on the state, so records and ids simply run ahead; mask words do depend on it.
+  Ahead q_cur = fetch(a.first), q_nxt = fetch(a.first + 1), q_nn = fetch(a.first + 2),
+        q_n3 = fetch(a.first + 3);
+  uint32_t id_cur[kRegChunks], id_nxt[kRegChunks], id_nn[kRegChunks];
+  MaskT m_cur[kRegChunks], m_nxt[kRegChunks];
+  load_ids(q_cur, id_cur); load_ids(q_nxt, id_nxt); load_ids(q_nn, id_nn);
+  load_masks(q_cur, id_cur, m_cur); load_masks(q_nxt, id_nxt, m_nxt);
   uint32_t hn0 = 0, hn1 = 0;   // prefix hits of the coming request, probed ahead
   bool reprobe = true;         // ... which must be probed again (always true for the first)
+  bool dirty_nxt = false;      // m_nxt was read before a commit that may have changed it
 
-  for (uint32_t j = 0; j < a.count; ++j) {
-    const uint32_t r = a.first + j;
-    const ReqRec rec = rec_cur;
-    const uint32_t n = rec.nblk, off = rec.off;
+  for (uint32_t r = a.first; r < end; ++r) {
+    const uint32_t n = q_cur.nblk, off = q_cur.off;
 
-    // ---- prefix hits of request r: computed while request r-1 was being decided (h_nxt), or
-    //      again now if r-1 may have changed a mask word of r
+    // ---- prefix hits of request r: probed while request r-1 was being decided, or again now
     uint32_t h0 = hn0, h1 = hn1;
-    if (reprobe) probe(rec, m_cur, h0, h1);
+    if (reprobe) probe(q_cur, m_cur, h0, h1);
     if (lane < R) cx.hits[lane] = h0;
     if (lane + 32u < R) cx.hits[lane + 32u] = h1;
     bar_arrive(kBarHits);                                 // the decide warp may score request r
     if (lane < R) st_probe += (h0 + 1 < n ? h0 + 1 : n);
     if (lane + 32u < R) st_probe += (h1 + 1 < n ? h1 + 1 : n);
 
-    // ---- while the decide warp works: early read of the mask words of request r+1, block ids
-    //      of request r+2, record of request r+3
-    const bool more = j + 1 < a.count;
-    MaskT m_nxt[kRegChunks];
-    uint32_t id_nn[kRegChunks];
-#pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) {
-      const uint32_t k = c * 32u + lane;
-      m_nxt[c] = (more && k < rec_nxt.nblk) ? mask_load<MaskT>(mask, id_nxt[c]) : (MaskT)0;
-      id_nn[c] = (j + 2 < a.count && k < rec_nn.nblk) ? ids[rec_nn.off + k] : 0u;
-    }
-    const ReqRec rec_n3 = req[min(r + 3, last_r)];
-    // probe request r+1 on those early words; valid unless request r changes one of them, and
-    // not attempted for prompts beyond the register window (their tail is read from memory)
-    const bool ahead = more && rec_nxt.nblk <= kRegChunks * 32u;
-    if (ahead) probe(rec_nxt, m_nxt, hn0, hn1);
+    // ---- while the decide warp works: mask words of r+2, ids of r+3, record of r+4 ...
+    MaskT m_nn[kRegChunks];
+    uint32_t id_n3[kRegChunks];
+    load_masks(q_nn, id_nn, m_nn);
+    load_ids(q_n3, id_n3);
+    const Ahead q_n4 = fetch(r + 4);
+    // ... and the probe of r+1 on the words read one request ago (read again first if the
+    // commit of r-1 may have changed them); prompts beyond the register window wait
+    const bool ahead = q_nxt.nblk <= kRegChunks * 32u;
+    if (dirty_nxt) load_masks(q_nxt, id_nxt, m_nxt);
+    if (ahead) probe(q_nxt, m_nxt, hn0, hn1);
 
     bar_wait(kBarRoute);                                  // the replica has been chosen
     const uint32_t istar = *cx.route;
     const MaskT bit = (MaskT)(((MaskT)1) << istar);
-    // request r+1 shares a block with r: its early mask read may miss the bits set below
-    bool redo = more && rec_nxt.prev_share == r;
 
     // ---- cache commit: set the replica's bit on the missing blocks
     uint32_t missing = 0;
@@ -692,14 +694,15 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     uint32_t occ = sm.occ[istar] + missing;
     uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
     uint32_t evicted = 0;
+    unsigned hit1 = 0, hit2 = 0;   // a victim's block occurs again in request r+1 / r+2
     if (need > 0) {
       uint32_t cr = sm.curreq[istar];
       int32_t cp = sm.curpos[istar];
-      unsigned hit_next = 0;     // a victim's block occurs again in request r+1
       // fast path: victims from the ring the scout warp keeps for this replica
       if (sm.act[istar]) {
         const uint4* lst = sm.lst + (size_t)istar * kListCap;
         uint32_t head = sm.ring_head[istar];
+        uint32_t last_e = kNone;   // ring slot of the last entry passed that was not void
         while (need > 0) {
           uint32_t avail = sm.ring_tail[istar] - head;
           for (uint32_t polls = 0; avail == 0 && polls < 64; ++polls) {
@@ -708,46 +711,66 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
           }
           if (avail == 0) break;                          // the scout is behind: walk ourselves
           __threadfence_block();
-          // up to 64 entries per round, two per lane, in ring order
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            if (need == 0 || avail <= 32u * u) break;
-            const uint32_t m = min(avail - 32u * u, 32u);
-            bool live = false, behind = false;
-            uint4 ent = make_uint4(0, 0, 0, 0);
-            if (lane < m) {
-              const uint32_t e = (head + lane) & (kListCap - 1);
-              ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
-              // entries the eviction cursor has already passed (after a walk of our own) are void
-              behind = ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
-              live = !behind;
-              if (live) {
-                if (ent.y == r) live = false;             // the block is in this very request
-                else if (ent.y < r) {                     // it came back in between: look again
-                  live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
-                  ent.y = r + 1;                          // where it goes next is unknown: assume r+1
-                }
-              }
-            }
-            const unsigned lv = __ballot_sync(kFull, live);
-            const uint32_t cnt = __popc(lv);
-            const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
-            const unsigned take = __ballot_sync(kFull, mine);
+          const uint32_t m = min(avail, 32u);
+          uint4 ent = make_uint4(0, kNone, 0, 0);
+          bool odd = false;      // void (behind the cursor) or touched again since it was listed
+          if (lane < m) {
+            const uint32_t e = (head + lane) & (kListCap - 1);
+            ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+            odd = ent.y <= r || ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
+          }
+          if (!__any_sync(kFull, odd)) {
+            // common case: the next entries are all live, the first `need` of them are victims
+            const uint32_t tk = min(need, m);
+            const bool mine = lane < tk;
             if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
-            hit_next |= __ballot_sync(kFull, mine && ent.y == r + 1);
-            const uint32_t tk = __popc(take);
-            // entries passed: the whole batch, or up to the last victim taken
-            const uint32_t passed = (cnt <= need) ? m : 32u - (uint32_t)__clz((int)take);
+            const unsigned soon = __ballot_sync(kFull, mine && ent.y - (r + 1) < 2u);
+            if (soon) {
+              hit1 |= __ballot_sync(kFull, mine && ent.y == r + 1);
+              hit2 |= __ballot_sync(kFull, mine && ent.y == r + 2);
+            }
             need -= tk;
             evicted += tk;
-            const uint32_t lastl = passed - 1;
-            const bool last_behind = __shfl_sync(kFull, (int)behind, lastl) != 0;
-            const uint32_t lw = __shfl_sync(kFull, ent.w, lastl);
-            const int32_t lz = (int32_t)__shfl_sync(kFull, ent.z, lastl);
-            if (!last_behind) { cr = lw; cp = lz - 1; }
-            head += passed;
-            if (passed < m) break;                        // stopped inside the batch
+            last_e = (head + tk - 1) & (kListCap - 1);
+            head += tk;
+            continue;
           }
+          bool live = false, unsure = false;
+          if (lane < m) {
+            // entries the eviction cursor has already passed (after a walk of our own) are void
+            live = !(ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp));
+            if (live && ent.y <= r) {
+              if (ent.y == r) live = false;               // the block is in this very request
+              else {                                      // it came back in between: look again
+                live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
+                unsure = true;                            // where it occurs next is not known here
+              }
+            }
+          }
+          const unsigned lv = __ballot_sync(kFull, live);
+          const uint32_t cnt = __popc(lv);
+          const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+          if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
+          hit1 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 1));
+          hit2 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 2));
+          // entries passed: the whole round, or up to the last victim taken
+          uint32_t passed = m, tk = cnt;
+          if (cnt > need) {
+            const unsigned take = __ballot_sync(kFull, mine);
+            passed = 32u - (uint32_t)__clz((int)take);
+            tk = need;
+          }
+          need -= tk;
+          evicted += tk;
+          // the cursor moves behind the last live entry passed (void ones lie behind it already)
+          const unsigned seen = lv & (passed >= 32u ? kFull : ((1u << passed) - 1u));
+          if (seen) last_e = (head + 31u - (uint32_t)__clz((int)seen)) & (kListCap - 1);
+          head += passed;
+        }
+        if (last_e != kNone) {
+          const uint4 le = a.lists_in_smem ? lst[last_e] : __ldcg(lst + last_e);
+          cr = le.w;
+          cp = (int32_t)le.z - 1;
         }
         if (lane == 0) sm.ring_head[istar] = head;
       }
@@ -786,14 +809,14 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
         const unsigned take = __ballot_sync(kFull, mine);
         if (mine) mask_clear_bit<MaskT>(mask, vid, bit);
-        hit_next |= __ballot_sync(kFull, mine && nxr == r + 1);
+        hit1 |= __ballot_sync(kFull, mine && nxr == r + 1);
+        hit2 |= __ballot_sync(kFull, mine && nxr == r + 2);
         cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
         const uint32_t tk = __popc(take);
         need -= tk;
         evicted += tk;
       }
       if (lane == 0) { sm.curreq[istar] = cr; sm.curpos[istar] = cp; }
-      redo = redo || (hit_next != 0);
     }
     occ -= evicted;
     st_evict += evicted;
@@ -819,22 +842,19 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     }
     __syncwarp();
 
-    // ---- move on: request r+1 becomes current (repeat its mask read if r may have changed it)
-    rec_cur = rec_nxt; rec_nxt = rec_nn; rec_nn = rec_n3;
+    // ---- did request r change a mask word that was read early?
+    const bool redo = q_nxt.prev_share == r || hit1 != 0;        // words of r+1 (already probed)
+    const bool dirty_nn = q_nn.prev_share == r || hit2 != 0;     // words of r+2 (read just now)
+    // ---- move on: request r+1 becomes current
+    q_cur = q_nxt; q_nxt = q_nn; q_nn = q_n3; q_n3 = q_n4;
 #pragma unroll
     for (int c = 0; c < kRegChunks; ++c) {
-      id_cur[c] = id_nxt[c];
-      id_nxt[c] = id_nn[c];
-      m_cur[c] = m_nxt[c];
+      id_cur[c] = id_nxt[c]; id_nxt[c] = id_nn[c]; id_nn[c] = id_n3[c];
+      m_cur[c] = m_nxt[c]; m_nxt[c] = m_nn[c];
     }
-    if (redo) {
-#pragma unroll
-      for (int c = 0; c < kRegChunks; ++c) {
-        const uint32_t k = c * 32u + lane;
-        m_cur[c] = (k < rec_cur.nblk) ? mask_load<MaskT>(mask, id_cur[c]) : (MaskT)0;
-      }
-    }
+    if (redo && r + 1 < end) load_masks(q_cur, id_cur, m_cur);
     reprobe = redo || !ahead;
+    dirty_nxt = dirty_nn;
   }
   st_probe = warp_sum_u64(st_probe);
   status = __reduce_min_sync(kFull, status);
