@@ -366,6 +366,12 @@ struct Ctx {
   volatile uint32_t* hits;     // [R]  prefix hit per replica of the current request
   volatile uint32_t* route;    // chosen replica of the current request
   volatile int32_t* status;    // first device-side limit hit by any warp
+  // staging of the coming requests by the probe warp (kStageDepth stages + one of the cache warp)
+  volatile uint32_t* st_ready; // [kStageDepth] request (+1) whose data the stage holds
+  volatile uint32_t* probe_gone;  // the probe warp has stopped
+  uint32_t* st_hits;           // [kStageDepth][R] prefix hits
+  uint32_t* st_ids;            // [kStageDepth+1][kStageBlocks] block ids
+  MaskT* st_mk;                // [kStageDepth+1][kStageBlocks] mask words
 };
 
 // Decide warp: queue signal, score, argmin, service model (paper Eq. 1-3).  Waits for the cache
@@ -554,11 +560,116 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
   }
 }
 
-// Cache warp: prefix probe of every replica's block cache, then, once the route is known, the
-// LRU commit on the chosen replica (set its bit on the missing blocks, evict down to capacity).
-// Mask words are read two requests ahead and probed one request ahead; such an early read is
-// repeated when a request committed in between can have changed one of the words (it shares a
-// block with the later request, or a victim evicted for it occurs in the later request).
+constexpr uint32_t kStageDepth = 4;                    // requests staged by the probe warp
+constexpr uint32_t kStageBlocks = kRegChunks * 32u;    // blocks of a request kept per stage
+constexpr uint32_t kWindow = 3;   // a staged read may be up to this many commits old
+
+// What a warp needs to know of a request ahead of time.
+struct Ahead { uint32_t off, nblk, prev_share; };
+__device__ __forceinline__ Ahead fetch_ahead(const ReqRec* req, uint32_t q, uint32_t end) {
+  Ahead h = {0u, 0u, kNone};
+  if (q < end) { const ReqRec x = req[q]; h.off = x.off; h.nblk = x.nblk; h.prev_share = x.prev_share; }
+  return h;
+}
+
+// Prefix probe on every replica from staged mask words: h_i = leading blocks whose mask has
+// bit i.  The first kStageBlocks words come from `smk`; longer prompts read the rest from memory.
+template <typename MaskT>
+__device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask,
+                                             const uint32_t* ids, const Ahead& q, uint32_t R,
+                                             uint32_t lane, uint32_t& h0, uint32_t& h1) {
+  h0 = 0; h1 = 0;   // this lane's replicas: lane and lane+32
+  const uint32_t n = q.nblk;
+  MaskT alive = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0 : (MaskT)((((MaskT)1) << (R & 63)) - 1);
+  for (uint32_t c = 0; c < n && alive != 0; c += 32) {
+    const uint32_t k = c + lane;
+    MaskT m = 0;
+    if (k < n) m = (c < kStageBlocks) ? smk[k] : mask_load<MaskT>(mask, ids[q.off + k]);
+    MaskT it = (MaskT)(shfl_mask<MaskT>(m, 0) & alive);
+    MaskT still = 0;
+    while (it != 0) {
+      const int i = first_bit<MaskT>(it);
+      it &= (MaskT)(it - 1);
+      const unsigned b = __ballot_sync(kFull, (m >> i) & 1);
+      const uint32_t run = (b == kFull) ? 32u : (uint32_t)__ffs((int)~b) - 1u;
+      if ((uint32_t)(i & 31) == lane) {
+        if (i < 32) h0 += run; else h1 += run;
+      }
+      if (run == 32u) still |= (MaskT)(((MaskT)1) << i);
+    }
+    alive = still;
+  }
+}
+
+// Probe warp: runs up to kWindow requests ahead of the cache warp.  For request q it reads the
+// block ids and the mask words (first kStageBlocks blocks), stages them in shared memory, probes
+// them and publishes the prefix hits.  Its reads may predate the commits of the last kWindow
+// requests; the cache warp knows which of those commits can have touched request q and then
+// repeats the work itself, so this warp is an accelerator only and may stop at any time.
+template <typename MaskT>
+__device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>& cx,
+                                           uint32_t lane) {
+  const Smem& sm = cx.sm;
+  const ReqRec* req = a.tr.req;
+  const uint32_t* ids = a.tr.ids;
+  const MaskT* mask = cx.mask;
+  const uint32_t R = a.m.R;
+  const uint32_t end = a.first + a.count;
+  Ahead q_a = fetch_ahead(req, a.first, end), q_n = fetch_ahead(req, a.first + 1, end);
+  Ahead q_b = q_a;
+  uint32_t id_a[kRegChunks], id_n[kRegChunks], id_b[kRegChunks];
+  MaskT m_a[kRegChunks], m_b[kRegChunks];
+#pragma unroll
+  for (int c = 0; c < kRegChunks; ++c) {
+    const uint32_t k = c * 32u + lane;
+    id_a[c] = (k < q_a.nblk) ? ids[q_a.off + k] : 0u;
+    id_b[c] = 0u; m_b[c] = (MaskT)0;
+  }
+  for (uint32_t qa = a.first; qa <= end; ++qa) {
+    if (qa < end) {
+      // room: the stage of request qa is free and its read is at most kWindow commits old once
+      // request qa - kWindow - 1 is committed, i.e. progress >= qa - kWindow
+      uint32_t polls = 0;
+      while ((int32_t)(*sm.progress - qa) < -(int32_t)kWindow) {
+        if (++polls > (1u << 22)) { *cx.probe_gone = 1; return; }   // bounded wait
+        __nanosleep(20);
+      }
+#pragma unroll
+      for (int c = 0; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        m_a[c] = (k < q_a.nblk) ? mask_load<MaskT>(mask, id_a[c]) : (MaskT)0;
+        id_n[c] = (k < q_n.nblk) ? ids[q_n.off + k] : 0u;     // ids of the request after
+      }
+    }
+    const Ahead q_nn = fetch_ahead(req, qa + 2, end);
+    if (qa > a.first) {
+      // stage and probe the previous request (its mask words were requested one round ago)
+      const uint32_t qb = qa - 1, slot = qb % kStageDepth;
+      uint32_t* sid = cx.st_ids + slot * kStageBlocks;
+      MaskT* smk = cx.st_mk + slot * kStageBlocks;
+#pragma unroll
+      for (int c = 0; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        if (k < q_b.nblk) { sid[k] = id_b[c]; smk[k] = m_b[c]; }
+      }
+      __syncwarp();
+      uint32_t h0, h1;
+      probe_staged<MaskT>(smk, mask, ids, q_b, R, lane, h0, h1);
+      if (lane < R) cx.st_hits[slot * R + lane] = h0;
+      if (lane + 32u < R) cx.st_hits[slot * R + lane + 32u] = h1;
+      __threadfence_block();
+      __syncwarp();
+      if (lane == 0) cx.st_ready[slot] = qb + 1;
+    }
+    q_b = q_a; q_a = q_n; q_n = q_nn;
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c) { id_b[c] = id_a[c]; m_b[c] = m_a[c]; id_a[c] = id_n[c]; }
+  }
+}
+
+// Cache warp: takes the staged prefix hits of request r (or reads and probes the mask words
+// itself when a recent commit can have changed them), and, once the route is known, does the
+// LRU commit on the chosen replica: set its bit on the missing blocks, evict down to capacity.
 template <typename MaskT>
 __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
                                            uint32_t lane) {
@@ -570,101 +681,55 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   MaskT* mask = cx.mask;
   uint32_t* lru_next = cx.lru_next;
   const uint8_t* route_log = cx.route_log;
-  const MaskT all_reps = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0
-                                                  : (MaskT)((((MaskT)1) << (R & 63)) - 1);
   int32_t status = 0;
   unsigned long long st_probe = 0, st_evict = 0;
   const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
   const uint32_t end = a.first + a.count;
 
-  // What the warp needs to know of a request ahead of time.
-  struct Ahead { uint32_t off, nblk, prev_share; };
-  auto fetch = [&](uint32_t q) {
-    Ahead h = {0u, 0u, kNone};
-    if (q < end) { const ReqRec x = req[q]; h.off = x.off; h.nblk = x.nblk; h.prev_share = x.prev_share; }
-    return h;
-  };
-  auto load_ids = [&](const Ahead& q, uint32_t (&dst)[kRegChunks]) {
-#pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) {
-      const uint32_t k = c * 32u + lane;
-      dst[c] = (k < q.nblk) ? ids[q.off + k] : 0u;
-    }
-  };
-  auto load_masks = [&](const Ahead& q, const uint32_t (&id)[kRegChunks], MaskT (&dst)[kRegChunks]) {
-#pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) {
-      const uint32_t k = c * 32u + lane;
-      dst[c] = (k < q.nblk) ? mask_load<MaskT>(mask, id[c]) : (MaskT)0;
-    }
-  };
-  // Prefix probe on every replica: h_i = leading blocks whose mask has bit i.  The first
-  // kRegChunks*32 mask words come in `mr`; longer prompts read the rest from memory.
-  auto probe = [&](const Ahead& q, const MaskT (&mr)[kRegChunks], uint32_t& h0, uint32_t& h1) {
-    h0 = 0; h1 = 0;   // this lane's replicas: lane and lane+32
-    const uint32_t n = q.nblk;
-    MaskT alive = all_reps;   // replicas whose cached prefix covers every block seen so far
-    auto probe_chunk = [&](MaskT m) {
-      MaskT it = (MaskT)(shfl_mask<MaskT>(m, 0) & alive);
-      MaskT still = 0;
-      while (it != 0) {
-        const int i = first_bit<MaskT>(it);
-        it &= (MaskT)(it - 1);
-        const unsigned b = __ballot_sync(kFull, (m >> i) & 1);
-        const uint32_t run = (b == kFull) ? 32u : (uint32_t)__ffs((int)~b) - 1u;
-        if ((uint32_t)(i & 31) == lane) {
-          if (i < 32) h0 += run; else h1 += run;
-        }
-        if (run == 32u) still |= (MaskT)(((MaskT)1) << i);
-      }
-      alive = still;
-    };
-#pragma unroll
-    for (int c = 0; c < kRegChunks; ++c)
-      if (c * 32u < n && alive != 0) probe_chunk(mr[c]);
-    for (uint32_t c = kRegChunks * 32u; c < n && alive != 0; c += 32) {   // very long prompts
-      const uint32_t k = c + lane;
-      MaskT m = 0;
-      if (k < n) m = mask_load<MaskT>(mask, ids[q.off + k]);
-      probe_chunk(m);
-    }
-  };
-
-  // Pipeline registers: request r (cur), r+1 (nxt), r+2 (nn), r+3 (n3).  The trace does not
-  // depend on the state, so records and ids simply run ahead; mask words do depend on it.
-  Ahead q_cur = fetch(a.first), q_nxt = fetch(a.first + 1), q_nn = fetch(a.first + 2),
-        q_n3 = fetch(a.first + 3);
-  uint32_t id_cur[kRegChunks], id_nxt[kRegChunks], id_nn[kRegChunks];
-  MaskT m_cur[kRegChunks], m_nxt[kRegChunks];
-  load_ids(q_cur, id_cur); load_ids(q_nxt, id_nxt); load_ids(q_nn, id_nn);
-  load_masks(q_cur, id_cur, m_cur); load_masks(q_nxt, id_nxt, m_nxt);
-  uint32_t hn0 = 0, hn1 = 0;   // prefix hits of the coming request, probed ahead
-  bool reprobe = true;         // ... which must be probed again (always true for the first)
-  bool dirty_nxt = false;      // m_nxt was read before a commit that may have changed it
+  Ahead q_cur = fetch_ahead(req, a.first, end), q_nxt = fetch_ahead(req, a.first + 1, end);
+  // latest earlier request sharing a block with r+1, r+2, r+3, and whether a commit since their
+  // staged read can have changed their mask words
+  uint32_t ps1 = q_nxt.prev_share, ps2 = fetch_ahead(req, a.first + 2, end).prev_share,
+           ps3 = fetch_ahead(req, a.first + 3, end).prev_share;
+  bool bad0 = false, bad1 = false, bad2 = false, bad3 = false;
 
   for (uint32_t r = a.first; r < end; ++r) {
     const uint32_t n = q_cur.nblk, off = q_cur.off;
+    const Ahead q_n2 = fetch_ahead(req, r + 2, end);          // used two rounds from now
+    const uint32_t ps4 = (r + 4 < end) ? req[r + 4].prev_share : kNone;
 
-    // ---- prefix hits of request r: probed while request r-1 was being decided, or again now
-    uint32_t h0 = hn0, h1 = hn1;
-    if (reprobe) probe(q_cur, m_cur, h0, h1);
+    // ---- prefix hits of request r: staged by the probe warp, or read and probed here
+    uint32_t slot = r % kStageDepth;
+    bool staged = false;
+    if (!bad0 && !*cx.probe_gone) {
+      uint32_t polls = 0;
+      while (cx.st_ready[slot] != r + 1 && !*cx.probe_gone && polls < 4096) { ++polls; __nanosleep(20); }
+      staged = cx.st_ready[slot] == r + 1;
+      __threadfence_block();
+    }
+    uint32_t h0 = 0, h1 = 0;
+    if (staged) {
+      if (lane < R) h0 = cx.st_hits[slot * R + lane];
+      if (lane + 32u < R) h1 = cx.st_hits[slot * R + lane + 32u];
+    } else {
+      slot = kStageDepth;                                     // this warp's own stage
+      uint32_t* sid = cx.st_ids + slot * kStageBlocks;
+      MaskT* smk = cx.st_mk + slot * kStageBlocks;
+#pragma unroll
+      for (int c = 0; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        if (k < n) { const uint32_t id = ids[off + k]; sid[k] = id; smk[k] = mask_load<MaskT>(mask, id); }
+      }
+      __syncwarp();
+      probe_staged<MaskT>(smk, mask, ids, q_cur, R, lane, h0, h1);
+    }
+    const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
+    const MaskT* smk = cx.st_mk + slot * kStageBlocks;
     if (lane < R) cx.hits[lane] = h0;
     if (lane + 32u < R) cx.hits[lane + 32u] = h1;
     bar_arrive(kBarHits);                                 // the decide warp may score request r
     if (lane < R) st_probe += (h0 + 1 < n ? h0 + 1 : n);
     if (lane + 32u < R) st_probe += (h1 + 1 < n ? h1 + 1 : n);
-
-    // ---- while the decide warp works: mask words of r+2, ids of r+3, record of r+4 ...
-    MaskT m_nn[kRegChunks];
-    uint32_t id_n3[kRegChunks];
-    load_masks(q_nn, id_nn, m_nn);
-    load_ids(q_n3, id_n3);
-    const Ahead q_n4 = fetch(r + 4);
-    // ... and the probe of r+1 on the words read one request ago (read again first if the
-    // commit of r-1 may have changed them); prompts beyond the register window wait
-    const bool ahead = q_nxt.nblk <= kRegChunks * 32u;
-    if (dirty_nxt) load_masks(q_nxt, id_nxt, m_nxt);
-    if (ahead) probe(q_nxt, m_nxt, hn0, hn1);
 
     bar_wait(kBarRoute);                                  // the replica has been chosen
     const uint32_t istar = *cx.route;
@@ -672,21 +737,14 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
 
     // ---- cache commit: set the replica's bit on the missing blocks
     uint32_t missing = 0;
-#pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) {
-      if (c * 32u < n) {
-        const uint32_t k = c * 32u + lane;
-        const bool miss = (k < n) && !(m_cur[c] & bit);
-        if (miss) mask_store<MaskT>(mask, id_cur[c], (MaskT)(m_cur[c] | bit));
-        missing += __popc(__ballot_sync(kFull, miss));
-      }
-    }
-    for (uint32_t c = kRegChunks * 32u; c < n; c += 32) {
+    for (uint32_t c = 0; c < n; c += 32) {
       const uint32_t k = c + lane;
       bool miss = false;
       if (k < n) {
-        const uint32_t id = ids[off + k];
-        const MaskT mv = mask_load<MaskT>(mask, id);
+        uint32_t id;
+        MaskT mv;
+        if (c < kStageBlocks) { id = sid[k]; mv = smk[k]; }
+        else { id = ids[off + k]; mv = mask_load<MaskT>(mask, id); }
         if (!(mv & bit)) { mask_store<MaskT>(mask, id, (MaskT)(mv | bit)); miss = true; }
       }
       missing += __popc(__ballot_sync(kFull, miss));
@@ -694,7 +752,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     uint32_t occ = sm.occ[istar] + missing;
     uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
     uint32_t evicted = 0;
-    unsigned hit1 = 0, hit2 = 0;   // a victim's block occurs again in request r+1 / r+2
+    unsigned hit1 = 0, hit2 = 0, hit3 = 0;   // a victim's block occurs again in request r+1/2/3
     if (need > 0) {
       uint32_t cr = sm.curreq[istar];
       int32_t cp = sm.curpos[istar];
@@ -724,10 +782,11 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
             const uint32_t tk = min(need, m);
             const bool mine = lane < tk;
             if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
-            const unsigned soon = __ballot_sync(kFull, mine && ent.y - (r + 1) < 2u);
+            const unsigned soon = __ballot_sync(kFull, mine && ent.y - (r + 1) < kWindow);
             if (soon) {
               hit1 |= __ballot_sync(kFull, mine && ent.y == r + 1);
               hit2 |= __ballot_sync(kFull, mine && ent.y == r + 2);
+              hit3 |= __ballot_sync(kFull, mine && ent.y == r + 3);
             }
             need -= tk;
             evicted += tk;
@@ -753,6 +812,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
           if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
           hit1 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 1));
           hit2 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 2));
+          hit3 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 3));
           // entries passed: the whole round, or up to the last victim taken
           uint32_t passed = m, tk = cnt;
           if (cnt > need) {
@@ -811,6 +871,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         if (mine) mask_clear_bit<MaskT>(mask, vid, bit);
         hit1 |= __ballot_sync(kFull, mine && nxr == r + 1);
         hit2 |= __ballot_sync(kFull, mine && nxr == r + 2);
+        hit3 |= __ballot_sync(kFull, mine && nxr == r + 3);
         cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
         const uint32_t tk = __popc(take);
         need -= tk;
@@ -842,19 +903,13 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     }
     __syncwarp();
 
-    // ---- did request r change a mask word that was read early?
-    const bool redo = q_nxt.prev_share == r || hit1 != 0;        // words of r+1 (already probed)
-    const bool dirty_nn = q_nn.prev_share == r || hit2 != 0;     // words of r+2 (read just now)
-    // ---- move on: request r+1 becomes current
-    q_cur = q_nxt; q_nxt = q_nn; q_nn = q_n3; q_n3 = q_n4;
-#pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) {
-      id_cur[c] = id_nxt[c]; id_nxt[c] = id_nn[c]; id_nn[c] = id_n3[c];
-      m_cur[c] = m_nxt[c]; m_nxt[c] = m_nn[c];
-    }
-    if (redo && r + 1 < end) load_masks(q_cur, id_cur, m_cur);
-    reprobe = redo || !ahead;
-    dirty_nxt = dirty_nn;
+    // ---- which staged reads did the commit of request r invalidate?  Then move on.
+    bad0 = bad1 || ps1 == r || hit1 != 0;
+    bad1 = bad2 || ps2 == r || hit2 != 0;
+    bad2 = bad3 || ps3 == r || hit3 != 0;
+    bad3 = false;
+    ps1 = ps2; ps2 = ps3; ps3 = ps4;
+    q_cur = q_nxt; q_nxt = q_n2;
   }
   st_probe = warp_sum_u64(st_probe);
   status = __reduce_min_sync(kFull, status);
@@ -868,8 +923,8 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   }
 }
 
-constexpr uint32_t kWarpDecide = 0, kWarpCache = 1, kWarpHelper = 2, kWarpScout0 = 3;
-constexpr uint32_t kReplayThreads = 32 * (3 + kScouts);
+constexpr uint32_t kWarpDecide = 0, kWarpCache = 1, kWarpProbe = 2, kWarpHelper = 3, kWarpScout0 = 4;
+constexpr uint32_t kReplayThreads = 32 * (4 + kScouts);
 
 template <typename MaskT>
 __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayArgs a) {
@@ -926,6 +981,14 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   sm.scan_cp = reinterpret_cast<volatile int32_t*>(sm.scan_cr + R);
   {
     uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R;
+    cx.st_ready = after;
+    cx.probe_gone = after + kStageDepth;
+    cx.st_hits = after + kStageDepth + 1;
+    cx.st_ids = cx.st_hits + kStageDepth * (size_t)R;
+    after = cx.st_ids + (kStageDepth + 1) * (size_t)kStageBlocks;
+    const uintptr_t a8 = (reinterpret_cast<uintptr_t>(after) + 7) & ~(uintptr_t)7;
+    cx.st_mk = reinterpret_cast<MaskT*>(a8);
+    after = reinterpret_cast<uint32_t*>(cx.st_mk + (kStageDepth + 1) * (size_t)kStageBlocks);
     const uintptr_t al = (reinterpret_cast<uintptr_t>(after) + 15) & ~(uintptr_t)15;
     sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(al)
                              : a.evict_lists + (size_t)p * R * kListCap;
@@ -959,11 +1022,13 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
     for (uint32_t x = threadIdx.x; x < 3 * RS; x += blockDim.x) slot_d[x] = g_slot_d[x];
     for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) slot_u[x] = g_slot_u[x];
   }
-  if (threadIdx.x == 0) { *sm.progress = a.first; *cx.status = 0; }
+  if (threadIdx.x == 0) { *sm.progress = a.first; *cx.status = 0; *cx.probe_gone = 0; }
+  if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
   __syncthreads();
 
   if (warp == kWarpDecide) decide_warp<MaskT>(a, cx, p, lane);
   else if (warp == kWarpCache) cache_warp<MaskT>(a, cx, p, lane);
+  else if (warp == kWarpProbe) probe_warp<MaskT>(a, cx, lane);
   else if (warp == kWarpHelper) helper_warp<MaskT>(a, sm, cx.mask, cx.lru_next, lane);
   else scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, warp - kWarpScout0);
   __syncthreads();
@@ -1121,7 +1186,9 @@ cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
   a.slots_in_smem = rs * 44 <= 44 * 1024 ? 1u : 0u;
   a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
-                (10 * (size_t)a.m.R + 3) * sizeof(uint32_t) + 16;
+                (10 * (size_t)a.m.R + 3) * sizeof(uint32_t) + 16 +
+                (kStageDepth + 1 + kStageDepth * (size_t)a.m.R + (kStageDepth + 1) * kStageBlocks) * sizeof(uint32_t) +
+                (kStageDepth + 1) * kStageBlocks * sizeof(MaskT) + 8;
   if (a.slots_in_smem) smem += rs * 44;
   if (a.lists_in_smem) smem += list_bytes;
   smem = (smem + 15) / 16 * 16;
