@@ -363,15 +363,17 @@ struct Ctx {
   // per-slot state (shared or global memory)
   double *free_at, *q0_fin, *q1_fin;
   uint32_t *q0_tok, *q1_tok, *q2_idx, *tail, *qcnt;
-  volatile uint32_t* hits;     // [R]  prefix hit per replica of the current request
   volatile uint32_t* route;    // chosen replica of the current request
   volatile int32_t* status;    // first device-side limit hit by any warp
   // staging of the coming requests by the probe warp (kStageDepth stages + one of the cache warp)
   volatile uint32_t* st_ready; // [kStageDepth] request (+1) whose data the stage holds
   volatile uint32_t* probe_gone;  // the probe warp has stopped
-  uint32_t* st_hits;           // [kStageDepth][R] prefix hits
-  uint32_t* st_ids;            // [kStageDepth+1][kStageBlocks] block ids
-  MaskT* st_mk;                // [kStageDepth+1][kStageBlocks] mask words
+  // (stages kStageDepth and kStageDepth+1 belong to the cache warp, used alternately)
+  uint32_t* st_hits;           // [kStageDepth+2][R] prefix hits
+  double* st_ab;               // [kStageDepth+2][R] (w_net*RTT + w_prefill*uncached) per replica
+  uint32_t* st_ids;            // [kStageDepth+2][kStageBlocks] block ids
+  MaskT* st_mk;                // [kStageDepth+2][kStageBlocks] mask words
+  volatile uint32_t* hit_slot; // stage that holds the current request's hits and scores
 };
 
 // Decide warp: queue signal, score, argmin, service model (paper Eq. 1-3).  Waits for the cache
@@ -475,35 +477,31 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
 
     bar_wait(kBarHits);                                   // prefix hits of request r are posted
 
-    // ---- score of Eq. 3 (fixed order, no FMA) and lowest-index argmin
+    // ---- score of Eq. 3 (fixed order, no FMA): the staged (w_net*RTT + w_prefill*uncached)
+    //      plus the queue term; lowest-index argmin
+    const uint32_t stage = *cx.hit_slot;
     uint64_t best_k = ~0ull;
     uint32_t best_i = kNone;
-    uint32_t unc0 = 0, unc1 = 0, h0 = 0, h1 = 0;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const uint32_t i = lane + 32u * half;
       if (i < R) {
-        const uint32_t h = cx.hits[i];
-        if (half) h1 = h; else h0 = h;
-        const unsigned long long hb = (unsigned long long)h * a.m.B;
-        const uint32_t unc = in_tok - (uint32_t)(hb < in_tok ? hb : in_tok);
-        if (half) unc1 = unc; else unc0 = unc;
-        double c = __dadd_rn(__dadd_rn(wrtt_row[i], __dmul_rn(w_pre, (double)unc)),
-                             half ? cq1 : cq0);
+        double c = __dadd_rn(cx.st_ab[stage * R + i], half ? cq1 : cq0);
         if (c != c) c = (i == 0) ? -d_inf() : d_inf();  // a NaN score wins only at index 0
         const uint64_t ck = order_key(c);
         if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i; }
       }
     }
     const uint32_t istar = warp_argmin_key(best_k, best_i);
+    const uint32_t hstar = cx.st_hits[stage * R + istar];   // read before the stage can be reused
     if (lane == 0) {
       *cx.route = istar;
       cx.route_log[r] = (uint8_t)istar;
     }
     bar_arrive(kBarRoute);                                // the cache warp may commit request r
 
-    const uint32_t hstar = __shfl_sync(kFull, istar < 32 ? h0 : h1, istar & 31);
-    const uint32_t uncstar = __shfl_sync(kFull, istar < 32 ? unc0 : unc1, istar & 31);
+    const unsigned long long hbstar = (unsigned long long)hstar * a.m.B;
+    const uint32_t uncstar = in_tok - (uint32_t)(hbstar < in_tok ? hbstar : in_tok);
 
     // ---- service commit: earliest-free slot, lowest index on ties
     uint64_t bk = ~0ull;
@@ -565,10 +563,14 @@ constexpr uint32_t kStageBlocks = kRegChunks * 32u;    // blocks of a request ke
 constexpr uint32_t kWindow = 3;   // a staged read may be up to this many commits old
 
 // What a warp needs to know of a request ahead of time.
-struct Ahead { uint32_t off, nblk, prev_share; };
+struct Ahead { uint32_t off, nblk, prev_share, in_tok, origin; };
 __device__ __forceinline__ Ahead fetch_ahead(const ReqRec* req, uint32_t q, uint32_t end) {
-  Ahead h = {0u, 0u, kNone};
-  if (q < end) { const ReqRec x = req[q]; h.off = x.off; h.nblk = x.nblk; h.prev_share = x.prev_share; }
+  Ahead h = {0u, 0u, kNone, 0u, 0u};
+  if (q < end) {
+    const ReqRec x = req[q];
+    h.off = x.off; h.nblk = x.nblk; h.prev_share = x.prev_share; h.in_tok = x.in_tok;
+    h.origin = x.origin;
+  }
   return h;
 }
 
@@ -598,6 +600,28 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
       if (run == 32u) still |= (MaskT)(((MaskT)1) << i);
     }
     alive = still;
+  }
+}
+
+// Stage the prefix hits of a request and the part of its score (Eq. 3) that depends on them:
+// ab_i = (w_net * RTT[g][i]) + (w_prefill * uncached_i), same operations and order as the score.
+template <typename MaskT>
+__device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<MaskT>& cx,
+                                             const Ahead& q, uint32_t slot, uint32_t h0,
+                                             uint32_t h1, uint32_t lane) {
+  const uint32_t R = a.m.R;
+  const double w_pre = cx.sm.w[1];
+  const double* wrtt_row = cx.sm.wrtt + (size_t)q.origin * R;
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const uint32_t i = lane + 32u * half;
+    if (i < R) {
+      const uint32_t h = half ? h1 : h0;
+      const unsigned long long hb = (unsigned long long)h * a.m.B;
+      const uint32_t unc = q.in_tok - (uint32_t)(hb < q.in_tok ? hb : q.in_tok);
+      cx.st_hits[slot * R + i] = h;
+      cx.st_ab[slot * R + i] = __dadd_rn(wrtt_row[i], __dmul_rn(w_pre, (double)unc));
+    }
   }
 }
 
@@ -655,8 +679,7 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
       __syncwarp();
       uint32_t h0, h1;
       probe_staged<MaskT>(smk, mask, ids, q_b, R, lane, h0, h1);
-      if (lane < R) cx.st_hits[slot * R + lane] = h0;
-      if (lane + 32u < R) cx.st_hits[slot * R + lane + 32u] = h1;
+      stage_scores<MaskT>(a, cx, q_b, slot, h0, h1, lane);
       __threadfence_block();
       __syncwarp();
       if (lane == 0) cx.st_ready[slot] = qb + 1;
@@ -712,7 +735,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       if (lane < R) h0 = cx.st_hits[slot * R + lane];
       if (lane + 32u < R) h1 = cx.st_hits[slot * R + lane + 32u];
     } else {
-      slot = kStageDepth;                                     // this warp's own stage
+      slot = kStageDepth + (r & 1u);                          // this warp's own stages
       uint32_t* sid = cx.st_ids + slot * kStageBlocks;
       MaskT* smk = cx.st_mk + slot * kStageBlocks;
 #pragma unroll
@@ -722,11 +745,11 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       }
       __syncwarp();
       probe_staged<MaskT>(smk, mask, ids, q_cur, R, lane, h0, h1);
+      stage_scores<MaskT>(a, cx, q_cur, slot, h0, h1, lane);
     }
     const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
     const MaskT* smk = cx.st_mk + slot * kStageBlocks;
-    if (lane < R) cx.hits[lane] = h0;
-    if (lane + 32u < R) cx.hits[lane + 32u] = h1;
+    if (lane == 0) *cx.hit_slot = slot;
     bar_arrive(kBarHits);                                 // the decide warp may score request r
     if (lane < R) st_probe += (h0 + 1 < n ? h0 + 1 : n);
     if (lane + 32u < R) st_probe += (h1 + 1 < n ? h1 + 1 : n);
@@ -973,8 +996,8 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   sm.progress = unext;
   cx.route = unext + 1;
   cx.status = reinterpret_cast<volatile int32_t*>(unext + 2);
-  cx.hits = unext + 3;                   // [R]
-  sm.act = unext + 3 + R;
+  cx.hit_slot = unext + 3;
+  sm.act = unext + 4;
   sm.ring_head = sm.act + R;
   sm.ring_tail = sm.ring_head + R;
   sm.scan_cr = sm.ring_tail + R;
@@ -984,11 +1007,12 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
     cx.st_ready = after;
     cx.probe_gone = after + kStageDepth;
     cx.st_hits = after + kStageDepth + 1;
-    cx.st_ids = cx.st_hits + kStageDepth * (size_t)R;
-    after = cx.st_ids + (kStageDepth + 1) * (size_t)kStageBlocks;
+    cx.st_ids = cx.st_hits + (kStageDepth + 2) * (size_t)R;
+    after = cx.st_ids + (kStageDepth + 2) * (size_t)kStageBlocks;
     const uintptr_t a8 = (reinterpret_cast<uintptr_t>(after) + 7) & ~(uintptr_t)7;
-    cx.st_mk = reinterpret_cast<MaskT*>(a8);
-    after = reinterpret_cast<uint32_t*>(cx.st_mk + (kStageDepth + 1) * (size_t)kStageBlocks);
+    cx.st_ab = reinterpret_cast<double*>(a8);
+    cx.st_mk = reinterpret_cast<MaskT*>(cx.st_ab + (kStageDepth + 2) * (size_t)R);
+    after = reinterpret_cast<uint32_t*>(cx.st_mk + (kStageDepth + 2) * (size_t)kStageBlocks);
     const uintptr_t al = (reinterpret_cast<uintptr_t>(after) + 15) & ~(uintptr_t)15;
     sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(al)
                              : a.evict_lists + (size_t)p * R * kListCap;
@@ -1186,9 +1210,10 @@ cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
   a.slots_in_smem = rs * 44 <= 44 * 1024 ? 1u : 0u;
   a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
-                (10 * (size_t)a.m.R + 3) * sizeof(uint32_t) + 16 +
-                (kStageDepth + 1 + kStageDepth * (size_t)a.m.R + (kStageDepth + 1) * kStageBlocks) * sizeof(uint32_t) +
-                (kStageDepth + 1) * kStageBlocks * sizeof(MaskT) + 8;
+                (9 * (size_t)a.m.R + 4) * sizeof(uint32_t) + 16 +
+                (kStageDepth + 1 + (kStageDepth + 2) * ((size_t)a.m.R + kStageBlocks)) * sizeof(uint32_t) +
+                8 + (kStageDepth + 2) * (size_t)a.m.R * sizeof(double) +
+                (kStageDepth + 2) * kStageBlocks * sizeof(MaskT) + 8;
   if (a.slots_in_smem) smem += rs * 44;
   if (a.lists_in_smem) smem += list_bytes;
   smem = (smem + 15) / 16 * 16;
