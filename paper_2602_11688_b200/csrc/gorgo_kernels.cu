@@ -715,6 +715,14 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   uint32_t ps1 = q_nxt.prev_share, ps2 = fetch_ahead(req, a.first + 2, end).prev_share,
            ps3 = fetch_ahead(req, a.first + 3, end).prev_share;
   bool bad0 = false, bad1 = false, bad2 = false, bad3 = false;
+  bool posted = false;         // the hits of the coming request were already handed over
+  // hand the staged hits of request q over to the decide warp and count its probes
+  auto hand_over = [&](uint32_t slot, uint32_t nblk) {
+    if (lane == 0) *cx.hit_slot = slot;
+    bar_arrive(kBarHits);                                 // the decide warp may score the request
+    if (lane < R) { const uint32_t h = cx.st_hits[slot * R + lane]; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+    if (lane + 32u < R) { const uint32_t h = cx.st_hits[slot * R + lane + 32u]; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+  };
 
   for (uint32_t r = a.first; r < end; ++r) {
     const uint32_t n = q_cur.nblk, off = q_cur.off;
@@ -723,18 +731,15 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
 
     // ---- prefix hits of request r: staged by the probe warp, or read and probed here
     uint32_t slot = r % kStageDepth;
-    bool staged = false;
-    if (!bad0 && !*cx.probe_gone) {
+    bool staged = posted;
+    if (!posted && !bad0 && !*cx.probe_gone) {
       uint32_t polls = 0;
       while (cx.st_ready[slot] != r + 1 && !*cx.probe_gone && polls < 4096) { ++polls; __nanosleep(20); }
       staged = cx.st_ready[slot] == r + 1;
       __threadfence_block();
     }
-    uint32_t h0 = 0, h1 = 0;
-    if (staged) {
-      if (lane < R) h0 = cx.st_hits[slot * R + lane];
-      if (lane + 32u < R) h1 = cx.st_hits[slot * R + lane + 32u];
-    } else {
+    if (!staged) {
+      uint32_t h0 = 0, h1 = 0;
       slot = kStageDepth + (r & 1u);                          // this warp's own stages
       uint32_t* sid = cx.st_ids + slot * kStageBlocks;
       MaskT* smk = cx.st_mk + slot * kStageBlocks;
@@ -749,10 +754,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     }
     const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
     const MaskT* smk = cx.st_mk + slot * kStageBlocks;
-    if (lane == 0) *cx.hit_slot = slot;
-    bar_arrive(kBarHits);                                 // the decide warp may score request r
-    if (lane < R) st_probe += (h0 + 1 < n ? h0 + 1 : n);
-    if (lane + 32u < R) st_probe += (h1 + 1 < n ? h1 + 1 : n);
+    if (!posted) hand_over(slot, n);
 
     bar_wait(kBarRoute);                                  // the replica has been chosen
     const uint32_t istar = *cx.route;
@@ -905,6 +907,21 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     occ -= evicted;
     st_evict += evicted;
 
+    // ---- which staged reads did the commit of request r invalidate?  If the next request's
+    //      are intact and staged, hand them over now: the decide warp works on r+1 while the
+    //      bookkeeping of r below finishes.
+    bad0 = bad1 || ps1 == r || hit1 != 0;
+    bad1 = bad2 || ps2 == r || hit2 != 0;
+    bad2 = bad3 || ps3 == r || hit3 != 0;
+    bad3 = false;
+    ps1 = ps2; ps2 = ps3; ps3 = ps4;
+    posted = false;
+    if (r + 1 < end && !bad0 && cx.st_ready[(r + 1) % kStageDepth] == r + 2) {
+      __threadfence_block();
+      hand_over((r + 1) % kStageDepth, q_nxt.nblk);
+      posted = true;
+    }
+
     if (lane == 0) {
       sm.occ[istar] = occ;
       // recency order of the replica: append this request
@@ -926,12 +943,6 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     }
     __syncwarp();
 
-    // ---- which staged reads did the commit of request r invalidate?  Then move on.
-    bad0 = bad1 || ps1 == r || hit1 != 0;
-    bad1 = bad2 || ps2 == r || hit2 != 0;
-    bad2 = bad3 || ps3 == r || hit3 != 0;
-    bad3 = false;
-    ps1 = ps2; ps2 = ps3; ps3 = ps4;
     q_cur = q_nxt; q_nxt = q_n2;
   }
   st_probe = warp_sum_u64(st_probe);
