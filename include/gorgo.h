@@ -165,6 +165,10 @@ int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
  * kernel (one launch per wave, at most 32 waves are timed).  gorgo_last_replay_ms waits for those
  * events and returns the summed device time of the replay launches of the most recent
  * evaluation and their number. */
+/* Measurement aid (no counterpart in the paper): how many candidates (CTAs of the replay kernel)
+ * one SM holds at once for this configuration, and the shared memory each takes.  A population
+ * larger than SMs x that number is replayed in successive rounds of CTAs. */
+int gorgo_replay_occupancy(gorgo_sim_t *sim, int32_t *ctas_per_sm, uint64_t *smem_bytes_per_cta);
 int gorgo_set_profiling(gorgo_sim_t *sim, int enable);
 int gorgo_last_replay_ms(gorgo_sim_t *sim, double *replay_ms, uint32_t *launches);
 

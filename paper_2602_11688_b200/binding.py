@@ -31,7 +31,7 @@ EXPORTS = [
     "gorgo_trace_info", "gorgo_workspace_bytes", "gorgo_eval_population",
     "gorgo_eval_population_host", "gorgo_state_bytes", "gorgo_sim_reset", "gorgo_route_batch",
     "gorgo_state_digest", "gorgo_state_status", "gorgo_set_profiling", "gorgo_last_replay_ms",
-    "gorgo_eval_population_static", "gorgo_strerror",
+    "gorgo_eval_population_static", "gorgo_replay_occupancy", "gorgo_strerror",
 ]
 
 
@@ -78,6 +78,7 @@ def load():
         "gorgo_state_digest": [vp, vp, u64, vp, vp],
         "gorgo_state_status": [vp, vp, u64, vp, pu64],
         "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp],
+        "gorgo_replay_occupancy": [vp, C.POINTER(C.c_int32), pu64],
         "gorgo_set_profiling": [vp, i32],
         "gorgo_last_replay_ms": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint32)],
     }
@@ -216,6 +217,13 @@ def gorgo_state_status(sim, state_workspace, stream: int = 0):
     rc = load().gorgo_state_status(sim, _dev_ptr(state_workspace), state_workspace.numel(),
                                    stream, C.byref(seen))
     return rc, seen.value
+
+
+def gorgo_replay_occupancy(sim):
+    """Returns (status, replay CTAs per SM, dynamic shared-memory bytes per CTA)."""
+    n, b = C.c_int32(), C.c_uint64()
+    rc = load().gorgo_replay_occupancy(sim, C.byref(n), C.byref(b))
+    return rc, n.value, b.value
 
 
 def gorgo_set_profiling(sim, enable: bool) -> int:

@@ -531,6 +531,16 @@ int gorgo_state_status(gorgo_sim_t* sim, void* state_workspace, uint64_t state_b
   return h.status;
 }
 
+int gorgo_replay_occupancy(gorgo_sim_t* sim, int32_t* ctas_per_sm, uint64_t* smem_bytes_per_cta) {
+  if (!sim || !ctas_per_sm) return GORGO_ERR_INVALID_ARG;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  const int n = replay_occupancy(sim->m, smem_bytes_per_cta);
+  if (n < 0) return GORGO_ERR_CUDA;
+  *ctas_per_sm = n;
+  return GORGO_OK;
+}
+
 int gorgo_set_profiling(gorgo_sim_t* sim, int enable) {
   if (!sim) return GORGO_ERR_INVALID_ARG;
   if (enable && sim->ev.empty()) {

@@ -125,5 +125,8 @@ cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st)
 cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st);
 uint32_t mask_bytes_for(uint32_t n_replicas);
 uint64_t evict_list_bytes(uint32_t n_replicas);
+// CTAs of the replay kernel that fit one SM for this model (-1: query failed), and the dynamic
+// shared memory one CTA asks for.
+int replay_occupancy(const Model& m, uint64_t* smem_bytes);
 
 }  // namespace gorgo

@@ -1215,7 +1215,7 @@ __global__ void __launch_bounds__(256) digest_kernel(const DigestArgs a) {
 }
 
 template <typename MaskT>
-cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
+size_t replay_smem_bytes(ReplayArgs& a) {
   const size_t rs = (size_t)a.m.R * a.m.S;
   const size_t list_bytes = (size_t)a.m.R * kListCap * sizeof(uint4);
   a.slots_in_smem = rs * 44 <= 44 * 1024 ? 1u : 0u;
@@ -1228,9 +1228,23 @@ cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
   if (a.slots_in_smem) smem += rs * 44;
   if (a.lists_in_smem) smem += list_bytes;
   smem = (smem + 15) / 16 * 16;
+  return smem;
+}
+
+template <typename MaskT>
+cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
+  const size_t smem = replay_smem_bytes<MaskT>(a);
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  // several candidates share an SM (P is usually larger than the SM count): ask for the largest
+  // shared-memory carve-out so that the per-CTA footprint, not the default split, decides
+  {
+    cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT>,
+                                         cudaFuncAttributePreferredSharedMemoryCarveout,
+                                         (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
   }
   replay_kernel<MaskT><<<n_cand, kReplayThreads, smem, st>>>(a);
@@ -1238,6 +1252,37 @@ cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
 }
 
 }  // namespace
+
+template <typename MaskT>
+int replay_occupancy_t(ReplayArgs a, size_t* smem_out) {
+  const size_t smem = replay_smem_bytes<MaskT>(a);
+  *smem_out = smem;
+  cudaFuncSetAttribute(replay_kernel<MaskT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaFuncSetAttribute(replay_kernel<MaskT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                       (int)cudaSharedmemCarveoutMaxShared);
+  int n = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, replay_kernel<MaskT>, (int)kReplayThreads,
+                                                    smem) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return n;
+}
+
+int replay_occupancy(const Model& m, uint64_t* smem_bytes) {
+  ReplayArgs a = {};
+  a.m = m;
+  int n;
+  size_t smem = 0;
+  switch (mask_bytes_for(m.R)) {
+    case 1: n = replay_occupancy_t<uint8_t>(a, &smem); break;
+    case 2: n = replay_occupancy_t<uint16_t>(a, &smem); break;
+    case 4: n = replay_occupancy_t<uint32_t>(a, &smem); break;
+    default: n = replay_occupancy_t<uint64_t>(a, &smem); break;
+  }
+  if (smem_bytes) *smem_bytes = smem;
+  return n;
+}
 
 uint64_t evict_list_bytes(uint32_t n_replicas) {
   return (uint64_t)n_replicas * kListCap * sizeof(uint4);
