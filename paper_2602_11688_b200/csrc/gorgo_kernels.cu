@@ -5,7 +5,7 @@
 //    the blocks of one conversation are runs of consecutive numbers);
 //  * per candidate ONE direct-indexed array `mask[id]` whose bit i says "block id is cached on
 //    replica i".  A request's prefix probe on all R replicas is one coalesced read of its n
-//    mask words, a prefix-AND across lanes and a few ballots;
+//    mask words and one ballot per replica that holds its first block;
 //  * exact LRU without per-block recency stamps: the recency order of replica i is the order of
 //    the requests routed to it (a linked list through `lru_next`), deepest block first inside a
 //    request.  An eviction cursor walks that order; a touch (request n, position k) is still the
@@ -14,10 +14,18 @@
 //    the cursor are the LRU victims; stale ones are skipped for good;
 //  * in-flight accounting through per-slot FIFO chains (finish times on one slot never
 //    decrease), with the earliest finish per replica cached so the common case is one compare.
-// One warp replays one candidate; requests are strictly ordered inside a candidate, so the
-// parallelism is across candidates, across the blocks of a request and across replicas.  A
-// second warp of the same CTA runs ahead through the (state-independent) trace and prefetches
-// what the replay warp will touch, since the replay is bound by memory latency, not bandwidth.
+// Requests are strictly ordered inside a candidate and every step depends on the one before, so
+// a replay is bound by the latency of that chain, not by bandwidth.  One CTA of five warps
+// replays one candidate and the warps split the chain:
+//   decide  queue signal, score (Eq. 3), argmin, service model, outputs;
+//   cache   validates the staged prefix hits, sizes and performs the eviction, recency list;
+//   probe   runs up to three requests ahead: reads block ids and mask words, probes them and
+//           stages hits and the hit-dependent part of the score in shared memory;
+//   scout   (two warps) validate touches ahead of every replica's eviction cursor and keep a
+//           ring of ready victims per replica.
+// A staged read may predate the commits of the last three requests; the cache warp knows which
+// of those commits can have touched the request (shared block, or evicted block that occurs in
+// it) and then repeats the read itself, so results never depend on the timing of the warps.
 #include "gorgo_internal.h"
 
 namespace gorgo {
@@ -99,9 +107,6 @@ __device__ __forceinline__ uint64_t mix64(uint64_t z) {  // splitmix64 finaliser
 }
 
 // ------------------------------------------------------------------------------ replay
-__device__ __forceinline__ void prefetch_l2(const void* p) {
-  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-}
 
 // Clear `bit` of mask[id] without reading it back (a reduction performed in L2).
 template <typename MaskT>
@@ -149,7 +154,6 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
 }
 
 constexpr int kRegChunks = 4;     // request blocks held in registers: 4 x 32 = 128
-constexpr uint32_t kAhead = 48;   // how far the helper warp runs ahead of the replay (requests)
 constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
 constexpr int kScoutBatches = 2;       // touches examined per lane and scout round
@@ -170,71 +174,6 @@ struct Smem {
   volatile uint32_t* scan_cr;     // scout's own cursor into the recency order (set at activation)
   volatile int32_t* scan_cp;
 };
-
-// Helper warp: runs ahead of the replay warp of the same candidate and pulls what it will touch
-// into L2 (mask words, next-occurrence links at the eviction cursors) and L1/L2 (request
-// records, block ids).  Pure prefetching: it changes no state and may stop at any time.
-template <typename MaskT>
-__device__ __forceinline__ void helper_warp(const ReplayArgs& a, const Smem& sm, const MaskT* mask,
-                            const uint32_t* lru_next, uint32_t lane) {
-  const ReqRec* req = a.tr.req;
-  const uint32_t* ids = a.tr.ids;
-  const uint32_t end = a.first + a.count;
-  const uint32_t R = a.m.R;
-  uint32_t pos = a.first;
-  uint32_t idle = 0;
-  constexpr uint32_t kLineShift = sizeof(MaskT) == 1 ? 5 : sizeof(MaskT) == 2 ? 4
-                                  : sizeof(MaskT) == 4 ? 3 : 2;   // ids per 32-byte sector
-  while (pos < end) {
-    const uint32_t cur = *sm.progress;
-    if (cur >= end) break;
-    if (pos < cur) pos = cur;                       // fell behind: skip what is already done
-    if (pos >= cur + kAhead) {
-      if (++idle > (1u << 24)) break;               // bounded wait; prefetching is optional
-      __nanosleep(256);
-      continue;
-    }
-    // one batch of up to 16 requests: every lane fetches one record, then the warp walks them
-    const uint32_t nb = min(16u, end - pos);
-    ReqRec mine = {};
-    if (lane < nb) mine = req[pos + lane];
-    for (uint32_t j = 0; j < nb; ++j) {
-      const uint32_t off = __shfl_sync(kFull, mine.off, j);
-      const uint32_t n = __shfl_sync(kFull, (uint32_t)mine.nblk, j);
-      for (uint32_t c = 0; c < n; c += 32) {
-        const uint32_t k = c + lane;
-        const uint32_t id = (k < n) ? ids[off + k] : 0u;
-        const uint32_t prev = __shfl_up_sync(kFull, id, 1);
-        if (k < n && (lane == 0 || (prev >> kLineShift) != (id >> kLineShift)))
-          prefetch_l2(mask + id);
-      }
-    }
-    // eviction cursors: the links and ids of the next touches of every replica
-    for (uint32_t i = lane; i < R; i += 32) {
-      uint32_t cr = sm.curreq[i];
-      int32_t cp = sm.curpos[i];
-      int32_t budget = 256;
-      for (int hop = 0; hop < 4 && cr != kNone && budget > 0; ++hop) {
-        if (hop > 0 || cp < 0) {
-          cr = lru_next[cr];
-          if (cr == kNone || cr >= cur) break;
-          cp = (int32_t)req[cr].nblk - 1;
-        }
-        if (cp < 0) continue;
-        const uint32_t coff = req[cr].off;
-        const int32_t lo = cp - budget + 1 > 0 ? cp - budget + 1 : 0;
-        for (int32_t k = lo & ~15; k <= cp; k += 16) {   // 16 links = 128 bytes
-          prefetch_l2(a.tr.occ_next + coff + k);
-          if ((k & 31) == 0 || k == (lo & ~15)) prefetch_l2(ids + coff + k);
-        }
-        budget -= cp - lo + 1;
-        cp = -1;
-      }
-    }
-    pos += nb;
-    idle = 0;
-  }
-}
 
 // Scout warp: for every replica whose cache is close to full it walks the recency order ahead
 // of the eviction cursor and appends to the replica's ring the touches that are still the latest
@@ -388,7 +327,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
   uint32_t *q0_tok = cx.q0_tok, *q1_tok = cx.q1_tok, *q2_idx = cx.q2_idx, *tail = cx.tail,
            *qcnt = cx.qcnt;
   uint4* qrec = cx.qrec;
-  const double w_pre = sm.w[1], w_que = sm.w[2];
+  const double w_que = sm.w[2];
   int32_t status = 0;
   unsigned long long st_hit = 0, st_blk = 0;
 
@@ -415,7 +354,6 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
     const double t = __dmul_rn(a.scale, rec.ts_ms);
     const uint32_t n = rec.nblk, in_tok = rec.in_tok;
     const double* rtt_row = sm.rtt + (size_t)rec.origin * R;
-    const double* wrtt_row = sm.wrtt + (size_t)rec.origin * R;
 
     // ---- queue signal: drop requests that completed by t (finish <= t)
     for (uint32_t i0 = 0; i0 < R; i0 += 32) {
@@ -957,8 +895,8 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   }
 }
 
-constexpr uint32_t kWarpDecide = 0, kWarpCache = 1, kWarpProbe = 2, kWarpHelper = 3, kWarpScout0 = 4;
-constexpr uint32_t kReplayThreads = 32 * (4 + kScouts);
+constexpr uint32_t kWarpDecide = 0, kWarpCache = 1, kWarpProbe = 2, kWarpScout0 = 3;
+constexpr uint32_t kReplayThreads = 32 * (3 + kScouts);
 
 template <typename MaskT>
 __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayArgs a) {
@@ -1064,7 +1002,6 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   if (warp == kWarpDecide) decide_warp<MaskT>(a, cx, p, lane);
   else if (warp == kWarpCache) cache_warp<MaskT>(a, cx, p, lane);
   else if (warp == kWarpProbe) probe_warp<MaskT>(a, cx, lane);
-  else if (warp == kWarpHelper) helper_warp<MaskT>(a, sm, cx.mask, cx.lru_next, lane);
   else scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, warp - kWarpScout0);
   __syncthreads();
 
