@@ -673,7 +673,8 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     if (!posted && !bad0 && !*cx.probe_gone) {
       uint32_t polls = 0;
       while (cx.st_ready[slot] != r + 1 && !*cx.probe_gone && polls < 4096) { ++polls; __nanosleep(20); }
-      staged = cx.st_ready[slot] == r + 1;
+      // (one lane decides: every lane must take the same path)
+      staged = __shfl_sync(kFull, cx.st_ready[slot], 0) == r + 1;
       __threadfence_block();
     }
     if (!staged) {
@@ -854,7 +855,8 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     bad3 = false;
     ps1 = ps2; ps2 = ps3; ps3 = ps4;
     posted = false;
-    if (r + 1 < end && !bad0 && cx.st_ready[(r + 1) % kStageDepth] == r + 2) {
+    if (r + 1 < end && !bad0 &&
+        __shfl_sync(kFull, cx.st_ready[(r + 1) % kStageDepth], 0) == r + 2) {
       __threadfence_block();
       hand_over((r + 1) % kStageDepth, q_nxt.nblk);
       posted = true;
