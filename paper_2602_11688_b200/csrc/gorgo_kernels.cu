@@ -156,7 +156,7 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
 constexpr int kRegChunks = 4;     // request blocks held in registers: 4 x 32 = 128
 constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
-constexpr int kScoutBatches = 2;       // touches examined per lane and scout round
+constexpr int kScoutBatches = 1;       // touches examined per lane and scout round
 constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is this close to full
 
 // Shared-memory view of one candidate's small state.
