@@ -34,6 +34,22 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
+// Optional cycle accounting of the replay warps (build with -DGORGO_PROF): every warp adds the
+// clock cycles it spends between the marks GORGO_PT(i) to counter i of its role, lane 0 adds them
+// to a global table at the end, `gorgo_prof_read` copies the table out.  Compiled out otherwise.
+#ifdef GORGO_PROF
+__device__ unsigned long long g_prof[256];
+#define GORGO_PROF_DECL long long pf_t = clock64(); unsigned long long pf[16] = {0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0};
+#define GORGO_PT(i) { const long long pf_n = clock64(); pf[i] += (unsigned long long)(pf_n - pf_t); pf_t = pf_n; }
+#define GORGO_PC(i, v) { pf[i] += (v); }
+#define GORGO_PROF_FLUSH(role) if (lane == 0) { for (int pf_i = 0; pf_i < 16; ++pf_i) atomicAdd(&g_prof[(role) * 16 + pf_i], pf[pf_i]); }
+#else
+#define GORGO_PROF_DECL
+#define GORGO_PT(i)
+#define GORGO_PC(i, v)
+#define GORGO_PROF_FLUSH(role)
+#endif
+
 __device__ __forceinline__ double d_inf() { return __longlong_as_double(0x7FF0000000000000LL); }
 
 template <typename T> struct MaskOps;
@@ -161,6 +177,7 @@ constexpr uint32_t kStages = kStageDepth + 2;          // + two stages for the r
 constexpr uint32_t kRouteRing = 32;                    // routed requests not yet served / committed
 constexpr uint32_t kExpRing = 16;                      // requests whose expiries are staged ahead
 constexpr uint32_t kInvalRing = 16;                    // > kWindow: requests whose staged read is void
+constexpr uint32_t kApplyRing = 8;                     // commits checked but not yet applied
 constexpr uint32_t kQueueWarps = 2;                    // replicas are split between them (i mod 2)
 constexpr uint32_t kProbeWarps = 2;                    // requests are split between them (r mod 2)
 constexpr uint32_t kScouts = 2;                        // scout warps (replicas split between them)
@@ -168,12 +185,15 @@ constexpr uint32_t kListCap = 256;                     // pre-validated eviction
 constexpr int kScoutBatches = 1;                       // touches examined per lane and scout round
 constexpr uint32_t kPostMargin = 512;                  // start pre-validating when a cache is this close to full
 constexpr uint32_t kSpinLimit = 1u << 24;              // polls after which a waiting warp gives up
+constexpr uint32_t kPollNs = 20;                       // pause between polls: keeps the waiting warps
+                                                       //   from flooding the shared-memory pipeline
 
 // Words of the control block (shared memory) through which the warps of a candidate pace each
 // other.  Counters hold request indices; they only grow.
 constexpr uint32_t kCtlRouted = 0;      // requests < this have a route (route warp)
 constexpr uint32_t kCtlApplied = 1;     // requests < this are fully committed to the cache state
 constexpr uint32_t kCtlChecked = 2;     // requests < this have their eviction victims determined
+constexpr uint32_t kCtlEnqueued = 3;    // requests < this have their commit handed to the apply warp
 constexpr uint32_t kCtlAbort = 4;       // a warp ran into a limit: everybody stops
 constexpr uint32_t kCtlStatus = 5;
 constexpr uint32_t kCtlProbeGone = 6;   // probe warps that have stopped
@@ -184,7 +204,10 @@ constexpr uint32_t kCtlWords = (kCtlServed + kQueueWarps + 1u) & ~1u;
 // Shared-memory view of one candidate's small state.
 struct Smem {
   double* rtt; double* wrtt; double* w; double* minfin; long long* load;
-  uint32_t* occ; uint32_t* curreq; int32_t* curpos; uint32_t* lrutail;
+  uint32_t* occ; uint32_t* curreq; int32_t* curpos;
+  volatile uint32_t* lrutail;     // last request appended to a replica's recency list (apply warp)
+  uint32_t* c_lrutail;            // last request routed to it as the check warp knows it
+  uint32_t* chead;                // ring entries taken by the check warp (>= ring_head)
   volatile uint32_t* progress;    // the kCtlApplied word
   volatile uint32_t* abort;       // the kCtlAbort word
   // eviction rings, one per replica: filled by a scout warp, drained by the cache warp.
@@ -192,7 +215,7 @@ struct Smem {
   //          position of the touch in its request, request of the touch), in eviction order
   uint4* lst;                     // [R][kListCap]
   volatile uint32_t* act;         // cache -> scout: the replica's cache is close to full
-  volatile uint32_t* ring_head;   // entries consumed (cache warp)
+  volatile uint32_t* ring_head;   // entries consumed and free for reuse (apply warp)
   volatile uint32_t* ring_tail;   // entries produced (scout warp)
   volatile uint32_t* scan_cr;     // scout's own cursor into the recency order (set at activation)
   volatile int32_t* scan_cp;
@@ -212,6 +235,7 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
   const uint32_t R = a.m.R;
   uint32_t idle = 0;
   uint32_t blocked0 = kNone - 1, blocked1 = kNone - 1;  // lru tail seen when the scan ran dry
+  GORGO_PROF_DECL
   while (true) {
     const uint32_t prog = *sm.progress;
     if (prog >= end || *sm.abort) break;
@@ -231,8 +255,10 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
     if (best == kNone || prog == a.first) {
       if (++idle > (1u << 26)) break;              // bounded wait
       __nanosleep(64);
+      GORGO_PT(0)
       continue;
     }
+    GORGO_PT(1)
     idle = 0;
     const uint32_t i = best & 255u;
     __threadfence_block();
@@ -301,7 +327,9 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
       if ((i & 31u) == lane) { if (i < 32) blocked0 = lt; else blocked1 = lt; }
     }
     __syncwarp();
+    GORGO_PT(2)
   }
+  GORGO_PROF_FLUSH(11 + which)
 }
 
 // Everything the warps of one candidate share.
@@ -318,6 +346,7 @@ struct Ctx {
   volatile uint32_t* ctl;         // [kCtlWords] control block
   volatile uint32_t* route_ring;  // [kRouteRing] replica | stage << 8 | prefix hit on it << 16
   long long* exp_sub;             // [kExpRing][R] tokens that stop being in flight at a request
+  uint4* apply_ring;              // [kApplyRing][2] work items of the apply warp (ApplyItem)
   volatile uint32_t* inval;       // [kInvalRing] request (+1) that lost a cached block to an eviction
                                   //   committed within the kWindow requests before it
   // staging of the coming requests by the probe warps (kStageDepth stages + two of the route warp)
@@ -328,6 +357,10 @@ struct Ctx {
   uint32_t* st_ids;               // [kStages][kStageBlocks] block ids
   MaskT* st_mk;                   // [kStages][kStageBlocks] mask words
 };
+
+// Keeps the compiler from moving ordinary loads above the polling of a flag that guards them
+// (the hardware issues a warp's shared-memory accesses in program order).
+__device__ __forceinline__ void compiler_fence() { asm volatile("" ::: "memory"); }
 
 // A warp that ran into a limit: record it and tell the other warps of the candidate to stop.
 __device__ __forceinline__ void give_up(volatile uint32_t* ctl, int32_t status, uint32_t lane) {
@@ -428,7 +461,9 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
     id_a[c] = (k < q_a.nblk) ? ids[q_a.off + k] : 0u;
     id_n[c] = 0u; id_b[c] = 0u; m_a[c] = (MaskT)0; m_b[c] = (MaskT)0;
   }
+  GORGO_PROF_DECL
   for (uint32_t qa = q0; qa < end + kProbeWarps; qa += kProbeWarps) {
+    GORGO_PT(0)
     if (qa > q0) {
       // stage and probe this warp's previous request (its mask words were requested a round ago)
       const uint32_t qb = qa - kProbeWarps, slot = qb % kStageDepth;
@@ -448,6 +483,7 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
       __syncwarp();
       if (lane == 0) cx.st_ready[slot] = qb + 1;
     }
+    GORGO_PT(1)
     if (qa < end) {
       // the stage of request qa is free, and its read at most kWindow commits old, once request
       // qa - kStageDepth is committed
@@ -462,6 +498,7 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
         pc = *sm.progress;
       }
       pc_a = pc;
+      GORGO_PT(2)
 #pragma unroll
       for (int c = 0; c < kRegChunks; ++c) {
         const uint32_t k = c * 32u + lane;
@@ -475,6 +512,7 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
 #pragma unroll
     for (int c = 0; c < kRegChunks; ++c) { id_b[c] = id_a[c]; m_b[c] = m_a[c]; id_a[c] = id_n[c]; }
   }
+  GORGO_PROF_FLUSH(7 + which)
 }
 
 // Route warp: the serial heart of a replay.  For request r it takes the staged prefix hits and
@@ -503,6 +541,7 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
   Ahead q0 = fetch_ahead(req, a.first, end), q1 = fetch_ahead(req, a.first + 1, end),
         q2 = fetch_ahead(req, a.first + 2, end);
 
+  GORGO_PROF_DECL
   for (uint32_t r = a.first; r < end; ++r) {
     const Ahead q = q0;
     q0 = q1; q1 = q2;
@@ -528,13 +567,21 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
         break;
       }
       if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
+      __nanosleep(kPollNs);
+#ifdef GORGO_PROF
+      if (!(mexp > r)) GORGO_PC(8, 1) else if (!(r - mserved < kRouteRing)) GORGO_PC(9, 1)
+      else if (!(ck >= r)) GORGO_PC(10, 1) else GORGO_PC(11, 1)
+#endif
     }
+    GORGO_PT(0)
     if (status) break;
+    compiler_fence();
     if (staged) {
       const uint32_t spc = cx.st_pc[slot];
       staged = (q.prev_share == kNone || q.prev_share < spc) && cx.inval[r % kInvalRing] != r + 1;
     }
     if (!staged) {
+      GORGO_PC(12, 1)
       // every earlier commit has to be in the masks before they are read here
       polls = 0;
       while (ctl[kCtlApplied] < r) {
@@ -557,6 +604,7 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
       __syncwarp();
     }
 
+    GORGO_PT(1)
     // ---- queue signal (Eq. 2): requests that completed by the arrival of r stop counting
     const volatile long long* sub = cx.exp_sub + (size_t)(r % kExpRing) * R;
     if (i0 < R) ld0 -= sub[i0];
@@ -581,7 +629,9 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
       const uint64_t ck = order_key(c);
       if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i1; }
     }
+    GORGO_PT(2)
     const uint32_t istar = warp_argmin_key(best_k, best_i);
+    GORGO_PT(3)
     const uint32_t hstar = cx.st_hits[slot * R + istar];
     if (lane == 0) {
       cx.route_ring[r % kRouteRing] = istar | (slot << 8) | (hstar << 16);
@@ -593,7 +643,9 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
     if ((istar & 31u) == lane) {
       if (istar < 32u) ld0 += (long long)q.in_tok; else ld1 += (long long)q.in_tok;
     }
+    GORGO_PT(4)
   }
+  GORGO_PROF_FLUSH(0)
   if (i0 < R) sm.load[i0] = ld0;
   if (i1 < R) sm.load[i1] = ld1;
   if (status != 0) give_up(ctl, status, lane);
@@ -650,8 +702,10 @@ __device__ __forceinline__ void queue_warp(const ReplayArgs& a, const Ctx<MaskT>
   uint32_t nd0 = a.need_svc[min(e, last_r)], nd1 = a.need_svc[min(e + 1, last_r)];
   uint32_t idle = 0;
 
+  GORGO_PROF_DECL
   while (ja < end || e < end) {
     const uint32_t routed = ctl[kCtlRouted];
+    GORGO_PT(0)
     if (e < end && e < routed + kExpRing && ja >= nd0) {
       // ---- (B) expiries at the arrival of request e
       const double t = te0;                        // = scale * ts[e]
@@ -714,6 +768,7 @@ __device__ __forceinline__ void queue_warp(const ReplayArgs& a, const Ctx<MaskT>
       te1 = a.tq[min(e + 1, last_r)];
       nd1 = a.need_svc[min(e + 1, last_r)];
       idle = 0;
+      GORGO_PT(1)
       if (__any_sync(kFull, status != 0)) break;
       continue;
     }
@@ -773,10 +828,15 @@ __device__ __forceinline__ void queue_warp(const ReplayArgs& a, const Ctx<MaskT>
       ra1 = req[min(ja + 1, last_r)];
       if (lane == 0) ctl[kCtlServed + which] = ja;
       idle = 0;
+#ifdef GORGO_PROF
+      if ((istar % kQueueWarps) == which) GORGO_PT(2) else GORGO_PT(3)
+#endif
       continue;
     }
     if (ctl[kCtlAbort] || ++idle > kSpinLimit) { status = -6; break; }
+    __nanosleep(2 * kPollNs);
   }
+  GORGO_PROF_FLUSH(3 + which)
   flush_pending();
   __syncwarp();
   status = __reduce_min_sync(kFull, status);
@@ -788,16 +848,32 @@ __device__ __forceinline__ void queue_warp(const ReplayArgs& a, const Ctx<MaskT>
   }
 }
 
-// Cache warp: commits routed request r to the chosen replica's cache: sets the replica's bit on
-// the missing blocks and evicts down to capacity (victims from the scout's ring, else by walking
-// the recency order itself).  A victim whose block occurs again in one of the next kWindow
-// requests voids that request's staged read: the request is flagged before the route warp is
-// told that the victims of r are known, which is all the route warp waits for.
+// The cache commit of a routed request is split between two warps.
+//
+// Check warp (on the serial path): from the staged mask words of request r it counts the blocks
+// missing on the chosen replica, sizes the eviction and takes the victims from the head of the
+// replica's ring.  A victim whose block occurs again in one of the next kWindow requests voids
+// that request's staged read: the request is flagged before the route warp is told that the
+// victims of r are known, which is all the route warp waits for.  In the common case this warp
+// touches shared memory only; the memory traffic of the commit is left to the apply warp as a
+// work item.  If the ring cannot serve the eviction as it stands (the scout is behind, or an
+// entry went stale), the warp waits until every earlier commit is applied and evicts by the
+// general procedure itself.
+//
+// Apply warp (behind): sets the replica's bit on the missing blocks, clears it on the victims,
+// appends the request to the replica's recency list and publishes the request as committed.
+struct ApplyItem {
+  uint32_t route;     // replica | stage << 8
+  uint32_t head0;     // ring index of the first victim left to this warp
+  uint32_t nvict;     // victims left to this warp (0: the check warp evicted itself)
+  uint32_t evicted;   // victims of the request in all (statistics)
+  uint32_t lru_prev;  // previous request routed to the replica (kNone: none)
+  uint32_t nblk, off, pad;
+};
+
 template <typename MaskT>
-__device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
-                                           uint32_t lane) {
+__device__ __forceinline__ void check_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t lane) {
   const Smem& sm = cx.sm;
-  const uint32_t R = a.m.R;
   const uint32_t N = a.tr.n_req;
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
@@ -806,106 +882,205 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   const uint8_t* route_log = cx.route_log;
   volatile uint32_t* ctl = cx.ctl;
   int32_t status = 0;
-  unsigned long long st_probe = 0, st_evict = 0;
   const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
   const uint32_t end = a.first + a.count;
 
   Ahead q_cur = fetch_ahead(req, a.first, end), q_nxt = fetch_ahead(req, a.first + 1, end);
 
+  GORGO_PROF_DECL
   for (uint32_t r = a.first; r < end; ++r) {
     const uint32_t n = q_cur.nblk, off = q_cur.off;
     const Ahead q_n2 = fetch_ahead(req, r + 2, end);          // used two rounds from now
 
-    // ---- wait for the route of request r
+    // ---- wait for the route of request r (and for room in the apply ring)
     uint32_t polls = 0;
-    while (ctl[kCtlRouted] <= r) {
+    while (ctl[kCtlRouted] <= r || r - ctl[kCtlApplied] >= kApplyRing) {
       if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
+      __nanosleep(kPollNs);
     }
+    GORGO_PT(0)
     if (status) break;
+    compiler_fence();
     const uint32_t ent0 = cx.route_ring[r % kRouteRing];
     const uint32_t istar = ent0 & 255u, slot = (ent0 >> 8) & 255u;
     const MaskT bit = (MaskT)(((MaskT)1) << istar);
-    const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
     const MaskT* smk = cx.st_mk + slot * kStageBlocks;
+    GORGO_PT(6)
 
-    // ---- cache commit: set the replica's bit on the missing blocks
+    // ---- blocks of r missing on the replica
     uint32_t missing = 0;
-    for (uint32_t c = 0; c < n; c += 32) {
-      const uint32_t k = c + lane;
-      bool miss = false;
-      if (k < n) {
-        uint32_t id;
-        MaskT mv;
-        if (c < kStageBlocks) { id = sid[k]; mv = smk[k]; }
-        else { id = ids[off + k]; mv = mask_load<MaskT>(mask, id); }
-        if (!(mv & bit)) { mask_store<MaskT>(mask, id, (MaskT)(mv | bit)); miss = true; }
+#pragma unroll
+    for (int c = 0; c < kRegChunks; ++c) {
+      if ((uint32_t)c * 32u < n) {
+        const uint32_t k = (uint32_t)c * 32u + lane;
+        const bool miss = k < n && !(smk[k] & bit);
+        missing += __popc(__ballot_sync(kFull, miss));
       }
+    }
+    for (uint32_t c = kStageBlocks; c < n; c += 32) {      // longer prompts: the rest from memory
+      const uint32_t k = c + lane;
+      const bool miss = k < n && !(mask_load<MaskT>(mask, ids[off + k]) & bit);
       missing += __popc(__ballot_sync(kFull, miss));
     }
+    GORGO_PT(1)
     uint32_t occ = sm.occ[istar] + missing;
     uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
-    uint32_t evicted = 0;
+    uint32_t evicted = 0, nvict = 0;
+    GORGO_PC(9, n) GORGO_PC(10, need)
+    const uint32_t head0 = sm.chead[istar];
     if (need > 0) {
       uint32_t cr = sm.curreq[istar];
       int32_t cp = sm.curpos[istar];
-      // fast path: victims from the ring the scout warp keeps for this replica
-      if (sm.act[istar]) {
-        const uint4* lst = sm.lst + (size_t)istar * kListCap;
-        uint32_t head = sm.ring_head[istar];
-        uint32_t last_e = kNone;   // ring slot of the last entry passed that was not void
-        while (need > 0) {
-          uint32_t avail = sm.ring_tail[istar] - head;
-          for (uint32_t polls2 = 0; avail == 0 && polls2 < 64; ++polls2) {
-            __nanosleep(20);
-            avail = sm.ring_tail[istar] - head;
-          }
-          if (avail == 0) break;                          // the scout is behind: walk ourselves
-          const uint32_t m = min(avail, 32u);
-          uint4 ent = make_uint4(0, kNone, 0, 0);
-          bool odd = false;      // void (behind the cursor) or touched again since it was listed
-          if (lane < m) {
-            const uint32_t e = (head + lane) & (kListCap - 1);
-            ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
-            odd = ent.y <= r || ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
-          }
-          if (!__any_sync(kFull, odd)) {
-            // common case: the next entries are all live, the first `need` of them are victims
-            const uint32_t tk = min(need, m);
-            const bool mine = lane < tk;
+      const uint4* lst = sm.lst + (size_t)istar * kListCap;
+      // ---- common case: the next `need` ring entries are all live; they are the victims
+      bool clean = sm.act[istar] != 0;
+      if (clean) {
+        uint32_t avail = sm.ring_tail[istar] - head0;
+        for (uint32_t polls2 = 0; avail < need && polls2 < 64; ++polls2) {
+          __nanosleep(20);
+          avail = sm.ring_tail[istar] - head0;
+          GORGO_PC(11, 1)
+        }
+        clean = avail >= need;
+        compiler_fence();
+      }
+      GORGO_PT(4)
+      uint32_t last_w = 0, last_z = 0;
+      for (uint32_t o = 0; clean && o < need; o += 32) {
+        const bool mine = o + lane < need;
+        uint4 ent = make_uint4(0, kNone, 0, 0);
+        bool odd = false;        // void (behind the cursor) or touched again since it was listed
+        if (mine) {
+          const uint32_t e = (head0 + o + lane) & (kListCap - 1);
+          ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+          odd = ent.y <= r || ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
+        }
+        if (__any_sync(kFull, odd)) { clean = false; break; }
+        // a victim that occurs again within the window voids that request's staged read
+        const bool soon = mine && ent.y - (r + 1) < kWindow;
+        if (__any_sync(kFull, soon)) {
+          if (soon) cx.inval[ent.y % kInvalRing] = ent.y + 1;
+          __threadfence_block();
+        }
+        const uint32_t lastl = min(need - o, 32u) - 1u;   // lane of the last victim of the round
+        last_w = __shfl_sync(kFull, ent.w, lastl);
+        last_z = __shfl_sync(kFull, ent.z, lastl);
+      }
+      GORGO_PT(5)
+      if (clean) {
+        cr = last_w;
+        cp = (int32_t)last_z - 1;
+        evicted = nvict = need;
+        need = 0;
+        if (lane == 0) sm.chead[istar] = head0 + nvict;
+      } else {
+        GORGO_PC(8, 1)
+        // ---- general procedure, by this warp, once every earlier commit is applied
+        polls = 0;
+        while (ctl[kCtlApplied] < r) {
+          if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
+        }
+        if (status) break;
+        __threadfence_block();
+        if (sm.act[istar]) {
+          uint32_t head = head0;     // == ring_head: the apply warp has caught up
+          uint32_t last_e = kNone;   // ring slot of the last entry passed that was not void
+          while (need > 0) {
+            uint32_t avail = sm.ring_tail[istar] - head;
+            for (uint32_t polls2 = 0; avail == 0 && polls2 < 64; ++polls2) {
+              __nanosleep(20);
+              avail = sm.ring_tail[istar] - head;
+            }
+            if (avail == 0) break;                          // the scout is behind: walk ourselves
+            const uint32_t m = min(avail, 32u);
+            uint4 ent = make_uint4(0, kNone, 0, 0);
+            bool live = false;
+            uint32_t nxr = kNone;      // request of the block's next occurrence after r
+            if (lane < m) {
+              const uint32_t e = (head + lane) & (kListCap - 1);
+              ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+              nxr = ent.y;
+              // entries the eviction cursor has already passed (after a walk of our own) are void
+              live = !(ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp));
+              if (live && ent.y <= r) {
+                // the block came back since the entry was made: follow its occurrences up to r
+                uint2 c = a.tr.occ_next[req[ent.w].off + ent.z];
+                nxr = kNone;
+                while (c.x != kNone) {
+                  if (c.y > r) { nxr = c.y; break; }
+                  const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
+                  if (rr == istar) { live = false; break; }
+                  c = a.tr.occ_next[c.x];
+                }
+              }
+            }
+            const unsigned lv = __ballot_sync(kFull, live);
+            const uint32_t cnt = __popc(lv);
+            const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
             if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
-            // a victim that occurs again within the window voids that request's staged read
-            const bool soon = mine && ent.y - (r + 1) < kWindow;
-            if (__any_sync(kFull, soon)) {
-              if (soon) cx.inval[ent.y % kInvalRing] = ent.y + 1;
-              __threadfence_block();
+            {
+              const bool soon = mine && nxr - (r + 1) < kWindow;
+              if (__any_sync(kFull, soon)) {
+                if (soon) cx.inval[nxr % kInvalRing] = nxr + 1;
+                __threadfence_block();
+              }
+            }
+            // entries passed: the whole round, or up to the last victim taken
+            uint32_t passed = m, tk = cnt;
+            if (cnt > need) {
+              const unsigned take = __ballot_sync(kFull, mine);
+              passed = 32u - (uint32_t)__clz((int)take);
+              tk = need;
             }
             need -= tk;
             evicted += tk;
-            last_e = (head + tk - 1) & (kListCap - 1);
-            head += tk;
+            // the cursor moves behind the last live entry passed (void ones lie behind it already)
+            const unsigned seen = lv & (passed >= 32u ? kFull : ((1u << passed) - 1u));
+            if (seen) last_e = (head + 31u - (uint32_t)__clz((int)seen)) & (kListCap - 1);
+            head += passed;
+          }
+          if (last_e != kNone) {
+            const uint4 le = a.lists_in_smem ? lst[last_e] : __ldcg(lst + last_e);
+            cr = le.w;
+            cp = (int32_t)le.z - 1;
+          }
+          if (lane == 0) { sm.chead[istar] = head; sm.ring_head[istar] = head; }
+        }
+        uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
+        unsigned long long guard = 0;
+        while (need > 0) {
+          if (++guard > evict_guard_max) { status = -6; break; }
+          if (cp < 0) {  // this request is used up: go to the next one routed here
+            const uint32_t nx = (cr == kNone) ? kNone : lru_next[cr];
+            if (nx == kNone) { status = -6; break; }
+            cr = nx;
+            const ReqRec cre = req[cr];
+            coff = cre.off;
+            cp = (int32_t)cre.nblk - 1;
             continue;
           }
+          // examine 32 touches, deepest position first
+          const int32_t k = cp - (int32_t)lane;
           bool live = false;
-          uint32_t nxr = ent.y;      // request of the block's next occurrence after r
-          if (lane < m) {
-            // entries the eviction cursor has already passed (after a walk of our own) are void
-            live = !(ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp));
-            if (live && ent.y <= r) {
-              // the block came back since the entry was made: follow its occurrences up to r
-              uint2 c = a.tr.occ_next[req[ent.w].off + ent.z];
-              nxr = kNone;
-              while (c.x != kNone) {
-                if (c.y > r) { nxr = c.y; break; }
-                const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
-                if (rr == istar) { live = false; break; }
-                c = a.tr.occ_next[c.x];
-              }
+          uint32_t vid = 0, nxr = kNone;
+          if (k >= 0) {
+            const uint32_t g = coff + (uint32_t)k;
+            vid = ids[g];
+            uint2 c = a.tr.occ_next[g];
+            live = true;
+            while (c.x != kNone && c.y <= r) {       // later occurrences of the block, up to r
+              const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
+              if (rr == istar) { live = false; break; }
+              c = a.tr.occ_next[c.x];
             }
+            if (live && c.x != kNone) nxr = c.y;     // its next occurrence after r
           }
           const unsigned lv = __ballot_sync(kFull, live);
           const uint32_t cnt = __popc(lv);
+          // the first `need` live touches in lane order are the victims
           const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
-          if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
+          const unsigned take = __ballot_sync(kFull, mine);
+          if (mine) mask_clear_bit<MaskT>(mask, vid, bit);
           {
             const bool soon = mine && nxr - (r + 1) < kWindow;
             if (__any_sync(kFull, soon)) {
@@ -913,94 +1088,28 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
               __threadfence_block();
             }
           }
-          // entries passed: the whole round, or up to the last victim taken
-          uint32_t passed = m, tk = cnt;
-          if (cnt > need) {
-            const unsigned take = __ballot_sync(kFull, mine);
-            passed = 32u - (uint32_t)__clz((int)take);
-            tk = need;
-          }
+          cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
+          const uint32_t tk = __popc(take);
           need -= tk;
           evicted += tk;
-          // the cursor moves behind the last live entry passed (void ones lie behind it already)
-          const unsigned seen = lv & (passed >= 32u ? kFull : ((1u << passed) - 1u));
-          if (seen) last_e = (head + 31u - (uint32_t)__clz((int)seen)) & (kListCap - 1);
-          head += passed;
         }
-        if (last_e != kNone) {
-          const uint4 le = a.lists_in_smem ? lst[last_e] : __ldcg(lst + last_e);
-          cr = le.w;
-          cp = (int32_t)le.z - 1;
-        }
-        if (lane == 0) sm.ring_head[istar] = head;
-      }
-      uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
-      unsigned long long guard = 0;
-      while (need > 0) {
-        if (++guard > evict_guard_max) { status = -6; break; }
-        if (cp < 0) {  // this request is used up: go to the next one routed here
-          const uint32_t nx = (cr == kNone) ? kNone : lru_next[cr];
-          if (nx == kNone) { status = -6; break; }
-          cr = nx;
-          const ReqRec cre = req[cr];
-          coff = cre.off;
-          cp = (int32_t)cre.nblk - 1;
-          continue;
-        }
-        // examine 32 touches, deepest position first
-        const int32_t k = cp - (int32_t)lane;
-        bool live = false;
-        uint32_t vid = 0, nxr = kNone;
-        if (k >= 0) {
-          const uint32_t g = coff + (uint32_t)k;
-          vid = ids[g];
-          uint2 c = a.tr.occ_next[g];
-          live = true;
-          while (c.x != kNone && c.y <= r) {       // later occurrences of the block, up to r
-            const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
-            if (rr == istar) { live = false; break; }
-            c = a.tr.occ_next[c.x];
-          }
-          if (live && c.x != kNone) nxr = c.y;     // its next occurrence after r
-        }
-        const unsigned lv = __ballot_sync(kFull, live);
-        const uint32_t cnt = __popc(lv);
-        // the first `need` live touches in lane order are the victims
-        const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
-        const unsigned take = __ballot_sync(kFull, mine);
-        if (mine) mask_clear_bit<MaskT>(mask, vid, bit);
-        {
-          const bool soon = mine && nxr - (r + 1) < kWindow;
-          if (__any_sync(kFull, soon)) {
-            if (soon) cx.inval[nxr % kInvalRing] = nxr + 1;
-            __threadfence_block();
-          }
-        }
-        cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
-        const uint32_t tk = __popc(take);
-        need -= tk;
-        evicted += tk;
+        __threadfence_block();                            // this warp's own reductions
       }
       if (lane == 0) { sm.curreq[istar] = cr; sm.curpos[istar] = cp; }
     }
     occ -= evicted;
-    st_evict += evicted;
 
-    // ---- the victims of r are known: the route warp may go on while the bookkeeping is done
+    // ---- the victims of r are known: the route warp may go on
     __syncwarp();
     if (lane == 0) ctl[kCtlChecked] = r + 1;
+    GORGO_PT(2)
 
-    if (lane < R) { const uint32_t h = cx.st_hits[slot * R + lane]; st_probe += (h + 1 < n ? h + 1 : n); }
-    if (lane + 32u < R) { const uint32_t h = cx.st_hits[slot * R + lane + 32u]; st_probe += (h + 1 < n ? h + 1 : n); }
-
+    // ---- hand the memory traffic of the commit to the apply warp
     if (lane == 0) {
       sm.occ[istar] = occ;
-      // recency order of the replica: append this request
-      const uint32_t lt = sm.lrutail[istar];
-      if (lt != kNone) lru_next[lt] = r;
-      lru_next[r] = kNone;
+      const uint32_t lt = sm.c_lrutail[istar];
+      sm.c_lrutail[istar] = r;
       if (sm.curreq[istar] == kNone) { sm.curreq[istar] = r; sm.curpos[istar] = (int32_t)n - 1; }
-      sm.lrutail[istar] = r;
       // hand the replica to the scout warp once its cache is close to full (before that no
       // eviction has happened here, so the scout starts from the eviction cursor)
       if (!sm.act[istar] && (uint64_t)occ + kPostMargin >= a.m.C) {
@@ -1009,17 +1118,95 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         __threadfence_block();
         sm.act[istar] = 1;
       }
+      uint4* item = cx.apply_ring + (size_t)(r % kApplyRing) * 2;
+      item[0] = make_uint4(istar | (slot << 8), head0, nvict, evicted);
+      item[1] = make_uint4(lt, n, off, 0u);
+      __threadfence_block();
+      ctl[kCtlEnqueued] = r + 1;
     }
-    __threadfence_block();                                // every lane's stores and reductions
-    __syncwarp();
-    if (lane == 0) ctl[kCtlApplied] = r + 1;              // request r is fully committed
     __syncwarp();
     if (__any_sync(kFull, status != 0)) break;
+    GORGO_PT(3)
 
     q_cur = q_nxt; q_nxt = q_n2;
   }
-  st_probe = warp_sum_u64(st_probe);
+  GORGO_PROF_FLUSH(1)
   status = __reduce_min_sync(kFull, status);
+  if (status != 0) give_up(ctl, status, lane);
+}
+
+template <typename MaskT>
+__device__ __forceinline__ void apply_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
+                                           uint32_t lane) {
+  const Smem& sm = cx.sm;
+  const uint32_t R = a.m.R;
+  const uint32_t* ids = a.tr.ids;
+  MaskT* mask = cx.mask;
+  uint32_t* lru_next = cx.lru_next;
+  volatile uint32_t* ctl = cx.ctl;
+  int32_t status = 0;
+  unsigned long long st_probe = 0, st_evict = 0;
+  const uint32_t end = a.first + a.count;
+
+  GORGO_PROF_DECL
+  for (uint32_t r = a.first; r < end; ++r) {
+    uint32_t polls = 0;
+    while (ctl[kCtlEnqueued] <= r) {
+      if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
+      __nanosleep(20);
+    }
+    GORGO_PT(0)
+    if (status) break;
+    compiler_fence();
+    const uint4* item = cx.apply_ring + (size_t)(r % kApplyRing) * 2;
+    const uint4 i0 = item[0], i1 = item[1];
+    const uint32_t istar = i0.x & 255u, slot = (i0.x >> 8) & 255u;
+    const uint32_t head0 = i0.y, nvict = i0.z, n = i1.y, off = i1.z;
+    const MaskT bit = (MaskT)(((MaskT)1) << istar);
+    const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
+    const MaskT* smk = cx.st_mk + slot * kStageBlocks;
+
+    // ---- set the replica's bit on the missing blocks
+    for (uint32_t c = 0; c < n; c += 32) {
+      const uint32_t k = c + lane;
+      if (k < n) {
+        uint32_t id;
+        MaskT mv;
+        if (c < kStageBlocks) { id = sid[k]; mv = smk[k]; }
+        else { id = ids[off + k]; mv = mask_load<MaskT>(mask, id); }
+        if (!(mv & bit)) mask_store<MaskT>(mask, id, (MaskT)(mv | bit));
+      }
+    }
+    GORGO_PT(1)
+    // ---- clear it on the victims the check warp took from the ring
+    const uint4* lst = sm.lst + (size_t)istar * kListCap;
+    for (uint32_t o = lane; o < nvict; o += 32) {
+      const uint32_t e = (head0 + o) & (kListCap - 1);
+      const uint4 ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+      mask_clear_bit<MaskT>(mask, ent.x, bit);
+    }
+    if (lane < R) { const uint32_t h = cx.st_hits[slot * R + lane]; st_probe += (h + 1 < n ? h + 1 : n); }
+    if (lane + 32u < R) { const uint32_t h = cx.st_hits[slot * R + lane + 32u]; st_probe += (h + 1 < n ? h + 1 : n); }
+    st_evict += i0.w;
+    if (lane == 0) {
+      // recency order of the replica: append this request
+      if (i1.x != kNone) lru_next[i1.x] = r;
+      lru_next[r] = kNone;
+    }
+    GORGO_PT(2)
+    __threadfence_block();                                // every lane's stores and reductions
+    __syncwarp();
+    GORGO_PT(3)
+    if (lane == 0) {
+      sm.lrutail[istar] = r;
+      if (nvict) sm.ring_head[istar] = head0 + nvict;     // the scout may reuse these entries
+      ctl[kCtlApplied] = r + 1;                           // request r is fully committed
+    }
+    __syncwarp();
+    GORGO_PT(4)
+  }
+  GORGO_PROF_FLUSH(2)
+  st_probe = warp_sum_u64(st_probe);
   if (status != 0) give_up(ctl, status, lane);
   if (lane == 0 && a.stats) {
     unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
@@ -1028,14 +1215,15 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   }
 }
 
-constexpr uint32_t kWarpRoute = 0, kWarpCache = 1, kWarpQueue0 = 2,
+constexpr uint32_t kWarpRoute = 0, kWarpCheck = 1, kWarpApply = 2, kWarpQueue0 = 3,
                    kWarpProbe0 = kWarpQueue0 + kQueueWarps, kWarpScout0 = kWarpProbe0 + kProbeWarps;
 constexpr uint32_t kReplayThreads = 32 * (kWarpScout0 + kScouts);
 
 // Byte offsets of the regions of a replay CTA's dynamic shared memory.
 struct SmemPlan {
   uint32_t rtt, wrtt, w, minfin, load, slot_d, exp_sub, st_ab, ctl, occ, curreq, curpos, lrutail,
-      slot_u, act, ring_head, ring_tail, scan_cr, scan_cp, route_ring, inval, st_ready, st_pc, st_hits,
+      slot_u, act, ring_head, ring_tail, scan_cr, scan_cp, c_lrutail, chead, route_ring, inval,
+      apply_ring, st_ready, st_pc, st_hits,
       st_ids, st_mk, lst, total;
 };
 __host__ __device__ inline SmemPlan smem_plan(uint32_t R, uint32_t G, uint32_t S, uint32_t K,
@@ -1065,6 +1253,8 @@ __host__ __device__ inline SmemPlan smem_plan(uint32_t R, uint32_t G, uint32_t S
   GORGO_TAKE(ring_tail, R * 4u, 4u)
   GORGO_TAKE(scan_cr, R * 4u, 4u)
   GORGO_TAKE(scan_cp, R * 4u, 4u)
+  GORGO_TAKE(c_lrutail, R * 4u, 4u)
+  GORGO_TAKE(chead, R * 4u, 4u)
   GORGO_TAKE(route_ring, kRouteRing * 4u, 4u)
   GORGO_TAKE(inval, kInvalRing * 4u, 4u)
   GORGO_TAKE(st_ready, kStageDepth * 4u, 4u)
@@ -1072,6 +1262,7 @@ __host__ __device__ inline SmemPlan smem_plan(uint32_t R, uint32_t G, uint32_t S
   GORGO_TAKE(st_hits, kStages * R * 4u, 4u)
   GORGO_TAKE(st_ids, kStages * kStageBlocks * 4u, 4u)
   GORGO_TAKE(st_mk, kStages * kStageBlocks * mask_bytes, 8u)
+  GORGO_TAKE(apply_ring, kApplyRing * 32u, 16u)
   GORGO_TAKE(lst, lists_in_smem ? R * kListCap * 16u : 0u, 16u)
 #undef GORGO_TAKE
   p.total = (o + 15u) / 16u * 16u;
@@ -1124,7 +1315,9 @@ __global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayA
   sm.occ = reinterpret_cast<uint32_t*>(smem_raw + pl.occ);
   sm.curreq = reinterpret_cast<uint32_t*>(smem_raw + pl.curreq);
   sm.curpos = reinterpret_cast<int32_t*>(smem_raw + pl.curpos);
-  sm.lrutail = reinterpret_cast<uint32_t*>(smem_raw + pl.lrutail);
+  sm.lrutail = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.lrutail);
+  sm.c_lrutail = reinterpret_cast<uint32_t*>(smem_raw + pl.c_lrutail);
+  sm.chead = reinterpret_cast<uint32_t*>(smem_raw + pl.chead);
   sm.act = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.act);
   sm.ring_head = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.ring_head);
   sm.ring_tail = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.ring_tail);
@@ -1132,6 +1325,7 @@ __global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayA
   sm.scan_cp = reinterpret_cast<volatile int32_t*>(smem_raw + pl.scan_cp);
   cx.route_ring = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.route_ring);
   cx.inval = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.inval);
+  cx.apply_ring = reinterpret_cast<uint4*>(smem_raw + pl.apply_ring);
   cx.st_ready = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.st_ready);
   cx.st_pc = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.st_pc);
   cx.st_hits = reinterpret_cast<uint32_t*>(smem_raw + pl.st_hits);
@@ -1162,6 +1356,7 @@ __global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayA
     const RepState rs = g_rep[i];
     sm.minfin[i] = rs.min_fin; sm.load[i] = rs.load; sm.occ[i] = rs.occ;
     sm.curreq[i] = rs.cur_req; sm.curpos[i] = rs.cur_pos; sm.lrutail[i] = rs.lru_tail;
+    sm.c_lrutail[i] = rs.lru_tail; sm.chead[i] = 0;
     sm.act[i] = 0; sm.ring_head[i] = 0; sm.ring_tail[i] = 0;
   }
   if (a.slots_in_smem) {
@@ -1171,6 +1366,7 @@ __global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayA
   if (threadIdx.x < kCtlWords) {
     uint32_t v = 0;
     if (threadIdx.x == kCtlRouted || threadIdx.x == kCtlApplied || threadIdx.x == kCtlChecked ||
+        threadIdx.x == kCtlEnqueued ||
         (threadIdx.x >= kCtlExp && threadIdx.x < kCtlServed + kQueueWarps))
       v = a.first;
     cx.ctl[threadIdx.x] = v;
@@ -1180,7 +1376,8 @@ __global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayA
   __syncthreads();
 
   if (warp == kWarpRoute) route_warp<MaskT>(a, cx, lane);
-  else if (warp == kWarpCache) cache_warp<MaskT>(a, cx, p, lane);
+  else if (warp == kWarpCheck) check_warp<MaskT>(a, cx, lane);
+  else if (warp == kWarpApply) apply_warp<MaskT>(a, cx, p, lane);
   else if (warp < kWarpProbe0) queue_warp<MaskT>(a, cx, p, lane, warp - kWarpQueue0);
   else if (warp < kWarpScout0) probe_warp<MaskT>(a, cx, lane, warp - kWarpProbe0);
   else scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, warp - kWarpScout0);
@@ -1488,3 +1685,18 @@ cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st)
 }
 
 }  // namespace gorgo
+
+#ifdef GORGO_PROF
+namespace gorgo {
+int prof_read(unsigned long long* out, int clear) {
+  cudaDeviceSynchronize();
+  if (cudaMemcpyFromSymbol(out, g_prof, sizeof(g_prof)) != cudaSuccess) return -1;
+  if (clear) {
+    static unsigned long long z[256];
+    cudaMemcpyToSymbol(g_prof, z, sizeof(z));
+  }
+  return 0;
+}
+}  // namespace gorgo
+extern "C" int gorgo_prof_read(unsigned long long* out, int clear) { return gorgo::prof_read(out, clear); }
+#endif
