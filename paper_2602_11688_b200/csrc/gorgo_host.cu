@@ -86,7 +86,7 @@ StateLayout make_layout(const Model& m) {
 
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
-  uint64_t params, rtt, status, p95, need, tq, masks, states, lists, qrec, lru_next, route_log,
+  uint64_t params, rtt, status, p95, masks, states, lists, qrec, lru_next, route_log,
       ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
@@ -103,8 +103,6 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.rtt = o; o = align_up(o + (uint64_t)m.G * m.R * 8);
   w.status = o; o = align_up(o + res * 4);
   w.p95 = o; o = align_up(o + res * 16);
-  w.need = o; o = align_up(o + N * 4);
-  w.tq = o; o = align_up(o + N * 8);
   w.masks = o; o = align_up(o + res * w.mask_stride);
   w.states = o; o = align_up(o + res * w.st.bytes);
   w.lists = o; o = align_up(o + res * evict_list_bytes(m.R));
@@ -197,8 +195,6 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
     a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
     a.route_log = route ? route + (size_t)p0 * N : base + w.route_log;
     a.route_log_stride = N;
-    a.need_svc = reinterpret_cast<uint32_t*>(base + w.need);
-    a.tq = reinterpret_cast<double*>(base + w.tq);
     a.route_out = nullptr;
     a.hit_out = hit ? hit + (size_t)p0 * N : nullptr;
     a.ttft_out = reinterpret_cast<double*>(base + w.ttft);
@@ -493,8 +489,6 @@ int gorgo_route_batch(gorgo_sim_t* sim, const double* params, double time_scale,
   a.qrec = reinterpret_cast<uint4*>(base + w.qrec);
   a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
   a.route_log = base + w.route_log; a.route_log_stride = N;
-  a.need_svc = reinterpret_cast<uint32_t*>(base + w.need);
-  a.tq = reinterpret_cast<double*>(base + w.tq);
   a.route_out = route; a.hit_out = hit_blocks; a.ttft_out = ttft_ms; a.e2e_out = e2e_ms;
   a.out_stride = count;
   a.stats = nullptr; a.status_out = nullptr;

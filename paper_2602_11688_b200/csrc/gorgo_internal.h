@@ -88,10 +88,6 @@ struct ReplayArgs {
   uint32_t* lru_next;             // next request routed to the same replica
   uint8_t* route_log;             // chosen replica of every request replayed so far
   uint64_t route_log_stride;      // elements between candidates
-  uint32_t* need_svc;             // [N] scratch shared by the candidates of a launch: per request,
-                                  //   one past the last earlier request that can have finished
-                                  //   by its arrival (filled by the launcher)
-  double* tq;                     // [N] scratch, same sharing: scaled arrival time of each request
   // outputs, candidate p at + p*out_stride, request r at + (r-first); any may be null
   uint8_t* route_out;
   uint16_t* hit_out;

@@ -34,22 +34,6 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
-// Optional cycle accounting of the replay warps (build with -DGORGO_PROF): every warp adds the
-// clock cycles it spends between the marks GORGO_PT(i) to counter i of its role, lane 0 adds them
-// to a global table at the end, `gorgo_prof_read` copies the table out.  Compiled out otherwise.
-#ifdef GORGO_PROF
-__device__ unsigned long long g_prof[256];
-#define GORGO_PROF_DECL long long pf_t = clock64(); unsigned long long pf[16] = {0,0,0,0,0,0,0,0,0,0,0,0,0,0,0,0};
-#define GORGO_PT(i) { const long long pf_n = clock64(); pf[i] += (unsigned long long)(pf_n - pf_t); pf_t = pf_n; }
-#define GORGO_PC(i, v) { pf[i] += (v); }
-#define GORGO_PROF_FLUSH(role) if (lane == 0) { for (int pf_i = 0; pf_i < 16; ++pf_i) atomicAdd(&g_prof[(role) * 16 + pf_i], pf[pf_i]); }
-#else
-#define GORGO_PROF_DECL
-#define GORGO_PT(i)
-#define GORGO_PC(i, v)
-#define GORGO_PROF_FLUSH(role)
-#endif
-
 __device__ __forceinline__ double d_inf() { return __longlong_as_double(0x7FF0000000000000LL); }
 
 template <typename T> struct MaskOps;
@@ -169,53 +153,23 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
   __stcg(reinterpret_cast<unsigned long long*>(mask) + id, (unsigned long long)v);
 }
 
-constexpr int kRegChunks = 8;                          // 32-block chunks of a request a probe warp holds
-constexpr uint32_t kStageBlocks = kRegChunks * 32u;    // blocks of a request kept per stage
-constexpr uint32_t kStageDepth = 8;                    // requests staged ahead of the cache warp
-constexpr uint32_t kWindow = kStageDepth - 1;          // a staged read is at most this many commits old
-constexpr uint32_t kStages = kStageDepth + 2;          // + two stages for the route warp's own probes
-constexpr uint32_t kRouteRing = 32;                    // routed requests not yet served / committed
-constexpr uint32_t kExpRing = 16;                      // requests whose expiries are staged ahead
-constexpr uint32_t kInvalRing = 16;                    // > kWindow: requests whose staged read is void
-constexpr uint32_t kApplyRing = 8;                     // commits checked but not yet applied
-constexpr uint32_t kQueueWarps = 2;                    // replicas are split between them (i mod 2)
-constexpr uint32_t kProbeWarps = 2;                    // requests are split between them (r mod 2)
-constexpr uint32_t kScouts = 2;                        // scout warps (replicas split between them)
-constexpr uint32_t kListCap = 256;                     // pre-validated eviction victims kept per replica
-constexpr int kScoutBatches = 1;                       // touches examined per lane and scout round
-constexpr uint32_t kPostMargin = 512;                  // start pre-validating when a cache is this close to full
-constexpr uint32_t kSpinLimit = 1u << 24;              // polls after which a waiting warp gives up
-constexpr uint32_t kPollNs = 20;                       // pause between polls: keeps the waiting warps
-                                                       //   from flooding the shared-memory pipeline
-
-// Words of the control block (shared memory) through which the warps of a candidate pace each
-// other.  Counters hold request indices; they only grow.
-constexpr uint32_t kCtlRouted = 0;      // requests < this have a route (route warp)
-constexpr uint32_t kCtlApplied = 1;     // requests < this are fully committed to the cache state
-constexpr uint32_t kCtlChecked = 2;     // requests < this have their eviction victims determined
-constexpr uint32_t kCtlEnqueued = 3;    // requests < this have their commit handed to the apply warp
-constexpr uint32_t kCtlAbort = 4;       // a warp ran into a limit: everybody stops
-constexpr uint32_t kCtlStatus = 5;
-constexpr uint32_t kCtlProbeGone = 6;   // probe warps that have stopped
-constexpr uint32_t kCtlExp = 8;         // [kQueueWarps] requests < this have their expiries staged
-constexpr uint32_t kCtlServed = kCtlExp + kQueueWarps;   // [kQueueWarps] requests < this are booked
-constexpr uint32_t kCtlWords = (kCtlServed + kQueueWarps + 1u) & ~1u;
+constexpr int kRegChunks = 4;     // request blocks held in registers: 4 x 32 = 128
+constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
+constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
+constexpr int kScoutBatches = 1;       // touches examined per lane and scout round
+constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is this close to full
 
 // Shared-memory view of one candidate's small state.
 struct Smem {
   double* rtt; double* wrtt; double* w; double* minfin; long long* load;
-  uint32_t* occ; uint32_t* curreq; int32_t* curpos;
-  volatile uint32_t* lrutail;     // last request appended to a replica's recency list (apply warp)
-  uint32_t* c_lrutail;            // last request routed to it as the check warp knows it
-  uint32_t* chead;                // ring entries taken by the check warp (>= ring_head)
-  volatile uint32_t* progress;    // the kCtlApplied word
-  volatile uint32_t* abort;       // the kCtlAbort word
-  // eviction rings, one per replica: filled by a scout warp, drained by the cache warp.
+  uint32_t* occ; uint32_t* curreq; int32_t* curpos; uint32_t* lrutail;
+  volatile uint32_t* progress;
+  // eviction rings, one per replica: filled by the scout warp, drained by the replay warp.
   // entry = (block id, request of the block's next occurrence after the entry was made or kNone,
   //          position of the touch in its request, request of the touch), in eviction order
   uint4* lst;                     // [R][kListCap]
-  volatile uint32_t* act;         // cache -> scout: the replica's cache is close to full
-  volatile uint32_t* ring_head;   // entries consumed and free for reuse (apply warp)
+  volatile uint32_t* act;         // replay -> scout: the replica's cache is close to full
+  volatile uint32_t* ring_head;   // entries consumed (replay warp)
   volatile uint32_t* ring_tail;   // entries produced (scout warp)
   volatile uint32_t* scan_cr;     // scout's own cursor into the recency order (set at activation)
   volatile int32_t* scan_cp;
@@ -223,9 +177,9 @@ struct Smem {
 
 // Scout warp: for every replica whose cache is close to full it walks the recency order ahead
 // of the eviction cursor and appends to the replica's ring the touches that are still the latest
-// touch of their block (the coming eviction victims, in order).  The cache warp evicts from the
-// ring instead of validating touches itself; entries that went stale after they were appended
-// are recognised there by their next-occurrence field.
+// touch of their block (the coming eviction victims, in order).  The replay warp evicts from the
+// ring instead of validating touches on its critical path; entries that went stale after they
+// were appended are recognised there by their next-occurrence field.
 template <typename MaskT>
 __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* lru_next,
                            const uint8_t* route_log, uint32_t lane, uint32_t which) {
@@ -235,10 +189,9 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
   const uint32_t R = a.m.R;
   uint32_t idle = 0;
   uint32_t blocked0 = kNone - 1, blocked1 = kNone - 1;  // lru tail seen when the scan ran dry
-  GORGO_PROF_DECL
   while (true) {
     const uint32_t prog = *sm.progress;
-    if (prog >= end || *sm.abort) break;
+    if (prog >= end) break;
     // the active replica with the emptiest ring that can still be extended
     uint32_t best = kNone;
 #pragma unroll
@@ -255,10 +208,8 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
     if (best == kNone || prog == a.first) {
       if (++idle > (1u << 26)) break;              // bounded wait
       __nanosleep(64);
-      GORGO_PT(0)
       continue;
     }
-    GORGO_PT(1)
     idle = 0;
     const uint32_t i = best & 255u;
     __threadfence_block();
@@ -315,7 +266,6 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
       }
       cp -= 32 * kScoutBatches;
       __threadfence_block();
-      __syncwarp();
       if (lane == 0) {
         sm.scan_cr[i] = cr;
         sm.scan_cp[i] = cp;
@@ -327,10 +277,25 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
       if ((i & 31u) == lane) { if (i < 32) blocked0 = lt; else blocked1 = lt; }
     }
     __syncwarp();
-    GORGO_PT(2)
   }
-  GORGO_PROF_FLUSH(11 + which)
 }
+
+// Holds the compiler back where shared-memory data is handed from one warp to another through a
+// flag: a warp's shared-memory accesses are performed in program order, and a hardware fence
+// would also wait for the warp's global loads in flight, which the pipelines below avoid.
+__device__ __forceinline__ void smem_order() { asm volatile("" ::: "memory"); }
+
+// Named CTA barriers pairing the decide warp and the cache warp (32 + 32 threads each).  The
+// barrier itself orders the arriving warp's earlier memory accesses before the waiting warp's
+// later ones.
+__device__ __forceinline__ void bar_arrive(int id) {
+  asm volatile("bar.arrive %0, 64;" ::"r"(id) : "memory");
+}
+__device__ __forceinline__ void bar_wait(int id) {
+  asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
+}
+constexpr int kBarHits = 1;    // cache warp -> decide warp: prefix hits of the request are posted
+constexpr int kBarRoute = 2;   // decide warp -> cache warp: the chosen replica is posted
 
 // Everything the warps of one candidate share.
 template <typename MaskT>
@@ -343,32 +308,203 @@ struct Ctx {
   // per-slot state (shared or global memory)
   double *free_at, *q0_fin, *q1_fin;
   uint32_t *q0_tok, *q1_tok, *q2_idx, *tail, *qcnt;
-  volatile uint32_t* ctl;         // [kCtlWords] control block
-  volatile uint32_t* route_ring;  // [kRouteRing] replica | stage << 8 | prefix hit on it << 16
-  long long* exp_sub;             // [kExpRing][R] tokens that stop being in flight at a request
-  uint4* apply_ring;              // [kApplyRing][2] work items of the apply warp (ApplyItem)
-  volatile uint32_t* inval;       // [kInvalRing] request (+1) that lost a cached block to an eviction
-                                  //   committed within the kWindow requests before it
-  // staging of the coming requests by the probe warps (kStageDepth stages + two of the route warp)
-  volatile uint32_t* st_ready;    // [kStageDepth] request (+1) whose data the stage holds
-  volatile uint32_t* st_pc;       // [kStageDepth] requests known committed before the masks were read
-  uint32_t* st_hits;              // [kStages][R] prefix hits
-  double* st_ab;                  // [kStages][R] (w_net*RTT + w_prefill*uncached) per replica
-  uint32_t* st_ids;               // [kStages][kStageBlocks] block ids
-  MaskT* st_mk;                   // [kStages][kStageBlocks] mask words
+  volatile uint32_t* route;    // chosen replica of the current request
+  volatile int32_t* status;    // first device-side limit hit by any warp
+  // staging of the coming requests by the probe warp (kStageDepth stages + one of the cache warp)
+  volatile uint32_t* st_ready; // [kStageDepth] request (+1) whose data the stage holds
+  volatile uint32_t* probe_gone;  // the probe warp has stopped
+  // (stages kStageDepth and kStageDepth+1 belong to the cache warp, used alternately)
+  uint32_t* st_hits;           // [kStageDepth+2][R] prefix hits
+  double* st_ab;               // [kStageDepth+2][R] (w_net*RTT + w_prefill*uncached) per replica
+  uint32_t* st_ids;            // [kStageDepth+2][kStageBlocks] block ids
+  MaskT* st_mk;                // [kStageDepth+2][kStageBlocks] mask words
+  volatile uint32_t* hit_slot; // stage that holds the current request's hits and scores
 };
 
-// Keeps the compiler from moving ordinary loads above the polling of a flag that guards them
-// (the hardware issues a warp's shared-memory accesses in program order).
-__device__ __forceinline__ void compiler_fence() { asm volatile("" ::: "memory"); }
+// Decide warp: queue signal, score, argmin, service model (paper Eq. 1-3).  Waits for the cache
+// warp's prefix hits of request r, publishes the route, then books the request on a slot.
+template <typename MaskT>
+__device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
+  const Smem& sm = cx.sm;
+  const uint32_t R = a.m.R, S = a.m.S, K = a.m.K;
+  const uint32_t N = a.tr.n_req;
+  const ReqRec* req = a.tr.req;
+  double *free_at = cx.free_at, *q0_fin = cx.q0_fin, *q1_fin = cx.q1_fin;
+  uint32_t *q0_tok = cx.q0_tok, *q1_tok = cx.q1_tok, *q2_idx = cx.q2_idx, *tail = cx.tail,
+           *qcnt = cx.qcnt;
+  uint4* qrec = cx.qrec;
+  const double w_que = sm.w[2];
+  int32_t status = 0;
+  unsigned long long st_hit = 0, st_blk = 0;
 
-// A warp that ran into a limit: record it and tell the other warps of the candidate to stop.
-__device__ __forceinline__ void give_up(volatile uint32_t* ctl, int32_t status, uint32_t lane) {
+  const uint32_t last_r = a.first + a.count - 1;
+  ReqRec rec_cur = req[a.first];
+  ReqRec rec_nxt = req[min(a.first + 1, last_r)];
+  // a queue refill whose load is in flight: slot index (kNone: none) and the record read
+  uint32_t pend_x = kNone;
+  uint4 pend_rec = make_uint4(0, 0, 0, 0);
+  auto flush_pending = [&]() {
+    if (pend_x != kNone) {
+      q1_fin[pend_x] = __hiloint2double((int)pend_rec.y, (int)pend_rec.x);
+      q2_idx[pend_x] = pend_rec.z;
+      q1_tok[pend_x] = pend_rec.w;
+      pend_x = kNone;
+    }
+  };
+
+  for (uint32_t j = 0; j < a.count; ++j) {
+    const uint32_t r = a.first + j;
+    const ReqRec rec = rec_cur;
+    rec_cur = rec_nxt;
+    rec_nxt = req[min(r + 2, last_r)];                   // in flight while this request runs
+    const double t = __dmul_rn(a.scale, rec.ts_ms);
+    const uint32_t n = rec.nblk, in_tok = rec.in_tok;
+    const double* rtt_row = sm.rtt + (size_t)rec.origin * R;
+
+    // ---- queue signal: drop requests that completed by t (finish <= t)
+    for (uint32_t i0 = 0; i0 < R; i0 += 32) {
+      const uint32_t i = i0 + lane;
+      unsigned due = __ballot_sync(kFull, i < R && sm.minfin[i] <= t);
+      while (due) {
+        const uint32_t ii = i0 + (uint32_t)__ffs((int)due) - 1;
+        due &= due - 1;
+        long long tok = 0;
+        double mn = d_inf();
+        for (uint32_t s = lane; s < S; s += 32) {
+          const uint32_t x = ii * S + s;
+          double hf = q0_fin[x];
+          if (hf <= t) {
+            uint32_t guard = 0;
+            uint32_t cnt = qcnt[x];
+            do {
+              if (pend_x == x) flush_pending();           // the second entry is still in flight
+              tok += (long long)q0_tok[x];
+              --cnt;
+              if (cnt == 0) { hf = d_inf(); }
+              else {
+                hf = q1_fin[x];                            // the second becomes the oldest
+                q0_tok[x] = q1_tok[x];
+                if (cnt >= 2) {                            // fetch the new second: consumed later
+                  flush_pending();
+                  pend_rec = qrec[q2_idx[x]];
+                  pend_x = x;
+                }
+              }
+              if (++guard > N) { status = -6; break; }
+            } while (hf <= t);
+            q0_fin[x] = hf;
+            qcnt[x] = cnt;
+          }
+          mn = fmin(mn, hf);
+        }
+        if (tok != 0)
+          atomicAdd(reinterpret_cast<unsigned long long*>(sm.load + ii), (unsigned long long)(-tok));
+        uint64_t mk = order_key(mn);
+        warp_argmin_key(mk, lane);
+        if (lane == 0) sm.minfin[ii] = order_value(mk);
+      }
+    }
+    __syncwarp();
+
+    // ---- the queue part of the score does not need the prefix hits
+    double cq0 = 0.0, cq1 = 0.0;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const uint32_t i = lane + 32u * half;
+      if (i < R) {
+        double q = (double)sm.load[i];
+        if (K != 3) q = __dmul_rn(q, sm.w[3 + i]);
+        const double c = __dmul_rn(w_que, q);
+        if (half) cq1 = c; else cq0 = c;
+      }
+    }
+
+    bar_wait(kBarHits);                                   // prefix hits of request r are posted
+
+    // ---- score of Eq. 3 (fixed order, no FMA): the staged (w_net*RTT + w_prefill*uncached)
+    //      plus the queue term; lowest-index argmin
+    const uint32_t stage = *cx.hit_slot;
+    uint64_t best_k = ~0ull;
+    uint32_t best_i = kNone;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const uint32_t i = lane + 32u * half;
+      if (i < R) {
+        double c = __dadd_rn(cx.st_ab[stage * R + i], half ? cq1 : cq0);
+        if (c != c) c = (i == 0) ? -d_inf() : d_inf();  // a NaN score wins only at index 0
+        const uint64_t ck = order_key(c);
+        if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i; }
+      }
+    }
+    const uint32_t istar = warp_argmin_key(best_k, best_i);
+    const uint32_t hstar = cx.st_hits[stage * R + istar];   // read before the stage can be reused
+    if (lane == 0) {
+      *cx.route = istar;
+      cx.route_log[r] = (uint8_t)istar;
+    }
+    bar_arrive(kBarRoute);                                // the cache warp may commit request r
+
+    const unsigned long long hbstar = (unsigned long long)hstar * a.m.B;
+    const uint32_t uncstar = in_tok - (uint32_t)(hbstar < in_tok ? hbstar : in_tok);
+
+    // ---- service commit: earliest-free slot, lowest index on ties
+    uint64_t bk = ~0ull;
+    uint32_t bs = kNone;
+    for (uint32_t s = lane; s < S; s += 32) {
+      const uint64_t vk = order_key(free_at[(size_t)istar * S + s]);
+      if (vk < bk || bs == kNone) { bk = vk; bs = s; }
+    }
+    bs = warp_argmin_key(bk, bs);
+    const double bv = free_at[(size_t)istar * S + bs];
+    const double arrive = __dadd_rn(t, rtt_row[istar]);
+    const double start = (bv > arrive) ? bv : arrive;
+    const double first = __dadd_rn(start, __dmul_rn(a.m.prefill_ms, (double)uncstar));
+    const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
+    const double finish = __dadd_rn(first, __dmul_rn(a.m.tpot_ms, (double)dec_tok));
+
+    flush_pending();
+    __syncwarp();
+    if (lane == 0) {
+      const size_t x = (size_t)istar * S + bs;
+      qrec[r] = make_uint4((uint32_t)__double2loint(finish), (uint32_t)__double2hiint(finish),
+                           kNone, in_tok);
+      const uint32_t cnt = qcnt[x];
+      if (cnt == 0) {
+        q0_fin[x] = finish; q0_tok[x] = in_tok;
+        sm.minfin[istar] = fmin(sm.minfin[istar], finish);
+      } else {
+        reinterpret_cast<uint32_t*>(qrec + tail[x])[2] = r;     // link behind the newest
+        if (cnt == 1) { q1_fin[x] = finish; q1_tok[x] = in_tok; q2_idx[x] = kNone; }
+        else if (cnt == 2) q2_idx[x] = r;
+      }
+      qcnt[x] = cnt + 1;
+      tail[x] = r;
+      free_at[x] = finish;
+      sm.load[istar] += (long long)in_tok;
+      const size_t o = (size_t)p * a.out_stride + j;
+      if (a.route_out) a.route_out[o] = (uint8_t)istar;
+      if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
+      if (a.ttft_out) a.ttft_out[o] = __dsub_rn(first, t);
+      if (a.e2e_out) a.e2e_out[o] = __dsub_rn(finish, t);
+      st_hit += hstar; st_blk += n;
+    }
+    __syncwarp();
+  }
+  flush_pending();
+  status = __reduce_min_sync(kFull, status);
   if (lane == 0) {
-    atomicMin(const_cast<int32_t*>(reinterpret_cast<volatile int32_t*>(ctl + kCtlStatus)), status);
-    ctl[kCtlAbort] = 1;
+    if (status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
+    if (a.stats) {
+      unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
+      atomicAdd(s4 + 1, st_hit);
+      atomicAdd(s4 + 2, st_blk);
+    }
   }
 }
+
+constexpr uint32_t kStageDepth = 4;                    // requests staged by the probe warp
+constexpr uint32_t kStageBlocks = kRegChunks * 32u;    // blocks of a request kept per stage
+constexpr uint32_t kWindow = 3;   // a staged read may be up to this many commits old
 
 // What a warp needs to know of a request ahead of time.
 struct Ahead { uint32_t off, nblk, prev_share, in_tok, origin; };
@@ -433,40 +569,50 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
   }
 }
 
-// Probe warp `which` of kProbeWarps: works on requests first+which, first+which+kProbeWarps, ...
-// up to kWindow requests ahead of the cache warp.  For request q it reads the block ids and the
-// mask words (first kStageBlocks blocks), stages them in shared memory, probes them and publishes
-// the prefix hits together with the number of requests known to be committed when the masks
-// were read.  Commits after that number may or may not show in the read; the route warp uses the
-// stage only if none of them can have touched a block of q, else it repeats the probe itself,
-// so results never depend on the timing of this warp, which may also stop at any time.
+// Probe warp: runs up to kWindow requests ahead of the cache warp.  For request q it reads the
+// block ids and the mask words (first kStageBlocks blocks), stages them in shared memory, probes
+// them and publishes the prefix hits.  Its reads may predate the commits of the last kWindow
+// requests; the cache warp knows which of those commits can have touched request q and then
+// repeats the work itself, so this warp is an accelerator only and may stop at any time.
 template <typename MaskT>
 __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>& cx,
-                                           uint32_t lane, uint32_t which) {
+                                           uint32_t lane) {
   const Smem& sm = cx.sm;
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
   const MaskT* mask = cx.mask;
   const uint32_t R = a.m.R;
   const uint32_t end = a.first + a.count;
-  const uint32_t q0 = a.first + which;
-  Ahead q_a = fetch_ahead(req, q0, end), q_n = fetch_ahead(req, q0 + kProbeWarps, end);
+  Ahead q_a = fetch_ahead(req, a.first, end), q_n = fetch_ahead(req, a.first + 1, end);
   Ahead q_b = q_a;
   uint32_t id_a[kRegChunks], id_n[kRegChunks], id_b[kRegChunks];
   MaskT m_a[kRegChunks], m_b[kRegChunks];
-  uint32_t pc_a = 0, pc_b = 0;
 #pragma unroll
   for (int c = 0; c < kRegChunks; ++c) {
     const uint32_t k = c * 32u + lane;
     id_a[c] = (k < q_a.nblk) ? ids[q_a.off + k] : 0u;
-    id_n[c] = 0u; id_b[c] = 0u; m_a[c] = (MaskT)0; m_b[c] = (MaskT)0;
+    id_b[c] = 0u; m_b[c] = (MaskT)0;
   }
-  GORGO_PROF_DECL
-  for (uint32_t qa = q0; qa < end + kProbeWarps; qa += kProbeWarps) {
-    GORGO_PT(0)
-    if (qa > q0) {
-      // stage and probe this warp's previous request (its mask words were requested a round ago)
-      const uint32_t qb = qa - kProbeWarps, slot = qb % kStageDepth;
+  for (uint32_t qa = a.first; qa <= end; ++qa) {
+    if (qa < end) {
+      // room: the stage of request qa is free and its read is at most kWindow commits old once
+      // request qa - kWindow - 1 is committed, i.e. progress >= qa - kWindow
+      uint32_t polls = 0;
+      while ((int32_t)(*sm.progress - qa) < -(int32_t)kWindow) {
+        if (++polls > (1u << 22)) { *cx.probe_gone = 1; return; }   // bounded wait
+        __nanosleep(20);
+      }
+#pragma unroll
+      for (int c = 0; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        m_a[c] = (k < q_a.nblk) ? mask_load<MaskT>(mask, id_a[c]) : (MaskT)0;
+        id_n[c] = (k < q_n.nblk) ? ids[q_n.off + k] : 0u;     // ids of the request after
+      }
+    }
+    const Ahead q_nn = fetch_ahead(req, qa + 2, end);
+    if (qa > a.first) {
+      // stage and probe the previous request (its mask words were requested one round ago)
+      const uint32_t qb = qa - 1, slot = qb % kStageDepth;
       uint32_t* sid = cx.st_ids + slot * kStageBlocks;
       MaskT* smk = cx.st_mk + slot * kStageBlocks;
 #pragma unroll
@@ -478,638 +624,258 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
       uint32_t h0, h1;
       probe_staged<MaskT>(smk, mask, ids, q_b, R, lane, h0, h1);
       stage_scores<MaskT>(a, cx, q_b, slot, h0, h1, lane);
-      if (lane == 0) cx.st_pc[slot] = pc_b;
-      __threadfence_block();                  // (no load of this warp is in flight here)
+      smem_order();
       __syncwarp();
       if (lane == 0) cx.st_ready[slot] = qb + 1;
     }
-    GORGO_PT(1)
-    if (qa < end) {
-      // the stage of request qa is free, and its read at most kWindow commits old, once request
-      // qa - kStageDepth is committed
-      uint32_t polls = 0;
-      uint32_t pc = *sm.progress;
-      while ((int32_t)(pc - qa) <= -(int32_t)kStageDepth) {
-        if (*sm.abort || ++polls > (1u << 22)) {           // bounded wait
-          if (lane == 0) atomicAdd(const_cast<uint32_t*>(cx.ctl + kCtlProbeGone), 1u);
-          return;
-        }
-        __nanosleep(20);
-        pc = *sm.progress;
-      }
-      pc_a = pc;
-      GORGO_PT(2)
-#pragma unroll
-      for (int c = 0; c < kRegChunks; ++c) {
-        const uint32_t k = c * 32u + lane;
-        m_a[c] = (k < q_a.nblk) ? mask_load<MaskT>(mask, id_a[c]) : (MaskT)0;
-        id_n[c] = (k < q_n.nblk) ? ids[q_n.off + k] : 0u;     // ids of this warp's next request
-      }
-    }
-    const Ahead q_nn = fetch_ahead(req, qa + 2 * kProbeWarps, end);
     q_b = q_a; q_a = q_n; q_n = q_nn;
-    pc_b = pc_a;
 #pragma unroll
     for (int c = 0; c < kRegChunks; ++c) { id_b[c] = id_a[c]; m_b[c] = m_a[c]; id_a[c] = id_n[c]; }
   }
-  GORGO_PROF_FLUSH(7 + which)
 }
 
-// Route warp: the serial heart of a replay.  For request r it takes the staged prefix hits and
-// hit-dependent score terms, applies the staged expiries to the in-flight token counts (kept in
-// registers: lane i owns replicas i and i+32), adds the queue term of Eq. 3, takes the
-// lowest-index argmin and publishes the route.  Everything else (service model, cache commit)
-// happens behind it in other warps.  A stage is used only if no commit since its masks were read
-// can have touched the request: no request since then shares a block with it (static field
-// `prev_share`) and the cache warp has not flagged the request (a block evicted by one of the
-// last kWindow commits occurs in it).  Otherwise the warp waits for the cache warp and probes
-// the request itself.
+// Cache warp: takes the staged prefix hits of request r (or reads and probes the mask words
+// itself when a recent commit can have changed them), and, once the route is known, does the
+// LRU commit on the chosen replica: set its bit on the missing blocks, evict down to capacity.
 template <typename MaskT>
-__device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t lane) {
+__device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
+                                           uint32_t lane) {
   const Smem& sm = cx.sm;
-  const uint32_t R = a.m.R, K = a.m.K;
-  const uint32_t end = a.first + a.count;
-  const ReqRec* req = a.tr.req;
-  const uint32_t* ids = a.tr.ids;
-  volatile uint32_t* ctl = cx.ctl;
-  const double w_que = sm.w[2];
-  const uint32_t i0 = lane, i1 = lane + 32u;
-  const double nrm0 = (K != 3 && i0 < R) ? sm.w[3 + i0] : 1.0;
-  const double nrm1 = (K != 3 && i1 < R) ? sm.w[3 + i1] : 1.0;
-  long long ld0 = i0 < R ? sm.load[i0] : 0, ld1 = i1 < R ? sm.load[i1] : 0;
-  int32_t status = 0;
-  Ahead q0 = fetch_ahead(req, a.first, end), q1 = fetch_ahead(req, a.first + 1, end),
-        q2 = fetch_ahead(req, a.first + 2, end);
-
-  GORGO_PROF_DECL
-  for (uint32_t r = a.first; r < end; ++r) {
-    const Ahead q = q0;
-    q0 = q1; q1 = q2;
-    q2 = fetch_ahead(req, r + 3, end);                   // in flight while three requests run
-    uint32_t slot = r % kStageDepth;
-
-    // ---- wait: expiries of r staged, room in the route ring, every earlier commit checked,
-    //      the stage of r filled (or no probe warp left to fill it)
-    uint32_t polls = 0;
-    bool staged = false;
-    while (true) {
-      uint32_t mexp = ctl[kCtlExp], mserved = ctl[kCtlServed];
-#pragma unroll
-      for (uint32_t w = 1; w < kQueueWarps; ++w) {
-        mexp = min(mexp, ctl[kCtlExp + w]);
-        mserved = min(mserved, ctl[kCtlServed + w]);
-      }
-      const uint32_t ck = ctl[kCtlChecked];
-      const uint32_t sready = cx.st_ready[slot];
-      const uint32_t gone = ctl[kCtlProbeGone];
-      if (mexp > r && r - mserved < kRouteRing && ck >= r && (sready == r + 1 || gone)) {
-        staged = sready == r + 1;
-        break;
-      }
-      if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
-      __nanosleep(kPollNs);
-#ifdef GORGO_PROF
-      if (!(mexp > r)) GORGO_PC(8, 1) else if (!(r - mserved < kRouteRing)) GORGO_PC(9, 1)
-      else if (!(ck >= r)) GORGO_PC(10, 1) else GORGO_PC(11, 1)
-#endif
-    }
-    GORGO_PT(0)
-    if (status) break;
-    compiler_fence();
-    if (staged) {
-      const uint32_t spc = cx.st_pc[slot];
-      staged = (q.prev_share == kNone || q.prev_share < spc) && cx.inval[r % kInvalRing] != r + 1;
-    }
-    if (!staged) {
-      GORGO_PC(12, 1)
-      // every earlier commit has to be in the masks before they are read here
-      polls = 0;
-      while (ctl[kCtlApplied] < r) {
-        if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
-      }
-      if (status) break;
-      __threadfence_block();
-      slot = kStageDepth + (r & 1u);
-      uint32_t* sid = cx.st_ids + slot * kStageBlocks;
-      MaskT* smk = cx.st_mk + slot * kStageBlocks;
-#pragma unroll
-      for (int c = 0; c < kRegChunks; ++c) {
-        const uint32_t k = c * 32u + lane;
-        if (k < q.nblk) { const uint32_t id = ids[q.off + k]; sid[k] = id; smk[k] = mask_load<MaskT>(cx.mask, id); }
-      }
-      __syncwarp();
-      uint32_t h0, h1;
-      probe_staged<MaskT>(smk, cx.mask, ids, q, R, lane, h0, h1);
-      stage_scores<MaskT>(a, cx, q, slot, h0, h1, lane);
-      __syncwarp();
-    }
-
-    GORGO_PT(1)
-    // ---- queue signal (Eq. 2): requests that completed by the arrival of r stop counting
-    const volatile long long* sub = cx.exp_sub + (size_t)(r % kExpRing) * R;
-    if (i0 < R) ld0 -= sub[i0];
-    if (i1 < R) ld1 -= sub[i1];
-
-    // ---- score of Eq. 3 (fixed order, no FMA): the staged (w_net*RTT + w_prefill*uncached)
-    //      plus the queue term; lowest-index argmin
-    uint64_t best_k = ~0ull;
-    uint32_t best_i = kNone;
-    if (i0 < R) {
-      double qv = (double)ld0;
-      if (K != 3) qv = __dmul_rn(qv, nrm0);
-      double c = __dadd_rn(cx.st_ab[slot * R + i0], __dmul_rn(w_que, qv));
-      if (c != c) c = (i0 == 0) ? -d_inf() : d_inf();    // a NaN score wins only at index 0
-      best_k = order_key(c); best_i = i0;
-    }
-    if (i1 < R) {
-      double qv = (double)ld1;
-      if (K != 3) qv = __dmul_rn(qv, nrm1);
-      double c = __dadd_rn(cx.st_ab[slot * R + i1], __dmul_rn(w_que, qv));
-      if (c != c) c = d_inf();
-      const uint64_t ck = order_key(c);
-      if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i1; }
-    }
-    GORGO_PT(2)
-    const uint32_t istar = warp_argmin_key(best_k, best_i);
-    GORGO_PT(3)
-    const uint32_t hstar = cx.st_hits[slot * R + istar];
-    if (lane == 0) {
-      cx.route_ring[r % kRouteRing] = istar | (slot << 8) | (hstar << 16);
-      cx.route_log[r] = (uint8_t)istar;
-    }
-    __threadfence_block();
-    __syncwarp();
-    if (lane == 0) ctl[kCtlRouted] = r + 1;
-    if ((istar & 31u) == lane) {
-      if (istar < 32u) ld0 += (long long)q.in_tok; else ld1 += (long long)q.in_tok;
-    }
-    GORGO_PT(4)
-  }
-  GORGO_PROF_FLUSH(0)
-  if (i0 < R) sm.load[i0] = ld0;
-  if (i1 < R) sm.load[i1] = ld1;
-  if (status != 0) give_up(ctl, status, lane);
-}
-
-// Queue warp `which` of kQueueWarps: owns the replicas i with i mod kQueueWarps == which.  It
-// does two things, both in request order:
-//  (A) books routed request j on its replica: earliest-free slot (lowest index on ties), start,
-//      first-token and finish times, outputs; the request joins the slot's FIFO of in-flight
-//      requests;
-//  (B) stages, for a coming request e, the tokens that stop being in flight on each of its
-//      replicas at the arrival of e (finish <= t'_e), for the route warp to subtract.
-// (B) for e may run ahead of the routing: it only needs (A) done for the requests that can
-// have finished by t'_e, which the static bound `need_svc[e]` gives (a request cannot finish
-// before its arrival plus its decode time).  (A) for j runs after (B) for j, so (B) never sees
-// a request that arrives later than e.
-template <typename MaskT>
-__device__ __forceinline__ void queue_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
-                                           uint32_t lane, uint32_t which) {
-  const Smem& sm = cx.sm;
-  const uint32_t R = a.m.R, S = a.m.S;
-  const uint32_t N = a.tr.n_req;
-  const ReqRec* req = a.tr.req;
-  double *free_at = cx.free_at, *q0_fin = cx.q0_fin, *q1_fin = cx.q1_fin;
-  uint32_t *q0_tok = cx.q0_tok, *q1_tok = cx.q1_tok, *q2_idx = cx.q2_idx, *tail = cx.tail,
-           *qcnt = cx.qcnt;
-  uint4* qrec = cx.qrec;
-  volatile uint32_t* ctl = cx.ctl;
-  int32_t status = 0;
-  unsigned long long st_hit = 0, st_blk = 0;
-  const uint32_t end = a.first + a.count;
-  const uint32_t last_r = end - 1;
-
-  // a slot whose second-oldest entry has to be refilled from the per-request records: slot index
-  // (kNone: none), record to read, whether the read has been issued, and the record read.  The
-  // read is issued after the expiries are published, so that nothing waits for it.
-  uint32_t pend_x = kNone, pend_idx = kNone;
-  bool pend_loaded = false;
-  uint4 pend_rec = make_uint4(0, 0, 0, 0);
-  auto flush_pending = [&]() {
-    if (pend_x != kNone) {
-      if (!pend_loaded) pend_rec = qrec[pend_idx];
-      q1_fin[pend_x] = __hiloint2double((int)pend_rec.y, (int)pend_rec.x);
-      q2_idx[pend_x] = pend_rec.z;
-      q1_tok[pend_x] = pend_rec.w;
-      pend_x = kNone;
-    }
-  };
-
-  uint32_t ja = a.first, e = a.first;
-  // static data of the coming requests, fetched two ahead of each cursor
-  ReqRec ra0 = req[min(ja, last_r)], ra1 = req[min(ja + 1, last_r)];
-  double te0 = a.tq[min(e, last_r)], te1 = a.tq[min(e + 1, last_r)];
-  uint32_t nd0 = a.need_svc[min(e, last_r)], nd1 = a.need_svc[min(e + 1, last_r)];
-  uint32_t idle = 0;
-
-  GORGO_PROF_DECL
-  while (ja < end || e < end) {
-    const uint32_t routed = ctl[kCtlRouted];
-    GORGO_PT(0)
-    if (e < end && e < routed + kExpRing && ja >= nd0) {
-      // ---- (B) expiries at the arrival of request e
-      const double t = te0;                        // = scale * ts[e]
-      long long* sub = cx.exp_sub + (size_t)(e % kExpRing) * R;
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const uint32_t i = lane + 32u * half;
-        if (i < R && (i % kQueueWarps) == which) sub[i] = 0;
-      }
-      __syncwarp();
-      for (uint32_t i0 = 0; i0 < R; i0 += 32) {
-        const uint32_t i = i0 + lane;
-        unsigned due = __ballot_sync(kFull, i < R && (i % kQueueWarps) == which && sm.minfin[i] <= t);
-        while (due) {
-          const uint32_t ii = i0 + (uint32_t)__ffs((int)due) - 1;
-          due &= due - 1;
-          long long tok = 0;
-          double mn = d_inf();
-          for (uint32_t s = lane; s < S; s += 32) {
-            const uint32_t x = ii * S + s;
-            double hf = q0_fin[x];
-            if (hf <= t) {
-              uint32_t guard = 0;
-              uint32_t cnt = qcnt[x];
-              do {
-                if (pend_x == x) flush_pending();           // the second entry is still in flight
-                tok += (long long)q0_tok[x];
-                --cnt;
-                if (cnt == 0) { hf = d_inf(); }
-                else {
-                  hf = q1_fin[x];                            // the second becomes the oldest
-                  q0_tok[x] = q1_tok[x];
-                  if (cnt >= 2) {                            // the new second is fetched later
-                    flush_pending();
-                    pend_x = x;
-                    pend_idx = q2_idx[x];
-                    pend_loaded = false;
-                  }
-                }
-                if (++guard > N) { status = -6; break; }
-              } while (hf <= t);
-              q0_fin[x] = hf;
-              qcnt[x] = cnt;
-            }
-            mn = fmin(mn, hf);
-          }
-          if (tok != 0)
-            atomicAdd(reinterpret_cast<unsigned long long*>(sub + ii), (unsigned long long)tok);
-          uint64_t mk = order_key(mn);
-          warp_argmin_key(mk, lane);
-          if (lane == 0) sm.minfin[ii] = order_value(mk);
-        }
-      }
-      __threadfence_block();
-      __syncwarp();
-      if (lane == 0) ctl[kCtlExp + which] = e + 1;
-      if (pend_x != kNone && !pend_loaded) { pend_rec = qrec[pend_idx]; pend_loaded = true; }
-      ++e;
-      te0 = te1; nd0 = nd1;
-      te1 = a.tq[min(e + 1, last_r)];
-      nd1 = a.need_svc[min(e + 1, last_r)];
-      idle = 0;
-      GORGO_PT(1)
-      if (__any_sync(kFull, status != 0)) break;
-      continue;
-    }
-    if (ja < routed && ja < e) {
-      // ---- (A) service commit of routed request ja, if its replica is one of this warp's
-      const uint32_t ent = cx.route_ring[ja % kRouteRing];
-      const uint32_t istar = ent & 255u, hstar = ent >> 16;
-      if ((istar % kQueueWarps) == which) {
-        const ReqRec rec = ra0;
-        const uint32_t r = ja, in_tok = rec.in_tok;
-        const double t = __dmul_rn(a.scale, rec.ts_ms);
-        const unsigned long long hbstar = (unsigned long long)hstar * a.m.B;
-        const uint32_t uncstar = in_tok - (uint32_t)(hbstar < in_tok ? hbstar : in_tok);
-        // earliest-free slot, lowest index on ties
-        uint64_t bk = ~0ull;
-        uint32_t bs = kNone;
-        for (uint32_t s = lane; s < S; s += 32) {
-          const uint64_t vk = order_key(free_at[(size_t)istar * S + s]);
-          if (vk < bk || bs == kNone) { bk = vk; bs = s; }
-        }
-        bs = warp_argmin_key(bk, bs);
-        const double bv = order_value(bk);
-        const double arrive = __dadd_rn(t, sm.rtt[(size_t)rec.origin * R + istar]);
-        const double start = (bv > arrive) ? bv : arrive;
-        const double first = __dadd_rn(start, __dmul_rn(a.m.prefill_ms, (double)uncstar));
-        const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
-        const double finish = __dadd_rn(first, __dmul_rn(a.m.tpot_ms, (double)dec_tok));
-        if (pend_x == istar * S + bs) flush_pending();   // the slot's own refill comes first
-        __syncwarp();
-        if (lane == 0) {
-          const size_t x = (size_t)istar * S + bs;
-          qrec[r] = make_uint4((uint32_t)__double2loint(finish), (uint32_t)__double2hiint(finish),
-                               kNone, in_tok);
-          const uint32_t cnt = qcnt[x];
-          if (cnt == 0) {
-            q0_fin[x] = finish; q0_tok[x] = in_tok;
-            sm.minfin[istar] = fmin(sm.minfin[istar], finish);
-          } else {
-            reinterpret_cast<uint32_t*>(qrec + tail[x])[2] = r;     // link behind the newest
-            if (cnt == 1) { q1_fin[x] = finish; q1_tok[x] = in_tok; q2_idx[x] = kNone; }
-            else if (cnt == 2) q2_idx[x] = r;
-          }
-          qcnt[x] = cnt + 1;
-          tail[x] = r;
-          free_at[x] = finish;
-          const size_t o = (size_t)p * a.out_stride + (r - a.first);
-          if (a.route_out) a.route_out[o] = (uint8_t)istar;
-          if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
-          if (a.ttft_out) a.ttft_out[o] = __dsub_rn(first, t);
-          if (a.e2e_out) a.e2e_out[o] = __dsub_rn(finish, t);
-          st_hit += hstar; st_blk += rec.nblk;
-        }
-        __syncwarp();
-      }
-      ++ja;
-      ra0 = ra1;
-      ra1 = req[min(ja + 1, last_r)];
-      if (lane == 0) ctl[kCtlServed + which] = ja;
-      idle = 0;
-#ifdef GORGO_PROF
-      if ((istar % kQueueWarps) == which) GORGO_PT(2) else GORGO_PT(3)
-#endif
-      continue;
-    }
-    if (ctl[kCtlAbort] || ++idle > kSpinLimit) { status = -6; break; }
-    __nanosleep(2 * kPollNs);
-  }
-  GORGO_PROF_FLUSH(3 + which)
-  flush_pending();
-  __syncwarp();
-  status = __reduce_min_sync(kFull, status);
-  if (status != 0) give_up(ctl, status, lane);
-  if (lane == 0 && a.stats) {
-    unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
-    atomicAdd(s4 + 1, st_hit);
-    atomicAdd(s4 + 2, st_blk);
-  }
-}
-
-// The cache commit of a routed request is split between two warps.
-//
-// Check warp (on the serial path): from the staged mask words of request r it counts the blocks
-// missing on the chosen replica, sizes the eviction and takes the victims from the head of the
-// replica's ring.  A victim whose block occurs again in one of the next kWindow requests voids
-// that request's staged read: the request is flagged before the route warp is told that the
-// victims of r are known, which is all the route warp waits for.  In the common case this warp
-// touches shared memory only; the memory traffic of the commit is left to the apply warp as a
-// work item.  If the ring cannot serve the eviction as it stands (the scout is behind, or an
-// entry went stale), the warp waits until every earlier commit is applied and evicts by the
-// general procedure itself.
-//
-// Apply warp (behind): sets the replica's bit on the missing blocks, clears it on the victims,
-// appends the request to the replica's recency list and publishes the request as committed.
-struct ApplyItem {
-  uint32_t route;     // replica | stage << 8
-  uint32_t head0;     // ring index of the first victim left to this warp
-  uint32_t nvict;     // victims left to this warp (0: the check warp evicted itself)
-  uint32_t evicted;   // victims of the request in all (statistics)
-  uint32_t lru_prev;  // previous request routed to the replica (kNone: none)
-  uint32_t nblk, off, pad;
-};
-
-template <typename MaskT>
-__device__ __forceinline__ void check_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t lane) {
-  const Smem& sm = cx.sm;
+  const uint32_t R = a.m.R;
   const uint32_t N = a.tr.n_req;
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
   MaskT* mask = cx.mask;
   uint32_t* lru_next = cx.lru_next;
   const uint8_t* route_log = cx.route_log;
-  volatile uint32_t* ctl = cx.ctl;
   int32_t status = 0;
+  unsigned long long st_probe = 0, st_evict = 0;
   const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
   const uint32_t end = a.first + a.count;
 
   Ahead q_cur = fetch_ahead(req, a.first, end), q_nxt = fetch_ahead(req, a.first + 1, end);
+  // latest earlier request sharing a block with r+1, r+2, r+3, and whether a commit since their
+  // staged read can have changed their mask words
+  uint32_t ps1 = q_nxt.prev_share, ps2 = fetch_ahead(req, a.first + 2, end).prev_share,
+           ps3 = fetch_ahead(req, a.first + 3, end).prev_share;
+  bool bad0 = false, bad1 = false, bad2 = false, bad3 = false;
+  bool posted = false;         // the hits of the coming request were already handed over
+  // hand the staged hits of request q over to the decide warp and count its probes
+  auto hand_over = [&](uint32_t slot, uint32_t nblk) {
+    if (lane == 0) *cx.hit_slot = slot;
+    bar_arrive(kBarHits);                                 // the decide warp may score the request
+    if (lane < R) { const uint32_t h = cx.st_hits[slot * R + lane]; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+    if (lane + 32u < R) { const uint32_t h = cx.st_hits[slot * R + lane + 32u]; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+  };
 
-  GORGO_PROF_DECL
   for (uint32_t r = a.first; r < end; ++r) {
     const uint32_t n = q_cur.nblk, off = q_cur.off;
     const Ahead q_n2 = fetch_ahead(req, r + 2, end);          // used two rounds from now
+    const uint32_t ps4 = (r + 4 < end) ? req[r + 4].prev_share : kNone;
 
-    // ---- wait for the route of request r (and for room in the apply ring)
-    uint32_t polls = 0;
-    while (ctl[kCtlRouted] <= r || r - ctl[kCtlApplied] >= kApplyRing) {
-      if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
-      __nanosleep(kPollNs);
+    // ---- prefix hits of request r: staged by the probe warp, or read and probed here
+    uint32_t slot = r % kStageDepth;
+    bool staged = posted;
+    if (!posted && !bad0 && !*cx.probe_gone) {
+      uint32_t polls = 0;
+      while (cx.st_ready[slot] != r + 1 && !*cx.probe_gone && polls < 4096) { ++polls; __nanosleep(20); }
+      // (one lane decides: every lane must take the same path)
+      staged = __shfl_sync(kFull, cx.st_ready[slot], 0) == r + 1;
+      smem_order();
     }
-    GORGO_PT(0)
-    if (status) break;
-    compiler_fence();
-    const uint32_t ent0 = cx.route_ring[r % kRouteRing];
-    const uint32_t istar = ent0 & 255u, slot = (ent0 >> 8) & 255u;
-    const MaskT bit = (MaskT)(((MaskT)1) << istar);
-    const MaskT* smk = cx.st_mk + slot * kStageBlocks;
-    GORGO_PT(6)
-
-    // ---- blocks of r missing on the replica
-    uint32_t missing = 0;
+    if (!staged) {
+      uint32_t h0 = 0, h1 = 0;
+      slot = kStageDepth + (r & 1u);                          // this warp's own stages
+      uint32_t* sid = cx.st_ids + slot * kStageBlocks;
+      MaskT* smk = cx.st_mk + slot * kStageBlocks;
 #pragma unroll
-    for (int c = 0; c < kRegChunks; ++c) {
-      if ((uint32_t)c * 32u < n) {
-        const uint32_t k = (uint32_t)c * 32u + lane;
-        const bool miss = k < n && !(smk[k] & bit);
-        missing += __popc(__ballot_sync(kFull, miss));
+      for (int c = 0; c < kRegChunks; ++c) {
+        const uint32_t k = c * 32u + lane;
+        if (k < n) { const uint32_t id = ids[off + k]; sid[k] = id; smk[k] = mask_load<MaskT>(mask, id); }
       }
+      __syncwarp();
+      probe_staged<MaskT>(smk, mask, ids, q_cur, R, lane, h0, h1);
+      stage_scores<MaskT>(a, cx, q_cur, slot, h0, h1, lane);
     }
-    for (uint32_t c = kStageBlocks; c < n; c += 32) {      // longer prompts: the rest from memory
+    const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
+    const MaskT* smk = cx.st_mk + slot * kStageBlocks;
+    if (!posted) hand_over(slot, n);
+
+    bar_wait(kBarRoute);                                  // the replica has been chosen
+    const uint32_t istar = *cx.route;
+    const MaskT bit = (MaskT)(((MaskT)1) << istar);
+
+    // ---- cache commit: set the replica's bit on the missing blocks
+    uint32_t missing = 0;
+    for (uint32_t c = 0; c < n; c += 32) {
       const uint32_t k = c + lane;
-      const bool miss = k < n && !(mask_load<MaskT>(mask, ids[off + k]) & bit);
+      bool miss = false;
+      if (k < n) {
+        uint32_t id;
+        MaskT mv;
+        if (c < kStageBlocks) { id = sid[k]; mv = smk[k]; }
+        else { id = ids[off + k]; mv = mask_load<MaskT>(mask, id); }
+        if (!(mv & bit)) { mask_store<MaskT>(mask, id, (MaskT)(mv | bit)); miss = true; }
+      }
       missing += __popc(__ballot_sync(kFull, miss));
     }
-    GORGO_PT(1)
     uint32_t occ = sm.occ[istar] + missing;
     uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
-    uint32_t evicted = 0, nvict = 0;
-    GORGO_PC(9, n) GORGO_PC(10, need)
-    const uint32_t head0 = sm.chead[istar];
+    uint32_t evicted = 0;
+    unsigned hit1 = 0, hit2 = 0, hit3 = 0;   // a victim's block occurs again in request r+1/2/3
     if (need > 0) {
       uint32_t cr = sm.curreq[istar];
       int32_t cp = sm.curpos[istar];
-      const uint4* lst = sm.lst + (size_t)istar * kListCap;
-      // ---- common case: the next `need` ring entries are all live; they are the victims
-      bool clean = sm.act[istar] != 0;
-      if (clean) {
-        uint32_t avail = sm.ring_tail[istar] - head0;
-        for (uint32_t polls2 = 0; avail < need && polls2 < 64; ++polls2) {
-          __nanosleep(20);
-          avail = sm.ring_tail[istar] - head0;
-          GORGO_PC(11, 1)
-        }
-        clean = avail >= need;
-        compiler_fence();
-      }
-      GORGO_PT(4)
-      uint32_t last_w = 0, last_z = 0;
-      for (uint32_t o = 0; clean && o < need; o += 32) {
-        const bool mine = o + lane < need;
-        uint4 ent = make_uint4(0, kNone, 0, 0);
-        bool odd = false;        // void (behind the cursor) or touched again since it was listed
-        if (mine) {
-          const uint32_t e = (head0 + o + lane) & (kListCap - 1);
-          ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
-          odd = ent.y <= r || ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
-        }
-        if (__any_sync(kFull, odd)) { clean = false; break; }
-        // a victim that occurs again within the window voids that request's staged read
-        const bool soon = mine && ent.y - (r + 1) < kWindow;
-        if (__any_sync(kFull, soon)) {
-          if (soon) cx.inval[ent.y % kInvalRing] = ent.y + 1;
-          __threadfence_block();
-        }
-        const uint32_t lastl = min(need - o, 32u) - 1u;   // lane of the last victim of the round
-        last_w = __shfl_sync(kFull, ent.w, lastl);
-        last_z = __shfl_sync(kFull, ent.z, lastl);
-      }
-      GORGO_PT(5)
-      if (clean) {
-        cr = last_w;
-        cp = (int32_t)last_z - 1;
-        evicted = nvict = need;
-        need = 0;
-        if (lane == 0) sm.chead[istar] = head0 + nvict;
-      } else {
-        GORGO_PC(8, 1)
-        // ---- general procedure, by this warp, once every earlier commit is applied
-        polls = 0;
-        while (ctl[kCtlApplied] < r) {
-          if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
-        }
-        if (status) break;
-        __threadfence_block();
-        if (sm.act[istar]) {
-          uint32_t head = head0;     // == ring_head: the apply warp has caught up
-          uint32_t last_e = kNone;   // ring slot of the last entry passed that was not void
-          while (need > 0) {
-            uint32_t avail = sm.ring_tail[istar] - head;
-            for (uint32_t polls2 = 0; avail == 0 && polls2 < 64; ++polls2) {
-              __nanosleep(20);
-              avail = sm.ring_tail[istar] - head;
-            }
-            if (avail == 0) break;                          // the scout is behind: walk ourselves
-            const uint32_t m = min(avail, 32u);
-            uint4 ent = make_uint4(0, kNone, 0, 0);
-            bool live = false;
-            uint32_t nxr = kNone;      // request of the block's next occurrence after r
-            if (lane < m) {
-              const uint32_t e = (head + lane) & (kListCap - 1);
-              ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
-              nxr = ent.y;
-              // entries the eviction cursor has already passed (after a walk of our own) are void
-              live = !(ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp));
-              if (live && ent.y <= r) {
-                // the block came back since the entry was made: follow its occurrences up to r
-                uint2 c = a.tr.occ_next[req[ent.w].off + ent.z];
-                nxr = kNone;
-                while (c.x != kNone) {
-                  if (c.y > r) { nxr = c.y; break; }
-                  const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
-                  if (rr == istar) { live = false; break; }
-                  c = a.tr.occ_next[c.x];
-                }
-              }
-            }
-            const unsigned lv = __ballot_sync(kFull, live);
-            const uint32_t cnt = __popc(lv);
-            const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+      // fast path: victims from the ring the scout warp keeps for this replica
+      if (sm.act[istar]) {
+        const uint4* lst = sm.lst + (size_t)istar * kListCap;
+        uint32_t head = sm.ring_head[istar];
+        uint32_t last_e = kNone;   // ring slot of the last entry passed that was not void
+        while (need > 0) {
+          uint32_t avail = sm.ring_tail[istar] - head;
+          for (uint32_t polls = 0; avail == 0 && polls < 64; ++polls) {
+            __nanosleep(20);
+            avail = sm.ring_tail[istar] - head;
+          }
+          if (avail == 0) break;                          // the scout is behind: walk ourselves
+          smem_order();
+          const uint32_t m = min(avail, 32u);
+          uint4 ent = make_uint4(0, kNone, 0, 0);
+          bool odd = false;      // void (behind the cursor) or touched again since it was listed
+          if (lane < m) {
+            const uint32_t e = (head + lane) & (kListCap - 1);
+            ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+            odd = ent.y <= r || ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
+          }
+          if (!__any_sync(kFull, odd)) {
+            // common case: the next entries are all live, the first `need` of them are victims
+            const uint32_t tk = min(need, m);
+            const bool mine = lane < tk;
             if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
-            {
-              const bool soon = mine && nxr - (r + 1) < kWindow;
-              if (__any_sync(kFull, soon)) {
-                if (soon) cx.inval[nxr % kInvalRing] = nxr + 1;
-                __threadfence_block();
-              }
-            }
-            // entries passed: the whole round, or up to the last victim taken
-            uint32_t passed = m, tk = cnt;
-            if (cnt > need) {
-              const unsigned take = __ballot_sync(kFull, mine);
-              passed = 32u - (uint32_t)__clz((int)take);
-              tk = need;
+            const unsigned soon = __ballot_sync(kFull, mine && ent.y - (r + 1) < kWindow);
+            if (soon) {
+              hit1 |= __ballot_sync(kFull, mine && ent.y == r + 1);
+              hit2 |= __ballot_sync(kFull, mine && ent.y == r + 2);
+              hit3 |= __ballot_sync(kFull, mine && ent.y == r + 3);
             }
             need -= tk;
             evicted += tk;
-            // the cursor moves behind the last live entry passed (void ones lie behind it already)
-            const unsigned seen = lv & (passed >= 32u ? kFull : ((1u << passed) - 1u));
-            if (seen) last_e = (head + 31u - (uint32_t)__clz((int)seen)) & (kListCap - 1);
-            head += passed;
-          }
-          if (last_e != kNone) {
-            const uint4 le = a.lists_in_smem ? lst[last_e] : __ldcg(lst + last_e);
-            cr = le.w;
-            cp = (int32_t)le.z - 1;
-          }
-          if (lane == 0) { sm.chead[istar] = head; sm.ring_head[istar] = head; }
-        }
-        uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
-        unsigned long long guard = 0;
-        while (need > 0) {
-          if (++guard > evict_guard_max) { status = -6; break; }
-          if (cp < 0) {  // this request is used up: go to the next one routed here
-            const uint32_t nx = (cr == kNone) ? kNone : lru_next[cr];
-            if (nx == kNone) { status = -6; break; }
-            cr = nx;
-            const ReqRec cre = req[cr];
-            coff = cre.off;
-            cp = (int32_t)cre.nblk - 1;
+            last_e = (head + tk - 1) & (kListCap - 1);
+            head += tk;
             continue;
           }
-          // examine 32 touches, deepest position first
-          const int32_t k = cp - (int32_t)lane;
-          bool live = false;
-          uint32_t vid = 0, nxr = kNone;
-          if (k >= 0) {
-            const uint32_t g = coff + (uint32_t)k;
-            vid = ids[g];
-            uint2 c = a.tr.occ_next[g];
-            live = true;
-            while (c.x != kNone && c.y <= r) {       // later occurrences of the block, up to r
-              const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
-              if (rr == istar) { live = false; break; }
-              c = a.tr.occ_next[c.x];
+          bool live = false, unsure = false;
+          if (lane < m) {
+            // entries the eviction cursor has already passed (after a walk of our own) are void
+            live = !(ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp));
+            if (live && ent.y <= r) {
+              if (ent.y == r) live = false;               // the block is in this very request
+              else {                                      // it came back in between: look again
+                live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
+                unsure = true;                            // where it occurs next is not known here
+              }
             }
-            if (live && c.x != kNone) nxr = c.y;     // its next occurrence after r
           }
           const unsigned lv = __ballot_sync(kFull, live);
           const uint32_t cnt = __popc(lv);
-          // the first `need` live touches in lane order are the victims
           const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
-          const unsigned take = __ballot_sync(kFull, mine);
-          if (mine) mask_clear_bit<MaskT>(mask, vid, bit);
-          {
-            const bool soon = mine && nxr - (r + 1) < kWindow;
-            if (__any_sync(kFull, soon)) {
-              if (soon) cx.inval[nxr % kInvalRing] = nxr + 1;
-              __threadfence_block();
-            }
+          if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
+          hit1 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 1));
+          hit2 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 2));
+          hit3 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 3));
+          // entries passed: the whole round, or up to the last victim taken
+          uint32_t passed = m, tk = cnt;
+          if (cnt > need) {
+            const unsigned take = __ballot_sync(kFull, mine);
+            passed = 32u - (uint32_t)__clz((int)take);
+            tk = need;
           }
-          cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
-          const uint32_t tk = __popc(take);
           need -= tk;
           evicted += tk;
+          // the cursor moves behind the last live entry passed (void ones lie behind it already)
+          const unsigned seen = lv & (passed >= 32u ? kFull : ((1u << passed) - 1u));
+          if (seen) last_e = (head + 31u - (uint32_t)__clz((int)seen)) & (kListCap - 1);
+          head += passed;
         }
-        __threadfence_block();                            // this warp's own reductions
+        if (last_e != kNone) {
+          const uint4 le = a.lists_in_smem ? lst[last_e] : __ldcg(lst + last_e);
+          cr = le.w;
+          cp = (int32_t)le.z - 1;
+        }
+        if (lane == 0) sm.ring_head[istar] = head;
+      }
+      uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
+      unsigned long long guard = 0;
+      while (need > 0) {
+        if (++guard > evict_guard_max) { status = -6; break; }
+        if (cp < 0) {  // this request is used up: go to the next one routed here
+          const uint32_t nx = (cr == kNone) ? kNone : lru_next[cr];
+          if (nx == kNone) { status = -6; break; }
+          cr = nx;
+          const ReqRec cre = req[cr];
+          coff = cre.off;
+          cp = (int32_t)cre.nblk - 1;
+          continue;
+        }
+        // examine 32 touches, deepest position first
+        const int32_t k = cp - (int32_t)lane;
+        bool live = false;
+        uint32_t vid = 0, nxr = kNone;
+        if (k >= 0) {
+          const uint32_t g = coff + (uint32_t)k;
+          vid = ids[g];
+          uint2 c = a.tr.occ_next[g];
+          live = true;
+          while (c.x != kNone && c.y <= r) {       // later occurrences of the block, up to r
+            const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
+            if (rr == istar) { live = false; break; }
+            c = a.tr.occ_next[c.x];
+          }
+          if (live && c.x != kNone) nxr = c.y;     // its next occurrence after r
+        }
+        const unsigned lv = __ballot_sync(kFull, live);
+        const uint32_t cnt = __popc(lv);
+        // the first `need` live touches in lane order are the victims
+        const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+        const unsigned take = __ballot_sync(kFull, mine);
+        if (mine) mask_clear_bit<MaskT>(mask, vid, bit);
+        hit1 |= __ballot_sync(kFull, mine && nxr == r + 1);
+        hit2 |= __ballot_sync(kFull, mine && nxr == r + 2);
+        hit3 |= __ballot_sync(kFull, mine && nxr == r + 3);
+        cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
+        const uint32_t tk = __popc(take);
+        need -= tk;
+        evicted += tk;
       }
       if (lane == 0) { sm.curreq[istar] = cr; sm.curpos[istar] = cp; }
     }
     occ -= evicted;
+    st_evict += evicted;
 
-    // ---- the victims of r are known: the route warp may go on
-    __syncwarp();
-    if (lane == 0) ctl[kCtlChecked] = r + 1;
-    GORGO_PT(2)
+    // ---- which staged reads did the commit of request r invalidate?  If the next request's
+    //      are intact and staged, hand them over now: the decide warp works on r+1 while the
+    //      bookkeeping of r below finishes.
+    bad0 = bad1 || ps1 == r || hit1 != 0;
+    bad1 = bad2 || ps2 == r || hit2 != 0;
+    bad2 = bad3 || ps3 == r || hit3 != 0;
+    bad3 = false;
+    ps1 = ps2; ps2 = ps3; ps3 = ps4;
+    posted = false;
+    if (r + 1 < end && !bad0 &&
+        __shfl_sync(kFull, cx.st_ready[(r + 1) % kStageDepth], 0) == r + 2) {
+      smem_order();
+      hand_over((r + 1) % kStageDepth, q_nxt.nblk);
+      posted = true;
+    }
 
-    // ---- hand the memory traffic of the commit to the apply warp
     if (lane == 0) {
       sm.occ[istar] = occ;
-      const uint32_t lt = sm.c_lrutail[istar];
-      sm.c_lrutail[istar] = r;
+      // recency order of the replica: append this request
+      const uint32_t lt = sm.lrutail[istar];
+      if (lt != kNone) lru_next[lt] = r;
+      lru_next[r] = kNone;
       if (sm.curreq[istar] == kNone) { sm.curreq[istar] = r; sm.curpos[istar] = (int32_t)n - 1; }
+      sm.lrutail[istar] = r;
       // hand the replica to the scout warp once its cache is close to full (before that no
       // eviction has happened here, so the scout starts from the eviction cursor)
       if (!sm.act[istar] && (uint64_t)occ + kPostMargin >= a.m.C) {
@@ -1118,159 +884,30 @@ __device__ __forceinline__ void check_warp(const ReplayArgs& a, const Ctx<MaskT>
         __threadfence_block();
         sm.act[istar] = 1;
       }
-      uint4* item = cx.apply_ring + (size_t)(r % kApplyRing) * 2;
-      item[0] = make_uint4(istar | (slot << 8), head0, nvict, evicted);
-      item[1] = make_uint4(lt, n, off, 0u);
       __threadfence_block();
-      ctl[kCtlEnqueued] = r + 1;
+      *sm.progress = r + 1;                               // request r is fully committed
     }
     __syncwarp();
-    if (__any_sync(kFull, status != 0)) break;
-    GORGO_PT(3)
 
     q_cur = q_nxt; q_nxt = q_n2;
   }
-  GORGO_PROF_FLUSH(1)
-  status = __reduce_min_sync(kFull, status);
-  if (status != 0) give_up(ctl, status, lane);
-}
-
-template <typename MaskT>
-__device__ __forceinline__ void apply_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
-                                           uint32_t lane) {
-  const Smem& sm = cx.sm;
-  const uint32_t R = a.m.R;
-  const uint32_t* ids = a.tr.ids;
-  MaskT* mask = cx.mask;
-  uint32_t* lru_next = cx.lru_next;
-  volatile uint32_t* ctl = cx.ctl;
-  int32_t status = 0;
-  unsigned long long st_probe = 0, st_evict = 0;
-  const uint32_t end = a.first + a.count;
-
-  GORGO_PROF_DECL
-  for (uint32_t r = a.first; r < end; ++r) {
-    uint32_t polls = 0;
-    while (ctl[kCtlEnqueued] <= r) {
-      if (ctl[kCtlAbort] || ++polls > kSpinLimit) { status = -6; break; }
-      __nanosleep(20);
-    }
-    GORGO_PT(0)
-    if (status) break;
-    compiler_fence();
-    const uint4* item = cx.apply_ring + (size_t)(r % kApplyRing) * 2;
-    const uint4 i0 = item[0], i1 = item[1];
-    const uint32_t istar = i0.x & 255u, slot = (i0.x >> 8) & 255u;
-    const uint32_t head0 = i0.y, nvict = i0.z, n = i1.y, off = i1.z;
-    const MaskT bit = (MaskT)(((MaskT)1) << istar);
-    const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
-    const MaskT* smk = cx.st_mk + slot * kStageBlocks;
-
-    // ---- set the replica's bit on the missing blocks
-    for (uint32_t c = 0; c < n; c += 32) {
-      const uint32_t k = c + lane;
-      if (k < n) {
-        uint32_t id;
-        MaskT mv;
-        if (c < kStageBlocks) { id = sid[k]; mv = smk[k]; }
-        else { id = ids[off + k]; mv = mask_load<MaskT>(mask, id); }
-        if (!(mv & bit)) mask_store<MaskT>(mask, id, (MaskT)(mv | bit));
-      }
-    }
-    GORGO_PT(1)
-    // ---- clear it on the victims the check warp took from the ring
-    const uint4* lst = sm.lst + (size_t)istar * kListCap;
-    for (uint32_t o = lane; o < nvict; o += 32) {
-      const uint32_t e = (head0 + o) & (kListCap - 1);
-      const uint4 ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
-      mask_clear_bit<MaskT>(mask, ent.x, bit);
-    }
-    if (lane < R) { const uint32_t h = cx.st_hits[slot * R + lane]; st_probe += (h + 1 < n ? h + 1 : n); }
-    if (lane + 32u < R) { const uint32_t h = cx.st_hits[slot * R + lane + 32u]; st_probe += (h + 1 < n ? h + 1 : n); }
-    st_evict += i0.w;
-    if (lane == 0) {
-      // recency order of the replica: append this request
-      if (i1.x != kNone) lru_next[i1.x] = r;
-      lru_next[r] = kNone;
-    }
-    GORGO_PT(2)
-    __threadfence_block();                                // every lane's stores and reductions
-    __syncwarp();
-    GORGO_PT(3)
-    if (lane == 0) {
-      sm.lrutail[istar] = r;
-      if (nvict) sm.ring_head[istar] = head0 + nvict;     // the scout may reuse these entries
-      ctl[kCtlApplied] = r + 1;                           // request r is fully committed
-    }
-    __syncwarp();
-    GORGO_PT(4)
-  }
-  GORGO_PROF_FLUSH(2)
   st_probe = warp_sum_u64(st_probe);
-  if (status != 0) give_up(ctl, status, lane);
-  if (lane == 0 && a.stats) {
-    unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
-    atomicAdd(s4 + 0, st_probe);
-    atomicAdd(s4 + 3, st_evict);
+  status = __reduce_min_sync(kFull, status);
+  if (lane == 0) {
+    if (status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
+    if (a.stats) {
+      unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
+      atomicAdd(s4 + 0, st_probe);
+      atomicAdd(s4 + 3, st_evict);
+    }
   }
 }
 
-constexpr uint32_t kWarpRoute = 0, kWarpCheck = 1, kWarpApply = 2, kWarpQueue0 = 3,
-                   kWarpProbe0 = kWarpQueue0 + kQueueWarps, kWarpScout0 = kWarpProbe0 + kProbeWarps;
-constexpr uint32_t kReplayThreads = 32 * (kWarpScout0 + kScouts);
-
-// Byte offsets of the regions of a replay CTA's dynamic shared memory.
-struct SmemPlan {
-  uint32_t rtt, wrtt, w, minfin, load, slot_d, exp_sub, st_ab, ctl, occ, curreq, curpos, lrutail,
-      slot_u, act, ring_head, ring_tail, scan_cr, scan_cp, c_lrutail, chead, route_ring, inval,
-      apply_ring, st_ready, st_pc, st_hits,
-      st_ids, st_mk, lst, total;
-};
-__host__ __device__ inline SmemPlan smem_plan(uint32_t R, uint32_t G, uint32_t S, uint32_t K,
-                                              uint32_t mask_bytes, bool slots_in_smem,
-                                              bool lists_in_smem) {
-  SmemPlan p;
-  uint32_t o = 0;
-  const uint32_t RS = R * S;
-#define GORGO_TAKE(field, bytes, align) \
-  o = (o + (align) - 1u) / (align) * (align); p.field = o; o += (uint32_t)(bytes);
-  GORGO_TAKE(rtt, G * R * 8u, 16u)
-  GORGO_TAKE(wrtt, G * R * 8u, 8u)
-  GORGO_TAKE(w, K * 8u, 8u)
-  GORGO_TAKE(minfin, R * 8u, 8u)
-  GORGO_TAKE(load, R * 8u, 8u)
-  GORGO_TAKE(slot_d, slots_in_smem ? 3u * RS * 8u : 0u, 8u)
-  GORGO_TAKE(exp_sub, kExpRing * R * 8u, 8u)
-  GORGO_TAKE(st_ab, kStages * R * 8u, 8u)
-  GORGO_TAKE(ctl, kCtlWords * 4u, 8u)
-  GORGO_TAKE(occ, R * 4u, 4u)
-  GORGO_TAKE(curreq, R * 4u, 4u)
-  GORGO_TAKE(curpos, R * 4u, 4u)
-  GORGO_TAKE(lrutail, R * 4u, 4u)
-  GORGO_TAKE(slot_u, slots_in_smem ? 5u * RS * 4u : 0u, 4u)
-  GORGO_TAKE(act, R * 4u, 4u)
-  GORGO_TAKE(ring_head, R * 4u, 4u)
-  GORGO_TAKE(ring_tail, R * 4u, 4u)
-  GORGO_TAKE(scan_cr, R * 4u, 4u)
-  GORGO_TAKE(scan_cp, R * 4u, 4u)
-  GORGO_TAKE(c_lrutail, R * 4u, 4u)
-  GORGO_TAKE(chead, R * 4u, 4u)
-  GORGO_TAKE(route_ring, kRouteRing * 4u, 4u)
-  GORGO_TAKE(inval, kInvalRing * 4u, 4u)
-  GORGO_TAKE(st_ready, kStageDepth * 4u, 4u)
-  GORGO_TAKE(st_pc, kStageDepth * 4u, 4u)
-  GORGO_TAKE(st_hits, kStages * R * 4u, 4u)
-  GORGO_TAKE(st_ids, kStages * kStageBlocks * 4u, 4u)
-  GORGO_TAKE(st_mk, kStages * kStageBlocks * mask_bytes, 8u)
-  GORGO_TAKE(apply_ring, kApplyRing * 32u, 16u)
-  GORGO_TAKE(lst, lists_in_smem ? R * kListCap * 16u : 0u, 16u)
-#undef GORGO_TAKE
-  p.total = (o + 15u) / 16u * 16u;
-  return p;
-}
+constexpr uint32_t kWarpDecide = 0, kWarpCache = 1, kWarpProbe = 2, kWarpScout0 = 3;
+constexpr uint32_t kReplayThreads = 32 * (3 + kScouts);
 
 template <typename MaskT>
-__global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayArgs a) {
+__global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayArgs a) {
   const uint32_t p = blockIdx.x;
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t warp = threadIdx.x >> 5;
@@ -1285,54 +922,58 @@ __global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayA
   uint32_t* g_slot_u = reinterpret_cast<uint32_t*>(st + a.lay.slot_u_off);  // 5 x [R*S] words
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const SmemPlan pl = smem_plan(R, G, S, K, (uint32_t)sizeof(MaskT), a.slots_in_smem != 0,
-                                a.lists_in_smem != 0);
   Ctx<MaskT> cx;
   Smem& sm = cx.sm;
-  sm.rtt = reinterpret_cast<double*>(smem_raw + pl.rtt);        // [G*R]
-  sm.wrtt = reinterpret_cast<double*>(smem_raw + pl.wrtt);      // [G*R]  w_net * rtt
-  sm.w = reinterpret_cast<double*>(smem_raw + pl.w);            // [K]
-  sm.minfin = reinterpret_cast<double*>(smem_raw + pl.minfin);  // [R]
-  sm.load = reinterpret_cast<long long*>(smem_raw + pl.load);   // [R]
+  sm.rtt = reinterpret_cast<double*>(smem_raw);            // [G*R]
+  sm.wrtt = sm.rtt + (size_t)G * R;                        // [G*R]  w_net * rtt
+  sm.w = sm.wrtt + (size_t)G * R;                          // [K]
+  sm.minfin = sm.w + K;                                    // [R]
+  sm.load = reinterpret_cast<long long*>(sm.minfin + R);   // [R]
+  double* dnext = reinterpret_cast<double*>(sm.load + R);
   // Per-slot state (in shared memory when it fits, else it stays in global memory).  A slot is a
   // FIFO of in-flight requests whose finish times never decrease; its two oldest entries are
   // kept here, the rest is reached through the per-request records in global memory.
-  double* slot_d = a.slots_in_smem ? reinterpret_cast<double*>(smem_raw + pl.slot_d) : g_slot_d;
-  uint32_t* slot_u = a.slots_in_smem ? reinterpret_cast<uint32_t*>(smem_raw + pl.slot_u) : g_slot_u;
+  double* slot_d = g_slot_d;
+  if (a.slots_in_smem) { slot_d = dnext; dnext += 3 * (size_t)RS; }
   cx.free_at = slot_d;                   // time the slot frees (finish of its newest request)
   cx.q0_fin = slot_d + RS;               // finish of the oldest in-flight request (+inf: none)
   cx.q1_fin = slot_d + 2 * (size_t)RS;   // finish of the second oldest
+  sm.occ = reinterpret_cast<uint32_t*>(dnext);             // [R]
+  sm.curreq = sm.occ + R;
+  sm.curpos = reinterpret_cast<int32_t*>(sm.curreq + R);
+  sm.lrutail = reinterpret_cast<uint32_t*>(sm.curpos + R);
+  uint32_t* unext = sm.lrutail + R;
+  uint32_t* slot_u = g_slot_u;
+  if (a.slots_in_smem) { slot_u = unext; unext += 5 * (size_t)RS; }
   cx.q0_tok = slot_u;                    // input tokens of the oldest
   cx.q1_tok = slot_u + RS;               //   and of the second oldest
   cx.q2_idx = slot_u + 2 * (size_t)RS;   // request index of the third oldest (kNone: none)
   cx.tail = slot_u + 3 * (size_t)RS;     // newest request queued on the slot
   cx.qcnt = slot_u + 4 * (size_t)RS;     // requests in flight on the slot
-  cx.exp_sub = reinterpret_cast<long long*>(smem_raw + pl.exp_sub);
-  cx.st_ab = reinterpret_cast<double*>(smem_raw + pl.st_ab);
-  cx.ctl = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.ctl);
-  sm.progress = cx.ctl + kCtlApplied;
-  sm.abort = cx.ctl + kCtlAbort;
-  sm.occ = reinterpret_cast<uint32_t*>(smem_raw + pl.occ);
-  sm.curreq = reinterpret_cast<uint32_t*>(smem_raw + pl.curreq);
-  sm.curpos = reinterpret_cast<int32_t*>(smem_raw + pl.curpos);
-  sm.lrutail = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.lrutail);
-  sm.c_lrutail = reinterpret_cast<uint32_t*>(smem_raw + pl.c_lrutail);
-  sm.chead = reinterpret_cast<uint32_t*>(smem_raw + pl.chead);
-  sm.act = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.act);
-  sm.ring_head = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.ring_head);
-  sm.ring_tail = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.ring_tail);
-  sm.scan_cr = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.scan_cr);
-  sm.scan_cp = reinterpret_cast<volatile int32_t*>(smem_raw + pl.scan_cp);
-  cx.route_ring = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.route_ring);
-  cx.inval = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.inval);
-  cx.apply_ring = reinterpret_cast<uint4*>(smem_raw + pl.apply_ring);
-  cx.st_ready = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.st_ready);
-  cx.st_pc = reinterpret_cast<volatile uint32_t*>(smem_raw + pl.st_pc);
-  cx.st_hits = reinterpret_cast<uint32_t*>(smem_raw + pl.st_hits);
-  cx.st_ids = reinterpret_cast<uint32_t*>(smem_raw + pl.st_ids);
-  cx.st_mk = reinterpret_cast<MaskT*>(smem_raw + pl.st_mk);
-  sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(smem_raw + pl.lst)
-                           : a.evict_lists + (size_t)p * R * kListCap;
+  sm.progress = unext;
+  cx.route = unext + 1;
+  cx.status = reinterpret_cast<volatile int32_t*>(unext + 2);
+  cx.hit_slot = unext + 3;
+  sm.act = unext + 4;
+  sm.ring_head = sm.act + R;
+  sm.ring_tail = sm.ring_head + R;
+  sm.scan_cr = sm.ring_tail + R;
+  sm.scan_cp = reinterpret_cast<volatile int32_t*>(sm.scan_cr + R);
+  {
+    uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R;
+    cx.st_ready = after;
+    cx.probe_gone = after + kStageDepth;
+    cx.st_hits = after + kStageDepth + 1;
+    cx.st_ids = cx.st_hits + (kStageDepth + 2) * (size_t)R;
+    after = cx.st_ids + (kStageDepth + 2) * (size_t)kStageBlocks;
+    const uintptr_t a8 = (reinterpret_cast<uintptr_t>(after) + 7) & ~(uintptr_t)7;
+    cx.st_ab = reinterpret_cast<double*>(a8);
+    cx.st_mk = reinterpret_cast<MaskT*>(cx.st_ab + (kStageDepth + 2) * (size_t)R);
+    after = reinterpret_cast<uint32_t*>(cx.st_mk + (kStageDepth + 2) * (size_t)kStageBlocks);
+    const uintptr_t al = (reinterpret_cast<uintptr_t>(after) + 15) & ~(uintptr_t)15;
+    sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(al)
+                             : a.evict_lists + (size_t)p * R * kListCap;
+  }
   cx.mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
   cx.qrec = a.qrec + (size_t)p * N;   // per request: (finish lo, finish hi, next on slot, tokens)
   cx.lru_next = a.lru_next + (size_t)p * N;
@@ -1356,30 +997,19 @@ __global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayA
     const RepState rs = g_rep[i];
     sm.minfin[i] = rs.min_fin; sm.load[i] = rs.load; sm.occ[i] = rs.occ;
     sm.curreq[i] = rs.cur_req; sm.curpos[i] = rs.cur_pos; sm.lrutail[i] = rs.lru_tail;
-    sm.c_lrutail[i] = rs.lru_tail; sm.chead[i] = 0;
     sm.act[i] = 0; sm.ring_head[i] = 0; sm.ring_tail[i] = 0;
   }
   if (a.slots_in_smem) {
     for (uint32_t x = threadIdx.x; x < 3 * RS; x += blockDim.x) slot_d[x] = g_slot_d[x];
     for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) slot_u[x] = g_slot_u[x];
   }
-  if (threadIdx.x < kCtlWords) {
-    uint32_t v = 0;
-    if (threadIdx.x == kCtlRouted || threadIdx.x == kCtlApplied || threadIdx.x == kCtlChecked ||
-        threadIdx.x == kCtlEnqueued ||
-        (threadIdx.x >= kCtlExp && threadIdx.x < kCtlServed + kQueueWarps))
-      v = a.first;
-    cx.ctl[threadIdx.x] = v;
-  }
-  if (threadIdx.x < kStageDepth) { cx.st_ready[threadIdx.x] = 0; cx.st_pc[threadIdx.x] = 0; }
-  if (threadIdx.x < kInvalRing) cx.inval[threadIdx.x] = 0;
+  if (threadIdx.x == 0) { *sm.progress = a.first; *cx.status = 0; *cx.probe_gone = 0; }
+  if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
   __syncthreads();
 
-  if (warp == kWarpRoute) route_warp<MaskT>(a, cx, lane);
-  else if (warp == kWarpCheck) check_warp<MaskT>(a, cx, lane);
-  else if (warp == kWarpApply) apply_warp<MaskT>(a, cx, p, lane);
-  else if (warp < kWarpProbe0) queue_warp<MaskT>(a, cx, p, lane, warp - kWarpQueue0);
-  else if (warp < kWarpScout0) probe_warp<MaskT>(a, cx, lane, warp - kWarpProbe0);
+  if (warp == kWarpDecide) decide_warp<MaskT>(a, cx, p, lane);
+  else if (warp == kWarpCache) cache_warp<MaskT>(a, cx, p, lane);
+  else if (warp == kWarpProbe) probe_warp<MaskT>(a, cx, lane);
   else scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, warp - kWarpScout0);
   __syncthreads();
 
@@ -1395,54 +1025,11 @@ __global__ void __launch_bounds__(kReplayThreads, 2) replay_kernel(const ReplayA
     for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) g_slot_u[x] = slot_u[x];
   }
   if (threadIdx.x == 0) {
-    const int32_t status = (int32_t)cx.ctl[kCtlStatus];
+    const int32_t status = *cx.status;
     hdr->processed = a.first + a.count;
     if (status != 0) hdr->status = status;
     if (a.status_out && (status != 0 || !a.check_order)) a.status_out[p] = status;
   }
-}
-
-// ---------------------------------------------------------------- expiry lower bound
-// need_svc[e] = one past the last request j < e (within the launch) that can have finished by
-// the arrival of e.  A request finishes no earlier than its arrival plus its decode time
-// (network, queueing and prefill only add to that, and every rounding is monotone), so with
-// lb_j = t'_j + tpot * max(out_j - 1, 0) and e_j = first request after j with t'_e >= lb_j,
-// need_svc[e] = max{ j + 1 : e_j <= e }.  Depends on the trace and the time scale only.
-__global__ void need_scatter_kernel(const ReqRec* req, double scale, double tpot_ms,
-                                    uint32_t first, uint32_t count, uint32_t* need, double* tq) {
-  const uint32_t x = blockIdx.x * blockDim.x + threadIdx.x;
-  if (x >= count) return;
-  const uint32_t j = first + x, end = first + count;
-  const ReqRec rec = req[j];
-  const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
-  const double t = __dmul_rn(scale, rec.ts_ms);          // scaled arrival, kept for the queue warps
-  tq[j] = t;
-  const double lb = __dadd_rn(t, __dmul_rn(tpot_ms, (double)dec_tok));
-  uint32_t lo = j + 1, hi = end;
-  while (lo < hi) {
-    const uint32_t mid = lo + (hi - lo) / 2;
-    if (__dmul_rn(scale, req[mid].ts_ms) >= lb) hi = mid; else lo = mid + 1;
-  }
-  if (lo < end) atomicMax(need + lo, j + 1);
-}
-
-constexpr int kScanThreads = 1024;
-__global__ void __launch_bounds__(kScanThreads) need_scan_kernel(uint32_t first, uint32_t count,
-                                                                 uint32_t* need) {
-  __shared__ uint32_t part[kScanThreads];
-  const uint32_t per = (count + kScanThreads - 1) / kScanThreads;
-  const uint32_t b = first + min(count, threadIdx.x * per), e = first + min(count, (threadIdx.x + 1) * per);
-  uint32_t m = 0;
-  for (uint32_t i = b; i < e; ++i) m = max(m, need[i]);
-  part[threadIdx.x] = m;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t run = 0;
-    for (int t = 0; t < kScanThreads; ++t) { const uint32_t v = part[t]; part[t] = run; run = max(run, v); }
-  }
-  __syncthreads();
-  m = part[threadIdx.x];                                  // maximum over the chunks before mine
-  for (uint32_t i = b; i < e; ++i) { m = max(m, need[i]); need[i] = m; }
 }
 
 // ------------------------------------------------------------------------------- reset
@@ -1578,8 +1165,15 @@ size_t replay_smem_bytes(ReplayArgs& a) {
   const size_t list_bytes = (size_t)a.m.R * kListCap * sizeof(uint4);
   a.slots_in_smem = rs * 44 <= 44 * 1024 ? 1u : 0u;
   a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
-  return smem_plan(a.m.R, a.m.G, a.m.S, a.m.K, (uint32_t)sizeof(MaskT), a.slots_in_smem != 0,
-                   a.lists_in_smem != 0).total;
+  size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
+                (9 * (size_t)a.m.R + 4) * sizeof(uint32_t) + 16 +
+                (kStageDepth + 1 + (kStageDepth + 2) * ((size_t)a.m.R + kStageBlocks)) * sizeof(uint32_t) +
+                8 + (kStageDepth + 2) * (size_t)a.m.R * sizeof(double) +
+                (kStageDepth + 2) * kStageBlocks * sizeof(MaskT) + 8;
+  if (a.slots_in_smem) smem += rs * 44;
+  if (a.lists_in_smem) smem += list_bytes;
+  smem = (smem + 15) / 16 * 16;
+  return smem;
 }
 
 template <typename MaskT>
@@ -1596,16 +1190,6 @@ cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
     cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT>,
                                          cudaFuncAttributePreferredSharedMemoryCarveout,
                                          (int)cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-  }
-  // which earlier requests can have finished by the arrival of each request (all candidates)
-  {
-    cudaError_t e = cudaMemsetAsync(a.need_svc + a.first, 0, (size_t)a.count * sizeof(uint32_t), st);
-    if (e != cudaSuccess) return e;
-    need_scatter_kernel<<<(a.count + 255) / 256, 256, 0, st>>>(a.tr.req, a.scale, a.m.tpot_ms,
-                                                               a.first, a.count, a.need_svc, a.tq);
-    need_scan_kernel<<<1, kScanThreads, 0, st>>>(a.first, a.count, a.need_svc);
-    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
   replay_kernel<MaskT><<<n_cand, kReplayThreads, smem, st>>>(a);
@@ -1685,18 +1269,3 @@ cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st)
 }
 
 }  // namespace gorgo
-
-#ifdef GORGO_PROF
-namespace gorgo {
-int prof_read(unsigned long long* out, int clear) {
-  cudaDeviceSynchronize();
-  if (cudaMemcpyFromSymbol(out, g_prof, sizeof(g_prof)) != cudaSuccess) return -1;
-  if (clear) {
-    static unsigned long long z[256];
-    cudaMemcpyToSymbol(g_prof, z, sizeof(z));
-  }
-  return 0;
-}
-}  // namespace gorgo
-extern "C" int gorgo_prof_read(unsigned long long* out, int clear) { return gorgo::prof_read(out, clear); }
-#endif
