@@ -160,6 +160,64 @@ int gorgo_state_digest(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
 int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_bytes,
                        void *cuda_stream, uint64_t *requests_seen);
 
+/* Rolling-window tuning objective (paper Section 4: the online tuner minimises the p95 TTFT of
+ * a rolling 128-request window with hop 32; the caption of its convergence figure reports the
+ * best window).  Window j covers requests [j*hop, j*hop + window) in trace order and its value is
+ * the nearest-rank p95 of their TTFTs, the k-th smallest with k = ceil(0.95 * window);
+ * n_windows = (N - window) / hop + 1 (gorgo_window_count), 0 when N < window.
+ * gorgo_eval_population_windows replays the population like gorgo_eval_population and reduces
+ * each candidate's TTFTs to: `win_p95_ttft_ms` DEVICE P*n_windows doubles, row-major, or NULL;
+ * `best_win_p95_ttft_ms` DEVICE P doubles, the smallest window value (required);
+ * `best_window` DEVICE P uint32, the first window that attains it, or NULL; `p95_ttft_ms` and
+ * `p95_e2e_ms` DEVICE P doubles each, the whole-replay p95s, both or neither NULL;
+ * `cand_status` DEVICE P int32 or NULL.  `params` HOST or DEVICE.  Work is enqueued on
+ * `cuda_stream`.  Errors: GORGO_ERR_INVALID_ARG for window = 0, hop = 0, window > 2048 or
+ * N < window; otherwise those of gorgo_eval_population. */
+int gorgo_window_count(uint64_t n_requests, uint32_t window, uint32_t hop, uint64_t *n_windows);
+int gorgo_eval_population_windows(gorgo_sim_t *sim, uint32_t n_candidates, const double *params,
+                                  double time_scale, void *workspace, uint64_t workspace_bytes,
+                                  void *cuda_stream, uint32_t window, uint32_t hop,
+                                  double *win_p95_ttft_ms, double *best_win_p95_ttft_ms,
+                                  uint32_t *best_window, double *p95_ttft_ms, double *p95_e2e_ms,
+                                  int32_t *cand_status);
+
+/* Evolution strategy of the tuner (paper Section 2.3: a (1+1)-ES perturbs each tuned weight
+ * multiplicatively in log space, Eq. 4  x' = clip(exp(ln x + sigma z), [lo, hi]), keeps the
+ * offspring when it beats the parent on the objective, and adapts sigma by Rechenberg's 1/5
+ * success rule; Section 4: W_rtt and W_queue start at 0.5 and 0.1 in [0.05, 2.0] and
+ * [0.05, 0.5], sigma0 = 0.5).  Here the strategy runs offline on the batched evaluator: step t
+ * draws `lambda` offspring of the parent (lambda = 1 is the paper's strategy), replays them over
+ * the uploaded trace in one population evaluation, takes the one with the smallest objective
+ * (lowest index among equals) and accepts it iff its objective is strictly smaller than the
+ * parent's.  The paper leaves the constants of the 1/5 rule open: sigma is multiplied by
+ * `sigma_up` after an accepted step and by sigma_up^(-1/4) after a rejected one, which leaves it
+ * unchanged at exactly one success in five.  The normal draws are an input: z[(t*lambda + l)*
+ * n_tuned + k] perturbs tuned parameter k of offspring l in step t.  Parameters not listed in
+ * `tuned` keep their value from x0.  The arithmetic of Eq. 4 is done on the host in double
+ * precision with the C library's exp and log; the sum ln x + sigma*z is two rounded operations.
+ * All pointers are HOST except `workspace` (DEVICE, as for gorgo_eval_population).  The call
+ * synchronises `cuda_stream` once per step.  `history`, if not NULL, receives per step
+ * 4 + n_tuned doubles: objective of the best offspring, 1.0 if it was accepted else 0.0, sigma
+ * after the step, objective of the parent after the step, tuned values of the parent after the
+ * step.  Errors: GORGO_ERR_INVALID_ARG (NULL, lambda = 0, n_tuned = 0 or > K, an index >= K,
+ * lo <= 0, hi < lo, x0 of a tuned parameter <= 0, objective > 1), GORGO_ERR_NONFINITE_PARAM,
+ * and those of gorgo_eval_population. */
+typedef struct {
+  uint32_t n_steps;        /* ES steps                                                       */
+  uint32_t lambda;         /* offspring per step                                             */
+  uint32_t n_tuned;        /* number of tuned parameters                                     */
+  uint32_t objective;      /* 0: p95 TTFT of the replay (the paper's), 1: p95 E2E            */
+  const uint32_t *tuned;   /* [n_tuned] their indices in the K-vector                        */
+  const double *lo;        /* [n_tuned] lower clamp, > 0                                     */
+  const double *hi;        /* [n_tuned] upper clamp, >= lo                                   */
+  double sigma0;           /* initial step size, > 0                                         */
+  double sigma_up;         /* > 1                                                            */
+  double time_scale;       /* as for gorgo_eval_population                                   */
+} gorgo_es_config_t;
+int gorgo_es_run(gorgo_sim_t *sim, const gorgo_es_config_t *cfg, const double *x0,
+                 const double *z, void *workspace, uint64_t workspace_bytes, void *cuda_stream,
+                 double *x_best, double *objective_best, double *sigma_final, double *history);
+
 /* Measurement aid (no counterpart in the paper).  With profiling enabled, gorgo_eval_population
  * records a CUDA event on `cuda_stream` directly before and after each launch of the replay
  * kernel (one launch per wave, at most 32 waves are timed).  gorgo_last_replay_ms waits for those

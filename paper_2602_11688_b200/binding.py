@@ -32,6 +32,7 @@ EXPORTS = [
     "gorgo_eval_population_host", "gorgo_state_bytes", "gorgo_sim_reset", "gorgo_route_batch",
     "gorgo_state_digest", "gorgo_state_status", "gorgo_set_profiling", "gorgo_last_replay_ms",
     "gorgo_eval_population_static", "gorgo_replay_occupancy", "gorgo_strerror",
+    "gorgo_window_count", "gorgo_eval_population_windows", "gorgo_es_run",
 ]
 
 
@@ -41,6 +42,13 @@ class gorgo_config_t(C.Structure):
                 ("cache_blocks", C.c_uint64), ("n_params", C.c_uint32), ("reserved", C.c_uint32),
                 ("prefill_ms_per_token", C.c_double), ("tpot_ms", C.c_double),
                 ("rtt_ms", C.c_void_p), ("device", C.c_int32)]
+
+
+class gorgo_es_config_t(C.Structure):
+    _fields_ = [("n_steps", C.c_uint32), ("lambda_", C.c_uint32), ("n_tuned", C.c_uint32),
+                ("objective", C.c_uint32), ("tuned", C.c_void_p), ("lo", C.c_void_p),
+                ("hi", C.c_void_p), ("sigma0", C.c_double), ("sigma_up", C.c_double),
+                ("time_scale", C.c_double)]
 
 
 class GorgoError(RuntimeError):
@@ -79,6 +87,11 @@ def load():
         "gorgo_state_status": [vp, vp, u64, vp, pu64],
         "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp],
         "gorgo_replay_occupancy": [vp, C.POINTER(C.c_int32), pu64],
+        "gorgo_window_count": [u64, u32, u32, pu64],
+        "gorgo_eval_population_windows": [vp, u32, vp, dbl, vp, u64, vp, u32, u32, vp, vp, vp, vp,
+                                          vp, vp],
+        "gorgo_es_run": [vp, C.POINTER(gorgo_es_config_t), vp, vp, vp, u64, vp, vp,
+                         C.POINTER(C.c_double), C.POINTER(C.c_double), vp],
         "gorgo_set_profiling": [vp, i32],
         "gorgo_last_replay_ms": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint32)],
     }
@@ -186,6 +199,48 @@ def gorgo_eval_population_static(sim, n_candidates, params, time_scale, stream, 
     return load().gorgo_eval_population_static(
         sim, int(n_candidates), pp, float(time_scale), stream, _dev_ptr(p95_ttft_ms),
         _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks))
+
+
+def gorgo_window_count(n_requests: int, window: int, hop: int):
+    out = C.c_uint64()
+    rc = load().gorgo_window_count(int(n_requests), int(window), int(hop), C.byref(out))
+    return rc, out.value
+
+
+def gorgo_eval_population_windows(sim, n_candidates, params, time_scale, workspace, stream, window,
+                                  hop, win_p95_ttft_ms, best_win_p95_ttft_ms, best_window=None,
+                                  p95_ttft_ms=None, p95_e2e_ms=None, cand_status=None) -> int:
+    """Population evaluation reduced to the rolling-window objective.  ``params``: float64 numpy
+    array (host) or torch CUDA tensor; every other array: torch CUDA tensor or None."""
+    pp = _np_ptr(params) if isinstance(params, np.ndarray) else _dev_ptr(params)
+    return load().gorgo_eval_population_windows(
+        sim, int(n_candidates), pp, float(time_scale), _dev_ptr(workspace), workspace.numel(),
+        stream, int(window), int(hop), _dev_ptr(win_p95_ttft_ms), _dev_ptr(best_win_p95_ttft_ms),
+        _dev_ptr(best_window), _dev_ptr(p95_ttft_ms), _dev_ptr(p95_e2e_ms), _dev_ptr(cand_status))
+
+
+def gorgo_es_run(sim, *, x0, z, tuned, lo, hi, sigma0, sigma_up, n_steps, lam, workspace, stream,
+                 time_scale=1.0, objective=0):
+    """Runs the evolution strategy; returns (status, x_best[K], objective_best, sigma_final,
+    history[n_steps, 4 + n_tuned]).  All array arguments are host numpy arrays except
+    ``workspace`` (torch CUDA tensor)."""
+    x0 = np.ascontiguousarray(x0, dtype=np.float64)
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    tuned = np.ascontiguousarray(tuned, dtype=np.uint32)
+    lo = np.ascontiguousarray(lo, dtype=np.float64)
+    hi = np.ascontiguousarray(hi, dtype=np.float64)
+    T = tuned.shape[0]
+    assert z.size == n_steps * lam * T and lo.shape == (T,) and hi.shape == (T,)
+    cfg = gorgo_es_config_t(int(n_steps), int(lam), int(T), int(objective), tuned.ctypes.data,
+                            lo.ctypes.data, hi.ctypes.data, float(sigma0), float(sigma_up),
+                            float(time_scale))
+    x_best = np.zeros_like(x0)
+    hist = np.zeros((int(n_steps), 4 + T), dtype=np.float64)
+    fb, sg = C.c_double(), C.c_double()
+    rc = load().gorgo_es_run(sim, C.byref(cfg), _np_ptr(x0), _np_ptr(z), _dev_ptr(workspace),
+                             workspace.numel(), stream, _np_ptr(x_best), C.byref(fb), C.byref(sg),
+                             _np_ptr(hist))
+    return rc, x_best, fb.value, sg.value, hist
 
 
 def gorgo_state_bytes(sim):

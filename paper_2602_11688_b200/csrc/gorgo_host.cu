@@ -129,13 +129,28 @@ bool all_finite(const double* v, uint64_t n) {
 
 bool finite_nonneg(double v) { return std::isfinite(v) && v >= 0.0; }
 
+// Rolling-window objective asked for with an evaluation (all pointers DEVICE).
+struct WindowSpec {
+  uint32_t window, hop;
+  double* win_p95;      // [P * n_windows] or null
+  double* best;         // [P]
+  uint32_t* best_win;   // [P] or null
+};
+
+uint64_t window_count(uint64_t n_requests, uint32_t window, uint32_t hop) {
+  return n_requests >= window ? (n_requests - window) / hop + 1 : 0;
+}
+
 int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, void* workspace,
               uint64_t workspace_bytes, cudaStream_t st, double* p95_ttft, double* p95_e2e,
               uint8_t* route, uint16_t* hit, uint64_t* digest, uint64_t* stats, int32_t* cand_status,
-              bool host_io) {
+              bool host_io, const WindowSpec* win = nullptr) {
   if (!sim || !params || !workspace || P == 0) return GORGO_ERR_INVALID_ARG;
-  if (!p95_ttft || !p95_e2e) return GORGO_ERR_INVALID_ARG;
+  if ((!p95_ttft || !p95_e2e) && !win) return GORGO_ERR_INVALID_ARG;
+  if (win && (win->window == 0 || win->hop == 0 || win->window > window_max() || !win->best))
+    return GORGO_ERR_INVALID_ARG;
   if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  if (win && sim->tr.n_req < win->window) return GORGO_ERR_INVALID_ARG;
   if (!finite_nonneg(scale)) return GORGO_ERR_NONFINITE_PARAM;
   if ((uintptr_t)workspace % kAlign) return GORGO_ERR_INVALID_ARG;
   DeviceGuard guard(sim->device);
@@ -210,11 +225,25 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
       sim->ev_used += 2;
     }
 
-    SelectArgs s = {};
-    s.ttft = a.ttft_out; s.e2e = a.e2e_out; s.stride = N; s.n = (uint32_t)N;
-    s.p95_ttft = host_io ? d_p95 : p95_ttft + p0;
-    s.p95_e2e = host_io ? d_p95 + res : p95_e2e + p0;
-    if (launch_select(s, pw, st) != cudaSuccess) return GORGO_ERR_CUDA;
+    if (p95_ttft && p95_e2e) {
+      SelectArgs s = {};
+      s.ttft = a.ttft_out; s.e2e = a.e2e_out; s.stride = N; s.n = (uint32_t)N;
+      s.p95_ttft = host_io ? d_p95 : p95_ttft + p0;
+      s.p95_e2e = host_io ? d_p95 + res : p95_e2e + p0;
+      if (launch_select(s, pw, st) != cudaSuccess) return GORGO_ERR_CUDA;
+    }
+    if (win) {
+      // window values go to the caller's array, else over the E2E scratch (no longer needed)
+      WindowArgs wa = {};
+      const uint64_t n_win = window_count(N, win->window, win->hop);
+      wa.values = a.ttft_out; wa.stride = N;
+      wa.window = win->window; wa.hop = win->hop; wa.n_win = (uint32_t)n_win;
+      wa.win_p95 = win->win_p95 ? win->win_p95 + (size_t)p0 * n_win : a.e2e_out;
+      wa.win_stride = win->win_p95 ? n_win : N;
+      wa.best = win->best + p0;
+      wa.best_win = win->best_win ? win->best_win + p0 : nullptr;
+      if (launch_window(wa, pw, st) != cudaSuccess) return GORGO_ERR_CUDA;
+    }
 
     if (digest) {
       DigestArgs d = {};
@@ -418,12 +447,105 @@ int gorgo_eval_population(gorgo_sim_t* sim, uint32_t n_candidates, const double*
                    hit_blocks, state_digest, stats, cand_status, false);
 }
 
+int gorgo_eval_population_windows(gorgo_sim_t* sim, uint32_t n_candidates, const double* params,
+                                  double time_scale, void* workspace, uint64_t workspace_bytes,
+                                  void* cuda_stream, uint32_t window, uint32_t hop,
+                                  double* win_p95_ttft_ms, double* best_win_p95_ttft_ms,
+                                  uint32_t* best_window, double* p95_ttft_ms, double* p95_e2e_ms,
+                                  int32_t* cand_status) {
+  WindowSpec w = {window, hop, win_p95_ttft_ms, best_win_p95_ttft_ms, best_window};
+  if ((p95_ttft_ms == nullptr) != (p95_e2e_ms == nullptr)) return GORGO_ERR_INVALID_ARG;
+  return eval_impl(sim, n_candidates, params, time_scale, workspace, workspace_bytes,
+                   static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, nullptr, nullptr,
+                   nullptr, nullptr, cand_status, false, &w);
+}
+
+int gorgo_window_count(uint64_t n_requests, uint32_t window, uint32_t hop, uint64_t* n_windows) {
+  if (!n_windows || window == 0 || hop == 0) return GORGO_ERR_INVALID_ARG;
+  *n_windows = window_count(n_requests, window, hop);
+  return GORGO_OK;
+}
+
 int gorgo_eval_population_host(gorgo_sim_t* sim, uint32_t n_candidates, const double* params,
                                double time_scale, void* workspace, uint64_t workspace_bytes,
                                void* cuda_stream, double* p95_ttft_ms, double* p95_e2e_ms) {
   return eval_impl(sim, n_candidates, params, time_scale, workspace, workspace_bytes,
                    static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, nullptr,
                    nullptr, nullptr, nullptr, nullptr, true);
+}
+
+// (1+lambda) evolution strategy of the paper's tuner (Section 2.3, Eq. 4) on top of the batched
+// evaluator: every step mutates the parent lambda times, replays all offspring in one population
+// evaluation, and keeps the best one if it beats the parent.  Host logic only; the replays and
+// their p95 reduction run on the device.
+int gorgo_es_run(gorgo_sim_t* sim, const gorgo_es_config_t* cfg, const double* x0, const double* z,
+                 void* workspace, uint64_t workspace_bytes, void* cuda_stream, double* x_best,
+                 double* objective_best, double* sigma_final, double* history) {
+  if (!sim || !cfg || !x0 || !z || !workspace || !x_best || !objective_best || !sigma_final)
+    return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  const uint32_t K = sim->m.K, T = cfg->n_tuned, L = cfg->lambda;
+  if (L == 0 || T == 0 || T > K || !cfg->tuned || !cfg->lo || !cfg->hi || cfg->objective > 1)
+    return GORGO_ERR_INVALID_ARG;
+  if (!(cfg->sigma0 > 0.0) || !std::isfinite(cfg->sigma0) || !(cfg->sigma_up > 1.0) ||
+      !std::isfinite(cfg->sigma_up))
+    return GORGO_ERR_NONFINITE_PARAM;
+  if (!all_finite(x0, K) || !all_finite(z, (uint64_t)cfg->n_steps * L * T))
+    return GORGO_ERR_NONFINITE_PARAM;
+  for (uint32_t k = 0; k < T; ++k) {
+    if (cfg->tuned[k] >= K) return GORGO_ERR_INVALID_ARG;
+    if (!(cfg->lo[k] > 0.0) || !(cfg->hi[k] >= cfg->lo[k]) || !std::isfinite(cfg->hi[k]))
+      return GORGO_ERR_INVALID_ARG;
+    if (!(x0[cfg->tuned[k]] > 0.0)) return GORGO_ERR_INVALID_ARG;   // ln(x) of Eq. 4
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  std::vector<double> parent(x0, x0 + K), pop((size_t)L * K), pt(L), pe(L);
+  // the parent's own objective
+  double ft = 0.0, fe = 0.0;
+  int rc = eval_impl(sim, 1, parent.data(), cfg->time_scale, workspace, workspace_bytes, st, &ft,
+                     &fe, nullptr, nullptr, nullptr, nullptr, nullptr, true);
+  if (rc != GORGO_OK) return rc;
+  double f_parent = cfg->objective == 0 ? ft : fe;
+  double sigma = cfg->sigma0;
+  const double down = std::pow(cfg->sigma_up, -0.25);   // one success in five keeps sigma in place
+  for (uint32_t t = 0; t < cfg->n_steps; ++t) {
+    for (uint32_t l = 0; l < L; ++l) {
+      double* x = pop.data() + (size_t)l * K;
+      std::copy(parent.begin(), parent.end(), x);
+      for (uint32_t k = 0; k < T; ++k) {
+        const double step = sigma * z[((size_t)t * L + l) * T + k];
+        double v = std::exp(std::log(parent[cfg->tuned[k]]) + step);     // Eq. 4
+        if (v < cfg->lo[k]) v = cfg->lo[k];
+        if (v > cfg->hi[k]) v = cfg->hi[k];
+        x[cfg->tuned[k]] = v;
+      }
+    }
+    rc = eval_impl(sim, L, pop.data(), cfg->time_scale, workspace, workspace_bytes, st, pt.data(),
+                   pe.data(), nullptr, nullptr, nullptr, nullptr, nullptr, true);
+    if (rc != GORGO_OK) return rc;
+    const std::vector<double>& f = cfg->objective == 0 ? pt : pe;
+    uint32_t best = 0;
+    for (uint32_t l = 1; l < L; ++l)
+      if (f[l] < f[best]) best = l;                 // lowest index among equals
+    const bool accept = f[best] < f_parent;         // the offspring has to beat the parent
+    const double f_best = f[best];
+    if (accept) {
+      std::copy(pop.begin() + (size_t)best * K, pop.begin() + (size_t)(best + 1) * K, parent.begin());
+      f_parent = f_best;
+      sigma *= cfg->sigma_up;
+    } else {
+      sigma *= down;
+    }
+    if (history) {
+      double* h = history + (size_t)t * (4 + T);
+      h[0] = f_best; h[1] = accept ? 1.0 : 0.0; h[2] = sigma; h[3] = f_parent;
+      for (uint32_t k = 0; k < T; ++k) h[4 + k] = parent[cfg->tuned[k]];
+    }
+  }
+  std::copy(parent.begin(), parent.end(), x_best);
+  *objective_best = f_parent;
+  *sigma_final = sigma;
+  return GORGO_OK;
 }
 
 int gorgo_state_bytes(const gorgo_sim_t* sim, uint64_t* bytes_out) {

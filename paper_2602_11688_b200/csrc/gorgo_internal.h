@@ -107,6 +107,16 @@ struct SelectArgs {
   double* p95_e2e;
 };
 
+struct WindowArgs {
+  const double* values;           // [P*stride] per-request values (TTFT), request order
+  uint64_t stride;
+  uint32_t window, hop, n_win;    // window j covers values [j*hop, j*hop + window)
+  double* win_p95;                // [P*win_stride] window values (output, also input of the best)
+  uint64_t win_stride;
+  double* best;                   // [P] smallest window value
+  uint32_t* best_win;             // [P] first window attaining it, or null
+};
+
 struct DigestArgs {
   Model m;
   TraceView tr;
@@ -123,6 +133,8 @@ cudaError_t launch_reset(unsigned char* masks, uint64_t mask_bytes_total, unsign
 cudaError_t launch_replay(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st);
+cudaError_t launch_window(const WindowArgs& a, uint32_t n_cand, cudaStream_t st);
+uint32_t window_max();          // largest window the window kernel handles
 uint32_t mask_bytes_for(uint32_t n_replicas);
 uint64_t evict_list_bytes(uint32_t n_replicas);
 // CTAs of the replay kernel that fit one SM for this model (-1: query failed), and the dynamic

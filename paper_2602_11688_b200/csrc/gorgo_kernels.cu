@@ -1120,6 +1120,69 @@ __global__ void __launch_bounds__(kSelectThreads) select_p95_kernel(const Select
   if (threadIdx.x == 0) *out = value_of(s_prefix);
 }
 
+// ------------------------------------------------------------------------ window objective
+// Rolling-window objective of the tuning loop (paper Section 4: p95 TTFT of a rolling 128-request
+// window with hop 32): window j covers requests [j*hop, j*hop + window); its value is the k-th
+// smallest of them, k = ceil(0.95 window) (nearest rank).  One CTA per (candidate, group of
+// windows); a window is copied to shared memory and every thread ranks its elements by counting
+// the smaller ones (ties broken by position), which is exact for any input.
+constexpr int kWindowThreads = 128;
+constexpr uint32_t kWindowMax = 2048;      // values of one window kept in shared memory
+
+__global__ void __launch_bounds__(kWindowThreads) window_p95_kernel(const WindowArgs a) {
+  __shared__ uint64_t keys[kWindowMax];
+  const uint32_t p = blockIdx.x;
+  const double* v = a.values + (size_t)p * a.stride;
+  double* out = a.win_p95 + (size_t)p * a.win_stride;
+  const uint32_t W = a.window;
+  const uint32_t rank = (uint32_t)((95ull * W + 99ull) / 100ull) - 1u;   // 0-based
+  for (uint32_t j = blockIdx.y; j < a.n_win; j += gridDim.y) {
+    const double* wv = v + (size_t)j * a.hop;
+    for (uint32_t i = threadIdx.x; i < W; i += blockDim.x) keys[i] = key_of(wv[i]);
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < W; i += blockDim.x) {
+      const uint64_t ki = keys[i];
+      uint32_t below = 0;
+      for (uint32_t x = 0; x < W; ++x) {
+        const uint64_t kx = keys[x];
+        below += (kx < ki || (kx == ki && x < i)) ? 1u : 0u;
+      }
+      if (below == rank) out[j] = value_of(ki);
+    }
+    __syncthreads();
+  }
+}
+
+// Smallest window value of every candidate and the first window that attains it.
+__global__ void __launch_bounds__(256) window_best_kernel(const WindowArgs a) {
+  const uint32_t p = blockIdx.x;
+  const double* w = a.win_p95 + (size_t)p * a.win_stride;
+  __shared__ uint64_t s_key[256];
+  __shared__ uint32_t s_idx[256];
+  uint64_t bk = ~0ull;
+  uint32_t bi = kNone;
+  for (uint32_t j = threadIdx.x; j < a.n_win; j += blockDim.x) {
+    const uint64_t k = key_of(w[j]);
+    if (k < bk) { bk = k; bi = j; }            // ascending j per thread: first minimum kept
+  }
+  s_key[threadIdx.x] = bk; s_idx[threadIdx.x] = bi;
+  __syncthreads();
+  for (uint32_t d = 128; d > 0; d >>= 1) {
+    if (threadIdx.x < d) {
+      const uint64_t ok = s_key[threadIdx.x + d];
+      const uint32_t oi = s_idx[threadIdx.x + d];
+      if (ok < s_key[threadIdx.x] || (ok == s_key[threadIdx.x] && oi < s_idx[threadIdx.x])) {
+        s_key[threadIdx.x] = ok; s_idx[threadIdx.x] = oi;
+      }
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    a.best[p] = a.n_win ? value_of(s_key[0]) : 0.0;
+    if (a.best_win) a.best_win[p] = s_idx[0];
+  }
+}
+
 // ------------------------------------------------------------------------------ digest
 // Per replica: occupancy and the sum over cached blocks of mix64(id ^ mix64(seq*65536+pos)).
 // A block's latest touch on its replica is cached iff it lies at or after the eviction cursor.
@@ -1257,6 +1320,17 @@ cudaError_t launch_replay(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st)
 
 cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st) {
   select_p95_kernel<<<dim3(n_cand, 2), kSelectThreads, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+uint32_t window_max() { return kWindowMax; }
+
+cudaError_t launch_window(const WindowArgs& a, uint32_t n_cand, cudaStream_t st) {
+  if (a.n_win > 0) {
+    const uint32_t groups = a.n_win < 1024u ? a.n_win : 1024u;
+    window_p95_kernel<<<dim3(n_cand, groups), kWindowThreads, 0, st>>>(a);
+  }
+  window_best_kernel<<<n_cand, 256, 0, st>>>(a);
   return cudaGetLastError();
 }
 
