@@ -229,6 +229,8 @@ int gorgo_es_run(gorgo_sim_t *sim, const gorgo_es_config_t *cfg, const double *x
 int gorgo_replay_occupancy(gorgo_sim_t *sim, int32_t *ctas_per_sm, uint64_t *smem_bytes_per_cta);
 int gorgo_set_profiling(gorgo_sim_t *sim, int enable);
 int gorgo_last_replay_ms(gorgo_sim_t *sim, double *replay_ms, uint32_t *launches);
+/* The same for the window-objective kernels of the most recent gorgo_eval_population_windows. */
+int gorgo_last_window_ms(gorgo_sim_t *sim, double *window_ms, uint32_t *launches);
 
 /* Population evaluation for callers that cannot allocate device memory (the paper has no
  * counterpart; this is a packaging variant of gorgo_eval_population).  Some hosts of this library

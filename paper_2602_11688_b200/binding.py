@@ -33,6 +33,7 @@ EXPORTS = [
     "gorgo_state_digest", "gorgo_state_status", "gorgo_set_profiling", "gorgo_last_replay_ms",
     "gorgo_eval_population_static", "gorgo_replay_occupancy", "gorgo_strerror",
     "gorgo_window_count", "gorgo_eval_population_windows", "gorgo_es_run",
+    "gorgo_last_window_ms",
 ]
 
 
@@ -94,6 +95,7 @@ def load():
                          C.POINTER(C.c_double), C.POINTER(C.c_double), vp],
         "gorgo_set_profiling": [vp, i32],
         "gorgo_last_replay_ms": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint32)],
+        "gorgo_last_window_ms": [vp, C.POINTER(C.c_double), C.POINTER(C.c_uint32)],
     }
     for name, argtypes in sig.items():
         fn = getattr(lib, name)
@@ -289,6 +291,14 @@ def gorgo_last_replay_ms(sim):
     """Returns (status, summed replay-kernel milliseconds, timed launches) of the last evaluation."""
     ms, n = C.c_double(), C.c_uint32()
     rc = load().gorgo_last_replay_ms(sim, C.byref(ms), C.byref(n))
+    return rc, ms.value, n.value
+
+
+def gorgo_last_window_ms(sim):
+    """Returns (status, summed window-kernel milliseconds, timed launches) of the last
+    gorgo_eval_population_windows."""
+    ms, n = C.c_double(), C.c_uint32()
+    rc = load().gorgo_last_window_ms(sim, C.byref(ms), C.byref(n))
     return rc, ms.value, n.value
 
 

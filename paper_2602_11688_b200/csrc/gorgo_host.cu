@@ -20,8 +20,10 @@ struct gorgo_sim {
   TraceView tr = {};
   // optional CUDA-event timing of the replay kernel (one pair per wave of the last evaluation)
   bool profiling = false;
-  std::vector<cudaEvent_t> ev;
+  std::vector<cudaEvent_t> ev;    // pairs around the replay launches
   uint32_t ev_used = 0;
+  std::vector<cudaEvent_t> wev;   // pairs around the window-objective launches
+  uint32_t wev_used = 0;
 };
 
 namespace {
@@ -181,6 +183,7 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
   std::vector<int32_t> h_status;
   if (host_io) h_status.assign(P, 0);
   sim->ev_used = 0;
+  sim->wev_used = 0;
 
   for (uint32_t p0 = 0; p0 < P; p0 += res) {
     const uint32_t pw = (P - p0 < res) ? (P - p0) : res;
@@ -242,7 +245,13 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
       wa.win_stride = win->win_p95 ? n_win : N;
       wa.best = win->best + p0;
       wa.best_win = win->best_win ? win->best_win + p0 : nullptr;
+      const bool wtimed = sim->profiling && sim->wev_used + 2 <= sim->wev.size();
+      if (wtimed && cudaEventRecord(sim->wev[sim->wev_used], st) != cudaSuccess) return GORGO_ERR_CUDA;
       if (launch_window(wa, pw, st) != cudaSuccess) return GORGO_ERR_CUDA;
+      if (wtimed) {
+        if (cudaEventRecord(sim->wev[sim->wev_used + 1], st) != cudaSuccess) return GORGO_ERR_CUDA;
+        sim->wev_used += 2;
+      }
     }
 
     if (digest) {
@@ -307,6 +316,7 @@ int gorgo_sim_destroy(gorgo_sim_t* sim) {
   if (!sim->ev.empty()) {
     DeviceGuard guard(sim->device);
     for (cudaEvent_t e : sim->ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : sim->wev) cudaEventDestroy(e);
   }
   delete sim;
   return GORGO_OK;
@@ -677,8 +687,38 @@ int gorgo_set_profiling(gorgo_sim_t* sim, int enable) {
       }
     }
   }
+  if (enable && sim->wev.empty()) {
+    DeviceGuard guard(sim->device);
+    if (!guard.ok) return GORGO_ERR_CUDA;
+    sim->wev.resize(64);
+    for (size_t i = 0; i < sim->wev.size(); ++i) {
+      if (cudaEventCreate(&sim->wev[i]) != cudaSuccess) {
+        for (size_t j = 0; j < i; ++j) cudaEventDestroy(sim->wev[j]);
+        sim->wev.clear();
+        return GORGO_ERR_CUDA;
+      }
+    }
+  }
   sim->profiling = enable != 0;
   sim->ev_used = 0;
+  sim->wev_used = 0;
+  return GORGO_OK;
+}
+
+int gorgo_last_window_ms(gorgo_sim_t* sim, double* window_ms, uint32_t* launches) {
+  if (!sim || !window_ms) return GORGO_ERR_INVALID_ARG;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  double sum = 0.0;
+  for (uint32_t i = 0; i + 1 < sim->wev_used; i += 2) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(sim->wev[i + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, sim->wev[i], sim->wev[i + 1]) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+    sum += ms;
+  }
+  *window_ms = sum;
+  if (launches) *launches = sim->wev_used / 2;
   return GORGO_OK;
 }
 
