@@ -81,6 +81,13 @@ struct Oracle {
     std::vector<Replica> rep;
     uint64_t next = 0;        // next request to process
     uint64_t stats[4] = {0, 0, 0, 0};  // sum_i min(h_i+1,n), sum h*, sum n, sum evicted
+    // Baseline policies of Section 4 inside the same simulator:
+    //  * queue signal counted in requests instead of tokens ("least-request": the replica with
+    //    the fewest in-flight requests from the proxy; in flight as for the token signal);
+    //  * routes fixed in advance, one per request ("simple-session-affinity", "random": the
+    //    choice does not depend on the simulator's state; the caller derives it).
+    bool queue_in_requests = false;
+    std::vector<uint8_t> forced_route;   // empty: route by the score
 };
 
 }  // namespace
@@ -174,7 +181,7 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
             while (hh < n && rp.cache.count(id[hh])) ++hh;
             hits[i] = hh;
             unc[i] = in - std::min<uint64_t>(hh * o->B, in);
-            double q = (double)rp.load;
+            double q = o->queue_in_requests ? (double)rp.inflight.size() : (double)rp.load;
             if (o->K != 3) q = q * w[3 + i];               // per-replica queue-load normaliser
             // Eq. 3 with explicit weights: three products, two sums, in this order
             const double a = w[0] * o->rtt[(size_t)g * R + i];
@@ -189,6 +196,7 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
         uint32_t best = 0;                                 // lowest index wins ties
         for (uint32_t i = 1; i < R; ++i)
             if (cost[i] < cost[best]) best = i;
+        if (!o->forced_route.empty()) best = o->forced_route[r];
 
         // ---- cache commit on the chosen replica (set semantics) ----
         Replica& rp = o->rep[best];
@@ -249,6 +257,20 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
         o->stats[3] += ev;
     }
     return done;
+}
+
+// Baseline-policy switches (see the Oracle struct).  `forced_route` holds one replica index per
+// request of the trace, or is NULL to route by the score again.  Returns 0, or -1 if an index is
+// out of range.
+int gorgo_oracle_set_policy(void* h, uint32_t queue_in_requests, const uint8_t* forced_route) {
+    Oracle* o = static_cast<Oracle*>(h);
+    if (forced_route)
+        for (uint64_t r = 0; r < o->N; ++r)
+            if (forced_route[r] >= o->R) return -1;
+    o->queue_in_requests = queue_in_requests != 0;
+    if (forced_route) o->forced_route.assign(forced_route, forced_route + o->N);
+    else o->forced_route.clear();
+    return 0;
 }
 
 // Nearest-rank percentile: the k-th smallest with k = ceil(0.95 n) in integers.

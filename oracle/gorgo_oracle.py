@@ -55,6 +55,8 @@ def _load():
         lib.gorgo_oracle_dump.argtypes = [vp, C.c_uint32, u64, vp, vp, vp]
         lib.gorgo_oracle_queues.argtypes = [vp, vp, vp, vp]
         lib.gorgo_oracle_stats.argtypes = [vp, vp]
+        lib.gorgo_oracle_set_policy.restype = C.c_int
+        lib.gorgo_oracle_set_policy.argtypes = [vp, C.c_uint32, vp]
         lib.gorgo_oracle_position.restype = u64
         lib.gorgo_oracle_position.argtypes = [vp]
         _lib = lib
@@ -123,6 +125,15 @@ class Oracle:
     def reset(self):
         self._lib.gorgo_oracle_reset(self._h)
 
+    def set_policy(self, queue_in_requests: bool = False, forced_route=None):
+        """Baseline policies of Section 4: queue signal in requests instead of tokens, and/or one
+        fixed replica per request (None: route by the score)."""
+        fr = None if forced_route is None else np.ascontiguousarray(forced_route, dtype=np.uint8)
+        assert fr is None or fr.shape == (self.N,)
+        rc = self._lib.gorgo_oracle_set_policy(self._h, int(bool(queue_in_requests)), _ptr(fr))
+        if rc != 0:
+            raise ValueError("forced route out of range")
+
     @property
     def position(self) -> int:
         return int(self._lib.gorgo_oracle_position(self._h))
@@ -171,11 +182,14 @@ class Oracle:
         return out
 
 
-def replay(workload, w, scale: float = 1.0, detail: bool = False):
+def replay(workload, w, scale: float = 1.0, detail: bool = False, queue_in_requests: bool = False,
+           forced_route=None):
     """Full replay of one candidate from the empty state: (RunResult, p95_ttft, p95_e2e,
     digest[R,2], stats[4])."""
     o = Oracle.from_workload(workload)
     try:
+        if queue_in_requests or forced_route is not None:
+            o.set_policy(queue_in_requests, forced_route)
         res = o.run(w, scale, detail=detail)
         return res, p95(res.ttft), p95(res.e2e), o.digest(), o.stats()
     finally:
