@@ -160,6 +160,37 @@ int gorgo_state_digest(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
 int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_bytes,
                        void *cuda_stream, uint64_t *requests_seen);
 
+/* Baseline routing policies of the paper (Section 4, "Baseline policies"; `random` is in its
+ * appendix tables) replayed through the same simulator, so that their TTFT/E2E can be set beside
+ * a tuned cost model's.  The paper runs them against live engines; inside the simulator they read:
+ *   LEAST_LOAD        fewest in-flight input tokens recorded by the proxy (the engine-side terms
+ *                     of the paper's sum do not exist here): the cost model with weights (0,0,1);
+ *   LEAST_REQUEST     fewest in-flight requests: the same with the queue signal counted in
+ *                     requests (in flight as for tokens: finish time > arrival);
+ *   PREFIX_CACHE      longest cached prefix: weights (0,1,0);
+ *   SESSION_AFFINITY  the paper hashes the first 256 tokens of the prompt; the id of the first
+ *                     block stands for them: replica = finaliser(id) mod R, with the 64-bit
+ *                     finaliser z ^= z>>30; z *= 0xbf58476d1ce4e5b9; z ^= z>>27;
+ *                     z *= 0x94d049bb133111eb; z ^= z>>31; replica 0 for a prompt without blocks;
+ *   RANDOM            replica = draws[r] mod R; `draws` HOST, one uint32 per request of the trace
+ *                     (the caller's random numbers; NULL for the other policies).
+ * Ties go to the lowest replica index.  One replay from the empty state; outputs as for
+ * gorgo_eval_population with one candidate: `p95_ttft_ms`, `p95_e2e_ms` DEVICE 1 double each,
+ * `route` DEVICE N bytes or NULL, `hit_blocks` DEVICE N uint16 or NULL, `state_digest` DEVICE
+ * R*2 uint64 or NULL, `cand_status` DEVICE 1 int32 or NULL.  `workspace` as for
+ * gorgo_eval_population with one resident candidate.  The call waits for `cuda_stream`. */
+enum {
+  GORGO_POLICY_LEAST_LOAD = 0,
+  GORGO_POLICY_LEAST_REQUEST = 1,
+  GORGO_POLICY_PREFIX_CACHE = 2,
+  GORGO_POLICY_SESSION_AFFINITY = 3,
+  GORGO_POLICY_RANDOM = 4
+};
+int gorgo_eval_policy(gorgo_sim_t *sim, uint32_t policy, const uint32_t *draws, double time_scale,
+                      void *workspace, uint64_t workspace_bytes, void *cuda_stream,
+                      double *p95_ttft_ms, double *p95_e2e_ms, uint8_t *route,
+                      uint16_t *hit_blocks, uint64_t *state_digest, int32_t *cand_status);
+
 /* Rolling-window tuning objective (paper Section 4: the online tuner minimises the p95 TTFT of
  * a rolling 128-request window with hop 32; the caption of its convergence figure reports the
  * best window).  Window j covers requests [j*hop, j*hop + window) in trace order and its value is

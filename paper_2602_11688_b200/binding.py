@@ -33,7 +33,7 @@ EXPORTS = [
     "gorgo_state_digest", "gorgo_state_status", "gorgo_set_profiling", "gorgo_last_replay_ms",
     "gorgo_eval_population_static", "gorgo_replay_occupancy", "gorgo_strerror",
     "gorgo_window_count", "gorgo_eval_population_windows", "gorgo_es_run",
-    "gorgo_last_window_ms",
+    "gorgo_last_window_ms", "gorgo_eval_policy",
 ]
 
 
@@ -89,6 +89,7 @@ def load():
         "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp],
         "gorgo_replay_occupancy": [vp, C.POINTER(C.c_int32), pu64],
         "gorgo_window_count": [u64, u32, u32, pu64],
+        "gorgo_eval_policy": [vp, u32, vp, dbl, vp, u64, vp, vp, vp, vp, vp, vp, vp],
         "gorgo_eval_population_windows": [vp, u32, vp, dbl, vp, u64, vp, u32, u32, vp, vp, vp, vp,
                                           vp, vp],
         "gorgo_es_run": [vp, C.POINTER(gorgo_es_config_t), vp, vp, vp, u64, vp, vp,
@@ -201,6 +202,23 @@ def gorgo_eval_population_static(sim, n_candidates, params, time_scale, stream, 
     return load().gorgo_eval_population_static(
         sim, int(n_candidates), pp, float(time_scale), stream, _dev_ptr(p95_ttft_ms),
         _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks))
+
+
+POLICIES = {"least-load": 0, "least-request": 1, "prefix-cache": 2, "session-affinity": 3,
+            "random": 4}
+
+
+def gorgo_eval_policy(sim, policy, draws, time_scale, workspace, stream, p95_ttft_ms, p95_e2e_ms,
+                      route=None, hit_blocks=None, state_digest=None, cand_status=None) -> int:
+    """One replay under a baseline policy (name from POLICIES or its number).  ``draws``: host
+    uint32 numpy array with one entry per request (``random`` only, else None); every other
+    array: torch CUDA tensor or None."""
+    pid = POLICIES[policy] if isinstance(policy, str) else int(policy)
+    d = None if draws is None else np.ascontiguousarray(draws, dtype=np.uint32)
+    return load().gorgo_eval_policy(
+        sim, pid, _np_ptr(d), float(time_scale), _dev_ptr(workspace), workspace.numel(), stream,
+        _dev_ptr(p95_ttft_ms), _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks),
+        _dev_ptr(state_digest), _dev_ptr(cand_status))
 
 
 def gorgo_window_count(n_requests: int, window: int, hop: int):

@@ -88,8 +88,8 @@ StateLayout make_layout(const Model& m) {
 
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
-  uint64_t params, rtt, status, p95, masks, states, lists, qrec, lru_next, route_log,
-      ttft, e2e, total;
+  uint64_t params, rtt, status, p95, forced, draws, masks, states, lists, qrec, lru_next,
+      route_log, ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
 };
@@ -105,6 +105,8 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.rtt = o; o = align_up(o + (uint64_t)m.G * m.R * 8);
   w.status = o; o = align_up(o + res * 4);
   w.p95 = o; o = align_up(o + res * 16);
+  w.forced = o; o = align_up(o + N);          // baseline policies: one route per request
+  w.draws = o; o = align_up(o + N * 4);       //   and the caller's draws for `random`
   w.masks = o; o = align_up(o + res * w.mask_stride);
   w.states = o; o = align_up(o + res * w.st.bytes);
   w.lists = o; o = align_up(o + res * evict_list_bytes(m.R));
@@ -132,6 +134,12 @@ bool all_finite(const double* v, uint64_t n) {
 bool finite_nonneg(double v) { return std::isfinite(v) && v >= 0.0; }
 
 // Rolling-window objective asked for with an evaluation (all pointers DEVICE).
+// Baseline policy asked for with an evaluation.
+struct PolicySpec {
+  bool queue_in_requests;
+  const uint8_t* forced_route;   // DEVICE [N] or null
+};
+
 struct WindowSpec {
   uint32_t window, hop;
   double* win_p95;      // [P * n_windows] or null
@@ -146,7 +154,7 @@ uint64_t window_count(uint64_t n_requests, uint32_t window, uint32_t hop) {
 int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, void* workspace,
               uint64_t workspace_bytes, cudaStream_t st, double* p95_ttft, double* p95_e2e,
               uint8_t* route, uint16_t* hit, uint64_t* digest, uint64_t* stats, int32_t* cand_status,
-              bool host_io, const WindowSpec* win = nullptr) {
+              bool host_io, const WindowSpec* win = nullptr, const PolicySpec* pol = nullptr) {
   if (!sim || !params || !workspace || P == 0) return GORGO_ERR_INVALID_ARG;
   if ((!p95_ttft || !p95_e2e) && !win) return GORGO_ERR_INVALID_ARG;
   if (win && (win->window == 0 || win->hop == 0 || win->window > window_max() || !win->best))
@@ -213,6 +221,8 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
     a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
     a.route_log = route ? route + (size_t)p0 * N : base + w.route_log;
     a.route_log_stride = N;
+    a.queue_in_requests = pol && pol->queue_in_requests ? 1u : 0u;
+    a.forced_route = pol ? pol->forced_route : nullptr;
     a.route_out = nullptr;
     a.hit_out = hit ? hit + (size_t)p0 * N : nullptr;
     a.ttft_out = reinterpret_cast<double*>(base + w.ttft);
@@ -468,6 +478,49 @@ int gorgo_eval_population_windows(gorgo_sim_t* sim, uint32_t n_candidates, const
   return eval_impl(sim, n_candidates, params, time_scale, workspace, workspace_bytes,
                    static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, nullptr, nullptr,
                    nullptr, nullptr, cand_status, false, &w);
+}
+
+int gorgo_eval_policy(gorgo_sim_t* sim, uint32_t policy, const uint32_t* draws, double time_scale,
+                      void* workspace, uint64_t workspace_bytes, void* cuda_stream,
+                      double* p95_ttft_ms, double* p95_e2e_ms, uint8_t* route, uint16_t* hit_blocks,
+                      uint64_t* state_digest, int32_t* cand_status) {
+  if (!sim || !workspace || policy > GORGO_POLICY_RANDOM) return GORGO_ERR_INVALID_ARG;
+  if (policy == GORGO_POLICY_RANDOM && !draws) return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  if ((uintptr_t)workspace % kAlign) return GORGO_ERR_INVALID_ARG;
+  const WsLayout w = make_ws(sim, 1, true);
+  if (w.total > workspace_bytes) return GORGO_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* base = static_cast<unsigned char*>(workspace);
+  const uint32_t K = sim->m.K;
+  // weights of the named policy: (w_net, w_prefill, w_queue), normalisers 1
+  std::vector<double> wts(K, 0.0);
+  for (uint32_t k = 3; k < K; ++k) wts[k] = 1.0;
+  PolicySpec ps = {false, nullptr};
+  switch (policy) {
+    case GORGO_POLICY_LEAST_LOAD: wts[2] = 1.0; break;
+    case GORGO_POLICY_LEAST_REQUEST: wts[2] = 1.0; ps.queue_in_requests = true; break;
+    case GORGO_POLICY_PREFIX_CACHE: wts[1] = 1.0; break;
+    default: {
+      DeviceGuard guard(sim->device);
+      if (!guard.ok) return GORGO_ERR_CUDA;
+      uint8_t* d_forced = base + w.forced;
+      uint32_t* d_draws = reinterpret_cast<uint32_t*>(base + w.draws);
+      const bool affinity = policy == GORGO_POLICY_SESSION_AFFINITY;
+      if (!affinity && cudaMemcpyAsync(d_draws, draws, (size_t)sim->tr.n_req * 4,
+                                       cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return GORGO_ERR_CUDA;
+      if (launch_policy_routes(sim->tr, sim->m.R, affinity, d_draws, d_forced, st) != cudaSuccess)
+        return GORGO_ERR_CUDA;
+      ps.forced_route = d_forced;
+    }
+  }
+  const int rc = eval_impl(sim, 1, wts.data(), time_scale, workspace, workspace_bytes, st,
+                           p95_ttft_ms, p95_e2e_ms, route, hit_blocks, state_digest, nullptr,
+                           cand_status, false, nullptr, &ps);
+  // `wts` and the caller's `draws` are host memory read by asynchronous copies
+  if (rc == GORGO_OK && cudaStreamSynchronize(st) != cudaSuccess) return GORGO_ERR_CUDA;
+  return rc;
 }
 
 int gorgo_window_count(uint64_t n_requests, uint32_t window, uint32_t hop, uint64_t* n_windows) {

@@ -88,6 +88,10 @@ struct ReplayArgs {
   uint32_t* lru_next;             // next request routed to the same replica
   uint8_t* route_log;             // chosen replica of every request replayed so far
   uint64_t route_log_stride;      // elements between candidates
+  // baseline policies: queue signal counted in requests instead of tokens; one fixed route per
+  // request of the trace (shared by the candidates of the launch) or null
+  uint32_t queue_in_requests;
+  const uint8_t* forced_route;
   // outputs, candidate p at + p*out_stride, request r at + (r-first); any may be null
   uint8_t* route_out;
   uint16_t* hit_out;
@@ -134,6 +138,8 @@ cudaError_t launch_replay(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st)
 cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_window(const WindowArgs& a, uint32_t n_cand, cudaStream_t st);
+cudaError_t launch_policy_routes(const TraceView& tr, uint32_t R, bool affinity,
+                                 const uint32_t* draws, uint8_t* route, cudaStream_t st);
 uint32_t window_max();          // largest window the window kernel handles
 uint32_t mask_bytes_for(uint32_t n_replicas);
 uint64_t evict_list_bytes(uint32_t n_replicas);

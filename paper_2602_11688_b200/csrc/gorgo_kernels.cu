@@ -162,6 +162,7 @@ constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is t
 // Shared-memory view of one candidate's small state.
 struct Smem {
   double* rtt; double* wrtt; double* w; double* minfin; long long* load;
+  int32_t* cnt;                   // in-flight requests per replica (kept when the queue signal counts requests)
   uint32_t* occ; uint32_t* curreq; int32_t* curpos; uint32_t* lrutail;
   volatile uint32_t* progress;
   // eviction rings, one per replica: filled by the scout warp, drained by the replay warp.
@@ -334,12 +335,16 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
            *qcnt = cx.qcnt;
   uint4* qrec = cx.qrec;
   const double w_que = sm.w[2];
+  const bool by_requests = a.queue_in_requests != 0;   // baseline "least-request" (Section 4)
   int32_t status = 0;
   unsigned long long st_hit = 0, st_blk = 0;
 
   const uint32_t last_r = a.first + a.count - 1;
   ReqRec rec_cur = req[a.first];
   ReqRec rec_nxt = req[min(a.first + 1, last_r)];
+  // routes fixed in advance (baselines that do not look at the state), fetched two ahead
+  uint32_t fr_cur = a.forced_route ? a.forced_route[a.first] : 0u;
+  uint32_t fr_nxt = a.forced_route ? a.forced_route[min(a.first + 1, last_r)] : 0u;
   // a queue refill whose load is in flight: slot index (kNone: none) and the record read
   uint32_t pend_x = kNone;
   uint4 pend_rec = make_uint4(0, 0, 0, 0);
@@ -369,6 +374,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
         const uint32_t ii = i0 + (uint32_t)__ffs((int)due) - 1;
         due &= due - 1;
         long long tok = 0;
+        int32_t gone = 0;
         double mn = d_inf();
         for (uint32_t s = lane; s < S; s += 32) {
           const uint32_t x = ii * S + s;
@@ -379,6 +385,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
             do {
               if (pend_x == x) flush_pending();           // the second entry is still in flight
               tok += (long long)q0_tok[x];
+              ++gone;
               --cnt;
               if (cnt == 0) { hf = d_inf(); }
               else {
@@ -399,6 +406,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
         }
         if (tok != 0)
           atomicAdd(reinterpret_cast<unsigned long long*>(sm.load + ii), (unsigned long long)(-tok));
+        if (by_requests && gone != 0) atomicSub(sm.cnt + ii, gone);
         uint64_t mk = order_key(mn);
         warp_argmin_key(mk, lane);
         if (lane == 0) sm.minfin[ii] = order_value(mk);
@@ -412,7 +420,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
     for (int half = 0; half < 2; ++half) {
       const uint32_t i = lane + 32u * half;
       if (i < R) {
-        double q = (double)sm.load[i];
+        double q = by_requests ? (double)sm.cnt[i] : (double)sm.load[i];
         if (K != 3) q = __dmul_rn(q, sm.w[3 + i]);
         const double c = __dmul_rn(w_que, q);
         if (half) cq1 = c; else cq0 = c;
@@ -436,7 +444,12 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
         if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i; }
       }
     }
-    const uint32_t istar = warp_argmin_key(best_k, best_i);
+    uint32_t istar = warp_argmin_key(best_k, best_i);
+    if (a.forced_route) {
+      istar = fr_cur;
+      fr_cur = fr_nxt;
+      fr_nxt = a.forced_route[min(r + 2, last_r)];
+    }
     const uint32_t hstar = cx.st_hits[stage * R + istar];   // read before the stage can be reused
     if (lane == 0) {
       *cx.route = istar;
@@ -481,6 +494,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
       tail[x] = r;
       free_at[x] = finish;
       sm.load[istar] += (long long)in_tok;
+      if (by_requests) sm.cnt[istar] += 1;
       const size_t o = (size_t)p * a.out_stride + j;
       if (a.route_out) a.route_out[o] = (uint8_t)istar;
       if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
@@ -960,7 +974,8 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   sm.scan_cr = sm.ring_tail + R;
   sm.scan_cp = reinterpret_cast<volatile int32_t*>(sm.scan_cr + R);
   {
-    uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R;
+    sm.cnt = reinterpret_cast<int32_t*>(const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R);
+    uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 3 * (size_t)R;
     cx.st_ready = after;
     cx.probe_gone = after + kStageDepth;
     cx.st_hits = after + kStageDepth + 1;
@@ -1004,6 +1019,12 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
     for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) slot_u[x] = g_slot_u[x];
   }
   if (threadIdx.x == 0) { *sm.progress = a.first; *cx.status = 0; *cx.probe_gone = 0; }
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {   // requests in flight per replica
+    int32_t c = 0;
+    for (uint32_t s2 = 0; s2 < S; ++s2) c += (int32_t)cx.qcnt[(size_t)i * S + s2];
+    sm.cnt[i] = c;
+  }
   if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
   __syncthreads();
 
@@ -1120,6 +1141,25 @@ __global__ void __launch_bounds__(kSelectThreads) select_p95_kernel(const Select
   if (threadIdx.x == 0) *out = value_of(s_prefix);
 }
 
+// ------------------------------------------------------------------------ baseline routes
+// Per-request routes of the baselines that do not look at the simulator's state (paper Section
+// 4): session affinity (the paper hashes the first 256 tokens of the prompt; the id of the first
+// block stands for them: finaliser of the caller's 64-bit id, modulo R; replica 0 for a prompt
+// without blocks) and random (one caller-supplied draw per request, modulo R).
+__global__ void policy_routes_kernel(TraceView tr, uint32_t R, uint32_t affinity,
+                                     const uint32_t* draws, uint8_t* route) {
+  const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= tr.n_req) return;
+  uint32_t i = 0;
+  if (affinity) {
+    const ReqRec q = tr.req[r];
+    if (q.nblk > 0) i = (uint32_t)(mix64(tr.raw_id[tr.ids[q.off]]) % R);
+  } else {
+    i = draws[r] % R;
+  }
+  route[r] = (uint8_t)i;
+}
+
 // ------------------------------------------------------------------------ window objective
 // Rolling-window objective of the tuning loop (paper Section 4: p95 TTFT of a rolling 128-request
 // window with hop 32): window j covers requests [j*hop, j*hop + window); its value is the k-th
@@ -1229,7 +1269,7 @@ size_t replay_smem_bytes(ReplayArgs& a) {
   a.slots_in_smem = rs * 44 <= 44 * 1024 ? 1u : 0u;
   a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
-                (9 * (size_t)a.m.R + 4) * sizeof(uint32_t) + 16 +
+                (10 * (size_t)a.m.R + 4) * sizeof(uint32_t) + 16 +
                 (kStageDepth + 1 + (kStageDepth + 2) * ((size_t)a.m.R + kStageBlocks)) * sizeof(uint32_t) +
                 8 + (kStageDepth + 2) * (size_t)a.m.R * sizeof(double) +
                 (kStageDepth + 2) * kStageBlocks * sizeof(MaskT) + 8;
@@ -1320,6 +1360,12 @@ cudaError_t launch_replay(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st)
 
 cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st) {
   select_p95_kernel<<<dim3(n_cand, 2), kSelectThreads, 0, st>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_policy_routes(const TraceView& tr, uint32_t R, bool affinity,
+                                 const uint32_t* draws, uint8_t* route, cudaStream_t st) {
+  policy_routes_kernel<<<(tr.n_req + 255) / 256, 256, 0, st>>>(tr, R, affinity ? 1u : 0u, draws, route);
   return cudaGetLastError();
 }
 
