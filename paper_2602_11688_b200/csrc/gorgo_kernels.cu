@@ -153,7 +153,7 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
   __stcg(reinterpret_cast<unsigned long long*>(mask) + id, (unsigned long long)v);
 }
 
-constexpr int kRegChunks = 4;     // request blocks held in registers: 4 x 32 = 128
+constexpr int kRegChunks = 8;     // request blocks held in registers: 8 x 32 = 256
 constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
 constexpr int kScoutBatches = 1;       // touches examined per lane and scout round
@@ -324,7 +324,9 @@ struct Ctx {
 
 // Decide warp: queue signal, score, argmin, service model (paper Eq. 1-3).  Waits for the cache
 // warp's prefix hits of request r, publishes the route, then books the request on a slot.
-template <typename MaskT>
+// kBaseline compiles in the two switches of the paper's baseline policies (Section 4): a queue
+// signal counted in requests, and routes fixed in advance; the cost-model replay is built without.
+template <typename MaskT, bool kBaseline>
 __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
   const Smem& sm = cx.sm;
   const uint32_t R = a.m.R, S = a.m.S, K = a.m.K;
@@ -335,7 +337,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
            *qcnt = cx.qcnt;
   uint4* qrec = cx.qrec;
   const double w_que = sm.w[2];
-  const bool by_requests = a.queue_in_requests != 0;   // baseline "least-request" (Section 4)
+  const bool by_requests = kBaseline && a.queue_in_requests != 0;   // baseline "least-request"
   int32_t status = 0;
   unsigned long long st_hit = 0, st_blk = 0;
 
@@ -343,8 +345,9 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
   ReqRec rec_cur = req[a.first];
   ReqRec rec_nxt = req[min(a.first + 1, last_r)];
   // routes fixed in advance (baselines that do not look at the state), fetched two ahead
-  uint32_t fr_cur = a.forced_route ? a.forced_route[a.first] : 0u;
-  uint32_t fr_nxt = a.forced_route ? a.forced_route[min(a.first + 1, last_r)] : 0u;
+  const uint8_t* forced = kBaseline ? a.forced_route : nullptr;
+  uint32_t fr_cur = forced ? forced[a.first] : 0u;
+  uint32_t fr_nxt = forced ? forced[min(a.first + 1, last_r)] : 0u;
   // a queue refill whose load is in flight: slot index (kNone: none) and the record read
   uint32_t pend_x = kNone;
   uint4 pend_rec = make_uint4(0, 0, 0, 0);
@@ -445,10 +448,10 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
       }
     }
     uint32_t istar = warp_argmin_key(best_k, best_i);
-    if (a.forced_route) {
+    if (kBaseline && forced) {
       istar = fr_cur;
       fr_cur = fr_nxt;
-      fr_nxt = a.forced_route[min(r + 2, last_r)];
+      fr_nxt = forced[min(r + 2, last_r)];
     }
     const uint32_t hstar = cx.st_hits[stage * R + istar];   // read before the stage can be reused
     if (lane == 0) {
@@ -920,7 +923,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
 constexpr uint32_t kWarpDecide = 0, kWarpCache = 1, kWarpProbe = 2, kWarpScout0 = 3;
 constexpr uint32_t kReplayThreads = 32 * (3 + kScouts);
 
-template <typename MaskT>
+template <typename MaskT, bool kBaseline>
 __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayArgs a) {
   const uint32_t p = blockIdx.x;
   const uint32_t lane = threadIdx.x & 31u;
@@ -1028,7 +1031,7 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
   __syncthreads();
 
-  if (warp == kWarpDecide) decide_warp<MaskT>(a, cx, p, lane);
+  if (warp == kWarpDecide) decide_warp<MaskT, kBaseline>(a, cx, p, lane);
   else if (warp == kWarpCache) cache_warp<MaskT>(a, cx, p, lane);
   else if (warp == kWarpProbe) probe_warp<MaskT>(a, cx, lane);
   else scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, warp - kWarpScout0);
@@ -1279,24 +1282,30 @@ size_t replay_smem_bytes(ReplayArgs& a) {
   return smem;
 }
 
-template <typename MaskT>
-cudaError_t launch_replay_t(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
+template <typename MaskT, bool kBaseline>
+cudaError_t launch_replay_tb(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
   const size_t smem = replay_smem_bytes<MaskT>(a);
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT>,
+    cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT, kBaseline>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   // several candidates share an SM (P is usually larger than the SM count): ask for the largest
   // shared-memory carve-out so that the per-CTA footprint, not the default split, decides
   {
-    cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT>,
+    cudaError_t e = cudaFuncSetAttribute(replay_kernel<MaskT, kBaseline>,
                                          cudaFuncAttributePreferredSharedMemoryCarveout,
                                          (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
   }
-  replay_kernel<MaskT><<<n_cand, kReplayThreads, smem, st>>>(a);
+  replay_kernel<MaskT, kBaseline><<<n_cand, kReplayThreads, smem, st>>>(a);
   return cudaGetLastError();
+}
+
+template <typename MaskT>
+cudaError_t launch_replay_t(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st) {
+  if (a.queue_in_requests || a.forced_route) return launch_replay_tb<MaskT, true>(a, n_cand, st);
+  return launch_replay_tb<MaskT, false>(a, n_cand, st);
 }
 
 }  // namespace
@@ -1305,11 +1314,11 @@ template <typename MaskT>
 int replay_occupancy_t(ReplayArgs a, size_t* smem_out) {
   const size_t smem = replay_smem_bytes<MaskT>(a);
   *smem_out = smem;
-  cudaFuncSetAttribute(replay_kernel<MaskT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  cudaFuncSetAttribute(replay_kernel<MaskT>, cudaFuncAttributePreferredSharedMemoryCarveout,
+  cudaFuncSetAttribute(replay_kernel<MaskT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaFuncSetAttribute(replay_kernel<MaskT, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
                        (int)cudaSharedmemCarveoutMaxShared);
   int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, replay_kernel<MaskT>, (int)kReplayThreads,
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, replay_kernel<MaskT, false>, (int)kReplayThreads,
                                                     smem) != cudaSuccess) {
     cudaGetLastError();
     return -1;
