@@ -190,7 +190,7 @@ def main():
     ap.add_argument("--requests", type=int, default=None, help="reduced trace length (debug)")
     ap.add_argument("--population", type=int, default=None)
     ap.add_argument("--cache-blocks", type=int, default=None)
-    ap.add_argument("--ref-requests", type=int, default=60_000,
+    ap.add_argument("--ref-requests", type=int, default=500_000,
                     help="requests per candidate in one reference/cpu-baseline step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -315,7 +315,7 @@ struct Ctx {
   volatile uint32_t* st_ready; // [kStageDepth] request (+1) whose data the stage holds
   volatile uint32_t* probe_gone;  // the probe warp has stopped
   // (stages kStageDepth and kStageDepth+1 belong to the cache warp, used alternately)
-  uint32_t* st_hits;           // [kStageDepth+2][R] prefix hits
+  uint32_t* st_hits;           // [kStageDepth+2][R] prefix hit | blocks present << 16
   double* st_ab;               // [kStageDepth+2][R] (w_net*RTT + w_prefill*uncached) per replica
   uint32_t* st_ids;            // [kStageDepth+2][kStageBlocks] block ids
   MaskT* st_mk;                // [kStageDepth+2][kStageBlocks] mask words
@@ -453,7 +453,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
       fr_cur = fr_nxt;
       fr_nxt = forced[min(r + 2, last_r)];
     }
-    const uint32_t hstar = cx.st_hits[stage * R + istar];   // read before the stage can be reused
+    const uint32_t hstar = cx.st_hits[stage * R + istar] & 0xFFFFu;   // read before the stage can be reused
     if (lane == 0) {
       *cx.route = istar;
       cx.route_log[r] = (uint8_t)istar;
@@ -535,28 +535,44 @@ __device__ __forceinline__ Ahead fetch_ahead(const ReqRec* req, uint32_t q, uint
   return h;
 }
 
-// Prefix probe on every replica from staged mask words: h_i = leading blocks whose mask has
-// bit i.  The first kStageBlocks words come from `smk`; longer prompts read the rest from memory.
+// Warp-wide OR of mask words.
+template <typename MaskT>
+__device__ __forceinline__ MaskT warp_or_mask(MaskT m) {
+  if (sizeof(MaskT) == 8) {
+    const uint32_t lo = __reduce_or_sync(kFull, (uint32_t)(uint64_t)m);
+    const uint32_t hi = __reduce_or_sync(kFull, (uint32_t)((uint64_t)m >> 32));
+    return (MaskT)(((uint64_t)hi << 32) | lo);
+  }
+  return (MaskT)__reduce_or_sync(kFull, (uint32_t)m);
+}
+
+// Probe of a request on every replica from staged mask words.  For this lane's replicas (lane
+// and lane+32): h = leading blocks whose mask has the replica's bit (the prefix hit), p = all
+// blocks of the request whose mask has it (what a commit there does not have to insert).  The
+// first kStageBlocks words come from `smk`; longer prompts read the rest from memory.
 template <typename MaskT>
 __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask,
                                              const uint32_t* ids, const Ahead& q, uint32_t R,
-                                             uint32_t lane, uint32_t& h0, uint32_t& h1) {
-  h0 = 0; h1 = 0;   // this lane's replicas: lane and lane+32
+                                             uint32_t lane, uint32_t& h0, uint32_t& h1,
+                                             uint32_t& p0, uint32_t& p1) {
+  h0 = 0; h1 = 0; p0 = 0; p1 = 0;
   const uint32_t n = q.nblk;
   MaskT alive = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0 : (MaskT)((((MaskT)1) << (R & 63)) - 1);
-  for (uint32_t c = 0; c < n && alive != 0; c += 32) {
+  for (uint32_t c = 0; c < n; c += 32) {
     const uint32_t k = c + lane;
     MaskT m = 0;
     if (k < n) m = (c < kStageBlocks) ? smk[k] : mask_load<MaskT>(mask, ids[q.off + k]);
-    MaskT it = (MaskT)(shfl_mask<MaskT>(m, 0) & alive);
+    MaskT it = warp_or_mask<MaskT>(m);      // replicas that hold any block of this chunk
     MaskT still = 0;
     while (it != 0) {
       const int i = first_bit<MaskT>(it);
       it &= (MaskT)(it - 1);
       const unsigned b = __ballot_sync(kFull, (m >> i) & 1);
-      const uint32_t run = (b == kFull) ? 32u : (uint32_t)__ffs((int)~b) - 1u;
+      const uint32_t cnt = __popc(b);
+      const bool running = (alive >> i) & 1;
+      const uint32_t run = !running ? 0u : (b == kFull) ? 32u : (uint32_t)__ffs((int)~b) - 1u;
       if ((uint32_t)(i & 31) == lane) {
-        if (i < 32) h0 += run; else h1 += run;
+        if (i < 32) { h0 += run; p0 += cnt; } else { h1 += run; p1 += cnt; }
       }
       if (run == 32u) still |= (MaskT)(((MaskT)1) << i);
     }
@@ -566,10 +582,11 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
 
 // Stage the prefix hits of a request and the part of its score (Eq. 3) that depends on them:
 // ab_i = (w_net * RTT[g][i]) + (w_prefill * uncached_i), same operations and order as the score.
+// st_hits packs (prefix hit, blocks present << 16) of a replica into one word.
 template <typename MaskT>
 __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<MaskT>& cx,
                                              const Ahead& q, uint32_t slot, uint32_t h0,
-                                             uint32_t h1, uint32_t lane) {
+                                             uint32_t h1, uint32_t p0, uint32_t p1, uint32_t lane) {
   const uint32_t R = a.m.R;
   const double w_pre = cx.sm.w[1];
   const double* wrtt_row = cx.sm.wrtt + (size_t)q.origin * R;
@@ -577,10 +594,10 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
   for (int half = 0; half < 2; ++half) {
     const uint32_t i = lane + 32u * half;
     if (i < R) {
-      const uint32_t h = half ? h1 : h0;
+      const uint32_t h = half ? h1 : h0, pr = half ? p1 : p0;
       const unsigned long long hb = (unsigned long long)h * a.m.B;
       const uint32_t unc = q.in_tok - (uint32_t)(hb < q.in_tok ? hb : q.in_tok);
-      cx.st_hits[slot * R + i] = h;
+      cx.st_hits[slot * R + i] = h | (pr << 16);
       cx.st_ab[slot * R + i] = __dadd_rn(wrtt_row[i], __dmul_rn(w_pre, (double)unc));
     }
   }
@@ -638,9 +655,9 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
         if (k < q_b.nblk) { sid[k] = id_b[c]; smk[k] = m_b[c]; }
       }
       __syncwarp();
-      uint32_t h0, h1;
-      probe_staged<MaskT>(smk, mask, ids, q_b, R, lane, h0, h1);
-      stage_scores<MaskT>(a, cx, q_b, slot, h0, h1, lane);
+      uint32_t h0, h1, p0, p1;
+      probe_staged<MaskT>(smk, mask, ids, q_b, R, lane, h0, h1, p0, p1);
+      stage_scores<MaskT>(a, cx, q_b, slot, h0, h1, p0, p1, lane);
       smem_order();
       __syncwarp();
       if (lane == 0) cx.st_ready[slot] = qb + 1;
@@ -681,8 +698,10 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   auto hand_over = [&](uint32_t slot, uint32_t nblk) {
     if (lane == 0) *cx.hit_slot = slot;
     bar_arrive(kBarHits);                                 // the decide warp may score the request
-    if (lane < R) { const uint32_t h = cx.st_hits[slot * R + lane]; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
-    if (lane + 32u < R) { const uint32_t h = cx.st_hits[slot * R + lane + 32u]; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+    if (a.stats) {                                        // probes the plain formula charges
+      if (lane < R) { const uint32_t h = cx.st_hits[slot * R + lane] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+      if (lane + 32u < R) { const uint32_t h = cx.st_hits[slot * R + lane + 32u] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+    }
   };
 
   for (uint32_t r = a.first; r < end; ++r) {
@@ -701,7 +720,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       smem_order();
     }
     if (!staged) {
-      uint32_t h0 = 0, h1 = 0;
+      uint32_t h0 = 0, h1 = 0, p0 = 0, p1 = 0;
       slot = kStageDepth + (r & 1u);                          // this warp's own stages
       uint32_t* sid = cx.st_ids + slot * kStageBlocks;
       MaskT* smk = cx.st_mk + slot * kStageBlocks;
@@ -711,8 +730,8 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         if (k < n) { const uint32_t id = ids[off + k]; sid[k] = id; smk[k] = mask_load<MaskT>(mask, id); }
       }
       __syncwarp();
-      probe_staged<MaskT>(smk, mask, ids, q_cur, R, lane, h0, h1);
-      stage_scores<MaskT>(a, cx, q_cur, slot, h0, h1, lane);
+      probe_staged<MaskT>(smk, mask, ids, q_cur, R, lane, h0, h1, p0, p1);
+      stage_scores<MaskT>(a, cx, q_cur, slot, h0, h1, p0, p1, lane);
     }
     const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
     const MaskT* smk = cx.st_mk + slot * kStageBlocks;
@@ -722,19 +741,18 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     const uint32_t istar = *cx.route;
     const MaskT bit = (MaskT)(((MaskT)1) << istar);
 
-    // ---- cache commit: set the replica's bit on the missing blocks
-    uint32_t missing = 0;
+    // ---- cache commit: set the replica's bit on the missing blocks (the probe counted the
+    //      blocks already present there)
+    const uint32_t missing = n - (cx.st_hits[slot * R + istar] >> 16);
     for (uint32_t c = 0; c < n; c += 32) {
       const uint32_t k = c + lane;
-      bool miss = false;
       if (k < n) {
         uint32_t id;
         MaskT mv;
         if (c < kStageBlocks) { id = sid[k]; mv = smk[k]; }
         else { id = ids[off + k]; mv = mask_load<MaskT>(mask, id); }
-        if (!(mv & bit)) { mask_store<MaskT>(mask, id, (MaskT)(mv | bit)); miss = true; }
+        if (!(mv & bit)) mask_store<MaskT>(mask, id, (MaskT)(mv | bit));
       }
-      missing += __popc(__ballot_sync(kFull, miss));
     }
     uint32_t occ = sm.occ[istar] + missing;
     uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
