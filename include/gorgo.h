@@ -160,6 +160,21 @@ int gorgo_state_digest(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
 int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_bytes,
                        void *cuda_stream, uint64_t *requests_seen);
 
+/* Population evaluation with one time scale per candidate (paper Section 3: the time between
+ * requests is scaled linearly to move the load; its load sweep replays one trace at several
+ * scales).  Candidate p is replayed with time_scales[p]; everything else is
+ * gorgo_eval_population.  A sweep of S scales over P parameter vectors is then ONE population of
+ * S*P (parameter vector, scale) pairs, which fills the GPU better than S evaluations of P: a
+ * replay occupies its share of an SM for the whole trace, so a population slightly larger than
+ * the number of replays the GPU holds at once costs two rounds.  `time_scales` HOST, P doubles,
+ * finite and >= 0; `params` HOST or DEVICE; outputs DEVICE as for gorgo_eval_population.  The
+ * call waits for `cuda_stream`. */
+int gorgo_eval_population_scales(gorgo_sim_t *sim, uint32_t n_candidates, const double *params,
+                                 const double *time_scales, void *workspace,
+                                 uint64_t workspace_bytes, void *cuda_stream, double *p95_ttft_ms,
+                                 double *p95_e2e_ms, uint8_t *route, uint16_t *hit_blocks,
+                                 uint64_t *state_digest, int32_t *cand_status);
+
 /* Baseline routing policies of the paper (Section 4, "Baseline policies"; `random` is in its
  * appendix tables) replayed through the same simulator, so that their TTFT/E2E can be set beside
  * a tuned cost model's.  The paper runs them against live engines; inside the simulator they read:

@@ -33,7 +33,7 @@ EXPORTS = [
     "gorgo_state_digest", "gorgo_state_status", "gorgo_set_profiling", "gorgo_last_replay_ms",
     "gorgo_eval_population_static", "gorgo_replay_occupancy", "gorgo_strerror",
     "gorgo_window_count", "gorgo_eval_population_windows", "gorgo_es_run",
-    "gorgo_last_window_ms", "gorgo_eval_policy",
+    "gorgo_last_window_ms", "gorgo_eval_policy", "gorgo_eval_population_scales",
 ]
 
 
@@ -89,6 +89,7 @@ def load():
         "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp],
         "gorgo_replay_occupancy": [vp, C.POINTER(C.c_int32), pu64],
         "gorgo_window_count": [u64, u32, u32, pu64],
+        "gorgo_eval_population_scales": [vp, u32, vp, vp, vp, u64, vp, vp, vp, vp, vp, vp, vp],
         "gorgo_eval_policy": [vp, u32, vp, dbl, vp, u64, vp, vp, vp, vp, vp, vp, vp],
         "gorgo_eval_population_windows": [vp, u32, vp, dbl, vp, u64, vp, u32, u32, vp, vp, vp, vp,
                                           vp, vp],
@@ -202,6 +203,21 @@ def gorgo_eval_population_static(sim, n_candidates, params, time_scale, stream, 
     return load().gorgo_eval_population_static(
         sim, int(n_candidates), pp, float(time_scale), stream, _dev_ptr(p95_ttft_ms),
         _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks))
+
+
+def gorgo_eval_population_scales(sim, n_candidates, params, time_scales, workspace, stream,
+                                 p95_ttft_ms, p95_e2e_ms, route=None, hit_blocks=None,
+                                 state_digest=None, cand_status=None) -> int:
+    """Population evaluation with one time scale per candidate.  ``params``: float64 numpy array
+    (host) or torch CUDA tensor; ``time_scales``: host float64 numpy array [P]; every other
+    array: torch CUDA tensor or None."""
+    pp = _np_ptr(params) if isinstance(params, np.ndarray) else _dev_ptr(params)
+    ts = np.ascontiguousarray(time_scales, dtype=np.float64)
+    assert ts.shape == (int(n_candidates),)
+    return load().gorgo_eval_population_scales(
+        sim, int(n_candidates), pp, _np_ptr(ts), _dev_ptr(workspace), workspace.numel(), stream,
+        _dev_ptr(p95_ttft_ms), _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks),
+        _dev_ptr(state_digest), _dev_ptr(cand_status))
 
 
 POLICIES = {"least-load": 0, "least-request": 1, "prefix-cache": 2, "session-affinity": 3,

@@ -88,7 +88,7 @@ StateLayout make_layout(const Model& m) {
 
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
-  uint64_t params, rtt, status, p95, forced, draws, masks, states, lists, qrec, lru_next,
+  uint64_t params, scales, rtt, status, p95, forced, draws, masks, states, lists, qrec, lru_next,
       route_log, ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
@@ -102,6 +102,7 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.mask_stride = align_up((uint64_t)s->tr.n_distinct * mask_bytes_for(m.R));
   uint64_t o = 0;
   w.params = o; o = align_up(o + res * m.K * 8);
+  w.scales = o; o = align_up(o + res * 8);       // one time scale per candidate (optional)
   w.rtt = o; o = align_up(o + (uint64_t)m.G * m.R * 8);
   w.status = o; o = align_up(o + res * 4);
   w.p95 = o; o = align_up(o + res * 16);
@@ -154,7 +155,8 @@ uint64_t window_count(uint64_t n_requests, uint32_t window, uint32_t hop) {
 int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, void* workspace,
               uint64_t workspace_bytes, cudaStream_t st, double* p95_ttft, double* p95_e2e,
               uint8_t* route, uint16_t* hit, uint64_t* digest, uint64_t* stats, int32_t* cand_status,
-              bool host_io, const WindowSpec* win = nullptr, const PolicySpec* pol = nullptr) {
+              bool host_io, const WindowSpec* win = nullptr, const PolicySpec* pol = nullptr,
+              const double* scales = nullptr /* HOST [P] or null */) {
   if (!sim || !params || !workspace || P == 0) return GORGO_ERR_INVALID_ARG;
   if ((!p95_ttft || !p95_e2e) && !win) return GORGO_ERR_INVALID_ARG;
   if (win && (win->window == 0 || win->hop == 0 || win->window > window_max() || !win->best))
@@ -162,6 +164,9 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
   if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
   if (win && sim->tr.n_req < win->window) return GORGO_ERR_INVALID_ARG;
   if (!finite_nonneg(scale)) return GORGO_ERR_NONFINITE_PARAM;
+  if (scales)
+    for (uint32_t p = 0; p < P; ++p)
+      if (!finite_nonneg(scales[p])) return GORGO_ERR_NONFINITE_PARAM;
   if ((uintptr_t)workspace % kAlign) return GORGO_ERR_INVALID_ARG;
   DeviceGuard guard(sim->device);
   if (!guard.ok) return GORGO_ERR_CUDA;
@@ -212,6 +217,13 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
 
     ReplayArgs a = {};
     a.m = m; a.tr = sim->tr; a.scale = scale;
+    if (scales) {
+      double* d_scales = reinterpret_cast<double*>(base + w.scales);
+      if (cudaMemcpyAsync(d_scales, scales + p0, (size_t)pw * 8, cudaMemcpyHostToDevice, st) !=
+          cudaSuccess)
+        return GORGO_ERR_CUDA;
+      a.scales = d_scales;
+    }
     a.first = 0; a.count = (uint32_t)N; a.check_order = 0;
     a.rtt = d_rtt; a.params = wave_params;
     a.masks = base + w.masks; a.mask_stride = w.mask_stride;
@@ -465,6 +477,21 @@ int gorgo_eval_population(gorgo_sim_t* sim, uint32_t n_candidates, const double*
   return eval_impl(sim, n_candidates, params, time_scale, workspace, workspace_bytes,
                    static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, route,
                    hit_blocks, state_digest, stats, cand_status, false);
+}
+
+int gorgo_eval_population_scales(gorgo_sim_t* sim, uint32_t n_candidates, const double* params,
+                                 const double* time_scales, void* workspace,
+                                 uint64_t workspace_bytes, void* cuda_stream, double* p95_ttft_ms,
+                                 double* p95_e2e_ms, uint8_t* route, uint16_t* hit_blocks,
+                                 uint64_t* state_digest, int32_t* cand_status) {
+  if (!time_scales) return GORGO_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int rc = eval_impl(sim, n_candidates, params, 1.0, workspace, workspace_bytes, st,
+                           p95_ttft_ms, p95_e2e_ms, route, hit_blocks, state_digest, nullptr,
+                           cand_status, false, nullptr, nullptr, time_scales);
+  // `time_scales` is host memory read by asynchronous copies
+  if (rc == GORGO_OK && cudaStreamSynchronize(st) != cudaSuccess) return GORGO_ERR_CUDA;
+  return rc;
 }
 
 int gorgo_eval_population_windows(gorgo_sim_t* sim, uint32_t n_candidates, const double* params,

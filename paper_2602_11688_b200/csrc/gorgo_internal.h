@@ -71,6 +71,7 @@ struct ReplayArgs {
   Model m;
   TraceView tr;
   double scale;
+  const double* scales;           // [P] device, one time scale per candidate, or null (use `scale`)
   uint32_t first, count;          // requests [first, first+count)
   uint32_t check_order;           // 1: refuse (status) unless header.processed == first
   uint32_t slots_in_smem;         // set by the launcher: per-slot state fits in shared memory

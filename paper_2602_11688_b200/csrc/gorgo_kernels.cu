@@ -337,6 +337,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
            *qcnt = cx.qcnt;
   uint4* qrec = cx.qrec;
   const double w_que = sm.w[2];
+  const double scale = a.scales ? a.scales[p] : a.scale;   // time scale of this candidate
   const bool by_requests = kBaseline && a.queue_in_requests != 0;   // baseline "least-request"
   int32_t status = 0;
   unsigned long long st_hit = 0, st_blk = 0;
@@ -365,7 +366,7 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
     const ReqRec rec = rec_cur;
     rec_cur = rec_nxt;
     rec_nxt = req[min(r + 2, last_r)];                   // in flight while this request runs
-    const double t = __dmul_rn(a.scale, rec.ts_ms);
+    const double t = __dmul_rn(scale, rec.ts_ms);
     const uint32_t n = rec.nblk, in_tok = rec.in_tok;
     const double* rtt_row = sm.rtt + (size_t)rec.origin * R;
 
