@@ -94,3 +94,10 @@ def test_policy_arguments():
         assert gb.gorgo_eval_policy(sim.h, "least-load", None, 1.0, sim.workspace, sim.stream, pt, pe) == gb.GORGO_OK
     finally:
         sim.close()
+
+
+def test_policies_under_eviction_pressure_at_a_larger_size():
+    # long prompts, full caches, scout rings in use: the policy build of the replay kernel at a
+    # size that spans many rounds of eviction (60,000 requests, 12,000 blocks per replica)
+    _check(W.make_workload("longctx", n_requests=60000, population=1, cache_blocks=12000), 0.5,
+           seed=3)
