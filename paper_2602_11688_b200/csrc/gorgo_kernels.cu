@@ -1185,33 +1185,40 @@ __global__ void policy_routes_kernel(TraceView tr, uint32_t R, uint32_t affinity
 // ------------------------------------------------------------------------ window objective
 // Rolling-window objective of the tuning loop (paper Section 4: p95 TTFT of a rolling 128-request
 // window with hop 32): window j covers requests [j*hop, j*hop + window); its value is the k-th
-// smallest of them, k = ceil(0.95 window) (nearest rank).  One CTA per (candidate, group of
-// windows); a window is copied to shared memory and every thread ranks its elements by counting
-// the smaller ones (ties broken by position), which is exact for any input.
-constexpr int kWindowThreads = 128;
-constexpr uint32_t kWindowMax = 2048;      // values of one window kept in shared memory
+// smallest of them, k = ceil(0.95 window) (nearest rank).  One warp per window: the window's
+// order-preserving keys are copied to the warp's piece of shared memory, padded to a power of two
+// with the largest key, sorted by a bitonic network (exact for any input) and read at rank k-1.
+constexpr int kWindowThreads = 128;                   // four windows in flight per CTA
+constexpr uint32_t kWindowMax = 2048;                 // longest window (its keys: 16 KB per warp)
 
-__global__ void __launch_bounds__(kWindowThreads) window_p95_kernel(const WindowArgs a) {
-  __shared__ uint64_t keys[kWindowMax];
+__global__ void __launch_bounds__(kWindowThreads) window_p95_kernel(const WindowArgs a,
+                                                                    uint32_t wpad) {
+  extern __shared__ __align__(16) unsigned char window_smem[];
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  const uint32_t warps = kWindowThreads / 32;
+  uint64_t* keys = reinterpret_cast<uint64_t*>(window_smem) + (size_t)warp * wpad;
   const uint32_t p = blockIdx.x;
   const double* v = a.values + (size_t)p * a.stride;
   double* out = a.win_p95 + (size_t)p * a.win_stride;
   const uint32_t W = a.window;
   const uint32_t rank = (uint32_t)((95ull * W + 99ull) / 100ull) - 1u;   // 0-based
-  for (uint32_t j = blockIdx.y; j < a.n_win; j += gridDim.y) {
+  for (uint32_t j = blockIdx.y * warps + warp; j < a.n_win; j += gridDim.y * warps) {
     const double* wv = v + (size_t)j * a.hop;
-    for (uint32_t i = threadIdx.x; i < W; i += blockDim.x) keys[i] = key_of(wv[i]);
-    __syncthreads();
-    for (uint32_t i = threadIdx.x; i < W; i += blockDim.x) {
-      const uint64_t ki = keys[i];
-      uint32_t below = 0;
-      for (uint32_t x = 0; x < W; ++x) {
-        const uint64_t kx = keys[x];
-        below += (kx < ki || (kx == ki && x < i)) ? 1u : 0u;
+    for (uint32_t i = lane; i < wpad; i += 32) keys[i] = i < W ? key_of(wv[i]) : ~0ull;
+    __syncwarp();
+    for (uint32_t size = 2; size <= wpad; size <<= 1) {
+      for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+        for (uint32_t t = lane; t < wpad / 2; t += 32) {
+          const uint32_t i = 2 * t - (t & (stride - 1));     // lower element of the t-th pair
+          const bool ascending = (i & size) == 0;
+          const uint64_t x = keys[i], y = keys[i + stride];
+          if ((x > y) == ascending) { keys[i] = y; keys[i + stride] = x; }
+        }
+        __syncwarp();
       }
-      if (below == rank) out[j] = value_of(ki);
     }
-    __syncthreads();
+    if (lane == 0) out[j] = value_of(keys[rank]);
+    __syncwarp();
   }
 }
 
@@ -1401,8 +1408,18 @@ uint32_t window_max() { return kWindowMax; }
 
 cudaError_t launch_window(const WindowArgs& a, uint32_t n_cand, cudaStream_t st) {
   if (a.n_win > 0) {
-    const uint32_t groups = a.n_win < 1024u ? a.n_win : 1024u;
-    window_p95_kernel<<<dim3(n_cand, groups), kWindowThreads, 0, st>>>(a);
+    uint32_t wpad = 1;
+    while (wpad < a.window) wpad <<= 1;
+    const uint32_t warps = kWindowThreads / 32;
+    const size_t smem = (size_t)warps * wpad * sizeof(uint64_t);
+    if (smem > 48 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(window_p95_kernel,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    const uint32_t groups_needed = (a.n_win + warps - 1) / warps;
+    const uint32_t groups = groups_needed < 1024u ? groups_needed : 1024u;
+    window_p95_kernel<<<dim3(n_cand, groups), kWindowThreads, smem, st>>>(a, wpad);
   }
   window_best_kernel<<<n_cand, 256, 0, st>>>(a);
   return cudaGetLastError();
