@@ -69,10 +69,6 @@ __device__ __forceinline__ uint64_t order_key(double v) {
   const uint64_t b = (uint64_t)__double_as_longlong(__dadd_rn(v, 0.0));
   return (b >> 63) ? ~b : (b | 0x8000000000000000ULL);
 }
-__device__ __forceinline__ double order_value(uint64_t k) {
-  const uint64_t b = (k >> 63) ? (k & 0x7FFFFFFFFFFFFFFFULL) : ~k;
-  return __longlong_as_double((long long)b);
-}
 // Warp-wide minimum of 64-bit keys with the lowest index among equal keys; lanes that do not
 // take part pass key = ~0 and idx = kNone.  Returns the winning index, the key through `key`.
 __device__ __forceinline__ uint32_t warp_argmin_key(uint64_t& key, uint32_t idx) {
@@ -411,9 +407,11 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
         if (tok != 0)
           atomicAdd(reinterpret_cast<unsigned long long*>(sm.load + ii), (unsigned long long)(-tok));
         if (by_requests && gone != 0) atomicSub(sm.cnt + ii, gone);
-        uint64_t mk = order_key(mn);
-        warp_argmin_key(mk, lane);
-        if (lane == 0) sm.minfin[ii] = order_value(mk);
+        // (times are >= 0 or +inf: their bit patterns order like the values)
+        const uint64_t mb = (uint64_t)__double_as_longlong(mn);
+        const uint32_t mh = __reduce_min_sync(kFull, (uint32_t)(mb >> 32));
+        const uint32_t ml = __reduce_min_sync(kFull, (uint32_t)(mb >> 32) == mh ? (uint32_t)mb : 0xFFFFFFFFu);
+        if (lane == 0) sm.minfin[ii] = __longlong_as_double((long long)(((uint64_t)mh << 32) | ml));
       }
     }
     __syncwarp();
@@ -468,11 +466,11 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
     uint64_t bk = ~0ull;
     uint32_t bs = kNone;
     for (uint32_t s = lane; s < S; s += 32) {
-      const uint64_t vk = order_key(free_at[(size_t)istar * S + s]);
+      const uint64_t vk = (uint64_t)__double_as_longlong(free_at[(size_t)istar * S + s]);   // >= 0
       if (vk < bk || bs == kNone) { bk = vk; bs = s; }
     }
     bs = warp_argmin_key(bk, bs);
-    const double bv = free_at[(size_t)istar * S + bs];
+    const double bv = __longlong_as_double((long long)bk);   // the slot's free time
     const double arrive = __dadd_rn(t, rtt_row[istar]);
     const double start = (bv > arrive) ? bv : arrive;
     const double first = __dadd_rn(start, __dmul_rn(a.m.prefill_ms, (double)uncstar));
