@@ -88,6 +88,10 @@ struct Oracle {
     //    choice does not depend on the simulator's state; the caller derives it).
     bool queue_in_requests = false;
     std::vector<uint8_t> forced_route;   // empty: route by the score
+    // Heterogeneous replicas (the paper's Section 7 names them as a limitation of its uniform
+    // fleet): per-replica prefill time per token and time per output token; empty = the uniform
+    // constants.  The cost model does not see them (the proxy has no such signal).
+    std::vector<double> rep_prefill_ms, rep_tpot_ms;
 };
 
 }  // namespace
@@ -237,10 +241,12 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
         for (uint32_t s = 1; s < o->S; ++s)
             if (rp.free_at[s] < rp.free_at[slot]) slot = s;
         const double start = std::max(arrive, rp.free_at[slot]);
-        const double prefill = o->prefill_ms * (double)unc[best];
+        const double prefill =
+            (o->rep_prefill_ms.empty() ? o->prefill_ms : o->rep_prefill_ms[best]) * (double)unc[best];
         const double first = start + prefill;
         const uint32_t out = o->out_tok[r];
-        const double decode = o->tpot_ms * (double)(out > 0 ? out - 1 : 0);
+        const double decode = (o->rep_tpot_ms.empty() ? o->tpot_ms : o->rep_tpot_ms[best]) *
+                              (double)(out > 0 ? out - 1 : 0);
         const double finish = first + decode;
         rp.free_at[slot] = finish;
         rp.inflight.emplace(finish, in);
@@ -270,6 +276,22 @@ int gorgo_oracle_set_policy(void* h, uint32_t queue_in_requests, const uint8_t* 
     o->queue_in_requests = queue_in_requests != 0;
     if (forced_route) o->forced_route.assign(forced_route, forced_route + o->N);
     else o->forced_route.clear();
+    return 0;
+}
+
+// Per-replica service speeds (R values each, NULL = the uniform constant).  Returns 0, or -1 for a
+// negative or non-finite value.
+int gorgo_oracle_set_replica_speeds(void* h, const double* prefill_ms_per_token,
+                                    const double* tpot_ms) {
+    Oracle* o = static_cast<Oracle*>(h);
+    for (uint32_t i = 0; i < o->R; ++i) {
+        if (prefill_ms_per_token && !(prefill_ms_per_token[i] >= 0.0 && std::isfinite(prefill_ms_per_token[i]))) return -1;
+        if (tpot_ms && !(tpot_ms[i] >= 0.0 && std::isfinite(tpot_ms[i]))) return -1;
+    }
+    if (prefill_ms_per_token) o->rep_prefill_ms.assign(prefill_ms_per_token, prefill_ms_per_token + o->R);
+    else o->rep_prefill_ms.clear();
+    if (tpot_ms) o->rep_tpot_ms.assign(tpot_ms, tpot_ms + o->R);
+    else o->rep_tpot_ms.clear();
     return 0;
 }
 

@@ -57,6 +57,8 @@ def _load():
         lib.gorgo_oracle_stats.argtypes = [vp, vp]
         lib.gorgo_oracle_set_policy.restype = C.c_int
         lib.gorgo_oracle_set_policy.argtypes = [vp, C.c_uint32, vp]
+        lib.gorgo_oracle_set_replica_speeds.restype = C.c_int
+        lib.gorgo_oracle_set_replica_speeds.argtypes = [vp, vp, vp]
         lib.gorgo_oracle_position.restype = u64
         lib.gorgo_oracle_position.argtypes = [vp]
         _lib = lib
@@ -134,6 +136,15 @@ class Oracle:
         if rc != 0:
             raise ValueError("forced route out of range")
 
+    def set_replica_speeds(self, prefill_ms_per_token=None, tpot_ms=None):
+        """Heterogeneous replicas: per-replica prefill time per token and time per output token
+        (None: the uniform constant)."""
+        a = None if prefill_ms_per_token is None else np.ascontiguousarray(prefill_ms_per_token, np.float64)
+        b = None if tpot_ms is None else np.ascontiguousarray(tpot_ms, np.float64)
+        assert (a is None or a.shape == (self.R,)) and (b is None or b.shape == (self.R,))
+        if self._lib.gorgo_oracle_set_replica_speeds(self._h, _ptr(a), _ptr(b)) != 0:
+            raise ValueError("replica speeds must be finite and >= 0")
+
     @property
     def position(self) -> int:
         return int(self._lib.gorgo_oracle_position(self._h))
@@ -183,13 +194,15 @@ class Oracle:
 
 
 def replay(workload, w, scale: float = 1.0, detail: bool = False, queue_in_requests: bool = False,
-           forced_route=None):
+           forced_route=None, rep_prefill_ms=None, rep_tpot_ms=None):
     """Full replay of one candidate from the empty state: (RunResult, p95_ttft, p95_e2e,
     digest[R,2], stats[4])."""
     o = Oracle.from_workload(workload)
     try:
         if queue_in_requests or forced_route is not None:
             o.set_policy(queue_in_requests, forced_route)
+        if rep_prefill_ms is not None or rep_tpot_ms is not None:
+            o.set_replica_speeds(rep_prefill_ms, rep_tpot_ms)
         res = o.run(w, scale, detail=detail)
         return res, p95(res.ttft), p95(res.e2e), o.digest(), o.stats()
     finally:
