@@ -160,6 +160,17 @@ int gorgo_state_digest(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
 int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_bytes,
                        void *cuda_stream, uint64_t *requests_seen);
 
+/* Heterogeneous replicas (the paper's Section 7 names a uniform fleet as a limitation of its
+ * cost model): per-replica service speeds for every later replay of this simulator.
+ * `prefill_ms_per_token` and `tpot_ms` are HOST arrays of R doubles, finite and >= 0, copied by
+ * the call; NULL restores the uniform constant of the configuration for that quantity.  Only the
+ * service model uses them (first-token time = start + prefill_i * uncached tokens, finish =
+ * first + tpot_i * max(out - 1, 0) on the chosen replica i); the score of Eq. 3 does not see
+ * them, as the paper's proxy has no such signal.  A persistent state (gorgo_route_batch) should
+ * keep one setting from reset to its last batch. */
+int gorgo_sim_set_replica_speeds(gorgo_sim_t *sim, const double *prefill_ms_per_token,
+                                 const double *tpot_ms);
+
 /* Population evaluation with one time scale per candidate (paper Section 3: the time between
  * requests is scaled linearly to move the load; its load sweep replays one trace at several
  * scales).  Candidate p is replayed with time_scales[p]; everything else is

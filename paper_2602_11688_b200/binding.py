@@ -34,6 +34,7 @@ EXPORTS = [
     "gorgo_eval_population_static", "gorgo_replay_occupancy", "gorgo_strerror",
     "gorgo_window_count", "gorgo_eval_population_windows", "gorgo_es_run",
     "gorgo_last_window_ms", "gorgo_eval_policy", "gorgo_eval_population_scales",
+    "gorgo_sim_set_replica_speeds",
 ]
 
 
@@ -89,6 +90,7 @@ def load():
         "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp],
         "gorgo_replay_occupancy": [vp, C.POINTER(C.c_int32), pu64],
         "gorgo_window_count": [u64, u32, u32, pu64],
+        "gorgo_sim_set_replica_speeds": [vp, vp, vp],
         "gorgo_eval_population_scales": [vp, u32, vp, vp, vp, u64, vp, vp, vp, vp, vp, vp, vp],
         "gorgo_eval_policy": [vp, u32, vp, dbl, vp, u64, vp, vp, vp, vp, vp, vp, vp],
         "gorgo_eval_population_windows": [vp, u32, vp, dbl, vp, u64, vp, u32, u32, vp, vp, vp, vp,
@@ -203,6 +205,14 @@ def gorgo_eval_population_static(sim, n_candidates, params, time_scale, stream, 
     return load().gorgo_eval_population_static(
         sim, int(n_candidates), pp, float(time_scale), stream, _dev_ptr(p95_ttft_ms),
         _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks))
+
+
+def gorgo_sim_set_replica_speeds(sim, prefill_ms_per_token=None, tpot_ms=None) -> int:
+    """Per-replica prefill time per token and time per output token (host float64 arrays of R
+    values, or None for the uniform constant) for every later replay of ``sim``."""
+    a = None if prefill_ms_per_token is None else np.ascontiguousarray(prefill_ms_per_token, np.float64)
+    b = None if tpot_ms is None else np.ascontiguousarray(tpot_ms, np.float64)
+    return load().gorgo_sim_set_replica_speeds(sim, _np_ptr(a), _np_ptr(b))
 
 
 def gorgo_eval_population_scales(sim, n_candidates, params, time_scales, workspace, stream,

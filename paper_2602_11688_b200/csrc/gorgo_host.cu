@@ -15,6 +15,7 @@ using namespace gorgo;
 struct gorgo_sim {
   Model m;
   std::vector<double> rtt;
+  std::vector<double> rep_prefill, rep_tpot;   // per-replica speeds; empty: the uniform constants
   int device = 0;
   bool has_trace = false;
   TraceView tr = {};
@@ -88,7 +89,7 @@ StateLayout make_layout(const Model& m) {
 
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
-  uint64_t params, scales, rtt, status, p95, forced, draws, masks, states, lists, qrec, lru_next,
+  uint64_t params, scales, rtt, speeds, status, p95, forced, draws, masks, states, lists, qrec, lru_next,
       route_log, ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
@@ -104,6 +105,7 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.params = o; o = align_up(o + res * m.K * 8);
   w.scales = o; o = align_up(o + res * 8);       // one time scale per candidate (optional)
   w.rtt = o; o = align_up(o + (uint64_t)m.G * m.R * 8);
+  w.speeds = o; o = align_up(o + (uint64_t)m.R * 16);   // per-replica speeds (optional)
   w.status = o; o = align_up(o + res * 4);
   w.p95 = o; o = align_up(o + res * 16);
   w.forced = o; o = align_up(o + N);          // baseline policies: one route per request
@@ -118,6 +120,24 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.e2e = o; if (with_latency) o = align_up(o + res * N * 8);
   w.total = o;
   return w;
+}
+
+// Copies the per-replica speeds (if set) into the workspace and points the launch at them.
+int attach_speeds(const gorgo_sim* sim, unsigned char* base, const WsLayout& w, cudaStream_t st,
+                  ReplayArgs* a) {
+  const uint32_t R = sim->m.R;
+  double* d = reinterpret_cast<double*>(base + w.speeds);
+  if (!sim->rep_prefill.empty()) {
+    if (cudaMemcpyAsync(d, sim->rep_prefill.data(), R * 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+    a->rep_prefill_ms = d;
+  }
+  if (!sim->rep_tpot.empty()) {
+    if (cudaMemcpyAsync(d + R, sim->rep_tpot.data(), R * 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+    a->rep_tpot_ms = d + R;
+  }
+  return GORGO_OK;
 }
 
 bool is_device_pointer(const void* p) {
@@ -235,6 +255,7 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
     a.route_log_stride = N;
     a.queue_in_requests = pol && pol->queue_in_requests ? 1u : 0u;
     a.forced_route = pol ? pol->forced_route : nullptr;
+    if (attach_speeds(sim, base, w, st, &a) != GORGO_OK) return GORGO_ERR_CUDA;
     a.route_out = nullptr;
     a.hit_out = hit ? hit + (size_t)p0 * N : nullptr;
     a.ttft_out = reinterpret_cast<double*>(base + w.ttft);
@@ -341,6 +362,21 @@ int gorgo_sim_destroy(gorgo_sim_t* sim) {
     for (cudaEvent_t e : sim->wev) cudaEventDestroy(e);
   }
   delete sim;
+  return GORGO_OK;
+}
+
+int gorgo_sim_set_replica_speeds(gorgo_sim_t* sim, const double* prefill_ms_per_token,
+                                 const double* tpot_ms) {
+  if (!sim) return GORGO_ERR_INVALID_ARG;
+  const uint32_t R = sim->m.R;
+  for (uint32_t i = 0; i < R; ++i) {
+    if (prefill_ms_per_token && !finite_nonneg(prefill_ms_per_token[i])) return GORGO_ERR_INVALID_ARG;
+    if (tpot_ms && !finite_nonneg(tpot_ms[i])) return GORGO_ERR_INVALID_ARG;
+  }
+  if (prefill_ms_per_token) sim->rep_prefill.assign(prefill_ms_per_token, prefill_ms_per_token + R);
+  else sim->rep_prefill.clear();
+  if (tpot_ms) sim->rep_tpot.assign(tpot_ms, tpot_ms + R);
+  else sim->rep_tpot.clear();
   return GORGO_OK;
 }
 
@@ -701,6 +737,7 @@ int gorgo_route_batch(gorgo_sim_t* sim, const double* params, double time_scale,
   a.qrec = reinterpret_cast<uint4*>(base + w.qrec);
   a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
   a.route_log = base + w.route_log; a.route_log_stride = N;
+  if (attach_speeds(sim, base, w, st, &a) != GORGO_OK) return GORGO_ERR_CUDA;
   a.route_out = route; a.hit_out = hit_blocks; a.ttft_out = ttft_ms; a.e2e_out = e2e_ms;
   a.out_stride = count;
   a.stats = nullptr; a.status_out = nullptr;

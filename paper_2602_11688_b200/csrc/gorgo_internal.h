@@ -93,6 +93,10 @@ struct ReplayArgs {
   // request of the trace (shared by the candidates of the launch) or null
   uint32_t queue_in_requests;
   const uint8_t* forced_route;
+  // heterogeneous replicas: per-replica prefill ms per token and ms per output token (device
+  // [R] each) or null for the uniform constants of the model
+  const double* rep_prefill_ms;
+  const double* rep_tpot_ms;
   // outputs, candidate p at + p*out_stride, request r at + (r-first); any may be null
   uint8_t* route_out;
   uint16_t* hit_out;

@@ -321,7 +321,8 @@ struct Ctx {
 // Decide warp: queue signal, score, argmin, service model (paper Eq. 1-3).  Waits for the cache
 // warp's prefix hits of request r, publishes the route, then books the request on a slot.
 // kBaseline compiles in the two switches of the paper's baseline policies (Section 4): a queue
-// signal counted in requests, and routes fixed in advance; the cost-model replay is built without.
+// signal counted in requests, and routes fixed in advance, and the per-replica service speeds of
+// a heterogeneous fleet; the plain cost-model replay is built without them.
 template <typename MaskT, bool kBaseline>
 __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
   const Smem& sm = cx.sm;
@@ -473,9 +474,12 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
     const double bv = __longlong_as_double((long long)bk);   // the slot's free time
     const double arrive = __dadd_rn(t, rtt_row[istar]);
     const double start = (bv > arrive) ? bv : arrive;
-    const double first = __dadd_rn(start, __dmul_rn(a.m.prefill_ms, (double)uncstar));
+    // (per-replica speeds, if any, only in the build that also carries the baseline switches)
+    const double pre_ms = (kBaseline && a.rep_prefill_ms) ? a.rep_prefill_ms[istar] : a.m.prefill_ms;
+    const double tok_ms = (kBaseline && a.rep_tpot_ms) ? a.rep_tpot_ms[istar] : a.m.tpot_ms;
+    const double first = __dadd_rn(start, __dmul_rn(pre_ms, (double)uncstar));
     const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
-    const double finish = __dadd_rn(first, __dmul_rn(a.m.tpot_ms, (double)dec_tok));
+    const double finish = __dadd_rn(first, __dmul_rn(tok_ms, (double)dec_tok));
 
     flush_pending();
     __syncwarp();
@@ -1328,7 +1332,8 @@ cudaError_t launch_replay_tb(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
 
 template <typename MaskT>
 cudaError_t launch_replay_t(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st) {
-  if (a.queue_in_requests || a.forced_route) return launch_replay_tb<MaskT, true>(a, n_cand, st);
+  if (a.queue_in_requests || a.forced_route || a.rep_prefill_ms || a.rep_tpot_ms)
+    return launch_replay_tb<MaskT, true>(a, n_cand, st);
   return launch_replay_tb<MaskT, false>(a, n_cand, st);
 }
 
