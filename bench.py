@@ -97,7 +97,7 @@ class ClockSampler:
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE replay-kernel launch on the
 # full workload, from the single-pass ncu capture summarised under profiles/.  Reported only
 # while the kernel source is the one that was captured (first 16 hex digits of its sha256).
-NCU_TRAFFIC = {"longctx": {"bytes": 140.18e9, "kernel_sha256_16": "f81acb8554437012"}}
+NCU_TRAFFIC = {"longctx": {"bytes": 140.07e9, "kernel_sha256_16": "103c6ccf1292f2db"}}
 
 
 def captured_traffic(workload: str, full_size: bool):
