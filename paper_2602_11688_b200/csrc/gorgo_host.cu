@@ -19,6 +19,7 @@ struct gorgo_sim {
   int device = 0;
   bool has_trace = false;
   TraceView tr = {};
+  uint32_t poll_limit = 1u << 24;   // bound of the device-side waits of one warp for another
   // optional CUDA-event timing of the replay kernel (one pair per wave of the last evaluation)
   bool profiling = false;
   std::vector<cudaEvent_t> ev;    // pairs around the replay launches
@@ -81,15 +82,14 @@ StateLayout make_layout(const Model& m) {
   uint64_t o = sizeof(CandHeader);
   l.rep_off = o; o += (uint64_t)m.R * sizeof(RepState);
   const uint64_t rs = (uint64_t)m.R * m.S;
-  l.slot_d_off = o; o += rs * 24;
-  l.slot_u_off = o; o += rs * 20;
+  l.slot_off = o; o += rs * 8;
   l.bytes = align_up(o);
   return l;
 }
 
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
-  uint64_t params, scales, rtt, speeds, status, p95, forced, draws, masks, states, lists, qrec, lru_next,
+  uint64_t params, scales, rtt, speeds, status, p95, forced, draws, masks, states, lists, exp_head, exp_rec, lru_next,
       route_log, ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
@@ -113,7 +113,8 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.masks = o; o = align_up(o + res * w.mask_stride);
   w.states = o; o = align_up(o + res * w.st.bytes);
   w.lists = o; o = align_up(o + res * evict_list_bytes(m.R));
-  w.qrec = o; o = align_up(o + res * N * 16);
+  w.exp_head = o; o = align_up(o + res * N * 4);
+  w.exp_rec = o; o = align_up(o + res * N * 16);
   w.lru_next = o; o = align_up(o + res * N * 4);
   w.route_log = o; o = align_up(o + res * N);
   w.ttft = o; if (with_latency) o = align_up(o + res * N * 8);
@@ -229,8 +230,9 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
         return GORGO_ERR_CUDA;
       wave_params = d_params;
     }
-    if (launch_reset(base + w.masks, (uint64_t)pw * w.mask_stride, base + w.states, w.st, m, pw,
-                     st) != cudaSuccess)
+    if (launch_reset(base + w.masks, (uint64_t)pw * w.mask_stride,
+                     reinterpret_cast<uint32_t*>(base + w.exp_head), (uint64_t)pw * N,
+                     base + w.states, w.st, m, pw, st) != cudaSuccess)
       return GORGO_ERR_CUDA;
     if (stats && cudaMemsetAsync(stats + (size_t)p0 * 4, 0, (size_t)pw * 32, st) != cudaSuccess)
       return GORGO_ERR_CUDA;
@@ -245,11 +247,13 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
       a.scales = d_scales;
     }
     a.first = 0; a.count = (uint32_t)N; a.check_order = 0;
+    a.poll_limit = sim->poll_limit;
     a.rtt = d_rtt; a.params = wave_params;
     a.masks = base + w.masks; a.mask_stride = w.mask_stride;
     a.states = base + w.states; a.lay = w.st;
     a.evict_lists = reinterpret_cast<uint4*>(base + w.lists);
-    a.qrec = reinterpret_cast<uint4*>(base + w.qrec);
+    a.exp_head = reinterpret_cast<uint32_t*>(base + w.exp_head);
+    a.exp_rec = reinterpret_cast<uint4*>(base + w.exp_rec);
     a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
     a.route_log = route ? route + (size_t)p0 * N : base + w.route_log;
     a.route_log_stride = N;
@@ -383,7 +387,8 @@ int gorgo_sim_set_replica_speeds(gorgo_sim_t* sim, const double* prefill_ms_per_
 int gorgo_trace_bytes(uint64_t n_requests, uint64_t n_block_ids, uint64_t* bytes_out) {
   if (!bytes_out) return GORGO_ERR_INVALID_ARG;
   *bytes_out = align_up(n_requests * sizeof(ReqRec)) + align_up(n_block_ids * 4) +
-               align_up(n_block_ids * 8) + align_up(n_block_ids * 8) + kAlign;
+               align_up(n_block_ids * 8) + align_up(n_block_ids * 8) + align_up(n_requests * 8) +
+               align_up((n_requests + 1) * 4) + kAlign;
   return GORGO_OK;
 }
 
@@ -461,6 +466,27 @@ int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_m
     }
   }
 
+  // time grid over the arrivals: grid[b] = first request with ts >= b * dt, b = 0..n_grid, with
+  // about one request per bucket; none when all requests arrive at one instant
+  uint32_t n_grid = 0;
+  double grid_dt = 0.0;
+  std::vector<uint32_t> grid;
+  {
+    const double span = ts_ms[N - 1];
+    const double dt = span / (double)N;
+    if (dt > 0.0 && std::isfinite(dt) && dt >= span * 0x1p-40) {
+      n_grid = (uint32_t)N;
+      grid_dt = dt;
+      grid.resize((size_t)n_grid + 1);
+      uint64_t r = 0;
+      for (uint32_t b = 0; b <= n_grid; ++b) {
+        const double edge = (double)b * dt;
+        while (r < N && ts_ms[r] < edge) ++r;
+        grid[b] = (uint32_t)(r < N ? r : N - 1);
+      }
+    }
+  }
+
   DeviceGuard guard(sim->device);
   if (!guard.ok) return GORGO_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -470,7 +496,12 @@ int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_m
   unsigned char* d_ids = base + o; o += align_up(T * 4);
   unsigned char* d_occ = base + o; o += align_up(T * 8);
   unsigned char* d_raw = base + o; o += align_up(D * 8);
+  unsigned char* d_ts = base + o; o += align_up(N * 8);
+  unsigned char* d_grid = base + o; o += align_up((N + 1) * 4);
   bool ok = cudaMemcpyAsync(d_req, req.data(), N * sizeof(ReqRec), cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(d_ts, ts_ms, N * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (n_grid > 0)
+    ok = ok && cudaMemcpyAsync(d_grid, grid.data(), ((size_t)n_grid + 1) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (T > 0) {
     ok = ok && cudaMemcpyAsync(d_ids, ids.data(), T * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(d_occ, occ.data(), T * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -482,6 +513,10 @@ int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_m
   sim->tr.ids = reinterpret_cast<const uint32_t*>(d_ids);
   sim->tr.occ_next = reinterpret_cast<const uint2*>(d_occ);
   sim->tr.raw_id = reinterpret_cast<const uint64_t*>(d_raw);
+  sim->tr.ts = reinterpret_cast<const double*>(d_ts);
+  sim->tr.grid = reinterpret_cast<const uint32_t*>(d_grid);
+  sim->tr.grid_dt = grid_dt;
+  sim->tr.grid_n = n_grid;
   sim->tr.n_req = (uint32_t)N; sim->tr.n_ids = (uint32_t)T; sim->tr.n_distinct = (uint32_t)D;
   sim->has_trace = true;
   return GORGO_OK;
@@ -698,7 +733,8 @@ int gorgo_sim_reset(gorgo_sim_t* sim, void* state_workspace, uint64_t state_byte
   DeviceGuard guard(sim->device);
   if (!guard.ok) return GORGO_ERR_CUDA;
   unsigned char* base = static_cast<unsigned char*>(state_workspace);
-  if (launch_reset(base + w.masks, w.mask_stride, base + w.states, w.st, sim->m, 1,
+  if (launch_reset(base + w.masks, w.mask_stride, reinterpret_cast<uint32_t*>(base + w.exp_head),
+                   sim->tr.n_req, base + w.states, w.st, sim->m, 1,
                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
     return GORGO_ERR_CUDA;
   return GORGO_OK;
@@ -730,11 +766,13 @@ int gorgo_route_batch(gorgo_sim_t* sim, const double* params, double time_scale,
   ReplayArgs a = {};
   a.m = sim->m; a.tr = sim->tr; a.scale = time_scale;
   a.first = (uint32_t)first; a.count = (uint32_t)count; a.check_order = 1;
+  a.poll_limit = sim->poll_limit;
   a.rtt = d_rtt; a.params = d_params;
   a.masks = base + w.masks; a.mask_stride = w.mask_stride;
   a.states = base + w.states; a.lay = w.st;
   a.evict_lists = reinterpret_cast<uint4*>(base + w.lists);
-  a.qrec = reinterpret_cast<uint4*>(base + w.qrec);
+  a.exp_head = reinterpret_cast<uint32_t*>(base + w.exp_head);
+  a.exp_rec = reinterpret_cast<uint4*>(base + w.exp_rec);
   a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
   a.route_log = base + w.route_log; a.route_log_stride = N;
   if (attach_speeds(sim, base, w, st, &a) != GORGO_OK) return GORGO_ERR_CUDA;
@@ -906,6 +944,18 @@ int gorgo_eval_population_static(gorgo_sim_t* sim, uint32_t n_candidates, const 
                    static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, route,
                    hit_blocks, nullptr, nullptr, nullptr, false);
 }
+
+#ifdef GORGO_PROF
+// Cycle-accounting build only (not declared in gorgo.h, not part of the product library):
+// waits for the device, copies the 64 phase accumulators out and clears them.
+int gorgo_debug_phase_cycles(gorgo_sim_t* sim, uint64_t* out64) {
+  if (!sim || !out64) return GORGO_ERR_INVALID_ARG;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return GORGO_ERR_CUDA;
+  return prof_read(reinterpret_cast<unsigned long long*>(out64), true) == cudaSuccess
+             ? GORGO_OK : GORGO_ERR_CUDA;
+}
+#endif
 
 const char* gorgo_strerror(int code) {
   switch (code) {

@@ -23,7 +23,7 @@ static_assert(sizeof(ReqRec) == 32, "ReqRec must be one sector");
 // Per-(candidate, replica) scalars kept in global memory between launches.
 struct __align__(32) RepState {
   long long load;     // in-flight input tokens
-  double min_fin;     // earliest finish among in-flight requests (+inf if none)
+  long long cnt;      // in-flight requests
   uint32_t occ;       // cached blocks
   uint32_t cur_req;   // eviction cursor: request whose touches are examined next (kNone: none yet)
   int32_t cur_pos;    //   next position of that request to examine (counts down; <0: exhausted)
@@ -45,6 +45,12 @@ struct TraceView {
   const uint2* occ_next;   // [T] (.x = flat index of the next occurrence of the same block or
                            //      kNone, .y = request of that occurrence)
   const uint64_t* raw_id;  // [D] caller's 64-bit id of each dense id
+  const double* ts;        // [N] arrival times (unscaled), the same values as in `req`
+  // time grid over the unscaled arrival times: grid[b] = first request with ts >= b * grid_dt,
+  // b = 0..grid_n (grid_n = 0: no grid, e.g. all arrivals at one instant)
+  const uint32_t* grid;
+  double grid_dt;
+  uint32_t grid_n;
   uint32_t n_req, n_ids, n_distinct;
 };
 
@@ -59,10 +65,7 @@ struct Model {
 // candidate lives in a separate region.
 struct StateLayout {
   uint64_t rep_off;        // RepState[R]
-  uint64_t slot_d_off;     // double[3][R*S]: slot free time, finish of its oldest and second
-                           //   oldest in-flight request
-  uint64_t slot_u_off;     // uint32[5][R*S]: tokens of the oldest and second oldest, request
-                           //   index of the third oldest, newest request, queue length
+  uint64_t slot_off;       // double[R*S]: time each slot frees (finish of its newest request)
   uint64_t bytes;          // size of the block (multiple of 256)
 };
 
@@ -74,6 +77,7 @@ struct ReplayArgs {
   const double* scales;           // [P] device, one time scale per candidate, or null (use `scale`)
   uint32_t first, count;          // requests [first, first+count)
   uint32_t check_order;           // 1: refuse (status) unless header.processed == first
+  uint32_t poll_limit;            // polls after which a warp stops waiting for another one
   uint32_t slots_in_smem;         // set by the launcher: per-slot state fits in shared memory
   uint32_t lists_in_smem;         // set by the launcher: eviction lists fit in shared memory
   uint4* evict_lists;             // [P * evict_list_bytes(R)] scratch used when they do not
@@ -84,8 +88,9 @@ struct ReplayArgs {
   unsigned char* states;          // [P * layout.bytes]
   StateLayout lay;
   // per-request arrays, candidate p at + p*N elements
-  uint4* qrec;                    // per request (finish lo, finish hi, next request queued on
-                                  //   the same replica slot, input tokens)
+  uint32_t* exp_head;             // [r]: first entry of the list of requests whose completion the
+                                  //   proxy sees when request r arrives (kNone: none)
+  uint4* exp_rec;                 // [j]: (next entry of j's list, input tokens of j, replica of j, -)
   uint32_t* lru_next;             // next request routed to the same replica
   uint8_t* route_log;             // chosen replica of every request replayed so far
   uint64_t route_log_stride;      // elements between candidates
@@ -136,15 +141,19 @@ struct DigestArgs {
   uint64_t* digest;               // [P*R*2], zeroed by the launcher
 };
 
-cudaError_t launch_reset(unsigned char* masks, uint64_t mask_bytes_total, unsigned char* states,
-                         const StateLayout& lay, const Model& m, uint32_t n_cand,
-                         cudaStream_t st);
+cudaError_t launch_reset(unsigned char* masks, uint64_t mask_bytes_total, uint32_t* exp_head,
+                         uint64_t exp_head_count, unsigned char* states, const StateLayout& lay,
+                         const Model& m, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_replay(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_select(const SelectArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_digest(const DigestArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_window(const WindowArgs& a, uint32_t n_cand, cudaStream_t st);
 cudaError_t launch_policy_routes(const TraceView& tr, uint32_t R, bool affinity,
                                  const uint32_t* draws, uint8_t* route, cudaStream_t st);
+#ifdef GORGO_PROF
+// Cycle accounting build only: the 64 accumulators (decide warp at 0, cache warp at 16).
+cudaError_t prof_read(unsigned long long* out64, bool reset);
+#endif
 uint32_t window_max();          // largest window the window kernel handles
 uint32_t mask_bytes_for(uint32_t n_replicas);
 uint64_t evict_list_bytes(uint32_t n_replicas);

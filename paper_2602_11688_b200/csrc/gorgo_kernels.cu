@@ -34,6 +34,22 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
+// Cycle accounting of the two serial warps (built only with -DGORGO_PROF; the normal library
+// carries none of it).  Every lap adds the SM clock ticks since the previous lap of the same
+// warp to one of 32 per-role accumulators; the totals of all candidates end up in g_prof.
+#ifdef GORGO_PROF
+__device__ unsigned long long g_prof[64];
+#define PROF_BEGIN() unsigned long long pf[16] = {}; long long pf_t = clock64()
+#define PROF_LAP(k) do { const long long pf_n = clock64(); pf[k] += (unsigned long long)(pf_n - pf_t); pf_t = pf_n; } while (0)
+#define PROF_ADD(k, v) pf[k] += (unsigned long long)(v)
+#define PROF_END(base) do { if (lane == 0) { _Pragma("unroll") for (int pf_i = 0; pf_i < 16; ++pf_i) atomicAdd(&g_prof[(base) + pf_i], pf[pf_i]); } } while (0)
+#else
+#define PROF_BEGIN() do {} while (0)
+#define PROF_LAP(k) do {} while (0)
+#define PROF_ADD(k, v) do {} while (0)
+#define PROF_END(base) do {} while (0)
+#endif
+
 __device__ __forceinline__ double d_inf() { return __longlong_as_double(0x7FF0000000000000LL); }
 
 template <typename T> struct MaskOps;
@@ -157,10 +173,17 @@ constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is t
 
 // Shared-memory view of one candidate's small state.
 struct Smem {
-  double* rtt; double* wrtt; double* w; double* minfin; long long* load;
-  int32_t* cnt;                   // in-flight requests per replica (kept when the queue signal counts requests)
+  double* rtt; double* wrtt; double* w;
+  long long* load;                // in-flight input tokens per replica (as of the last launch; the route warp keeps the live value)
+  long long* cnt;                 // in-flight requests per replica (kept when the queue signal counts requests)
   uint32_t* occ; uint32_t* curreq; int32_t* curpos; uint32_t* lrutail;
   volatile uint32_t* progress;
+  // hand-over between the route, service and expiry warps
+  volatile uint32_t* routed;      // requests routed so far
+  volatile uint32_t* serviced;    // requests whose service commit is done and whose completion is filed
+  volatile uint32_t* exp_ready;   // requests whose completion sums are published
+  uint32_t* route_ring;           // [kRouteRing] chosen replica | prefix hit there << 8
+  long long* exp_sum;             // [kExpRing][R] tokens (or requests) that completed by the request's arrival
   // eviction rings, one per replica: filled by the scout warp, drained by the replay warp.
   // entry = (block id, request of the block's next occurrence after the entry was made or kNone,
   //          position of the touch in its request, request of the touch), in eviction order
@@ -299,14 +322,14 @@ template <typename MaskT>
 struct Ctx {
   Smem sm;
   MaskT* mask;
-  uint4* qrec;
+  uint32_t* exp_head;
+  uint4* exp_rec;
   uint32_t* lru_next;
   uint8_t* route_log;
-  // per-slot state (shared or global memory)
-  double *free_at, *q0_fin, *q1_fin;
-  uint32_t *q0_tok, *q1_tok, *q2_idx, *tail, *qcnt;
+  double* free_at;             // [R*S] time each slot frees (shared or global memory)
   volatile uint32_t* route;    // chosen replica of the current request
   volatile int32_t* status;    // first device-side limit hit by any warp
+  volatile uint32_t* abort_flag;  // a bounded wait ran out: the other waits stop too
   // staging of the coming requests by the probe warp (kStageDepth stages + one of the cache warp)
   volatile uint32_t* st_ready; // [kStageDepth] request (+1) whose data the stage holds
   volatile uint32_t* probe_gone;  // the probe warp has stopped
@@ -318,26 +341,50 @@ struct Ctx {
   volatile uint32_t* hit_slot; // stage that holds the current request's hits and scores
 };
 
-// Decide warp: queue signal, score, argmin, service model (paper Eq. 1-3).  Waits for the cache
-// warp's prefix hits of request r, publishes the route, then books the request on a slot.
+// (forward) rings between the route, service and expiry warps
+constexpr uint32_t kRouteRing = 32;   // routes handed from the route warp to the service warp
+constexpr uint32_t kRouteLead = 24;   // the route warp runs at most this far ahead of the service warp
+constexpr uint32_t kExpRing = 8;      // completion sums published ahead of the route warp
+
+// Bounded wait of one warp for a counter another warp of the candidate advances: polls until
+// (int)(counter - want) >= 0.  If the limit runs out (or another warp already gave up) the
+// candidate is marked failed and every later wait returns at once, so the CTA still terminates.
+__device__ __forceinline__ uint32_t wait_counter(volatile uint32_t* counter, uint32_t want,
+                                                 volatile uint32_t* abort_flag, uint32_t limit,
+                                                 int32_t& status) {
+  uint32_t v = *counter;
+  uint32_t polls = 0;
+  while ((int32_t)(v - want) < 0) {
+    if (*abort_flag) break;
+    if (++polls > limit) { status = -6; *abort_flag = 1; break; }
+    __nanosleep(20);
+    v = *counter;
+  }
+  return v;
+}
+
+// Route warp: the serial chain of a replay.  Per request it adds the queue term to the staged
+// part of the score of Eq. 3, takes the lowest-index argmin and posts the route.  Lane i (and
+// i+32) keeps replica i's in-flight signal in registers: tokens (or requests) dispatched there,
+// minus what the expiry warp reports as completed by this request's arrival.  The service model
+// (slots, times) is not on this chain: it runs behind in the service warp.
 // kBaseline compiles in the two switches of the paper's baseline policies (Section 4): a queue
-// signal counted in requests, and routes fixed in advance, and the per-replica service speeds of
-// a heterogeneous fleet; the plain cost-model replay is built without them.
+// signal counted in requests, and routes fixed in advance; the plain cost-model replay is built
+// without them.
 template <typename MaskT, bool kBaseline>
-__device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
+__device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
   const Smem& sm = cx.sm;
-  const uint32_t R = a.m.R, S = a.m.S, K = a.m.K;
-  const uint32_t N = a.tr.n_req;
+  const uint32_t R = a.m.R, K = a.m.K;
   const ReqRec* req = a.tr.req;
-  double *free_at = cx.free_at, *q0_fin = cx.q0_fin, *q1_fin = cx.q1_fin;
-  uint32_t *q0_tok = cx.q0_tok, *q1_tok = cx.q1_tok, *q2_idx = cx.q2_idx, *tail = cx.tail,
-           *qcnt = cx.qcnt;
-  uint4* qrec = cx.qrec;
   const double w_que = sm.w[2];
-  const double scale = a.scales ? a.scales[p] : a.scale;   // time scale of this candidate
   const bool by_requests = kBaseline && a.queue_in_requests != 0;   // baseline "least-request"
   int32_t status = 0;
   unsigned long long st_hit = 0, st_blk = 0;
+  const uint32_t i0 = lane, i1 = lane + 32u;
+  long long ld0 = 0, ld1 = 0;          // in-flight signal of replicas lane and lane+32
+  double nrm0 = 1.0, nrm1 = 1.0;       // their queue-load normalisers
+  if (i0 < R) { ld0 = by_requests ? sm.cnt[i0] : sm.load[i0]; if (K != 3) nrm0 = sm.w[3 + i0]; }
+  if (i1 < R) { ld1 = by_requests ? sm.cnt[i1] : sm.load[i1]; if (K != 3) nrm1 = sm.w[3 + i1]; }
 
   const uint32_t last_r = a.first + a.count - 1;
   ReqRec rec_cur = req[a.first];
@@ -346,91 +393,36 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
   const uint8_t* forced = kBaseline ? a.forced_route : nullptr;
   uint32_t fr_cur = forced ? forced[a.first] : 0u;
   uint32_t fr_nxt = forced ? forced[min(a.first + 1, last_r)] : 0u;
-  // a queue refill whose load is in flight: slot index (kNone: none) and the record read
-  uint32_t pend_x = kNone;
-  uint4 pend_rec = make_uint4(0, 0, 0, 0);
-  auto flush_pending = [&]() {
-    if (pend_x != kNone) {
-      q1_fin[pend_x] = __hiloint2double((int)pend_rec.y, (int)pend_rec.x);
-      q2_idx[pend_x] = pend_rec.z;
-      q1_tok[pend_x] = pend_rec.w;
-      pend_x = kNone;
-    }
-  };
+  uint32_t exp_seen = a.first, srv_seen = a.first;
 
+  PROF_BEGIN();
   for (uint32_t j = 0; j < a.count; ++j) {
     const uint32_t r = a.first + j;
     const ReqRec rec = rec_cur;
     rec_cur = rec_nxt;
     rec_nxt = req[min(r + 2, last_r)];                   // in flight while this request runs
-    const double t = __dmul_rn(scale, rec.ts_ms);
     const uint32_t n = rec.nblk, in_tok = rec.in_tok;
-    const double* rtt_row = sm.rtt + (size_t)rec.origin * R;
 
-    // ---- queue signal: drop requests that completed by t (finish <= t)
-    for (uint32_t i0 = 0; i0 < R; i0 += 32) {
-      const uint32_t i = i0 + lane;
-      unsigned due = __ballot_sync(kFull, i < R && sm.minfin[i] <= t);
-      while (due) {
-        const uint32_t ii = i0 + (uint32_t)__ffs((int)due) - 1;
-        due &= due - 1;
-        long long tok = 0;
-        int32_t gone = 0;
-        double mn = d_inf();
-        for (uint32_t s = lane; s < S; s += 32) {
-          const uint32_t x = ii * S + s;
-          double hf = q0_fin[x];
-          if (hf <= t) {
-            uint32_t guard = 0;
-            uint32_t cnt = qcnt[x];
-            do {
-              if (pend_x == x) flush_pending();           // the second entry is still in flight
-              tok += (long long)q0_tok[x];
-              ++gone;
-              --cnt;
-              if (cnt == 0) { hf = d_inf(); }
-              else {
-                hf = q1_fin[x];                            // the second becomes the oldest
-                q0_tok[x] = q1_tok[x];
-                if (cnt >= 2) {                            // fetch the new second: consumed later
-                  flush_pending();
-                  pend_rec = qrec[q2_idx[x]];
-                  pend_x = x;
-                }
-              }
-              if (++guard > N) { status = -6; break; }
-            } while (hf <= t);
-            q0_fin[x] = hf;
-            qcnt[x] = cnt;
-          }
-          mn = fmin(mn, hf);
-        }
-        if (tok != 0)
-          atomicAdd(reinterpret_cast<unsigned long long*>(sm.load + ii), (unsigned long long)(-tok));
-        if (by_requests && gone != 0) atomicSub(sm.cnt + ii, gone);
-        // (times are >= 0 or +inf: their bit patterns order like the values)
-        const uint64_t mb = (uint64_t)__double_as_longlong(mn);
-        const uint32_t mh = __reduce_min_sync(kFull, (uint32_t)(mb >> 32));
-        const uint32_t ml = __reduce_min_sync(kFull, (uint32_t)(mb >> 32) == mh ? (uint32_t)mb : 0xFFFFFFFFu);
-        if (lane == 0) sm.minfin[ii] = __longlong_as_double((long long)(((uint64_t)mh << 32) | ml));
-      }
-    }
-    __syncwarp();
+    // ---- completions the proxy has seen by this arrival (published by the expiry warp), and
+    //      room in the ring of routes the service warp has not taken yet
+    if ((int32_t)(exp_seen - (r + 1)) < 0)
+      exp_seen = wait_counter(sm.exp_ready, r + 1, cx.abort_flag, a.poll_limit, status);
+    if (r - srv_seen >= kRouteLead)
+      srv_seen = wait_counter(sm.serviced, r + 1 - kRouteLead, cx.abort_flag, a.poll_limit, status);
+    smem_order();
+    PROF_LAP(0);
+    const long long* gone = sm.exp_sum + (size_t)(r % kExpRing) * R;
+    if (i0 < R) ld0 -= gone[i0];
+    if (i1 < R) ld1 -= gone[i1];
 
     // ---- the queue part of the score does not need the prefix hits
     double cq0 = 0.0, cq1 = 0.0;
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const uint32_t i = lane + 32u * half;
-      if (i < R) {
-        double q = by_requests ? (double)sm.cnt[i] : (double)sm.load[i];
-        if (K != 3) q = __dmul_rn(q, sm.w[3 + i]);
-        const double c = __dmul_rn(w_que, q);
-        if (half) cq1 = c; else cq0 = c;
-      }
-    }
+    if (i0 < R) { double q = (double)ld0; if (K != 3) q = __dmul_rn(q, nrm0); cq0 = __dmul_rn(w_que, q); }
+    if (i1 < R) { double q = (double)ld1; if (K != 3) q = __dmul_rn(q, nrm1); cq1 = __dmul_rn(w_que, q); }
+    PROF_LAP(1);
 
     bar_wait(kBarHits);                                   // prefix hits of request r are posted
+    PROF_LAP(2);
 
     // ---- score of Eq. 3 (fixed order, no FMA): the staged (w_net*RTT + w_prefill*uncached)
     //      plus the queue term; lowest-index argmin
@@ -447,70 +439,33 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
         if (ck < best_k || best_i == kNone) { best_k = ck; best_i = i; }
       }
     }
+    PROF_LAP(3);
     uint32_t istar = warp_argmin_key(best_k, best_i);
     if (kBaseline && forced) {
       istar = fr_cur;
       fr_cur = fr_nxt;
       fr_nxt = forced[min(r + 2, last_r)];
     }
+    PROF_LAP(4);
     const uint32_t hstar = cx.st_hits[stage * R + istar] & 0xFFFFu;   // read before the stage can be reused
     if (lane == 0) {
       *cx.route = istar;
       cx.route_log[r] = (uint8_t)istar;
+      sm.route_ring[r % kRouteRing] = istar | (hstar << 8);
+      smem_order();
+      *sm.routed = r + 1;
     }
     bar_arrive(kBarRoute);                                // the cache warp may commit request r
-
-    const unsigned long long hbstar = (unsigned long long)hstar * a.m.B;
-    const uint32_t uncstar = in_tok - (uint32_t)(hbstar < in_tok ? hbstar : in_tok);
-
-    // ---- service commit: earliest-free slot, lowest index on ties
-    uint64_t bk = ~0ull;
-    uint32_t bs = kNone;
-    for (uint32_t s = lane; s < S; s += 32) {
-      const uint64_t vk = (uint64_t)__double_as_longlong(free_at[(size_t)istar * S + s]);   // >= 0
-      if (vk < bk || bs == kNone) { bk = vk; bs = s; }
-    }
-    bs = warp_argmin_key(bk, bs);
-    const double bv = __longlong_as_double((long long)bk);   // the slot's free time
-    const double arrive = __dadd_rn(t, rtt_row[istar]);
-    const double start = (bv > arrive) ? bv : arrive;
-    // (per-replica speeds, if any, only in the build that also carries the baseline switches)
-    const double pre_ms = (kBaseline && a.rep_prefill_ms) ? a.rep_prefill_ms[istar] : a.m.prefill_ms;
-    const double tok_ms = (kBaseline && a.rep_tpot_ms) ? a.rep_tpot_ms[istar] : a.m.tpot_ms;
-    const double first = __dadd_rn(start, __dmul_rn(pre_ms, (double)uncstar));
-    const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
-    const double finish = __dadd_rn(first, __dmul_rn(tok_ms, (double)dec_tok));
-
-    flush_pending();
-    __syncwarp();
-    if (lane == 0) {
-      const size_t x = (size_t)istar * S + bs;
-      qrec[r] = make_uint4((uint32_t)__double2loint(finish), (uint32_t)__double2hiint(finish),
-                           kNone, in_tok);
-      const uint32_t cnt = qcnt[x];
-      if (cnt == 0) {
-        q0_fin[x] = finish; q0_tok[x] = in_tok;
-        sm.minfin[istar] = fmin(sm.minfin[istar], finish);
-      } else {
-        reinterpret_cast<uint32_t*>(qrec + tail[x])[2] = r;     // link behind the newest
-        if (cnt == 1) { q1_fin[x] = finish; q1_tok[x] = in_tok; q2_idx[x] = kNone; }
-        else if (cnt == 2) q2_idx[x] = r;
-      }
-      qcnt[x] = cnt + 1;
-      tail[x] = r;
-      free_at[x] = finish;
-      sm.load[istar] += (long long)in_tok;
-      if (by_requests) sm.cnt[istar] += 1;
-      const size_t o = (size_t)p * a.out_stride + j;
-      if (a.route_out) a.route_out[o] = (uint8_t)istar;
-      if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
-      if (a.ttft_out) a.ttft_out[o] = __dsub_rn(first, t);
-      if (a.e2e_out) a.e2e_out[o] = __dsub_rn(finish, t);
-      st_hit += hstar; st_blk += n;
-    }
-    __syncwarp();
+    PROF_LAP(5);
+    const long long add = by_requests ? 1ll : (long long)in_tok;
+    if (istar == i0) ld0 += add;
+    if (istar == i1) ld1 += add;
+    st_hit += hstar; st_blk += n;
   }
-  flush_pending();
+  PROF_END(0);
+  // the signal as of the last request routed
+  if (i0 < R) { if (by_requests) sm.cnt[i0] = ld0; else sm.load[i0] = ld0; }
+  if (i1 < R) { if (by_requests) sm.cnt[i1] = ld1; else sm.load[i1] = ld1; }
   status = __reduce_min_sync(kFull, status);
   if (lane == 0) {
     if (status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
@@ -520,6 +475,266 @@ __device__ __forceinline__ void decide_warp(const ReplayArgs& a, const Ctx<MaskT
       atomicAdd(s4 + 2, st_blk);
     }
   }
+}
+
+// First request x in [lo, hi] whose scaled arrival time is >= f; the caller knows that request
+// hi qualifies.  Every lane walks the same bisection (broadcast loads).
+__device__ __forceinline__ uint32_t first_arrival_at_or_after(const double* ts, double scale, double f,
+                                                              uint32_t lo, uint32_t hi) {
+  while (lo < hi) {                                       // at most 32 rounds
+    const uint32_t mid = lo + ((hi - lo) >> 1);
+    if (__dmul_rn(scale, ts[mid]) >= f) hi = mid; else lo = mid + 1;
+  }
+  return lo;
+}
+
+// Service warp: the service model of a routed request (paper Eq. 1: network, queue wait,
+// prefill), a few requests behind the route warp.  It takes the slot of the chosen replica that
+// frees first, computes start, first-token and finish times, writes the outputs, and files the
+// request under the first later request x that arrives at or after its finish time: that is
+// when the proxy has seen its completion event, i.e. when it stops counting as in flight
+// (signal of Eq. 2).  The search for x (a time grid over the arrivals, then a 32-wide window)
+// and the list insertion need three dependent memory round trips; they run as a three-stage
+// pipeline over consecutive requests so that none of them is waited for.
+template <typename MaskT, bool kBaseline>
+__device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
+  const Smem& sm = cx.sm;
+  const uint32_t R = a.m.R, S = a.m.S;
+  const uint32_t N = a.tr.n_req;
+  const ReqRec* req = a.tr.req;
+  double* free_at = cx.free_at;
+  const double scale = a.scales ? a.scales[p] : a.scale;   // time scale of this candidate
+  const uint32_t end = a.first + a.count;
+  const double t_last = __dmul_rn(scale, a.tr.ts[N - 1]);
+  // grid bucket of a time: (time / scale) / grid_dt, as one multiplication; the search starts one
+  // bucket early, which covers the rounding of this product many times over
+  const bool use_grid = a.tr.grid_n > 0 && scale * a.tr.grid_dt >= 1e-280;
+  const double to_bucket = use_grid ? 1.0 / (scale * a.tr.grid_dt) : 0.0;
+  int32_t status = 0;
+
+  // pipeline registers (uniform over the warp unless noted)
+  uint32_t j1 = kNone, lo1 = 0, g1 = 0, tok1 = 0, rep1 = 0;  double f1 = 0.0;   // grid entry in flight (g1: lane 0)
+  uint32_t j2 = kNone, lo2 = 0, tok2 = 0, rep2 = 0;  double f2 = 0.0, win2 = 0.0;   // window in flight (win2: per lane)
+  uint32_t j3 = kNone, tok3 = 0, rep3 = 0, old3 = kNone;                       // list head exchange in flight (old3: lane 0)
+  bool ins1 = false, ins2 = false, ins3 = false;   // the request gets a list entry (it completes before the trace ends)
+  uint32_t s = a.first;
+  uint32_t routed_seen = a.first;
+  ReqRec rec_nxt = req[a.first];
+  uint32_t idle = 0;
+  bool failed = false;
+
+  PROF_BEGIN();
+  while (true) {
+    // ---- what arrived since the last round
+    uint32_t fin = kNone;
+    if (j3 != kNone) {
+      if (ins3 && lane == 0) cx.exp_rec[j3] = make_uint4(old3, tok3, rep3, 0u);
+      fin = j3 + 1;
+    }
+    uint32_t x2 = kNone;
+    if (j2 != kNone && ins2) {
+      const bool ok = lo2 + lane < N && __dmul_rn(scale, win2) >= f2;
+      const unsigned b = __ballot_sync(kFull, ok);
+      if (b) x2 = lo2 + (uint32_t)__ffs((int)b) - 1u;
+      else x2 = first_arrival_at_or_after(a.tr.ts, scale, f2, min(lo2 + 32u, N - 1), N - 1);
+    }
+    const uint32_t g = __shfl_sync(kFull, g1, 0);
+    PROF_LAP(0);
+    // ---- publish the requests whose list entry is linked
+    if (fin != kNone && lane == 0) {
+      __threadfence_block();
+      *sm.serviced = fin;
+    }
+    if (fin == end) break;
+    PROF_LAP(1);
+    // ---- next stage of each request in the pipeline
+    j3 = j2; tok3 = tok2; rep3 = rep2; ins3 = ins2;
+    if (j3 != kNone && ins3 && lane == 0) old3 = atomicExch(cx.exp_head + x2, j3);
+    j2 = j1; tok2 = tok1; rep2 = rep1; f2 = f1; ins2 = ins1;
+    if (j2 != kNone && ins2) {
+      lo2 = max(lo1, use_grid ? g : 0u);
+      win2 = lo2 + lane < N ? a.tr.ts[lo2 + lane] : 0.0;
+    }
+    j1 = kNone; ins1 = false;
+    PROF_LAP(2);
+
+    // ---- service model of the next routed request, if there is one
+    if (s < end) {
+      if ((int32_t)(routed_seen - (s + 1)) < 0) routed_seen = *sm.routed;
+      if ((int32_t)(routed_seen - (s + 1)) >= 0) {
+        smem_order();
+        idle = 0;
+        const ReqRec rec = rec_nxt;
+        rec_nxt = req[min(s + 1, end - 1)];
+        const uint32_t rq = sm.route_ring[s % kRouteRing];
+        const uint32_t istar = rq & 0xFFu, hstar = rq >> 8;
+        const double t = __dmul_rn(scale, rec.ts_ms);
+        const uint32_t in_tok = rec.in_tok;
+        const unsigned long long hb = (unsigned long long)hstar * a.m.B;
+        const uint32_t unc = in_tok - (uint32_t)(hb < in_tok ? hb : in_tok);
+        // earliest-free slot, lowest index on ties (times are >= 0: bit patterns order like values)
+        uint64_t bk = ~0ull;
+        uint32_t bs = kNone;
+        const double* fa = free_at + (size_t)istar * S;
+        if (S <= 32) {
+          if (lane < S) { bk = (uint64_t)__double_as_longlong(fa[lane]); bs = lane; }
+        } else {
+          for (uint32_t s2 = lane; s2 < S; s2 += 32) {
+            const uint64_t vk = (uint64_t)__double_as_longlong(fa[s2]);
+            if (vk < bk || bs == kNone) { bk = vk; bs = s2; }
+          }
+        }
+        bs = warp_argmin_key(bk, bs);
+        PROF_LAP(3);
+        const double bv = __longlong_as_double((long long)bk);   // the slot's free time
+        const double arrive = __dadd_rn(t, sm.rtt[(size_t)rec.origin * R + istar]);
+        const double start = (bv > arrive) ? bv : arrive;
+        // (per-replica speeds, if any, only in the build that also carries the baseline switches)
+        const double pre_ms = (kBaseline && a.rep_prefill_ms) ? a.rep_prefill_ms[istar] : a.m.prefill_ms;
+        const double tok_ms = (kBaseline && a.rep_tpot_ms) ? a.rep_tpot_ms[istar] : a.m.tpot_ms;
+        const double first = __dadd_rn(start, __dmul_rn(pre_ms, (double)unc));
+        const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
+        const double finish = __dadd_rn(first, __dmul_rn(tok_ms, (double)dec_tok));
+        if (lane == 0) {
+          free_at[(size_t)istar * S + bs] = finish;
+          const size_t o = (size_t)p * a.out_stride + (s - a.first);
+          if (a.route_out) a.route_out[o] = (uint8_t)istar;
+          if (a.hit_out) a.hit_out[o] = (uint16_t)hstar;
+          if (a.ttft_out) a.ttft_out[o] = __dsub_rn(first, t);
+          if (a.e2e_out) a.e2e_out[o] = __dsub_rn(finish, t);
+        }
+        // the request stops counting at the first later arrival at or after `finish`
+        j1 = s; f1 = finish; tok1 = in_tok; rep1 = istar;
+        ins1 = s + 1 < N && t_last >= finish;
+        lo1 = s + 1;
+        if (ins1 && use_grid && lane == 0) {
+          const double bf = __dmul_rn(finish, to_bucket);
+          uint32_t b = 0;
+          if (bf >= 2.0) b = (bf >= (double)a.tr.grid_n ? a.tr.grid_n : (uint32_t)bf) - 1u;
+          g1 = a.tr.grid[b];
+        }
+        ++s;
+        __syncwarp();
+        PROF_LAP(4);
+        continue;
+      }
+    }
+    if (j2 == kNone && j3 == kNone) {        // nothing in flight and no route to take: wait
+      if (*cx.abort_flag) failed = true;
+      if (++idle > a.poll_limit) { status = -6; *cx.abort_flag = 1; failed = true; }
+      if (failed) break;
+      __nanosleep(40);
+    }
+    PROF_LAP(5);
+  }
+  PROF_END(16);
+  status = __reduce_min_sync(kFull, status);
+  if (lane == 0 && status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
+}
+
+// Expiry warp: for every request r, ahead of the route warp, the in-flight tokens (or requests)
+// per replica whose completion the proxy has seen by r's arrival: the sum over r's list, filed by
+// the service warp.  The list of r can only gain entries from requests j < r with finish <= t_r.
+// finish_j >= t_j + tpot * decode tokens (network, waiting and prefill only add to it), so once
+// every j < r whose bound lb_j = t_j + tpot*dec_j is <= t_r has been serviced, the list is
+// final and is walked: one lane per request, eight requests in flight, one list hop per round.
+template <bool kBaseline>
+__device__ __forceinline__ void expiry_warp(const ReplayArgs& a, const Smem& sm, const uint32_t* exp_head,
+                                            const uint4* exp_rec, volatile uint32_t* abort_flag,
+                                            volatile int32_t* cta_status, uint32_t p, uint32_t lane) {
+  const uint32_t R = a.m.R;
+  const ReqRec* req = a.tr.req;
+  const double scale = a.scales ? a.scales[p] : a.scale;
+  const uint32_t end = a.first + a.count;
+  const bool by_requests = kBaseline && a.queue_in_requests != 0;
+  // smallest time per output token over the replicas (a lower bound of every decode time)
+  double tok_ms = a.m.tpot_ms;
+  if (kBaseline && a.rep_tpot_ms) {
+    tok_ms = a.rep_tpot_ms[0];
+    for (uint32_t i = 1; i < R; ++i) tok_ms = fmin(tok_ms, a.rep_tpot_ms[i]);
+  }
+  int32_t status = 0;
+  double lb = d_inf();                 // bound of the latest request j with j % 32 == lane (none yet: +inf)
+  uint32_t next_r = a.first;           // next request whose list walk starts
+  uint32_t published = a.first;        // requests whose sums are published
+  uint32_t my_r = kNone;               // lanes 0..7: request whose list this lane walks (kNone: idle)
+  uint32_t e = kNone;                  //   entry whose record is in flight (kNone with my_r set: walk done)
+  bool head_pending = false;           //   the list head is in flight
+  uint32_t head_val = kNone;
+  uint4 rec_val = make_uint4(kNone, 0u, 0u, 0u);
+  uint32_t srv_seen = a.first, routed_seen = a.first;
+  ReqRec rq_nxt = req[a.first];
+  uint32_t idle = 0;
+
+  while (published < end) {
+    bool progress = false;
+    // ---- what arrived: the head of a list, or one entry of it
+    if (my_r != kNone) {
+      if (head_pending) { e = head_val; head_pending = false; }
+      else if (e != kNone) {
+        long long* row = sm.exp_sum + (size_t)(my_r % kExpRing) * R;
+        row[rec_val.z] += by_requests ? 1ll : (long long)rec_val.y;
+        e = rec_val.x;
+      }
+    }
+    // ---- publish finished walks in request order
+    {
+      const bool fin = my_r != kNone && !head_pending && e == kNone;
+      unsigned m = __ballot_sync(kFull, fin) & 0xFFu;
+      while (m & (1u << (published % kExpRing))) {          // the lane of request `published` is done
+        if (lane == published % kExpRing) my_r = kNone;
+        m &= ~(1u << (published % kExpRing));
+        ++published;
+        progress = true;
+      }
+      if (progress && lane == 0) { smem_order(); *sm.exp_ready = published; }
+    }
+    // ---- start the walks of up to two more requests
+    for (int k = 0; k < 2 && next_r < end; ++k) {
+      const uint32_t owner = next_r % kExpRing;
+      // the ring row is free once the route warp has used its previous occupant
+      if (next_r >= kExpRing + a.first && (int32_t)(routed_seen - (next_r - kExpRing + 1)) < 0) {
+        routed_seen = *sm.routed;
+        if ((int32_t)(routed_seen - (next_r - kExpRing + 1)) < 0) break;
+      }
+      if (__shfl_sync(kFull, my_r, owner) != kNone) break;    // its lane still walks (cannot happen once the row is free)
+      const double t = __dmul_rn(scale, rq_nxt.ts_ms);
+      // requests j in [next_r-32, next_r) whose completion may be visible at t: all up to the
+      // latest of them must have been serviced
+      const unsigned hz = __ballot_sync(kFull, lb <= t);
+      const uint32_t rot = next_r & 31u;
+      const unsigned in_order = __funnelshift_r(hz, hz, rot);   // bit k: request next_r - 32 + k
+      const long long need = (long long)next_r - (long long)__clz((int)in_order);
+      if ((long long)srv_seen < need) {
+        srv_seen = *sm.serviced;
+        if ((long long)srv_seen < need) break;
+      }
+      __threadfence_block();   // the service warp's list stores before `serviced` are visible from here on
+      // clear the row, start the walk
+      long long* row = sm.exp_sum + (size_t)owner * R;
+      if (lane < R) row[lane] = 0;
+      if (lane + 32u < R) row[lane + 32u] = 0;
+      __syncwarp();
+      if (lane == owner) { my_r = next_r; head_pending = true; e = kNone; head_val = __ldcg(exp_head + next_r); }
+      if (lane == rot) {
+        const uint32_t dec_tok = rq_nxt.out_tok > 0 ? rq_nxt.out_tok - 1 : 0;
+        lb = __dadd_rn(t, __dmul_rn(tok_ms, (double)dec_tok));
+      }
+      ++next_r;
+      rq_nxt = req[min(next_r, end - 1)];
+      progress = true;
+    }
+    // ---- next hop of every walk
+    if (my_r != kNone && !head_pending && e != kNone) rec_val = __ldcg(exp_rec + e);
+    if (progress) idle = 0;
+    else {
+      if (*abort_flag) break;
+      if (++idle > a.poll_limit) { status = -6; *abort_flag = 1; break; }
+      __nanosleep(40);
+    }
+  }
+  status = __reduce_min_sync(kFull, status);
+  if (lane == 0 && status != 0) atomicMin(const_cast<int32_t*>(cta_status), status);
 }
 
 constexpr uint32_t kStageDepth = 4;                    // requests staged by the probe warp
@@ -707,6 +922,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     }
   };
 
+  PROF_BEGIN();
   for (uint32_t r = a.first; r < end; ++r) {
     const uint32_t n = q_cur.nblk, off = q_cur.off;
     const Ahead q_n2 = fetch_ahead(req, r + 2, end);          // used two rounds from now
@@ -723,6 +939,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       smem_order();
     }
     if (!staged) {
+      PROF_ADD(11, 1);
       uint32_t h0 = 0, h1 = 0, p0 = 0, p1 = 0;
       slot = kStageDepth + (r & 1u);                          // this warp's own stages
       uint32_t* sid = cx.st_ids + slot * kStageBlocks;
@@ -738,9 +955,12 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     }
     const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
     const MaskT* smk = cx.st_mk + slot * kStageBlocks;
+    PROF_LAP(0);
     if (!posted) hand_over(slot, n);
+    PROF_LAP(1);
 
     bar_wait(kBarRoute);                                  // the replica has been chosen
+    PROF_LAP(2);
     const uint32_t istar = *cx.route;
     const MaskT bit = (MaskT)(((MaskT)1) << istar);
 
@@ -757,8 +977,11 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         if (!(mv & bit)) mask_store<MaskT>(mask, id, (MaskT)(mv | bit));
       }
     }
+    PROF_LAP(3);
     uint32_t occ = sm.occ[istar] + missing;
     uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
+    PROF_ADD(12, need > 0 ? 1 : 0);
+    PROF_ADD(15, need);
     uint32_t evicted = 0;
     unsigned hit1 = 0, hit2 = 0, hit3 = 0;   // a victim's block occurs again in request r+1/2/3
     if (need > 0) {
@@ -842,6 +1065,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         }
         if (lane == 0) sm.ring_head[istar] = head;
       }
+      PROF_ADD(13, need > 0 ? 1 : 0);
       uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
       unsigned long long guard = 0;
       while (need > 0) {
@@ -889,6 +1113,7 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
     }
     occ -= evicted;
     st_evict += evicted;
+    PROF_LAP(4);
 
     // ---- which staged reads did the commit of request r invalidate?  If the next request's
     //      are intact and staged, hand them over now: the decide warp works on r+1 while the
@@ -904,7 +1129,9 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
       smem_order();
       hand_over((r + 1) % kStageDepth, q_nxt.nblk);
       posted = true;
+      PROF_ADD(14, 1);
     }
+    PROF_LAP(5);
 
     if (lane == 0) {
       sm.occ[istar] = occ;
@@ -922,13 +1149,16 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         __threadfence_block();
         sm.act[istar] = 1;
       }
+      PROF_LAP(6);
       __threadfence_block();
       *sm.progress = r + 1;                               // request r is fully committed
     }
     __syncwarp();
+    PROF_LAP(7);
 
     q_cur = q_nxt; q_nxt = q_n2;
   }
+  PROF_END(32);
   st_probe = warp_sum_u64(st_probe);
   status = __reduce_min_sync(kFull, status);
   if (lane == 0) {
@@ -941,8 +1171,9 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   }
 }
 
-constexpr uint32_t kWarpDecide = 0, kWarpCache = 1, kWarpProbe = 2, kWarpScout0 = 3;
-constexpr uint32_t kReplayThreads = 32 * (3 + kScouts);
+constexpr uint32_t kWarpRoute = 0, kWarpCache = 1, kWarpProbe = 2, kWarpScout0 = 3;
+constexpr uint32_t kWarpService = 3 + kScouts, kWarpExpiry = 4 + kScouts;
+constexpr uint32_t kReplayThreads = 32 * (5 + kScouts);
 
 template <typename MaskT, bool kBaseline>
 __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayArgs a) {
@@ -956,8 +1187,7 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   unsigned char* st = a.states + (size_t)p * a.lay.bytes;
   CandHeader* hdr = reinterpret_cast<CandHeader*>(st);
   RepState* g_rep = reinterpret_cast<RepState*>(st + a.lay.rep_off);
-  double* g_slot_d = reinterpret_cast<double*>(st + a.lay.slot_d_off);     // 3 x [R*S] doubles
-  uint32_t* g_slot_u = reinterpret_cast<uint32_t*>(st + a.lay.slot_u_off);  // 5 x [R*S] words
+  double* g_slot = reinterpret_cast<double*>(st + a.lay.slot_off);     // [R*S] slot free times
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Ctx<MaskT> cx;
@@ -965,41 +1195,34 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   sm.rtt = reinterpret_cast<double*>(smem_raw);            // [G*R]
   sm.wrtt = sm.rtt + (size_t)G * R;                        // [G*R]  w_net * rtt
   sm.w = sm.wrtt + (size_t)G * R;                          // [K]
-  sm.minfin = sm.w + K;                                    // [R]
-  sm.load = reinterpret_cast<long long*>(sm.minfin + R);   // [R]
-  double* dnext = reinterpret_cast<double*>(sm.load + R);
-  // Per-slot state (in shared memory when it fits, else it stays in global memory).  A slot is a
-  // FIFO of in-flight requests whose finish times never decrease; its two oldest entries are
-  // kept here, the rest is reached through the per-request records in global memory.
-  double* slot_d = g_slot_d;
-  if (a.slots_in_smem) { slot_d = dnext; dnext += 3 * (size_t)RS; }
-  cx.free_at = slot_d;                   // time the slot frees (finish of its newest request)
-  cx.q0_fin = slot_d + RS;               // finish of the oldest in-flight request (+inf: none)
-  cx.q1_fin = slot_d + 2 * (size_t)RS;   // finish of the second oldest
+  sm.load = reinterpret_cast<long long*>(sm.w + K);        // [R]
+  sm.cnt = sm.load + R;                                    // [R]
+  sm.exp_sum = sm.cnt + R;                                 // [kExpRing][R]
+  double* dnext = reinterpret_cast<double*>(sm.exp_sum + (size_t)kExpRing * R);
+  // slot free times (in shared memory when they fit, else they stay in global memory)
+  cx.free_at = g_slot;
+  if (a.slots_in_smem) { cx.free_at = dnext; dnext += RS; }
   sm.occ = reinterpret_cast<uint32_t*>(dnext);             // [R]
   sm.curreq = sm.occ + R;
   sm.curpos = reinterpret_cast<int32_t*>(sm.curreq + R);
   sm.lrutail = reinterpret_cast<uint32_t*>(sm.curpos + R);
   uint32_t* unext = sm.lrutail + R;
-  uint32_t* slot_u = g_slot_u;
-  if (a.slots_in_smem) { slot_u = unext; unext += 5 * (size_t)RS; }
-  cx.q0_tok = slot_u;                    // input tokens of the oldest
-  cx.q1_tok = slot_u + RS;               //   and of the second oldest
-  cx.q2_idx = slot_u + 2 * (size_t)RS;   // request index of the third oldest (kNone: none)
-  cx.tail = slot_u + 3 * (size_t)RS;     // newest request queued on the slot
-  cx.qcnt = slot_u + 4 * (size_t)RS;     // requests in flight on the slot
   sm.progress = unext;
   cx.route = unext + 1;
   cx.status = reinterpret_cast<volatile int32_t*>(unext + 2);
   cx.hit_slot = unext + 3;
-  sm.act = unext + 4;
+  sm.routed = unext + 4;
+  sm.serviced = unext + 5;
+  sm.exp_ready = unext + 6;
+  cx.abort_flag = unext + 7;
+  sm.route_ring = unext + 8;                               // [kRouteRing]
+  sm.act = sm.route_ring + kRouteRing;
   sm.ring_head = sm.act + R;
   sm.ring_tail = sm.ring_head + R;
   sm.scan_cr = sm.ring_tail + R;
   sm.scan_cp = reinterpret_cast<volatile int32_t*>(sm.scan_cr + R);
   {
-    sm.cnt = reinterpret_cast<int32_t*>(const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R);
-    uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 3 * (size_t)R;
+    uint32_t* after = const_cast<uint32_t*>(sm.scan_cr) + 2 * (size_t)R;
     cx.st_ready = after;
     cx.probe_gone = after + kStageDepth;
     cx.st_hits = after + kStageDepth + 1;
@@ -1014,7 +1237,8 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
                              : a.evict_lists + (size_t)p * R * kListCap;
   }
   cx.mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
-  cx.qrec = a.qrec + (size_t)p * N;   // per request: (finish lo, finish hi, next on slot, tokens)
+  cx.exp_head = a.exp_head + (size_t)p * N;
+  cx.exp_rec = a.exp_rec + (size_t)p * N;
   cx.lru_next = a.lru_next + (size_t)p * N;
   cx.route_log = a.route_log + (size_t)p * a.route_log_stride;
 
@@ -1034,41 +1258,37 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   for (uint32_t i = threadIdx.x; i < K; i += blockDim.x) sm.w[i] = a.params[(size_t)p * K + i];
   for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
     const RepState rs = g_rep[i];
-    sm.minfin[i] = rs.min_fin; sm.load[i] = rs.load; sm.occ[i] = rs.occ;
+    sm.load[i] = rs.load; sm.cnt[i] = rs.cnt; sm.occ[i] = rs.occ;
     sm.curreq[i] = rs.cur_req; sm.curpos[i] = rs.cur_pos; sm.lrutail[i] = rs.lru_tail;
     sm.act[i] = 0; sm.ring_head[i] = 0; sm.ring_tail[i] = 0;
   }
-  if (a.slots_in_smem) {
-    for (uint32_t x = threadIdx.x; x < 3 * RS; x += blockDim.x) slot_d[x] = g_slot_d[x];
-    for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) slot_u[x] = g_slot_u[x];
-  }
-  if (threadIdx.x == 0) { *sm.progress = a.first; *cx.status = 0; *cx.probe_gone = 0; }
-  __syncthreads();
-  for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {   // requests in flight per replica
-    int32_t c = 0;
-    for (uint32_t s2 = 0; s2 < S; ++s2) c += (int32_t)cx.qcnt[(size_t)i * S + s2];
-    sm.cnt[i] = c;
+  if (a.slots_in_smem)
+    for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) cx.free_at[x] = g_slot[x];
+  if (threadIdx.x == 0) {
+    *sm.progress = a.first; *cx.status = 0; *cx.probe_gone = 0; *cx.abort_flag = 0;
+    *sm.routed = a.first; *sm.serviced = a.first; *sm.exp_ready = a.first;
   }
   if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
   __syncthreads();
 
-  if (warp == kWarpDecide) decide_warp<MaskT, kBaseline>(a, cx, p, lane);
+  if (warp == kWarpRoute) route_warp<MaskT, kBaseline>(a, cx, p, lane);
   else if (warp == kWarpCache) cache_warp<MaskT>(a, cx, p, lane);
   else if (warp == kWarpProbe) probe_warp<MaskT>(a, cx, lane);
+  else if (warp == kWarpService) service_warp<MaskT, kBaseline>(a, cx, p, lane);
+  else if (warp == kWarpExpiry)
+    expiry_warp<kBaseline>(a, sm, cx.exp_head, cx.exp_rec, cx.abort_flag, cx.status, p, lane);
   else scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, warp - kWarpScout0);
   __syncthreads();
 
   // ---- write the small state back
   for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
     RepState rs;
-    rs.min_fin = sm.minfin[i]; rs.load = sm.load[i]; rs.occ = sm.occ[i];
+    rs.load = sm.load[i]; rs.cnt = sm.cnt[i]; rs.occ = sm.occ[i];
     rs.cur_req = sm.curreq[i]; rs.cur_pos = sm.curpos[i]; rs.lru_tail = sm.lrutail[i];
     g_rep[i] = rs;
   }
-  if (a.slots_in_smem) {
-    for (uint32_t x = threadIdx.x; x < 3 * RS; x += blockDim.x) g_slot_d[x] = slot_d[x];
-    for (uint32_t x = threadIdx.x; x < 5 * RS; x += blockDim.x) g_slot_u[x] = slot_u[x];
-  }
+  if (a.slots_in_smem)
+    for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) g_slot[x] = cx.free_at[x];
   if (threadIdx.x == 0) {
     const int32_t status = *cx.status;
     hdr->processed = a.first + a.count;
@@ -1090,22 +1310,13 @@ __global__ void reset_states_kernel(unsigned char* states, StateLayout lay, uint
   RepState* rep = reinterpret_cast<RepState*>(st + lay.rep_off);
   for (uint32_t i = threadIdx.x; i < R; i += blockDim.x) {
     RepState rs;
-    rs.load = 0; rs.min_fin = d_inf(); rs.occ = 0; rs.cur_req = kNone; rs.cur_pos = -1;
+    rs.load = 0; rs.cnt = 0; rs.occ = 0; rs.cur_req = kNone; rs.cur_pos = -1;
     rs.lru_tail = kNone;
     rep[i] = rs;
   }
-  double* slot_d = reinterpret_cast<double*>(st + lay.slot_d_off);
-  uint32_t* slot_u = reinterpret_cast<uint32_t*>(st + lay.slot_u_off);
+  double* slot = reinterpret_cast<double*>(st + lay.slot_off);
   const uint32_t RS = R * S;
-  for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) {
-    slot_d[x] = 0.0;                    // free_at
-    slot_d[RS + x] = d_inf();           // q0_fin
-    slot_d[2 * (size_t)RS + x] = d_inf();   // q1_fin
-    slot_u[x] = 0; slot_u[RS + x] = 0;  // q0_tok, q1_tok
-    slot_u[2 * (size_t)RS + x] = kNone; // q2_idx
-    slot_u[3 * (size_t)RS + x] = kNone; // tail
-    slot_u[4 * (size_t)RS + x] = 0;     // qcnt
-  }
+  for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) slot[x] = 0.0;   // free from time 0
 }
 
 // ------------------------------------------------------------------------------ select
@@ -1297,14 +1508,14 @@ template <typename MaskT>
 size_t replay_smem_bytes(ReplayArgs& a) {
   const size_t rs = (size_t)a.m.R * a.m.S;
   const size_t list_bytes = (size_t)a.m.R * kListCap * sizeof(uint4);
-  a.slots_in_smem = rs * 44 <= 44 * 1024 ? 1u : 0u;
+  a.slots_in_smem = rs * 8 <= 40 * 1024 ? 1u : 0u;
   a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
-  size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + 2 * (size_t)a.m.R) * sizeof(double) +
-                (10 * (size_t)a.m.R + 4) * sizeof(uint32_t) + 16 +
+  size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + (2 + kExpRing) * (size_t)a.m.R) * sizeof(double) +
+                (9 * (size_t)a.m.R + 8 + kRouteRing) * sizeof(uint32_t) + 16 +
                 (kStageDepth + 1 + (kStageDepth + 2) * ((size_t)a.m.R + kStageBlocks)) * sizeof(uint32_t) +
                 8 + (kStageDepth + 2) * (size_t)a.m.R * sizeof(double) +
                 (kStageDepth + 2) * kStageBlocks * sizeof(MaskT) + 8;
-  if (a.slots_in_smem) smem += rs * 44;
+  if (a.slots_in_smem) smem += rs * 8;
   if (a.lists_in_smem) smem += list_bytes;
   smem = (smem + 15) / 16 * 16;
   return smem;
@@ -1378,10 +1589,12 @@ uint32_t mask_bytes_for(uint32_t n_replicas) {
   return n_replicas <= 8 ? 1u : n_replicas <= 16 ? 2u : n_replicas <= 32 ? 4u : 8u;
 }
 
-cudaError_t launch_reset(unsigned char* masks, uint64_t mask_bytes_total, unsigned char* states,
-                         const StateLayout& lay, const Model& m, uint32_t n_cand,
-                         cudaStream_t st) {
+cudaError_t launch_reset(unsigned char* masks, uint64_t mask_bytes_total, uint32_t* exp_head,
+                         uint64_t exp_head_count, unsigned char* states, const StateLayout& lay,
+                         const Model& m, uint32_t n_cand, cudaStream_t st) {
   cudaError_t e = cudaMemsetAsync(masks, 0, mask_bytes_total, st);
+  if (e != cudaSuccess) return e;
+  e = cudaMemsetAsync(exp_head, 0xFF, exp_head_count * sizeof(uint32_t), st);   // kNone: empty lists
   if (e != cudaSuccess) return e;
   reset_states_kernel<<<n_cand, 128, 0, st>>>(states, lay, m.R, m.S, n_cand);
   return cudaGetLastError();
@@ -1406,6 +1619,15 @@ cudaError_t launch_policy_routes(const TraceView& tr, uint32_t R, bool affinity,
   policy_routes_kernel<<<(tr.n_req + 255) / 256, 256, 0, st>>>(tr, R, affinity ? 1u : 0u, draws, route);
   return cudaGetLastError();
 }
+
+#ifdef GORGO_PROF
+cudaError_t prof_read(unsigned long long* out64, bool reset) {
+  cudaError_t e = cudaMemcpyFromSymbol(out64, g_prof, sizeof(g_prof));
+  if (e != cudaSuccess || !reset) return e;
+  unsigned long long zero[64] = {};
+  return cudaMemcpyToSymbol(g_prof, zero, sizeof(zero));
+}
+#endif
 
 uint32_t window_max() { return kWindowMax; }
 

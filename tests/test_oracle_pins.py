@@ -74,6 +74,8 @@ def test_w1_handworked_trace():
     ids, seq, pos = o.dump(0)
     assert [inv[int(b)] for b in ids] == ["F", "C", "B", "A"]
     assert seq.tolist() == [3, 4, 4, 4] and pos.tolist() == [2, 2, 1, 0]
+    # the four counters the byte model of the benchmark is built from, counted by hand
+    assert o.stats().tolist() == e["counters"]
 
 
 def test_w2_equal_costs_go_to_lowest_index():
@@ -139,6 +141,37 @@ def test_prefix_hits_and_lru_against_recency_list_model(seed, structured):
         assert [int(b) for b in ids] == lists[i]
         assert len(ids) <= C
     assert (res.occ_after <= C).all()
+
+
+@pytest.mark.parametrize("seed,structured", [(5, True), (6, False), (7, True)])
+def test_counters_recomputed_from_per_request_outputs_and_the_recency_list_model(seed, structured):
+    """Oracle.stats() = [sum_r sum_i min(h_{r,i}+1, n_r), sum_r h_{r,i*}, sum_r n_r, sum_r E_r].
+    Recomputed twice without the oracle's own accumulators: from its per-request outputs, and
+    from the independent recency-list cache model driven by the routes alone."""
+    reqs = small_trace(seed, n_req=400, n_sessions=10, max_blocks=7, structured=structured)
+    R, C = 3, 11
+    w = W.handmade(np.array([20.0, 35.0, 50.0]), reqs, slots=2, cache_blocks=C,
+                   params=[[1.0, 0.05, 0.001]])
+    o = O.Oracle.from_workload(w)
+    res = o.run(w.params[0], 1.0, detail=True)
+    st = o.stats().tolist()
+    n = np.array([len(q[3]) for q in reqs], dtype=np.int64)
+    probes = np.minimum(res.hit_all.astype(np.int64) + 1, n[:, None]).sum()
+    chosen = res.hit_all[np.arange(len(reqs)), res.route].astype(np.int64)
+    assert (chosen == res.hit).all()
+    assert st == [int(probes), int(chosen.sum()), int(n.sum()), int(res.evicted.sum())]
+    model, _ = recency_list_replay(reqs, res.route.tolist(), R, C)
+    m_probes = sum(min(h + 1, len(q[3])) for (hits, _, _), q in zip(model, reqs) for h in hits)
+    m_hit = sum(hits[i] for (hits, _, _), i in zip(model, res.route.tolist()))
+    m_ev = sum(ev for (_, _, ev) in model)
+    assert st == [m_probes, m_hit, int(n.sum()), m_ev]
+    assert m_ev > 0 and m_hit > 0
+    # a second run continues the sums; a reset clears them
+    o.reset()
+    assert o.stats().tolist() == [0, 0, 0, 0]
+    o.run(w.params[0], 1.0, count=150)
+    o.run(w.params[0], 1.0)
+    assert o.stats().tolist() == st
 
 
 def test_prefix_hit_brute_force_without_eviction():
