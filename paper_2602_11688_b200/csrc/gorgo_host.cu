@@ -20,6 +20,8 @@ struct gorgo_sim {
   bool has_trace = false;
   TraceView tr = {};
   uint32_t poll_limit = 1u << 24;   // bound of the device-side waits of one warp for another
+  uint32_t ring_polls = 64;         // polls for the scout's victims before a commit warp walks itself
+  uint32_t probe_off = 0, scout_off = 0;   // test switches (gorgo_debug_set)
   // optional CUDA-event timing of the replay kernel (one pair per wave of the last evaluation)
   bool profiling = false;
   std::vector<cudaEvent_t> ev;    // pairs around the replay launches
@@ -247,7 +249,8 @@ int eval_impl(gorgo_sim* sim, uint32_t P, const double* params, double scale, vo
       a.scales = d_scales;
     }
     a.first = 0; a.count = (uint32_t)N; a.check_order = 0;
-    a.poll_limit = sim->poll_limit;
+    a.poll_limit = sim->poll_limit; a.ring_polls = sim->ring_polls;
+    a.probe_off = sim->probe_off; a.scout_off = sim->scout_off;
     a.rtt = d_rtt; a.params = wave_params;
     a.masks = base + w.masks; a.mask_stride = w.mask_stride;
     a.states = base + w.states; a.lay = w.st;
@@ -766,7 +769,8 @@ int gorgo_route_batch(gorgo_sim_t* sim, const double* params, double time_scale,
   ReplayArgs a = {};
   a.m = sim->m; a.tr = sim->tr; a.scale = time_scale;
   a.first = (uint32_t)first; a.count = (uint32_t)count; a.check_order = 1;
-  a.poll_limit = sim->poll_limit;
+  a.poll_limit = sim->poll_limit; a.ring_polls = sim->ring_polls;
+  a.probe_off = sim->probe_off; a.scout_off = sim->scout_off;
   a.rtt = d_rtt; a.params = d_params;
   a.masks = base + w.masks; a.mask_stride = w.mask_stride;
   a.states = base + w.states; a.lay = w.st;

@@ -78,6 +78,8 @@ struct ReplayArgs {
   uint32_t first, count;          // requests [first, first+count)
   uint32_t check_order;           // 1: refuse (status) unless header.processed == first
   uint32_t poll_limit;            // polls after which a warp stops waiting for another one
+  uint32_t ring_polls;            // polls of a commit warp for the scout's next victims before it walks itself
+  uint32_t probe_off, scout_off;  // test switches: run without the probe warp / without the scout warps
   uint32_t slots_in_smem;         // set by the launcher: per-slot state fits in shared memory
   uint32_t lists_in_smem;         // set by the launcher: eviction lists fit in shared memory
   uint4* evict_lists;             // [P * evict_list_bytes(R)] scratch used when they do not

@@ -131,7 +131,18 @@ __device__ __forceinline__ void mask_clear_bit(MaskT* mask, uint32_t id, MaskT b
     atomicAnd(reinterpret_cast<unsigned int*>(addr & ~(uintptr_t)3), ~((uint32_t)bit << sh));
   }
 }
-// Mask words are read and written around L1: they are also changed by reductions in L2.
+// Set `bit` of mask[id] the same way.
+template <typename MaskT>
+__device__ __forceinline__ void mask_set_bit(MaskT* mask, uint32_t id, MaskT bit) {
+  if (sizeof(MaskT) == 8) {
+    atomicOr(reinterpret_cast<unsigned long long*>(mask) + id, (unsigned long long)bit);
+  } else {
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(mask + id);
+    const uint32_t sh = (uint32_t)(addr & 3u) * 8u;
+    atomicOr(reinterpret_cast<unsigned int*>(addr & ~(uintptr_t)3), (uint32_t)bit << sh);
+  }
+}
+// Mask words are read around L1: they are changed by reductions in L2.
 template <typename MaskT>
 __device__ __forceinline__ MaskT mask_load(const MaskT* mask, uint32_t id) {
   return __ldcg(mask + id);
@@ -165,11 +176,20 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
   __stcg(reinterpret_cast<unsigned long long*>(mask) + id, (unsigned long long)v);
 }
 
-constexpr int kRegChunks = 8;     // request blocks held in registers: 8 x 32 = 256
+constexpr int kRegChunks = 4;     // request blocks held in registers: 4 x 32 = 128
 constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
 constexpr int kScoutBatches = 1;       // touches examined per lane and scout round
 constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is this close to full
+
+// rings and counts of the warps of one candidate
+constexpr uint32_t kRouteRing = 32;   // routes handed from the route warp to the service warp
+constexpr uint32_t kRouteLead = 24;   // the route warp runs at most this far ahead of the service warp
+constexpr uint32_t kExpRing = 8;      // completion sums published ahead of the route warp
+constexpr uint32_t kCommitWarps = 3;  // commit warps per candidate (replicas split between them)
+constexpr uint32_t kJobRing = 32;     // routed requests handed from the gate warp to the commit warps
+constexpr uint32_t kHitRing = 16;     // tags of requests hit by a recent eviction (> kWindow)
+constexpr uint32_t kServices = 2;      // service warps per candidate (replicas split between them)
 
 // Shared-memory view of one candidate's small state.
 struct Smem {
@@ -177,10 +197,13 @@ struct Smem {
   long long* load;                // in-flight input tokens per replica (as of the last launch; the route warp keeps the live value)
   long long* cnt;                 // in-flight requests per replica (kept when the queue signal counts requests)
   uint32_t* occ; uint32_t* curreq; int32_t* curpos; uint32_t* lrutail;
-  volatile uint32_t* progress;
+  volatile uint32_t* progress;    // [kCommitWarps] requests each commit warp has passed
+  volatile uint32_t* abort_flag;  // a bounded wait ran out: the other waits stop too
+  volatile uint32_t* jobs;        // requests handed to the commit warps
+  uint32_t* job;                  // [kJobRing] replica | stage << 8 | blocks << 16
   // hand-over between the route, service and expiry warps
   volatile uint32_t* routed;      // requests routed so far
-  volatile uint32_t* serviced;    // requests whose service commit is done and whose completion is filed
+  volatile uint32_t* serviced;    // [kServices] requests each service warp has passed (serviced and filed, or not its own)
   volatile uint32_t* exp_ready;   // requests whose completion sums are published
   uint32_t* route_ring;           // [kRouteRing] chosen replica | prefix hit there << 8
   long long* exp_sum;             // [kExpRing][R] tokens (or requests) that completed by the request's arrival
@@ -194,6 +217,42 @@ struct Smem {
   volatile uint32_t* scan_cr;     // scout's own cursor into the recency order (set at activation)
   volatile int32_t* scan_cp;
 };
+
+// Requests committed on every replica: the slowest commit warp's position.
+__device__ __forceinline__ uint32_t committed(const Smem& sm) {
+  uint32_t v = sm.progress[0];
+#pragma unroll
+  for (uint32_t k = 1; k < kCommitWarps; ++k) v = min(v, sm.progress[k]);
+  return v;
+}
+// Bounded wait until every request < want is committed.
+__device__ __forceinline__ void wait_committed(const Smem& sm, uint32_t want, uint32_t limit, int32_t& status) {
+  uint32_t polls = 0;
+  while ((int32_t)(committed(sm) - want) < 0) {
+    if (*sm.abort_flag) break;
+    if (++polls > limit) { status = -6; *sm.abort_flag = 1; break; }
+    __nanosleep(20);
+  }
+}
+
+// Requests every service warp has passed.
+__device__ __forceinline__ uint32_t serviced_all(const Smem& sm) {
+  uint32_t v = sm.serviced[0];
+#pragma unroll
+  for (uint32_t k = 1; k < kServices; ++k) v = min(v, sm.serviced[k]);
+  return v;
+}
+__device__ __forceinline__ uint32_t wait_serviced(const Smem& sm, uint32_t want, uint32_t limit, int32_t& status) {
+  uint32_t polls = 0;
+  uint32_t v = serviced_all(sm);
+  while ((int32_t)(v - want) < 0) {
+    if (*sm.abort_flag) break;
+    if (++polls > limit) { status = -6; *sm.abort_flag = 1; break; }
+    __nanosleep(20);
+    v = serviced_all(sm);
+  }
+  return v;
+}
 
 // Scout warp: for every replica whose cache is close to full it walks the recency order ahead
 // of the eviction cursor and appends to the replica's ring the touches that are still the latest
@@ -209,9 +268,10 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
   const uint32_t R = a.m.R;
   uint32_t idle = 0;
   uint32_t blocked0 = kNone - 1, blocked1 = kNone - 1;  // lru tail seen when the scan ran dry
+  if (a.scout_off) return;                               // (test switch: the commit warps find their victims themselves)
   while (true) {
-    const uint32_t prog = *sm.progress;
-    if (prog >= end) break;
+    const uint32_t prog = committed(sm);
+    if (prog >= end || *sm.abort_flag) break;
     // the active replica with the emptiest ring that can still be extended
     uint32_t best = kNone;
 #pragma unroll
@@ -329,22 +389,18 @@ struct Ctx {
   double* free_at;             // [R*S] time each slot frees (shared or global memory)
   volatile uint32_t* route;    // chosen replica of the current request
   volatile int32_t* status;    // first device-side limit hit by any warp
-  volatile uint32_t* abort_flag;  // a bounded wait ran out: the other waits stop too
   // staging of the coming requests by the probe warp (kStageDepth stages + one of the cache warp)
   volatile uint32_t* st_ready; // [kStageDepth] request (+1) whose data the stage holds
   volatile uint32_t* probe_gone;  // the probe warp has stopped
   // (stages kStageDepth and kStageDepth+1 belong to the cache warp, used alternately)
   uint32_t* st_hits;           // [kStageDepth+2][R] prefix hit | blocks present << 16
   double* st_ab;               // [kStageDepth+2][R] (w_net*RTT + w_prefill*uncached) per replica
+  unsigned long long* st_where;  // [kStageDepth+2] replicas that held any block of the request when it was read
+  volatile uint32_t* evhit;    // [kHitRing] evhit[q % kHitRing] == q: a recent eviction took a block of request q
   uint32_t* st_ids;            // [kStageDepth+2][kStageBlocks] block ids
   MaskT* st_mk;                // [kStageDepth+2][kStageBlocks] mask words
   volatile uint32_t* hit_slot; // stage that holds the current request's hits and scores
 };
-
-// (forward) rings between the route, service and expiry warps
-constexpr uint32_t kRouteRing = 32;   // routes handed from the route warp to the service warp
-constexpr uint32_t kRouteLead = 24;   // the route warp runs at most this far ahead of the service warp
-constexpr uint32_t kExpRing = 8;      // completion sums published ahead of the route warp
 
 // Bounded wait of one warp for a counter another warp of the candidate advances: polls until
 // (int)(counter - want) >= 0.  If the limit runs out (or another warp already gave up) the
@@ -406,9 +462,9 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
     // ---- completions the proxy has seen by this arrival (published by the expiry warp), and
     //      room in the ring of routes the service warp has not taken yet
     if ((int32_t)(exp_seen - (r + 1)) < 0)
-      exp_seen = wait_counter(sm.exp_ready, r + 1, cx.abort_flag, a.poll_limit, status);
+      exp_seen = wait_counter(sm.exp_ready, r + 1, sm.abort_flag, a.poll_limit, status);
     if (r - srv_seen >= kRouteLead)
-      srv_seen = wait_counter(sm.serviced, r + 1 - kRouteLead, cx.abort_flag, a.poll_limit, status);
+      srv_seen = wait_serviced(sm, r + 1 - kRouteLead, a.poll_limit, status);
     smem_order();
     PROF_LAP(0);
     const long long* gone = sm.exp_sum + (size_t)(r % kExpRing) * R;
@@ -497,7 +553,8 @@ __device__ __forceinline__ uint32_t first_arrival_at_or_after(const double* ts, 
 // and the list insertion need three dependent memory round trips; they run as a three-stage
 // pipeline over consecutive requests so that none of them is waited for.
 template <typename MaskT, bool kBaseline>
-__device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
+__device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane,
+                                             uint32_t which) {
   const Smem& sm = cx.sm;
   const uint32_t R = a.m.R, S = a.m.S;
   const uint32_t N = a.tr.n_req;
@@ -518,19 +575,15 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
   uint32_t j3 = kNone, tok3 = 0, rep3 = 0, old3 = kNone;                       // list head exchange in flight (old3: lane 0)
   bool ins1 = false, ins2 = false, ins3 = false;   // the request gets a list entry (it completes before the trace ends)
   uint32_t s = a.first;
-  uint32_t routed_seen = a.first;
-  ReqRec rec_nxt = req[a.first];
+  uint32_t routed_seen = a.first, published = a.first;
   uint32_t idle = 0;
   bool failed = false;
 
   PROF_BEGIN();
   while (true) {
     // ---- what arrived since the last round
-    uint32_t fin = kNone;
-    if (j3 != kNone) {
-      if (ins3 && lane == 0) cx.exp_rec[j3] = make_uint4(old3, tok3, rep3, 0u);
-      fin = j3 + 1;
-    }
+    const bool retired = j3 != kNone;
+    if (retired && ins3 && lane == 0) cx.exp_rec[j3] = make_uint4(old3, tok3, rep3, 0u);
     uint32_t x2 = kNone;
     if (j2 != kNone && ins2) {
       const bool ok = lo2 + lane < N && __dmul_rn(scale, win2) >= f2;
@@ -540,12 +593,19 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
     }
     const uint32_t g = __shfl_sync(kFull, g1, 0);
     PROF_LAP(0);
-    // ---- publish the requests whose list entry is linked
-    if (fin != kNone && lane == 0) {
-      __threadfence_block();
-      *sm.serviced = fin;
+    // ---- publish how far this warp has got: every request before the oldest one it still works
+    //      on is filed, or belongs to the other service warp
+    {
+      const uint32_t upto = j2 != kNone ? j2 : j1 != kNone ? j1 : s;
+      if (upto != published) {
+        published = upto;
+        if (lane == 0) {
+          if (retired) __threadfence_block();
+          sm.serviced[which] = upto;
+        }
+      }
+      if (upto == end) break;
     }
-    if (fin == end) break;
     PROF_LAP(1);
     // ---- next stage of each request in the pipeline
     j3 = j2; tok3 = tok2; rep3 = rep2; ins3 = ins2;
@@ -558,14 +618,15 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
     j1 = kNone; ins1 = false;
     PROF_LAP(2);
 
-    // ---- service model of the next routed request, if there is one
+    // ---- service model of the next routed request of this warp's replicas, if there is one
+    if (s < end && (int32_t)(routed_seen - (s + 1)) < 0) routed_seen = *sm.routed;
+    smem_order();
+    while (s < end && (int32_t)(routed_seen - (s + 1)) >= 0 &&
+           (sm.route_ring[s % kRouteRing] & 0xFFu) % kServices != which) ++s;   // the other warp's
     if (s < end) {
-      if ((int32_t)(routed_seen - (s + 1)) < 0) routed_seen = *sm.routed;
       if ((int32_t)(routed_seen - (s + 1)) >= 0) {
-        smem_order();
         idle = 0;
-        const ReqRec rec = rec_nxt;
-        rec_nxt = req[min(s + 1, end - 1)];
+        const ReqRec rec = req[s];
         const uint32_t rq = sm.route_ring[s % kRouteRing];
         const uint32_t istar = rq & 0xFFu, hstar = rq >> 8;
         const double t = __dmul_rn(scale, rec.ts_ms);
@@ -619,9 +680,9 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
         continue;
       }
     }
-    if (j2 == kNone && j3 == kNone) {        // nothing in flight and no route to take: wait
-      if (*cx.abort_flag) failed = true;
-      if (++idle > a.poll_limit) { status = -6; *cx.abort_flag = 1; failed = true; }
+    if (j2 == kNone && j3 == kNone && s < end) {   // nothing in flight and no route to take: wait
+      if (*sm.abort_flag) failed = true;
+      if (++idle > a.poll_limit) { status = -6; *sm.abort_flag = 1; failed = true; }
       if (failed) break;
       __nanosleep(40);
     }
@@ -706,7 +767,7 @@ __device__ __forceinline__ void expiry_warp(const ReplayArgs& a, const Smem& sm,
       const unsigned in_order = __funnelshift_r(hz, hz, rot);   // bit k: request next_r - 32 + k
       const long long need = (long long)next_r - (long long)__clz((int)in_order);
       if ((long long)srv_seen < need) {
-        srv_seen = *sm.serviced;
+        srv_seen = serviced_all(sm);
         if ((long long)srv_seen < need) break;
       }
       __threadfence_block();   // the service warp's list stores before `serviced` are visible from here on
@@ -737,9 +798,10 @@ __device__ __forceinline__ void expiry_warp(const ReplayArgs& a, const Smem& sm,
   if (lane == 0 && status != 0) atomicMin(const_cast<int32_t*>(cta_status), status);
 }
 
-constexpr uint32_t kStageDepth = 4;                    // requests staged by the probe warp
+constexpr uint32_t kStageDepth = 14;                   // requests staged by the probe warps (> kWindow)
 constexpr uint32_t kStageBlocks = kRegChunks * 32u;    // blocks of a request kept per stage
-constexpr uint32_t kWindow = 3;   // a staged read may be up to this many commits old
+constexpr uint32_t kWindow = 12;  // a staged read may be up to this many commits old (<= 32)
+constexpr uint32_t kProbes = 2;   // probe warps per candidate (requests alternate between them)
 
 // What a warp needs to know of a request ahead of time.
 struct Ahead { uint32_t off, nblk, prev_share, in_tok, origin; };
@@ -772,8 +834,8 @@ template <typename MaskT>
 __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask,
                                              const uint32_t* ids, const Ahead& q, uint32_t R,
                                              uint32_t lane, uint32_t& h0, uint32_t& h1,
-                                             uint32_t& p0, uint32_t& p1) {
-  h0 = 0; h1 = 0; p0 = 0; p1 = 0;
+                                             uint32_t& p0, uint32_t& p1, unsigned long long& where) {
+  h0 = 0; h1 = 0; p0 = 0; p1 = 0; where = 0;
   const uint32_t n = q.nblk;
   MaskT alive = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0 : (MaskT)((((MaskT)1) << (R & 63)) - 1);
   for (uint32_t c = 0; c < n; c += 32) {
@@ -781,6 +843,7 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
     MaskT m = 0;
     if (k < n) m = (c < kStageBlocks) ? smk[k] : mask_load<MaskT>(mask, ids[q.off + k]);
     MaskT it = warp_or_mask<MaskT>(m);      // replicas that hold any block of this chunk
+    where |= (unsigned long long)it;
     MaskT still = 0;
     while (it != 0) {
       const int i = first_bit<MaskT>(it);
@@ -804,8 +867,10 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
 template <typename MaskT>
 __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<MaskT>& cx,
                                              const Ahead& q, uint32_t slot, uint32_t h0,
-                                             uint32_t h1, uint32_t p0, uint32_t p1, uint32_t lane) {
+                                             uint32_t h1, uint32_t p0, uint32_t p1,
+                                             unsigned long long where, uint32_t lane) {
   const uint32_t R = a.m.R;
+  if (lane == 0) cx.st_where[slot] = where;
   const double w_pre = cx.sm.w[1];
   const double* wrtt_row = cx.sm.wrtt + (size_t)q.origin * R;
 #pragma unroll
@@ -828,14 +893,16 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
 // repeats the work itself, so this warp is an accelerator only and may stop at any time.
 template <typename MaskT>
 __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>& cx,
-                                           uint32_t lane) {
+                                           uint32_t lane, uint32_t which) {
   const Smem& sm = cx.sm;
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
   const MaskT* mask = cx.mask;
   const uint32_t R = a.m.R;
   const uint32_t end = a.first + a.count;
-  Ahead q_a = fetch_ahead(req, a.first, end), q_n = fetch_ahead(req, a.first + 1, end);
+  if (a.probe_off) { if (lane == 0) *cx.probe_gone = 1; return; }   // (test switch: the gate warp probes every request)
+  const uint32_t q0 = a.first + which;                  // this warp takes requests q0, q0 + kProbes, ...
+  Ahead q_a = fetch_ahead(req, q0, end), q_n = fetch_ahead(req, q0 + kProbes, end);
   Ahead q_b = q_a;
   uint32_t id_a[kRegChunks], id_n[kRegChunks], id_b[kRegChunks];
   MaskT m_a[kRegChunks], m_b[kRegChunks];
@@ -845,13 +912,13 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
     id_a[c] = (k < q_a.nblk) ? ids[q_a.off + k] : 0u;
     id_b[c] = 0u; m_b[c] = (MaskT)0;
   }
-  for (uint32_t qa = a.first; qa <= end; ++qa) {
+  for (uint32_t qa = q0; qa < end + kProbes; qa += kProbes) {
     if (qa < end) {
       // room: the stage of request qa is free and its read is at most kWindow commits old once
       // request qa - kWindow - 1 is committed, i.e. progress >= qa - kWindow
       uint32_t polls = 0;
-      while ((int32_t)(*sm.progress - qa) < -(int32_t)kWindow) {
-        if (++polls > (1u << 22)) { *cx.probe_gone = 1; return; }   // bounded wait
+      while ((int32_t)(committed(sm) - qa) < -(int32_t)kWindow) {
+        if (++polls > (1u << 22) || *sm.abort_flag) { *cx.probe_gone = 1; return; }   // bounded wait
         __nanosleep(20);
       }
 #pragma unroll
@@ -861,10 +928,10 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
         id_n[c] = (k < q_n.nblk) ? ids[q_n.off + k] : 0u;     // ids of the request after
       }
     }
-    const Ahead q_nn = fetch_ahead(req, qa + 2, end);
-    if (qa > a.first) {
-      // stage and probe the previous request (its mask words were requested one round ago)
-      const uint32_t qb = qa - 1, slot = qb % kStageDepth;
+    const Ahead q_nn = fetch_ahead(req, qa + 2 * kProbes, end);
+    if (qa > q0) {
+      // stage and probe this warp's previous request (its mask words were requested one round ago)
+      const uint32_t qb = qa - kProbes, slot = qb % kStageDepth;
       uint32_t* sid = cx.st_ids + slot * kStageBlocks;
       MaskT* smk = cx.st_mk + slot * kStageBlocks;
 #pragma unroll
@@ -874,8 +941,9 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
       }
       __syncwarp();
       uint32_t h0, h1, p0, p1;
-      probe_staged<MaskT>(smk, mask, ids, q_b, R, lane, h0, h1, p0, p1);
-      stage_scores<MaskT>(a, cx, q_b, slot, h0, h1, p0, p1, lane);
+      unsigned long long where;
+      probe_staged<MaskT>(smk, mask, ids, q_b, R, lane, h0, h1, p0, p1, where);
+      stage_scores<MaskT>(a, cx, q_b, slot, h0, h1, p0, p1, where, lane);
       smem_order();
       __syncwarp();
       if (lane == 0) cx.st_ready[slot] = qb + 1;
@@ -886,12 +954,146 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
   }
 }
 
-// Cache warp: takes the staged prefix hits of request r (or reads and probes the mask words
-// itself when a recent commit can have changed them), and, once the route is known, does the
-// LRU commit on the chosen replica: set its bit on the missing blocks, evict down to capacity.
+// Gate warp: the partner of the route warp.  For every request it decides whether the prefix
+// hits the probe warp staged are still exact, hands them to the route warp, and passes the routed
+// request on to the commit warps.  A staged read of request q may predate the commits of the
+// kWindow requests before q.  Such a commit can have changed q's hits only if it (a) shares a
+// block with q -- known from the trace: `prev_share` -- or (b) evicted a block of q, which needs
+// the commit to have been routed to a replica that held one of q's blocks when they were read
+// (`st_where`).  If neither can be the case the staged hits go out the moment the previous route
+// is known; otherwise the gate waits for the commits in question and looks at what they report
+// (`evhit`), and if need be reads and probes the mask words again itself.
 template <typename MaskT>
-__device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
-                                           uint32_t lane) {
+__device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
+                                          uint32_t lane) {
+  const Smem& sm = cx.sm;
+  const uint32_t R = a.m.R;
+  const ReqRec* req = a.tr.req;
+  const uint32_t* ids = a.tr.ids;
+  const MaskT* mask = cx.mask;
+  int32_t status = 0;
+  unsigned long long st_probe = 0;
+  const uint32_t end = a.first + a.count;
+
+  Ahead q_cur = fetch_ahead(req, a.first, end), q_nxt = fetch_ahead(req, a.first + 1, end);
+  uint32_t my_req = kNone, my_rep = 0;   // lane l: the latest routed request with index % 32 == l, and its replica
+  bool posted = false;             // the hits of the coming request were already handed over
+  uint32_t slot = 0;               // stage that holds the current request's ids, mask words and hits
+  // hand the hits of a request over to the route warp and count its probes
+  auto hand_over = [&](uint32_t sl, uint32_t nblk) {
+    if (lane == 0) *cx.hit_slot = sl;
+    bar_arrive(kBarHits);                                 // the route warp may score the request
+    if (a.stats) {                                        // probes the plain formula charges
+      if (lane < R) { const uint32_t h = cx.st_hits[sl * R + lane] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+      if (lane + 32u < R) { const uint32_t h = cx.st_hits[sl * R + lane + 32u] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+    }
+  };
+  // latest request among the kWindow before q that was routed to a replica in `where` (kNone: none)
+  auto conflict = [&](uint32_t q, unsigned long long where) -> uint32_t {
+    const bool hit = my_req != kNone && q - 1u - my_req < kWindow && ((where >> my_rep) & 1ull);
+    if (!__any_sync(kFull, hit)) return kNone;
+    return __reduce_max_sync(kFull, hit ? my_req : 0u);
+  };
+  // does a commit since its staged read share a block with the request?
+  auto shares = [&](const Ahead& q, uint32_t idx) {
+    return q.prev_share != kNone && q.prev_share + kWindow >= idx;
+  };
+
+  PROF_BEGIN();
+  for (uint32_t r = a.first; r < end; ++r) {
+    const Ahead q_n2 = fetch_ahead(req, r + 2, end);          // used two rounds from now
+    const uint32_t n = q_cur.nblk;
+
+    // ---- prefix hits of request r, unless they went out right after the previous route
+    if (!posted) {
+      const bool sh = shares(q_cur, r);
+      bool staged = false;
+      uint32_t done_to = sh ? r : 0u;                         // requests < done_to must be committed
+      if (!sh && !*cx.probe_gone) {
+        const uint32_t ss = r % kStageDepth;
+        uint32_t polls = 0;
+        while (cx.st_ready[ss] != r + 1 && !*cx.probe_gone && polls < 4096) { ++polls; __nanosleep(20); }
+        // (one lane decides: every lane must take the same path)
+        staged = __shfl_sync(kFull, cx.st_ready[ss], 0) == r + 1;
+        smem_order();
+        if (staged) {
+          const uint32_t c = conflict(r, cx.st_where[ss]);
+          if (c != kNone) done_to = c + 1;
+        }
+      }
+      if (!staged) done_to = r;
+      PROF_LAP(3);
+      if (done_to > a.first) wait_committed(sm, done_to, a.poll_limit, status);
+      smem_order();
+      PROF_LAP(4);
+      if (staged && (done_to <= a.first || cx.evhit[r % kHitRing] != r)) {
+        slot = r % kStageDepth;
+      } else {
+        // read and probe here, after every earlier request is committed
+        PROF_ADD(11, 1);
+        if (done_to < r) wait_committed(sm, r, a.poll_limit, status);
+        uint32_t h0 = 0, h1 = 0, p0 = 0, p1 = 0;
+        slot = kStageDepth + (r & 1u);                          // this warp's own stages
+        uint32_t* sid = cx.st_ids + slot * kStageBlocks;
+        MaskT* smk = cx.st_mk + slot * kStageBlocks;
+        for (uint32_t c = 0; c < n && c < kStageBlocks; c += 32) {
+          const uint32_t k = c + lane;
+          if (k < n) { const uint32_t id = ids[q_cur.off + k]; sid[k] = id; smk[k] = mask_load<MaskT>(mask, id); }
+        }
+        __syncwarp();
+        unsigned long long where = 0;
+        probe_staged<MaskT>(smk, mask, ids, q_cur, R, lane, h0, h1, p0, p1, where);
+        stage_scores<MaskT>(a, cx, q_cur, slot, h0, h1, p0, p1, where, lane);
+        __syncwarp();
+      }
+      hand_over(slot, n);
+    }
+    PROF_LAP(0);
+
+    bar_wait(kBarRoute);                                  // the replica has been chosen
+    PROF_LAP(1);
+    const uint32_t istar = *cx.route;
+    if (lane == 0) {
+      sm.job[r % kJobRing] = istar | (slot << 8) | (n << 16);
+      smem_order();
+      *sm.jobs = r + 1;                                   // the commit warps may take request r
+    }
+    if (lane == (r & 31u)) { my_req = r; my_rep = istar; }
+
+    // ---- the next request's hits go out now if no commit since their read can have touched them
+    posted = false;
+    if (r + 1 < end && !shares(q_nxt, r + 1)) {
+      const uint32_t ss = (r + 1) % kStageDepth;
+      if (__shfl_sync(kFull, cx.st_ready[ss], 0) == r + 2) {
+        smem_order();
+        if (conflict(r + 1, cx.st_where[ss]) == kNone) {
+          slot = ss;
+          hand_over(slot, q_nxt.nblk);
+          posted = true;
+          PROF_ADD(14, 1);
+        } else PROF_ADD(13, 1);
+      } else PROF_ADD(12, 1);
+    } else PROF_ADD(10, 1);
+    PROF_LAP(2);
+    q_cur = q_nxt; q_nxt = q_n2;
+  }
+  PROF_END(32);
+  st_probe = warp_sum_u64(st_probe);
+  status = __reduce_min_sync(kFull, status);
+  if (lane == 0) {
+    if (status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
+    if (a.stats) atomicAdd(reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4, st_probe);
+  }
+}
+
+// Commit warp `which` of kCommitWarps: the LRU commits of the requests routed to replicas
+// i % kCommitWarps == which, in request order.  Commits on different replicas touch different
+// bits of the mask words (set and cleared by reductions) and different recency lists, so the
+// warps need no order among themselves; `progress[which]` says how far this one has got, and a
+// request counts as committed once every warp has passed it.
+template <typename MaskT>
+__device__ __forceinline__ void commit_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
+                                            uint32_t lane, uint32_t which) {
   const Smem& sm = cx.sm;
   const uint32_t R = a.m.R;
   const uint32_t N = a.tr.n_req;
@@ -901,237 +1103,208 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
   uint32_t* lru_next = cx.lru_next;
   const uint8_t* route_log = cx.route_log;
   int32_t status = 0;
-  unsigned long long st_probe = 0, st_evict = 0;
+  unsigned long long st_evict = 0;
   const unsigned long long evict_guard_max = (unsigned long long)N + a.tr.n_ids / 16u + 64u;
   const uint32_t end = a.first + a.count;
-
-  Ahead q_cur = fetch_ahead(req, a.first, end), q_nxt = fetch_ahead(req, a.first + 1, end);
-  // latest earlier request sharing a block with r+1, r+2, r+3, and whether a commit since their
-  // staged read can have changed their mask words
-  uint32_t ps1 = q_nxt.prev_share, ps2 = fetch_ahead(req, a.first + 2, end).prev_share,
-           ps3 = fetch_ahead(req, a.first + 3, end).prev_share;
-  bool bad0 = false, bad1 = false, bad2 = false, bad3 = false;
-  bool posted = false;         // the hits of the coming request were already handed over
-  // hand the staged hits of request q over to the decide warp and count its probes
-  auto hand_over = [&](uint32_t slot, uint32_t nblk) {
-    if (lane == 0) *cx.hit_slot = slot;
-    bar_arrive(kBarHits);                                 // the decide warp may score the request
-    if (a.stats) {                                        // probes the plain formula charges
-      if (lane < R) { const uint32_t h = cx.st_hits[slot * R + lane] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
-      if (lane + 32u < R) { const uint32_t h = cx.st_hits[slot * R + lane + 32u] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
-    }
-  };
+  uint32_t jobs_seen = a.first;
+  // a victim's block occurs again in request q soon after r: tell the gate warp
+  auto mark_hit = [&](uint32_t q) { cx.evhit[q % kHitRing] = q; };
 
   PROF_BEGIN();
   for (uint32_t r = a.first; r < end; ++r) {
-    const uint32_t n = q_cur.nblk, off = q_cur.off;
-    const Ahead q_n2 = fetch_ahead(req, r + 2, end);          // used two rounds from now
-    const uint32_t ps4 = (r + 4 < end) ? req[r + 4].prev_share : kNone;
-
-    // ---- prefix hits of request r: staged by the probe warp, or read and probed here
-    uint32_t slot = r % kStageDepth;
-    bool staged = posted;
-    if (!posted && !bad0 && !*cx.probe_gone) {
-      uint32_t polls = 0;
-      while (cx.st_ready[slot] != r + 1 && !*cx.probe_gone && polls < 4096) { ++polls; __nanosleep(20); }
-      // (one lane decides: every lane must take the same path)
-      staged = __shfl_sync(kFull, cx.st_ready[slot], 0) == r + 1;
-      smem_order();
+    if ((int32_t)(jobs_seen - (r + 1)) < 0) {
+      jobs_seen = wait_counter(sm.jobs, r + 1, sm.abort_flag, a.poll_limit, status);
+      if ((int32_t)(jobs_seen - (r + 1)) < 0) break;        // gave up
     }
-    if (!staged) {
-      PROF_ADD(11, 1);
-      uint32_t h0 = 0, h1 = 0, p0 = 0, p1 = 0;
-      slot = kStageDepth + (r & 1u);                          // this warp's own stages
-      uint32_t* sid = cx.st_ids + slot * kStageBlocks;
-      MaskT* smk = cx.st_mk + slot * kStageBlocks;
-#pragma unroll
-      for (int c = 0; c < kRegChunks; ++c) {
-        const uint32_t k = c * 32u + lane;
-        if (k < n) { const uint32_t id = ids[off + k]; sid[k] = id; smk[k] = mask_load<MaskT>(mask, id); }
-      }
-      __syncwarp();
-      probe_staged<MaskT>(smk, mask, ids, q_cur, R, lane, h0, h1, p0, p1);
-      stage_scores<MaskT>(a, cx, q_cur, slot, h0, h1, p0, p1, lane);
+    smem_order();
+    PROF_LAP(0);
+    const uint32_t job = sm.job[r % kJobRing];
+    const uint32_t istar = job & 0xFFu;
+    if (istar % kCommitWarps != which) {                    // another warp's replica
+      if (lane == 0) sm.progress[which] = r + 1;
+      PROF_LAP(4);
+      continue;
     }
+    const uint32_t slot = (job >> 8) & 0xFFu, n = job >> 16;
+    const MaskT bit = (MaskT)(((MaskT)1) << istar);
     const uint32_t* sid = cx.st_ids + slot * kStageBlocks;
     const MaskT* smk = cx.st_mk + slot * kStageBlocks;
-    PROF_LAP(0);
-    if (!posted) hand_over(slot, n);
+
+    // ---- how many blocks the commit inserts (the probe counted the blocks already present on
+    //      the replica) and how many it has to evict first
+    const uint32_t missing = n - (cx.st_hits[slot * R + istar] >> 16);
+    uint32_t occ = sm.occ[istar] + missing;
+    uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
+    PROF_ADD(12, need > 0 ? 1 : 0);
+    PROF_ADD(15, need);
+    uint32_t evicted = 0;
+    if (need > 0) {
+      uint32_t cr = sm.curreq[istar];
+      int32_t cp = sm.curpos[istar];
+      bool clean = false;
+      // clean case: the scout's ring already holds `need` entries, none of them void or touched
+      // again since it was listed; then exactly these are the victims
+      if (sm.act[istar] && need <= 96u) {
+        const uint32_t head = sm.ring_head[istar];
+        if (sm.ring_tail[istar] - head >= need) {
+          smem_order();
+          const uint4* lst = sm.lst + (size_t)istar * kListCap;
+          uint4 v0 = make_uint4(0, kNone, 0, 0), v1 = v0, v2 = v0;
+          bool odd = false;
+          auto look = [&](uint32_t idx, uint4& v) {
+            if (idx < need) {
+              const uint32_t e = (head + idx) & (kListCap - 1);
+              v = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+              odd = odd || v.y <= r || v.w < cr || (v.w == cr && (int32_t)v.z > cp);
+            }
+          };
+          look(lane, v0);
+          if (need > 32u) look(lane + 32u, v1);
+          if (need > 64u) look(lane + 64u, v2);
+          if (!__any_sync(kFull, odd)) {
+            if (lane < need) { mask_clear_bit<MaskT>(mask, v0.x, bit); if (v0.y - (r + 1) < kWindow) mark_hit(v0.y); }
+            if (lane + 32u < need) { mask_clear_bit<MaskT>(mask, v1.x, bit); if (v1.y - (r + 1) < kWindow) mark_hit(v1.y); }
+            if (lane + 64u < need) { mask_clear_bit<MaskT>(mask, v2.x, bit); if (v2.y - (r + 1) < kWindow) mark_hit(v2.y); }
+            // the eviction cursor moves behind the last victim
+            const uint32_t li = need - 1;
+            if (lane == (li & 31u)) {
+              const uint4 le = li < 32u ? v0 : li < 64u ? v1 : v2;
+              sm.curreq[istar] = le.w;
+              sm.curpos[istar] = (int32_t)le.z - 1;
+            }
+            if (lane == 0) sm.ring_head[istar] = head + need;
+            evicted = need;
+            need = 0;
+            clean = true;
+            PROF_ADD(8, 1);
+          } else PROF_ADD(9, 1);
+        } else PROF_ADD(10, 1);
+      } else PROF_ADD(11, 1);
+      if (!clean) {
+        // victims from the ring the scout warp keeps for this replica, entry by entry
+        if (sm.act[istar]) {
+          const uint4* lst = sm.lst + (size_t)istar * kListCap;
+          uint32_t head = sm.ring_head[istar];
+          uint32_t last_e = kNone;   // ring slot of the last entry passed that was not void
+          while (need > 0) {
+            uint32_t avail = sm.ring_tail[istar] - head;
+            for (uint32_t polls = 0; avail == 0 && polls < a.ring_polls; ++polls) {
+              __nanosleep(20);
+              avail = sm.ring_tail[istar] - head;
+              PROF_ADD(14, 1);
+            }
+            if (avail == 0) break;                          // the scout is behind: walk ourselves
+            smem_order();
+            const uint32_t m = min(avail, 32u);
+            uint4 ent = make_uint4(0, kNone, 0, 0);
+            bool live = false, unsure = false;
+            if (lane < m) {
+              const uint32_t e = (head + lane) & (kListCap - 1);
+              ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
+              // entries the eviction cursor has already passed (after a walk of our own) are void
+              live = !(ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp));
+              if (live && ent.y <= r) {
+                if (ent.y == r) live = false;               // the block is in this very request
+                else {                                      // it came back in between: look again
+                  live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
+                  unsure = true;                            // where it occurs next is not known here
+                }
+              }
+            }
+            const unsigned lv = __ballot_sync(kFull, live);
+            const uint32_t cnt = __popc(lv);
+            const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+            if (mine) {
+              mask_clear_bit<MaskT>(mask, ent.x, bit);
+              if (unsure) { for (uint32_t q = r + 1; q <= r + kWindow; ++q) mark_hit(q); }
+              else if (ent.y - (r + 1) < kWindow) mark_hit(ent.y);
+            }
+            // entries passed: the whole round, or up to the last victim taken
+            uint32_t passed = m, tk = cnt;
+            if (cnt > need) {
+              const unsigned take = __ballot_sync(kFull, mine);
+              passed = 32u - (uint32_t)__clz((int)take);
+              tk = need;
+            }
+            need -= tk;
+            evicted += tk;
+            // the cursor moves behind the last live entry passed (void ones lie behind it already)
+            const unsigned seen = lv & (passed >= 32u ? kFull : ((1u << passed) - 1u));
+            if (seen) last_e = (head + 31u - (uint32_t)__clz((int)seen)) & (kListCap - 1);
+            head += passed;
+          }
+          if (last_e != kNone) {
+            const uint4 le = a.lists_in_smem ? lst[last_e] : __ldcg(lst + last_e);
+            cr = le.w;
+            cp = (int32_t)le.z - 1;
+          }
+          if (lane == 0) sm.ring_head[istar] = head;
+        }
+        PROF_ADD(13, need > 0 ? 1 : 0);
+        // whatever is still needed: walk the recency order from the cursor and validate touches here
+        uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
+        unsigned long long guard = 0;
+        while (need > 0) {
+          if (++guard > evict_guard_max) { status = -6; break; }
+          if (cp < 0) {  // this request is used up: go to the next one routed here
+            const uint32_t nx = (cr == kNone) ? kNone : lru_next[cr];
+            if (nx == kNone) { status = -6; break; }
+            cr = nx;
+            const ReqRec cre = req[cr];
+            coff = cre.off;
+            cp = (int32_t)cre.nblk - 1;
+            continue;
+          }
+          // examine 32 touches, deepest position first
+          const int32_t k = cp - (int32_t)lane;
+          bool live = false;
+          uint32_t vid = 0, nxr = kNone;
+          if (k >= 0) {
+            const uint32_t g = coff + (uint32_t)k;
+            vid = ids[g];
+            uint2 c = a.tr.occ_next[g];
+            live = true;
+            while (c.x != kNone && c.y <= r) {       // later occurrences of the block, up to r
+              const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
+              if (rr == istar) { live = false; break; }
+              c = a.tr.occ_next[c.x];
+            }
+            if (live && c.x != kNone) nxr = c.y;     // its next occurrence after r
+          }
+          const unsigned lv = __ballot_sync(kFull, live);
+          const uint32_t cnt = __popc(lv);
+          // the first `need` live touches in lane order are the victims
+          const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
+          const unsigned take = __ballot_sync(kFull, mine);
+          if (mine) {
+            mask_clear_bit<MaskT>(mask, vid, bit);
+            if (nxr - (r + 1) < kWindow) mark_hit(nxr);
+          }
+          cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
+          const uint32_t tk = __popc(take);
+          need -= tk;
+          evicted += tk;
+        }
+        if (lane == 0) { sm.curreq[istar] = cr; sm.curpos[istar] = cp; }
+      }
+    }
+    occ -= evicted;
+    st_evict += evicted;
     PROF_LAP(1);
 
-    bar_wait(kBarRoute);                                  // the replica has been chosen
-    PROF_LAP(2);
-    const uint32_t istar = *cx.route;
-    const MaskT bit = (MaskT)(((MaskT)1) << istar);
-
-    // ---- cache commit: set the replica's bit on the missing blocks (the probe counted the
-    //      blocks already present there)
-    const uint32_t missing = n - (cx.st_hits[slot * R + istar] >> 16);
+    // ---- set the replica's bit on the blocks the request inserts
     for (uint32_t c = 0; c < n; c += 32) {
       const uint32_t k = c + lane;
       if (k < n) {
         uint32_t id;
         MaskT mv;
         if (c < kStageBlocks) { id = sid[k]; mv = smk[k]; }
-        else { id = ids[off + k]; mv = mask_load<MaskT>(mask, id); }
-        if (!(mv & bit)) mask_store<MaskT>(mask, id, (MaskT)(mv | bit));
+        else { id = ids[req[r].off + k]; mv = mask_load<MaskT>(mask, id); }
+        if (!(mv & bit)) mask_set_bit<MaskT>(mask, id, bit);
       }
     }
-    PROF_LAP(3);
-    uint32_t occ = sm.occ[istar] + missing;
-    uint32_t need = occ > a.m.C ? (uint32_t)(occ - a.m.C) : 0u;
-    PROF_ADD(12, need > 0 ? 1 : 0);
-    PROF_ADD(15, need);
-    uint32_t evicted = 0;
-    unsigned hit1 = 0, hit2 = 0, hit3 = 0;   // a victim's block occurs again in request r+1/2/3
-    if (need > 0) {
-      uint32_t cr = sm.curreq[istar];
-      int32_t cp = sm.curpos[istar];
-      // fast path: victims from the ring the scout warp keeps for this replica
-      if (sm.act[istar]) {
-        const uint4* lst = sm.lst + (size_t)istar * kListCap;
-        uint32_t head = sm.ring_head[istar];
-        uint32_t last_e = kNone;   // ring slot of the last entry passed that was not void
-        while (need > 0) {
-          uint32_t avail = sm.ring_tail[istar] - head;
-          for (uint32_t polls = 0; avail == 0 && polls < 64; ++polls) {
-            __nanosleep(20);
-            avail = sm.ring_tail[istar] - head;
-          }
-          if (avail == 0) break;                          // the scout is behind: walk ourselves
-          smem_order();
-          const uint32_t m = min(avail, 32u);
-          uint4 ent = make_uint4(0, kNone, 0, 0);
-          bool odd = false;      // void (behind the cursor) or touched again since it was listed
-          if (lane < m) {
-            const uint32_t e = (head + lane) & (kListCap - 1);
-            ent = a.lists_in_smem ? lst[e] : __ldcg(lst + e);
-            odd = ent.y <= r || ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp);
-          }
-          if (!__any_sync(kFull, odd)) {
-            // common case: the next entries are all live, the first `need` of them are victims
-            const uint32_t tk = min(need, m);
-            const bool mine = lane < tk;
-            if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
-            const unsigned soon = __ballot_sync(kFull, mine && ent.y - (r + 1) < kWindow);
-            if (soon) {
-              hit1 |= __ballot_sync(kFull, mine && ent.y == r + 1);
-              hit2 |= __ballot_sync(kFull, mine && ent.y == r + 2);
-              hit3 |= __ballot_sync(kFull, mine && ent.y == r + 3);
-            }
-            need -= tk;
-            evicted += tk;
-            last_e = (head + tk - 1) & (kListCap - 1);
-            head += tk;
-            continue;
-          }
-          bool live = false, unsure = false;
-          if (lane < m) {
-            // entries the eviction cursor has already passed (after a walk of our own) are void
-            live = !(ent.w < cr || (ent.w == cr && (int32_t)ent.z > cp));
-            if (live && ent.y <= r) {
-              if (ent.y == r) live = false;               // the block is in this very request
-              else {                                      // it came back in between: look again
-                live = !touch_is_stale(a.tr, route_log, req[ent.w].off + ent.z, istar, r, istar);
-                unsure = true;                            // where it occurs next is not known here
-              }
-            }
-          }
-          const unsigned lv = __ballot_sync(kFull, live);
-          const uint32_t cnt = __popc(lv);
-          const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
-          if (mine) mask_clear_bit<MaskT>(mask, ent.x, bit);
-          hit1 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 1));
-          hit2 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 2));
-          hit3 |= __ballot_sync(kFull, mine && (unsure || ent.y == r + 3));
-          // entries passed: the whole round, or up to the last victim taken
-          uint32_t passed = m, tk = cnt;
-          if (cnt > need) {
-            const unsigned take = __ballot_sync(kFull, mine);
-            passed = 32u - (uint32_t)__clz((int)take);
-            tk = need;
-          }
-          need -= tk;
-          evicted += tk;
-          // the cursor moves behind the last live entry passed (void ones lie behind it already)
-          const unsigned seen = lv & (passed >= 32u ? kFull : ((1u << passed) - 1u));
-          if (seen) last_e = (head + 31u - (uint32_t)__clz((int)seen)) & (kListCap - 1);
-          head += passed;
-        }
-        if (last_e != kNone) {
-          const uint4 le = a.lists_in_smem ? lst[last_e] : __ldcg(lst + last_e);
-          cr = le.w;
-          cp = (int32_t)le.z - 1;
-        }
-        if (lane == 0) sm.ring_head[istar] = head;
-      }
-      PROF_ADD(13, need > 0 ? 1 : 0);
-      uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
-      unsigned long long guard = 0;
-      while (need > 0) {
-        if (++guard > evict_guard_max) { status = -6; break; }
-        if (cp < 0) {  // this request is used up: go to the next one routed here
-          const uint32_t nx = (cr == kNone) ? kNone : lru_next[cr];
-          if (nx == kNone) { status = -6; break; }
-          cr = nx;
-          const ReqRec cre = req[cr];
-          coff = cre.off;
-          cp = (int32_t)cre.nblk - 1;
-          continue;
-        }
-        // examine 32 touches, deepest position first
-        const int32_t k = cp - (int32_t)lane;
-        bool live = false;
-        uint32_t vid = 0, nxr = kNone;
-        if (k >= 0) {
-          const uint32_t g = coff + (uint32_t)k;
-          vid = ids[g];
-          uint2 c = a.tr.occ_next[g];
-          live = true;
-          while (c.x != kNone && c.y <= r) {       // later occurrences of the block, up to r
-            const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
-            if (rr == istar) { live = false; break; }
-            c = a.tr.occ_next[c.x];
-          }
-          if (live && c.x != kNone) nxr = c.y;     // its next occurrence after r
-        }
-        const unsigned lv = __ballot_sync(kFull, live);
-        const uint32_t cnt = __popc(lv);
-        // the first `need` live touches in lane order are the victims
-        const bool mine = live && (uint32_t)__popc(lv & ((1u << lane) - 1u)) < need;
-        const unsigned take = __ballot_sync(kFull, mine);
-        if (mine) mask_clear_bit<MaskT>(mask, vid, bit);
-        hit1 |= __ballot_sync(kFull, mine && nxr == r + 1);
-        hit2 |= __ballot_sync(kFull, mine && nxr == r + 2);
-        hit3 |= __ballot_sync(kFull, mine && nxr == r + 3);
-        cp -= (cnt <= need) ? 32 : 32 - __clz((int)take);
-        const uint32_t tk = __popc(take);
-        need -= tk;
-        evicted += tk;
-      }
-      if (lane == 0) { sm.curreq[istar] = cr; sm.curpos[istar] = cp; }
-    }
-    occ -= evicted;
-    st_evict += evicted;
-    PROF_LAP(4);
-
-    // ---- which staged reads did the commit of request r invalidate?  If the next request's
-    //      are intact and staged, hand them over now: the decide warp works on r+1 while the
-    //      bookkeeping of r below finishes.
-    bad0 = bad1 || ps1 == r || hit1 != 0;
-    bad1 = bad2 || ps2 == r || hit2 != 0;
-    bad2 = bad3 || ps3 == r || hit3 != 0;
-    bad3 = false;
-    ps1 = ps2; ps2 = ps3; ps3 = ps4;
-    posted = false;
-    if (r + 1 < end && !bad0 &&
-        __shfl_sync(kFull, cx.st_ready[(r + 1) % kStageDepth], 0) == r + 2) {
-      smem_order();
-      hand_over((r + 1) % kStageDepth, q_nxt.nblk);
-      posted = true;
-      PROF_ADD(14, 1);
-    }
-    PROF_LAP(5);
+    __syncwarp();
+    PROF_LAP(2);
 
     if (lane == 0) {
       sm.occ[istar] = occ;
@@ -1149,34 +1322,41 @@ __device__ __forceinline__ void cache_warp(const ReplayArgs& a, const Ctx<MaskT>
         __threadfence_block();
         sm.act[istar] = 1;
       }
-      PROF_LAP(6);
       __threadfence_block();
-      *sm.progress = r + 1;                               // request r is fully committed
+      sm.progress[which] = r + 1;                         // request r is committed
     }
     __syncwarp();
-    PROF_LAP(7);
-
-    q_cur = q_nxt; q_nxt = q_n2;
+    PROF_LAP(3);
   }
-  PROF_END(32);
-  st_probe = warp_sum_u64(st_probe);
+  PROF_END(48);
   status = __reduce_min_sync(kFull, status);
   if (lane == 0) {
     if (status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
-    if (a.stats) {
-      unsigned long long* s4 = reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4;
-      atomicAdd(s4 + 0, st_probe);
-      atomicAdd(s4 + 3, st_evict);
-    }
+    if (a.stats) atomicAdd(reinterpret_cast<unsigned long long*>(a.stats) + (size_t)p * 4 + 3, st_evict);
   }
 }
 
-constexpr uint32_t kWarpRoute = 0, kWarpCache = 1, kWarpProbe = 2, kWarpScout0 = 3;
-constexpr uint32_t kWarpService = 3 + kScouts, kWarpExpiry = 4 + kScouts;
-constexpr uint32_t kReplayThreads = 32 * (5 + kScouts);
+// Roles of the twelve warps of a candidate.  Warp w issues from scheduler w % 4 of the SM, and a
+// scheduler's instruction cache is small, so warps that run the same code sit on one scheduler:
+//   scheduler 0: route, expiry, scout     scheduler 1: gate, service, service
+//   scheduler 2: probe, probe, scout      scheduler 3: commit, commit, commit
+enum Role : uint32_t { kRoleRoute, kRoleGate, kRoleProbe, kRoleScout, kRoleService, kRoleExpiry, kRoleCommit, kRoleNone };
+constexpr uint32_t kReplayWarps = 12;
+constexpr uint32_t kReplayThreads = 32 * kReplayWarps;
+__device__ __forceinline__ void role_of(uint32_t warp, Role& role, uint32_t& which) {
+  const uint32_t sched = warp & 3u, k = warp >> 2;
+  which = k;
+  if (sched == 0) role = k == 0 ? kRoleRoute : k == 1 ? kRoleExpiry : kRoleScout;
+  else if (sched == 1) { role = k == 0 ? kRoleGate : kRoleService; which = k - 1; }
+  else if (sched == 2) role = k < kProbes ? kRoleProbe : kRoleScout;
+  else role = kRoleCommit;
+  if (role == kRoleScout) which = sched >> 1;      // scout 0 and scout 1
+}
+static_assert(kScouts == 2 && kProbes == 2 && kCommitWarps == 3, "role map");
+constexpr int kReplayMinCtas = 2;   // registers capped so that two candidates share an SM
 
 template <typename MaskT, bool kBaseline>
-__global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayArgs a) {
+__global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(const ReplayArgs a) {
   const uint32_t p = blockIdx.x;
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t warp = threadIdx.x >> 5;
@@ -1207,16 +1387,19 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   sm.curpos = reinterpret_cast<int32_t*>(sm.curreq + R);
   sm.lrutail = reinterpret_cast<uint32_t*>(sm.curpos + R);
   uint32_t* unext = sm.lrutail + R;
-  sm.progress = unext;
-  cx.route = unext + 1;
-  cx.status = reinterpret_cast<volatile int32_t*>(unext + 2);
-  cx.hit_slot = unext + 3;
-  sm.routed = unext + 4;
-  sm.serviced = unext + 5;
-  sm.exp_ready = unext + 6;
-  cx.abort_flag = unext + 7;
-  sm.route_ring = unext + 8;                               // [kRouteRing]
-  sm.act = sm.route_ring + kRouteRing;
+  sm.progress = unext;                                     // [kCommitWarps] (<= 3)
+  cx.route = unext + 3;
+  cx.status = reinterpret_cast<volatile int32_t*>(unext + 4);
+  cx.hit_slot = unext + 5;
+  sm.routed = unext + 6;
+  sm.exp_ready = unext + 7;
+  sm.abort_flag = unext + 8;
+  sm.jobs = unext + 9;
+  sm.serviced = unext + 10;                                // [kServices] (<= 2)
+  sm.route_ring = unext + 12;                              // [kRouteRing]
+  sm.job = sm.route_ring + kRouteRing;                     // [kJobRing]
+  cx.evhit = sm.job + kJobRing;                            // [kHitRing]
+  sm.act = const_cast<uint32_t*>(cx.evhit) + kHitRing;
   sm.ring_head = sm.act + R;
   sm.ring_tail = sm.ring_head + R;
   sm.scan_cr = sm.ring_tail + R;
@@ -1230,7 +1413,8 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
     after = cx.st_ids + (kStageDepth + 2) * (size_t)kStageBlocks;
     const uintptr_t a8 = (reinterpret_cast<uintptr_t>(after) + 7) & ~(uintptr_t)7;
     cx.st_ab = reinterpret_cast<double*>(a8);
-    cx.st_mk = reinterpret_cast<MaskT*>(cx.st_ab + (kStageDepth + 2) * (size_t)R);
+    cx.st_where = reinterpret_cast<unsigned long long*>(cx.st_ab + (kStageDepth + 2) * (size_t)R);
+    cx.st_mk = reinterpret_cast<MaskT*>(cx.st_where + (kStageDepth + 2));
     after = reinterpret_cast<uint32_t*>(cx.st_mk + (kStageDepth + 2) * (size_t)kStageBlocks);
     const uintptr_t al = (reinterpret_cast<uintptr_t>(after) + 15) & ~(uintptr_t)15;
     sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(al)
@@ -1265,19 +1449,27 @@ __global__ void __launch_bounds__(kReplayThreads, 1) replay_kernel(const ReplayA
   if (a.slots_in_smem)
     for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) cx.free_at[x] = g_slot[x];
   if (threadIdx.x == 0) {
-    *sm.progress = a.first; *cx.status = 0; *cx.probe_gone = 0; *cx.abort_flag = 0;
-    *sm.routed = a.first; *sm.serviced = a.first; *sm.exp_ready = a.first;
+    *cx.status = 0; *cx.probe_gone = 0; *sm.abort_flag = 0;
+    *sm.routed = a.first; *sm.exp_ready = a.first; *sm.jobs = a.first;
+    sm.serviced[0] = a.first; sm.serviced[1] = a.first;
   }
+  if (threadIdx.x < kCommitWarps) sm.progress[threadIdx.x] = a.first;
   if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
+  if (threadIdx.x < kJobRing) sm.job[threadIdx.x] = 0;
+  if (threadIdx.x < kHitRing) cx.evhit[threadIdx.x] = kNone;
   __syncthreads();
 
-  if (warp == kWarpRoute) route_warp<MaskT, kBaseline>(a, cx, p, lane);
-  else if (warp == kWarpCache) cache_warp<MaskT>(a, cx, p, lane);
-  else if (warp == kWarpProbe) probe_warp<MaskT>(a, cx, lane);
-  else if (warp == kWarpService) service_warp<MaskT, kBaseline>(a, cx, p, lane);
-  else if (warp == kWarpExpiry)
-    expiry_warp<kBaseline>(a, sm, cx.exp_head, cx.exp_rec, cx.abort_flag, cx.status, p, lane);
-  else scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, warp - kWarpScout0);
+  Role role;
+  uint32_t which;
+  role_of(warp, role, which);
+  if (role == kRoleRoute) route_warp<MaskT, kBaseline>(a, cx, p, lane);
+  else if (role == kRoleGate) gate_warp<MaskT>(a, cx, p, lane);
+  else if (role == kRoleCommit) commit_warp<MaskT>(a, cx, p, lane, which);
+  else if (role == kRoleProbe) probe_warp<MaskT>(a, cx, lane, which);
+  else if (role == kRoleService) service_warp<MaskT, kBaseline>(a, cx, p, lane, which);
+  else if (role == kRoleExpiry)
+    expiry_warp<kBaseline>(a, sm, cx.exp_head, cx.exp_rec, sm.abort_flag, cx.status, p, lane);
+  else if (role == kRoleScout) scout_warp<MaskT>(a, sm, cx.lru_next, cx.route_log, lane, which);
   __syncthreads();
 
   // ---- write the small state back
@@ -1511,7 +1703,8 @@ size_t replay_smem_bytes(ReplayArgs& a) {
   a.slots_in_smem = rs * 8 <= 40 * 1024 ? 1u : 0u;
   a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + (2 + kExpRing) * (size_t)a.m.R) * sizeof(double) +
-                (9 * (size_t)a.m.R + 8 + kRouteRing) * sizeof(uint32_t) + 16 +
+                (9 * (size_t)a.m.R + 12 + kRouteRing + kJobRing + kHitRing) * sizeof(uint32_t) + 16 +
+                (kStageDepth + 2) * sizeof(unsigned long long) +
                 (kStageDepth + 1 + (kStageDepth + 2) * ((size_t)a.m.R + kStageBlocks)) * sizeof(uint32_t) +
                 8 + (kStageDepth + 2) * (size_t)a.m.R * sizeof(double) +
                 (kStageDepth + 2) * kStageBlocks * sizeof(MaskT) + 8;

@@ -23,11 +23,19 @@ ROLES = {
     "service": (16, ["retire: list entry, window vote, grid value", "fence and publish",
                      "issue list exchange and window loads", "slot argmin",
                      "times, outputs, grid load", "idle round"]),
-    "cache": (32, ["take staged hits / probe", "hand hits over (not posted early)",
-                   "wait for the route", "mask stores", "eviction", "invalidation check, early hand-over",
-                   "recency list", "fence and progress", None, None, None, "#probes redone here",
-                   "#requests that evict", "#evictions finished by own walk",
-                   "#hits handed over early", "#blocks evicted"]),
+    "gate": (32, ["hand-over at the request's own turn (rest)", "wait for the route",
+                  "job, early hand-over of the next request", "own turn: wait for the staged read",
+                  "own turn: wait for commits", None, None, None, None, None,
+                  "#not early: shares a block with a recent request", "#probes redone here",
+                  "#not early: not staged yet", "#not early: recent route to a holder of its blocks",
+                  "#hits handed over early"]),
+    "commit (all warps)": (48, ["wait for the next routed request", "need and eviction",
+                                "mask bits of the inserted blocks", "recency list, progress",
+                                "requests of other warps' replicas", None,
+                                None, None, "#evictions: clean case", "#evictions: an entry was void or touched again",
+                                "#evictions: ring held too few entries", "#evictions: more than 96 victims or ring not in use",
+                                "#requests that evict", "#evictions finished by own walk", "#polls for ring entries",
+                                "#blocks evicted"]),
 }
 
 
