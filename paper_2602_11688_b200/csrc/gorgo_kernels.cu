@@ -182,6 +182,11 @@ constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas sp
 constexpr int kScoutBatches = 1;       // touches examined per lane and scout round
 constexpr uint32_t kPostMargin = 512;  // start pre-validating when a cache is this close to full
 
+constexpr uint32_t kStageDepth = 14;                   // requests staged by the probe warps (> kWindow)
+constexpr uint32_t kStageBlocks = kRegChunks * 32u;    // blocks of a request kept per stage
+constexpr uint32_t kWindow = 12;  // a staged read may be up to this many commits old (<= 32)
+constexpr uint32_t kProbes = 2;   // probe warps per candidate (requests alternate between them)
+
 // rings and counts of the warps of one candidate
 constexpr uint32_t kRouteRing = 32;   // routes handed from the route warp to the service warp
 constexpr uint32_t kRouteLead = 24;   // the route warp runs at most this far ahead of the service warp
@@ -395,6 +400,7 @@ struct Ctx {
   // (stages kStageDepth and kStageDepth+1 belong to the cache warp, used alternately)
   uint32_t* st_hits;           // [kStageDepth+2][R] prefix hit | blocks present << 16
   double* st_ab;               // [kStageDepth+2][R] (w_net*RTT + w_prefill*uncached) per replica
+  uint4* st_meta;              // [kStageDepth+2] (input tokens, blocks | origin << 16, latest earlier request sharing a block, offset of its ids)
   unsigned long long* st_where;  // [kStageDepth+2] replicas that held any block of the request when it was read
   volatile uint32_t* evhit;    // [kHitRing] evhit[q % kHitRing] == q: a recent eviction took a block of request q
   uint32_t* st_ids;            // [kStageDepth+2][kStageBlocks] block ids
@@ -431,20 +437,18 @@ template <typename MaskT, bool kBaseline>
 __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p, uint32_t lane) {
   const Smem& sm = cx.sm;
   const uint32_t R = a.m.R, K = a.m.K;
-  const ReqRec* req = a.tr.req;
   const double w_que = sm.w[2];
   const bool by_requests = kBaseline && a.queue_in_requests != 0;   // baseline "least-request"
   int32_t status = 0;
   unsigned long long st_hit = 0, st_blk = 0;
+  constexpr bool kWide = sizeof(MaskT) == 8;   // more than 32 replicas: two per lane
   const uint32_t i0 = lane, i1 = lane + 32u;
   long long ld0 = 0, ld1 = 0;          // in-flight signal of replicas lane and lane+32
   double nrm0 = 1.0, nrm1 = 1.0;       // their queue-load normalisers
   if (i0 < R) { ld0 = by_requests ? sm.cnt[i0] : sm.load[i0]; if (K != 3) nrm0 = sm.w[3 + i0]; }
-  if (i1 < R) { ld1 = by_requests ? sm.cnt[i1] : sm.load[i1]; if (K != 3) nrm1 = sm.w[3 + i1]; }
+  if (kWide && i1 < R) { ld1 = by_requests ? sm.cnt[i1] : sm.load[i1]; if (K != 3) nrm1 = sm.w[3 + i1]; }
 
   const uint32_t last_r = a.first + a.count - 1;
-  ReqRec rec_cur = req[a.first];
-  ReqRec rec_nxt = req[min(a.first + 1, last_r)];
   // routes fixed in advance (baselines that do not look at the state), fetched two ahead
   const uint8_t* forced = kBaseline ? a.forced_route : nullptr;
   uint32_t fr_cur = forced ? forced[a.first] : 0u;
@@ -454,10 +458,6 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
   PROF_BEGIN();
   for (uint32_t j = 0; j < a.count; ++j) {
     const uint32_t r = a.first + j;
-    const ReqRec rec = rec_cur;
-    rec_cur = rec_nxt;
-    rec_nxt = req[min(r + 2, last_r)];                   // in flight while this request runs
-    const uint32_t n = rec.nblk, in_tok = rec.in_tok;
 
     // ---- completions the proxy has seen by this arrival (published by the expiry warp), and
     //      room in the ring of routes the service warp has not taken yet
@@ -469,12 +469,12 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
     PROF_LAP(0);
     const long long* gone = sm.exp_sum + (size_t)(r % kExpRing) * R;
     if (i0 < R) ld0 -= gone[i0];
-    if (i1 < R) ld1 -= gone[i1];
+    if (kWide && i1 < R) ld1 -= gone[i1];
 
     // ---- the queue part of the score does not need the prefix hits
     double cq0 = 0.0, cq1 = 0.0;
     if (i0 < R) { double q = (double)ld0; if (K != 3) q = __dmul_rn(q, nrm0); cq0 = __dmul_rn(w_que, q); }
-    if (i1 < R) { double q = (double)ld1; if (K != 3) q = __dmul_rn(q, nrm1); cq1 = __dmul_rn(w_que, q); }
+    if (kWide && i1 < R) { double q = (double)ld1; if (K != 3) q = __dmul_rn(q, nrm1); cq1 = __dmul_rn(w_que, q); }
     PROF_LAP(1);
 
     bar_wait(kBarHits);                                   // prefix hits of request r are posted
@@ -483,10 +483,12 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
     // ---- score of Eq. 3 (fixed order, no FMA): the staged (w_net*RTT + w_prefill*uncached)
     //      plus the queue term; lowest-index argmin
     const uint32_t stage = *cx.hit_slot;
+    const uint4 meta = cx.st_meta[stage];                 // (this warp reads no global memory in its loop)
+    const uint32_t in_tok = meta.x, n = meta.y & 0xFFFFu;
     uint64_t best_k = ~0ull;
     uint32_t best_i = kNone;
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
+    for (int half = 0; half < (kWide ? 2 : 1); ++half) {
       const uint32_t i = lane + 32u * half;
       if (i < R) {
         double c = __dadd_rn(cx.st_ab[stage * R + i], half ? cq1 : cq0);
@@ -515,13 +517,13 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
     PROF_LAP(5);
     const long long add = by_requests ? 1ll : (long long)in_tok;
     if (istar == i0) ld0 += add;
-    if (istar == i1) ld1 += add;
+    if (kWide && istar == i1) ld1 += add;
     st_hit += hstar; st_blk += n;
   }
   PROF_END(0);
   // the signal as of the last request routed
   if (i0 < R) { if (by_requests) sm.cnt[i0] = ld0; else sm.load[i0] = ld0; }
-  if (i1 < R) { if (by_requests) sm.cnt[i1] = ld1; else sm.load[i1] = ld1; }
+  if (kWide && i1 < R) { if (by_requests) sm.cnt[i1] = ld1; else sm.load[i1] = ld1; }
   status = __reduce_min_sync(kFull, status);
   if (lane == 0) {
     if (status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
@@ -798,11 +800,6 @@ __device__ __forceinline__ void expiry_warp(const ReplayArgs& a, const Smem& sm,
   if (lane == 0 && status != 0) atomicMin(const_cast<int32_t*>(cta_status), status);
 }
 
-constexpr uint32_t kStageDepth = 14;                   // requests staged by the probe warps (> kWindow)
-constexpr uint32_t kStageBlocks = kRegChunks * 32u;    // blocks of a request kept per stage
-constexpr uint32_t kWindow = 12;  // a staged read may be up to this many commits old (<= 32)
-constexpr uint32_t kProbes = 2;   // probe warps per candidate (requests alternate between them)
-
 // What a warp needs to know of a request ahead of time.
 struct Ahead { uint32_t off, nblk, prev_share, in_tok, origin; };
 __device__ __forceinline__ Ahead fetch_ahead(const ReqRec* req, uint32_t q, uint32_t end) {
@@ -853,7 +850,7 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
       const bool running = (alive >> i) & 1;
       const uint32_t run = !running ? 0u : (b == kFull) ? 32u : (uint32_t)__ffs((int)~b) - 1u;
       if ((uint32_t)(i & 31) == lane) {
-        if (i < 32) { h0 += run; p0 += cnt; } else { h1 += run; p1 += cnt; }
+        if (sizeof(MaskT) != 8 || i < 32) { h0 += run; p0 += cnt; } else { h1 += run; p1 += cnt; }
       }
       if (run == 32u) still |= (MaskT)(((MaskT)1) << i);
     }
@@ -870,11 +867,14 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
                                              uint32_t h1, uint32_t p0, uint32_t p1,
                                              unsigned long long where, uint32_t lane) {
   const uint32_t R = a.m.R;
-  if (lane == 0) cx.st_where[slot] = where;
+  if (lane == 0) {
+    cx.st_where[slot] = where;
+    cx.st_meta[slot] = make_uint4(q.in_tok, q.nblk | (q.origin << 16), q.prev_share, q.off);
+  }
   const double w_pre = cx.sm.w[1];
   const double* wrtt_row = cx.sm.wrtt + (size_t)q.origin * R;
 #pragma unroll
-  for (int half = 0; half < 2; ++half) {
+  for (int half = 0; half < (sizeof(MaskT) == 8 ? 2 : 1); ++half) {
     const uint32_t i = lane + 32u * half;
     if (i < R) {
       const uint32_t h = half ? h1 : h0, pr = half ? p1 : p0;
@@ -975,7 +975,6 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
   unsigned long long st_probe = 0;
   const uint32_t end = a.first + a.count;
 
-  Ahead q_cur = fetch_ahead(req, a.first, end), q_nxt = fetch_ahead(req, a.first + 1, end);
   uint32_t my_req = kNone, my_rep = 0;   // lane l: the latest routed request with index % 32 == l, and its replica
   bool posted = false;             // the hits of the coming request were already handed over
   uint32_t slot = 0;               // stage that holds the current request's ids, mask words and hits
@@ -985,7 +984,7 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
     bar_arrive(kBarHits);                                 // the route warp may score the request
     if (a.stats) {                                        // probes the plain formula charges
       if (lane < R) { const uint32_t h = cx.st_hits[sl * R + lane] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
-      if (lane + 32u < R) { const uint32_t h = cx.st_hits[sl * R + lane + 32u] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
+      if (sizeof(MaskT) == 8 && lane + 32u < R) { const uint32_t h = cx.st_hits[sl * R + lane + 32u] & 0xFFFFu; st_probe += (h + 1 < nblk ? h + 1 : nblk); }
     }
   };
   // latest request among the kWindow before q that was routed to a replica in `where` (kNone: none)
@@ -994,28 +993,37 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
     if (!__any_sync(kFull, hit)) return kNone;
     return __reduce_max_sync(kFull, hit ? my_req : 0u);
   };
-  // does a commit since its staged read share a block with the request?
-  auto shares = [&](const Ahead& q, uint32_t idx) {
-    return q.prev_share != kNone && q.prev_share + kWindow >= idx;
-  };
+  // does a commit since its staged read share a block with request idx?  (prev: the latest earlier
+  // request that shares a block with it)
+  auto shares = [&](uint32_t prev, uint32_t idx) { return prev != kNone && prev + kWindow >= idx; };
+  uint32_t n = 0;                  // blocks of the current request
 
   PROF_BEGIN();
   for (uint32_t r = a.first; r < end; ++r) {
-    const Ahead q_n2 = fetch_ahead(req, r + 2, end);          // used two rounds from now
-    const uint32_t n = q_cur.nblk;
-
     // ---- prefix hits of request r, unless they went out right after the previous route
     if (!posted) {
-      const bool sh = shares(q_cur, r);
-      bool staged = false;
-      uint32_t done_to = sh ? r : 0u;                         // requests < done_to must be committed
-      if (!sh && !*cx.probe_gone) {
-        const uint32_t ss = r % kStageDepth;
-        uint32_t polls = 0;
-        while (cx.st_ready[ss] != r + 1 && !*cx.probe_gone && polls < 4096) { ++polls; __nanosleep(20); }
-        // (one lane decides: every lane must take the same path)
-        staged = __shfl_sync(kFull, cx.st_ready[ss], 0) == r + 1;
+      const uint32_t ss = r % kStageDepth;
+      bool staged = __shfl_sync(kFull, cx.st_ready[ss], 0) == r + 1;
+      Ahead q_cur;
+      if (staged) {
         smem_order();
+        const uint4 meta = cx.st_meta[ss];
+        q_cur.in_tok = meta.x; q_cur.nblk = meta.y & 0xFFFFu; q_cur.origin = meta.y >> 16;
+        q_cur.prev_share = meta.z; q_cur.off = meta.w;
+      } else {
+        q_cur = fetch_ahead(req, r, end);
+      }
+      n = q_cur.nblk;
+      const bool sh = shares(q_cur.prev_share, r);
+      uint32_t done_to = sh ? r : 0u;                         // requests < done_to must be committed
+      if (!sh) {
+        if (!staged && !*cx.probe_gone) {
+          uint32_t polls = 0;
+          while (cx.st_ready[ss] != r + 1 && !*cx.probe_gone && polls < 4096) { ++polls; __nanosleep(20); }
+          // (one lane decides: every lane must take the same path)
+          staged = __shfl_sync(kFull, cx.st_ready[ss], 0) == r + 1;
+          smem_order();
+        }
         if (staged) {
           const uint32_t c = conflict(r, cx.st_where[ss]);
           if (c != kNone) done_to = c + 1;
@@ -1026,8 +1034,8 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
       if (done_to > a.first) wait_committed(sm, done_to, a.poll_limit, status);
       smem_order();
       PROF_LAP(4);
-      if (staged && (done_to <= a.first || cx.evhit[r % kHitRing] != r)) {
-        slot = r % kStageDepth;
+      if (!sh && staged && (done_to <= a.first || cx.evhit[r % kHitRing] != r)) {
+        slot = ss;
       } else {
         // read and probe here, after every earlier request is committed
         PROF_ADD(11, 1);
@@ -1062,20 +1070,28 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
 
     // ---- the next request's hits go out now if no commit since their read can have touched them
     posted = false;
-    if (r + 1 < end && !shares(q_nxt, r + 1)) {
+    if (r + 1 < end) {
       const uint32_t ss = (r + 1) % kStageDepth;
       if (__shfl_sync(kFull, cx.st_ready[ss], 0) == r + 2) {
         smem_order();
-        if (conflict(r + 1, cx.st_where[ss]) == kNone) {
+        const uint4 meta = cx.st_meta[ss];
+        bool okk = !shares(meta.z, r + 1);
+        if (okk) {
+          // a commit routed to a holder of its blocks is no obstacle once it is done and did not
+          // evict any of them
+          const uint32_t c = conflict(r + 1, cx.st_where[ss]);
+          if (c != kNone) okk = (int32_t)(committed(sm) - (c + 1)) >= 0 && cx.evhit[(r + 1) % kHitRing] != r + 1;
+        }
+        if (okk) {
           slot = ss;
-          hand_over(slot, q_nxt.nblk);
+          n = meta.y & 0xFFFFu;
+          hand_over(slot, n);
           posted = true;
           PROF_ADD(14, 1);
         } else PROF_ADD(13, 1);
       } else PROF_ADD(12, 1);
-    } else PROF_ADD(10, 1);
+    }
     PROF_LAP(2);
-    q_cur = q_nxt; q_nxt = q_n2;
   }
   PROF_END(32);
   st_probe = warp_sum_u64(st_probe);
@@ -1414,7 +1430,11 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
     const uintptr_t a8 = (reinterpret_cast<uintptr_t>(after) + 7) & ~(uintptr_t)7;
     cx.st_ab = reinterpret_cast<double*>(a8);
     cx.st_where = reinterpret_cast<unsigned long long*>(cx.st_ab + (kStageDepth + 2) * (size_t)R);
-    cx.st_mk = reinterpret_cast<MaskT*>(cx.st_where + (kStageDepth + 2));
+    {
+      const uintptr_t m16 = (reinterpret_cast<uintptr_t>(cx.st_where + (kStageDepth + 2)) + 15) & ~(uintptr_t)15;
+      cx.st_meta = reinterpret_cast<uint4*>(m16);
+    }
+    cx.st_mk = reinterpret_cast<MaskT*>(cx.st_meta + (kStageDepth + 2));
     after = reinterpret_cast<uint32_t*>(cx.st_mk + (kStageDepth + 2) * (size_t)kStageBlocks);
     const uintptr_t al = (reinterpret_cast<uintptr_t>(after) + 15) & ~(uintptr_t)15;
     sm.lst = a.lists_in_smem ? reinterpret_cast<uint4*>(al)
@@ -1704,7 +1724,7 @@ size_t replay_smem_bytes(ReplayArgs& a) {
   a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + (2 + kExpRing) * (size_t)a.m.R) * sizeof(double) +
                 (9 * (size_t)a.m.R + 12 + kRouteRing + kJobRing + kHitRing) * sizeof(uint32_t) + 16 +
-                (kStageDepth + 2) * sizeof(unsigned long long) +
+                (kStageDepth + 2) * (sizeof(unsigned long long) + sizeof(uint4)) + 16 +
                 (kStageDepth + 1 + (kStageDepth + 2) * ((size_t)a.m.R + kStageBlocks)) * sizeof(uint32_t) +
                 8 + (kStageDepth + 2) * (size_t)a.m.R * sizeof(double) +
                 (kStageDepth + 2) * kStageBlocks * sizeof(MaskT) + 8;

@@ -19,13 +19,15 @@ import numpy as np
 ROLES = {
     "route": (0, ["wait for completion sums / ring room", "completion sums, queue term of the score",
                   "wait for the prefix hits", "score and order key", "argmin over replicas",
-                  "hit of the chosen replica, route stores, barrier"]),
+                  "hit of the chosen replica, route stores, barrier", None, None,
+                  "gate's hand-over stamp -> route warp past the barrier"]),
     "service": (16, ["retire: list entry, window vote, grid value", "fence and publish",
                      "issue list exchange and window loads", "slot argmin",
                      "times, outputs, grid load", "idle round"]),
     "gate": (32, ["hand-over at the request's own turn (rest)", "wait for the route",
                   "job, early hand-over of the next request", "own turn: wait for the staged read",
-                  "own turn: wait for commits", None, None, None, None, None,
+                  "own turn: wait for commits", "early: route read, job post", "early: staged?", "early: shares/conflict",
+                  "route warp's stamp -> gate warp past the barrier", None,
                   "#not early: shares a block with a recent request", "#probes redone here",
                   "#not early: not staged yet", "#not early: recent route to a holder of its blocks",
                   "#hits handed over early"]),
