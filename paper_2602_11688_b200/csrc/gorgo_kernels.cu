@@ -103,6 +103,7 @@ __device__ __forceinline__ bool touch_is_stale(const TraceView& tr, const uint8_
                                                uint32_t g, uint32_t rep, uint32_t r_now,
                                                uint32_t rep_now) {
   uint2 nx = tr.occ_next[g];
+  #pragma unroll 1
   while (nx.x != kNone && nx.y <= r_now) {
     const uint32_t rt = (nx.y == r_now) ? rep_now : (uint32_t)route_log[nx.y];
     if (rt == rep) return true;
@@ -176,7 +177,7 @@ __device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id
   __stcg(reinterpret_cast<unsigned long long*>(mask) + id, (unsigned long long)v);
 }
 
-constexpr int kRegChunks = 4;     // request blocks held in registers: 4 x 32 = 128
+constexpr int kRegChunks = 2;     // request blocks held in registers: 2 x 32 = 64
 constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
 constexpr int kScoutBatches = 1;       // touches examined per lane and scout round
@@ -194,7 +195,7 @@ constexpr uint32_t kExpRing = 8;      // completion sums published ahead of the 
 constexpr uint32_t kCommitWarps = 3;  // commit warps per candidate (replicas split between them)
 constexpr uint32_t kJobRing = 32;     // routed requests handed from the gate warp to the commit warps
 constexpr uint32_t kHitRing = 16;     // tags of requests hit by a recent eviction (> kWindow)
-constexpr uint32_t kServices = 2;      // service warps per candidate (replicas split between them)
+constexpr uint32_t kServices = 1;      // service warps per candidate (replicas split between them)
 
 // Shared-memory view of one candidate's small state.
 struct Smem {
@@ -305,6 +306,7 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
     uint32_t tail = sm.ring_tail[i];
     uint4* out = sm.lst + (size_t)i * kListCap;
     bool dry = false;
+    #pragma unroll 1
     for (uint32_t round = 0; round < 6; ++round) {
       const uint32_t room = kListCap - (tail - sm.ring_head[i]);
       if (room < 32u * kScoutBatches) break;
@@ -338,6 +340,7 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
         uint32_t nxr = kNone;
         if (live) {
           uint2 cc = c[u];
+          #pragma unroll 1
           while (cc.x != kNone && cc.y <= rs) {       // later occurrences up to rs
             if ((uint32_t)__ldcg(route_log + cc.y) == i) { live = false; break; }
             cc = a.tr.occ_next[cc.x];
@@ -539,6 +542,7 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
 // hi qualifies.  Every lane walks the same bisection (broadcast loads).
 __device__ __forceinline__ uint32_t first_arrival_at_or_after(const double* ts, double scale, double f,
                                                               uint32_t lo, uint32_t hi) {
+  #pragma unroll 1
   while (lo < hi) {                                       // at most 32 rounds
     const uint32_t mid = lo + ((hi - lo) >> 1);
     if (__dmul_rn(scale, ts[mid]) >= f) hi = mid; else lo = mid + 1;
@@ -623,6 +627,7 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
     // ---- service model of the next routed request of this warp's replicas, if there is one
     if (s < end && (int32_t)(routed_seen - (s + 1)) < 0) routed_seen = *sm.routed;
     smem_order();
+    #pragma unroll 1
     while (s < end && (int32_t)(routed_seen - (s + 1)) >= 0 &&
            (sm.route_ring[s % kRouteRing] & 0xFFu) % kServices != which) ++s;   // the other warp's
     if (s < end) {
@@ -642,6 +647,7 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
         if (S <= 32) {
           if (lane < S) { bk = (uint64_t)__double_as_longlong(fa[lane]); bs = lane; }
         } else {
+          #pragma unroll 1
           for (uint32_t s2 = lane; s2 < S; s2 += 32) {
             const uint64_t vk = (uint64_t)__double_as_longlong(fa[s2]);
             if (vk < bk || bs == kNone) { bk = vk; bs = s2; }
@@ -744,6 +750,7 @@ __device__ __forceinline__ void expiry_warp(const ReplayArgs& a, const Smem& sm,
     {
       const bool fin = my_r != kNone && !head_pending && e == kNone;
       unsigned m = __ballot_sync(kFull, fin) & 0xFFu;
+      #pragma unroll 1
       while (m & (1u << (published % kExpRing))) {          // the lane of request `published` is done
         if (lane == published % kExpRing) my_r = kNone;
         m &= ~(1u << (published % kExpRing));
@@ -753,6 +760,7 @@ __device__ __forceinline__ void expiry_warp(const ReplayArgs& a, const Smem& sm,
       if (progress && lane == 0) { smem_order(); *sm.exp_ready = published; }
     }
     // ---- start the walks of up to two more requests
+    #pragma unroll 1
     for (int k = 0; k < 2 && next_r < end; ++k) {
       const uint32_t owner = next_r % kExpRing;
       // the ring row is free once the route warp has used its previous occupant
@@ -835,6 +843,7 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
   h0 = 0; h1 = 0; p0 = 0; p1 = 0; where = 0;
   const uint32_t n = q.nblk;
   MaskT alive = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0 : (MaskT)((((MaskT)1) << (R & 63)) - 1);
+  #pragma unroll 1
   for (uint32_t c = 0; c < n; c += 32) {
     const uint32_t k = c + lane;
     MaskT m = 0;
@@ -842,6 +851,7 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
     MaskT it = warp_or_mask<MaskT>(m);      // replicas that hold any block of this chunk
     where |= (unsigned long long)it;
     MaskT still = 0;
+    #pragma unroll 1
     while (it != 0) {
       const int i = first_bit<MaskT>(it);
       it &= (MaskT)(it - 1);
@@ -1044,6 +1054,7 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
         slot = kStageDepth + (r & 1u);                          // this warp's own stages
         uint32_t* sid = cx.st_ids + slot * kStageBlocks;
         MaskT* smk = cx.st_mk + slot * kStageBlocks;
+        #pragma unroll 1
         for (uint32_t c = 0; c < n && c < kStageBlocks; c += 32) {
           const uint32_t k = c + lane;
           if (k < n) { const uint32_t id = ids[q_cur.off + k]; sid[k] = id; smk[k] = mask_load<MaskT>(mask, id); }
@@ -1202,6 +1213,7 @@ __device__ __forceinline__ void commit_warp(const ReplayArgs& a, const Ctx<MaskT
           const uint4* lst = sm.lst + (size_t)istar * kListCap;
           uint32_t head = sm.ring_head[istar];
           uint32_t last_e = kNone;   // ring slot of the last entry passed that was not void
+          #pragma unroll 1
           while (need > 0) {
             uint32_t avail = sm.ring_tail[istar] - head;
             for (uint32_t polls = 0; avail == 0 && polls < a.ring_polls; ++polls) {
@@ -1260,6 +1272,7 @@ __device__ __forceinline__ void commit_warp(const ReplayArgs& a, const Ctx<MaskT
         // whatever is still needed: walk the recency order from the cursor and validate touches here
         uint32_t coff = (cr != kNone && need > 0) ? req[cr].off : 0u;
         unsigned long long guard = 0;
+        #pragma unroll 1
         while (need > 0) {
           if (++guard > evict_guard_max) { status = -6; break; }
           if (cp < 0) {  // this request is used up: go to the next one routed here
@@ -1280,6 +1293,7 @@ __device__ __forceinline__ void commit_warp(const ReplayArgs& a, const Ctx<MaskT
             vid = ids[g];
             uint2 c = a.tr.occ_next[g];
             live = true;
+            #pragma unroll 1
             while (c.x != kNone && c.y <= r) {       // later occurrences of the block, up to r
               const uint32_t rr = (c.y == r) ? istar : (uint32_t)route_log[c.y];
               if (rr == istar) { live = false; break; }
@@ -1309,6 +1323,7 @@ __device__ __forceinline__ void commit_warp(const ReplayArgs& a, const Ctx<MaskT
     PROF_LAP(1);
 
     // ---- set the replica's bit on the blocks the request inserts
+    #pragma unroll 1
     for (uint32_t c = 0; c < n; c += 32) {
       const uint32_t k = c + lane;
       if (k < n) {
@@ -1354,8 +1369,8 @@ __device__ __forceinline__ void commit_warp(const ReplayArgs& a, const Ctx<MaskT
 
 // Roles of the twelve warps of a candidate.  Warp w issues from scheduler w % 4 of the SM, and a
 // scheduler's instruction cache is small, so warps that run the same code sit on one scheduler:
-//   scheduler 0: route, expiry, scout     scheduler 1: gate, service, service
-//   scheduler 2: probe, probe, scout      scheduler 3: commit, commit, commit
+//   scheduler 0: route, expiry, scout     scheduler 1: gate, service, scout
+//   scheduler 2: probe, probe             scheduler 3: commit, commit, commit
 enum Role : uint32_t { kRoleRoute, kRoleGate, kRoleProbe, kRoleScout, kRoleService, kRoleExpiry, kRoleCommit, kRoleNone };
 constexpr uint32_t kReplayWarps = 12;
 constexpr uint32_t kReplayThreads = 32 * kReplayWarps;
@@ -1363,12 +1378,12 @@ __device__ __forceinline__ void role_of(uint32_t warp, Role& role, uint32_t& whi
   const uint32_t sched = warp & 3u, k = warp >> 2;
   which = k;
   if (sched == 0) role = k == 0 ? kRoleRoute : k == 1 ? kRoleExpiry : kRoleScout;
-  else if (sched == 1) { role = k == 0 ? kRoleGate : kRoleService; which = k - 1; }
-  else if (sched == 2) role = k < kProbes ? kRoleProbe : kRoleScout;
-  else role = kRoleCommit;
-  if (role == kRoleScout) which = sched >> 1;      // scout 0 and scout 1
+  else if (sched == 1) { role = k == 0 ? kRoleGate : (k - 1 < kServices ? kRoleService : kRoleScout); which = k - 1; }
+  else if (sched == 2) role = k < kProbes ? kRoleProbe : (kServices == 2 && k == 2 ? kRoleScout : kRoleNone);
+  else role = k < kCommitWarps ? kRoleCommit : kRoleNone;
+  if (role == kRoleScout) which = sched == 0 ? 0 : 1;      // scout 0 and scout 1
 }
-static_assert(kScouts == 2 && kProbes == 2 && kCommitWarps == 3, "role map");
+static_assert(kScouts == 2 && kProbes <= 3 && kCommitWarps <= 3 && kServices <= 2, "role map");
 constexpr int kReplayMinCtas = 2;   // registers capped so that two candidates share an SM
 
 template <typename MaskT, bool kBaseline>
@@ -1471,7 +1486,7 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
   if (threadIdx.x == 0) {
     *cx.status = 0; *cx.probe_gone = 0; *sm.abort_flag = 0;
     *sm.routed = a.first; *sm.exp_ready = a.first; *sm.jobs = a.first;
-    sm.serviced[0] = a.first; sm.serviced[1] = a.first;
+    sm.serviced[0] = a.first; if (kServices > 1) sm.serviced[1] = a.first;
   }
   if (threadIdx.x < kCommitWarps) sm.progress[threadIdx.x] = a.first;
   if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
