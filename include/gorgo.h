@@ -275,19 +275,51 @@ int gorgo_es_run(gorgo_sim_t *sim, const gorgo_es_config_t *cfg, const double *x
                  const double *z, void *workspace, uint64_t workspace_bytes, void *cuda_stream,
                  double *x_best, double *objective_best, double *sigma_final, double *history);
 
+/* Measurement aid (no counterpart in the paper): how many candidates (CTAs of the replay kernel)
+ * one SM holds at once for this configuration, and the shared memory each takes.  A population
+ * larger than SMs x that number is replayed in successive rounds of CTAs. */
+int gorgo_replay_occupancy(gorgo_sim_t *sim, int32_t *ctas_per_sm, uint64_t *smem_bytes_per_cta);
 /* Measurement aid (no counterpart in the paper).  With profiling enabled, gorgo_eval_population
  * records a CUDA event on `cuda_stream` directly before and after each launch of the replay
  * kernel (one launch per wave, at most 32 waves are timed).  gorgo_last_replay_ms waits for those
  * events and returns the summed device time of the replay launches of the most recent
  * evaluation and their number. */
-/* Measurement aid (no counterpart in the paper): how many candidates (CTAs of the replay kernel)
- * one SM holds at once for this configuration, and the shared memory each takes.  A population
- * larger than SMs x that number is replayed in successive rounds of CTAs. */
-int gorgo_replay_occupancy(gorgo_sim_t *sim, int32_t *ctas_per_sm, uint64_t *smem_bytes_per_cta);
 int gorgo_set_profiling(gorgo_sim_t *sim, int enable);
 int gorgo_last_replay_ms(gorgo_sim_t *sim, double *replay_ms, uint32_t *launches);
 /* The same for the window-objective kernels of the most recent gorgo_eval_population_windows. */
 int gorgo_last_window_ms(gorgo_sim_t *sim, double *window_ms, uint32_t *launches);
+
+/* Measurement aid (no counterpart in the paper): the rate at which this GPU serves independent
+ * 32-byte reads (one sector each) at pseudo-random positions of a footprint of `footprint_bytes`,
+ * in GB/s of sectors (reads x 32 bytes / time; best of three timed launches after a warm-up, CUDA
+ * events on `cuda_stream`).  With a footprint far larger than the L2 cache this is the random-sector
+ * DRAM rate, with a footprint inside it the L2 rate: the two yardsticks a gather-bound kernel can be
+ * held against besides the streaming copy bandwidth.  `buffer` DEVICE, 256-byte aligned,
+ * `buffer_bytes` >= footprint_bytes + 256 (its contents are read, and four bytes behind the
+ * footprint may be written); footprint_bytes >= 4096.  The call waits for its launches. */
+int gorgo_measure_gather(int device, void *buffer, uint64_t buffer_bytes, uint64_t footprint_bytes,
+                         void *cuda_stream, double *sectors_gb_per_s);
+
+/* Test aid (no counterpart in the paper).  Inside the replay kernel the warps of one candidate
+ * wait for one another with bounded polls, and two kinds of helper warps only prepare work
+ * ahead of the warps that must do it anyway (the probe warps stage prefix hits, the scout warps
+ * pre-validate eviction victims).  These switches let a test take those paths on purpose; none
+ * of them makes a kernel fault or hang.  They apply to every later launch of `sim`.
+ *   GORGO_DEBUG_POLL_LIMIT  polls after which a warp gives up waiting (default 2^24).  With 0 the
+ *                           first wait that is not already satisfied gives up: the candidate
+ *                           finishes with wrong results and status GORGO_ERR_DEVICE_LIMIT.
+ *   GORGO_DEBUG_RING_POLLS  polls of a commit warp for the scout's next victim before it looks for
+ *                           victims itself (default 64; results do not depend on it).
+ *   GORGO_DEBUG_PROBE_OFF   nonzero: no probe warps; every request is probed where it is needed
+ *                           (results do not depend on it).
+ *   GORGO_DEBUG_SCOUT_OFF   nonzero: no scout warps (results do not depend on it). */
+enum {
+  GORGO_DEBUG_POLL_LIMIT = 0,
+  GORGO_DEBUG_RING_POLLS = 1,
+  GORGO_DEBUG_PROBE_OFF = 2,
+  GORGO_DEBUG_SCOUT_OFF = 3
+};
+int gorgo_debug_set(gorgo_sim_t *sim, uint32_t what, uint32_t value);
 
 /* Population evaluation for callers that cannot allocate device memory (the paper has no
  * counterpart; this is a packaging variant of gorgo_eval_population).  Some hosts of this library
@@ -300,13 +332,15 @@ int gorgo_last_window_ms(gorgo_sim_t *sim, double *window_ms, uint32_t *launches
  * the library holds until the process exits.  The call allocates and frees nothing, on host
  * paths of the CUDA runtime included: no cudaMalloc, cudaFree or allocating library routine.
  *
- * Arguments are those of gorgo_eval_population without the workspace, digest, counters and
- * status: `params` HOST or DEVICE (P*K doubles), `p95_ttft_ms` / `p95_e2e_ms` DEVICE (P doubles
- * each), `route` DEVICE P*N bytes or NULL, `hit_blocks` DEVICE P*N uint16 or NULL.
+ * Arguments are those of gorgo_eval_population without the workspace, digest and counters:
+ * `params` HOST or DEVICE (P*K doubles), `p95_ttft_ms` / `p95_e2e_ms` DEVICE (P doubles
+ * each), `route` DEVICE P*N bytes or NULL, `hit_blocks` DEVICE P*N uint16 or NULL, `cand_status`
+ * DEVICE P int32 or NULL: 0, or GORGO_ERR_DEVICE_LIMIT for a candidate whose replay gave up on a
+ * bounded wait (its outputs are then meaningless; read it after synchronising the stream).
  * Limit: the scratch of ONE candidate, gorgo_workspace_bytes(sim, 1), must not exceed
  * GORGO_STATIC_SCRATCH_BYTES, else GORGO_ERR_STATIC_LIMIT and nothing runs; a population whose
  * candidates do not all fit at once is evaluated in waves.  (Per candidate the scratch is about
- * 33 bytes per request plus 1 to 8 bytes per distinct block id.)
+ * 41 bytes per request plus 1 to 8 bytes per distinct block id.)
  * The first call on a device looks up the array's device address; make that first call outside
  * any stream capture.  All calls in a process share the one array per GPU and it keeps what the
  * previous call left there; each call clears what it needs to start from zero, but two calls
@@ -315,7 +349,8 @@ int gorgo_last_window_ms(gorgo_sim_t *sim, double *window_ms, uint32_t *launches
 #define GORGO_STATIC_SCRATCH_BYTES (64u << 20)
 int gorgo_eval_population_static(gorgo_sim_t *sim, uint32_t n_candidates, const double *params,
                                  double time_scale, void *cuda_stream, double *p95_ttft_ms,
-                                 double *p95_e2e_ms, uint8_t *route, uint16_t *hit_blocks);
+                                 double *p95_e2e_ms, uint8_t *route, uint16_t *hit_blocks,
+                                 int32_t *cand_status);
 
 const char *gorgo_strerror(int code);
 

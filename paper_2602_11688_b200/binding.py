@@ -34,8 +34,9 @@ EXPORTS = [
     "gorgo_eval_population_static", "gorgo_replay_occupancy", "gorgo_strerror",
     "gorgo_window_count", "gorgo_eval_population_windows", "gorgo_es_run",
     "gorgo_last_window_ms", "gorgo_eval_policy", "gorgo_eval_population_scales",
-    "gorgo_sim_set_replica_speeds",
+    "gorgo_sim_set_replica_speeds", "gorgo_debug_set", "gorgo_measure_gather",
 ]
+GORGO_DEBUG_POLL_LIMIT, GORGO_DEBUG_RING_POLLS, GORGO_DEBUG_PROBE_OFF, GORGO_DEBUG_SCOUT_OFF = 0, 1, 2, 3
 
 
 class gorgo_config_t(C.Structure):
@@ -87,7 +88,9 @@ def load():
         "gorgo_route_batch": [vp, vp, dbl, u64, u64, vp, u64, vp, vp, vp, vp, vp],
         "gorgo_state_digest": [vp, vp, u64, vp, vp],
         "gorgo_state_status": [vp, vp, u64, vp, pu64],
-        "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp],
+        "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp, vp],
+        "gorgo_debug_set": [vp, u32, u32],
+        "gorgo_measure_gather": [i32, vp, u64, u64, vp, C.POINTER(C.c_double)],
         "gorgo_replay_occupancy": [vp, C.POINTER(C.c_int32), pu64],
         "gorgo_window_count": [u64, u32, u32, pu64],
         "gorgo_sim_set_replica_speeds": [vp, vp, vp],
@@ -195,8 +198,22 @@ def gorgo_eval_population_host(sim, n_candidates, params, time_scale, workspace,
         workspace.numel(), stream, host_ptr(p95_ttft_ms), host_ptr(p95_e2e_ms))
 
 
+def gorgo_measure_gather(device: int, buffer, footprint_bytes: int, stream: int = 0):
+    """Random 32-byte-sector read rate over the first ``footprint_bytes`` of ``buffer`` (a torch CUDA
+    uint8 tensor at least 256 bytes longer).  Returns (status, GB/s of sectors)."""
+    out = C.c_double()
+    rc = load().gorgo_measure_gather(int(device), _dev_ptr(buffer), buffer.numel(),
+                                     int(footprint_bytes), stream, C.byref(out))
+    return rc, out.value
+
+
+def gorgo_debug_set(sim, what: int, value: int) -> int:
+    """Test switches of the replay kernel (GORGO_DEBUG_* constants)."""
+    return load().gorgo_debug_set(sim, int(what), int(value))
+
+
 def gorgo_eval_population_static(sim, n_candidates, params, time_scale, stream, p95_ttft_ms,
-                                 p95_e2e_ms, route=None, hit_blocks=None) -> int:
+                                 p95_e2e_ms, route=None, hit_blocks=None, cand_status=None) -> int:
     """Evaluation that uses the scratch array built into the library instead of a workspace, for
     callers that may not allocate device memory.  ``params``: float64 numpy array (host) or torch
     CUDA tensor; outputs: torch CUDA tensors.  Returns GORGO_ERR_STATIC_LIMIT when one
@@ -204,7 +221,7 @@ def gorgo_eval_population_static(sim, n_candidates, params, time_scale, stream, 
     pp = _np_ptr(params) if isinstance(params, np.ndarray) else _dev_ptr(params)
     return load().gorgo_eval_population_static(
         sim, int(n_candidates), pp, float(time_scale), stream, _dev_ptr(p95_ttft_ms),
-        _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks))
+        _dev_ptr(p95_e2e_ms), _dev_ptr(route), _dev_ptr(hit_blocks), _dev_ptr(cand_status))
 
 
 def gorgo_sim_set_replica_speeds(sim, prefill_ms_per_token=None, tpot_ms=None) -> int:

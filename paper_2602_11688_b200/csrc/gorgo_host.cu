@@ -832,6 +832,55 @@ int gorgo_replay_occupancy(gorgo_sim_t* sim, int32_t* ctas_per_sm, uint64_t* sme
   return GORGO_OK;
 }
 
+int gorgo_measure_gather(int device, void* buffer, uint64_t buffer_bytes, uint64_t footprint_bytes,
+                         void* cuda_stream, double* sectors_gb_per_s) {
+  if (!buffer || !sectors_gb_per_s || (uintptr_t)buffer % kAlign) return GORGO_ERR_INVALID_ARG;
+  if (footprint_bytes < 4096 || footprint_bytes + 256 > buffer_bytes) return GORGO_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return GORGO_ERR_CUDA;
+  const uint32_t blocks = (uint32_t)prop.multiProcessorCount * 8u;   // 2,048 threads per SM
+  const uint32_t per_thread = 256;
+  const uint64_t n_sectors = footprint_bytes / 32;
+  uint32_t* sink = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(buffer) + footprint_bytes / 256 * 256);
+  cudaEvent_t e0, e1;
+  if (cudaEventCreate(&e0) != cudaSuccess) return GORGO_ERR_CUDA;
+  if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return GORGO_ERR_CUDA; }
+  int rc = GORGO_OK;
+  float best_ms = 0.f;
+  for (int rep = 0; rep < 4 && rc == GORGO_OK; ++rep) {        // first pass warms up
+    if (cudaEventRecord(e0, st) != cudaSuccess ||
+        launch_gather(buffer, n_sectors, per_thread, blocks, sink, st) != cudaSuccess ||
+        cudaEventRecord(e1, st) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) {
+      rc = GORGO_ERR_CUDA;
+      break;
+    }
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) { rc = GORGO_ERR_CUDA; break; }
+    if (rep > 0 && (best_ms == 0.f || ms < best_ms)) best_ms = ms;
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (rc != GORGO_OK) { cudaGetLastError(); return rc; }
+  const double sectors = (double)blocks * 256.0 * per_thread;
+  *sectors_gb_per_s = sectors * 32.0 / (best_ms * 1e-3) / 1e9;
+  return GORGO_OK;
+}
+
+int gorgo_debug_set(gorgo_sim_t* sim, uint32_t what, uint32_t value) {
+  if (!sim) return GORGO_ERR_INVALID_ARG;
+  switch (what) {
+    case GORGO_DEBUG_POLL_LIMIT: sim->poll_limit = value; break;
+    case GORGO_DEBUG_RING_POLLS: sim->ring_polls = value; break;
+    case GORGO_DEBUG_PROBE_OFF: sim->probe_off = value ? 1u : 0u; break;
+    case GORGO_DEBUG_SCOUT_OFF: sim->scout_off = value ? 1u : 0u; break;
+    default: return GORGO_ERR_INVALID_ARG;
+  }
+  return GORGO_OK;
+}
+
 int gorgo_set_profiling(gorgo_sim_t* sim, int enable) {
   if (!sim) return GORGO_ERR_INVALID_ARG;
   if (enable && sim->ev.empty()) {
@@ -929,7 +978,8 @@ int static_scratch_address(int device, void** out) {
 
 int gorgo_eval_population_static(gorgo_sim_t* sim, uint32_t n_candidates, const double* params,
                                  double time_scale, void* cuda_stream, double* p95_ttft_ms,
-                                 double* p95_e2e_ms, uint8_t* route, uint16_t* hit_blocks) {
+                                 double* p95_e2e_ms, uint8_t* route, uint16_t* hit_blocks,
+                                 int32_t* cand_status) {
   if (!sim) return GORGO_ERR_INVALID_ARG;
   if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
   // one candidate's replay state must fit; a larger population then runs in waves inside it
@@ -946,7 +996,7 @@ int gorgo_eval_population_static(gorgo_sim_t* sim, uint32_t n_candidates, const 
   // so whatever an earlier call left in the array is never read
   return eval_impl(sim, n_candidates, params, time_scale, scratch, GORGO_STATIC_SCRATCH_BYTES,
                    static_cast<cudaStream_t>(cuda_stream), p95_ttft_ms, p95_e2e_ms, route,
-                   hit_blocks, nullptr, nullptr, nullptr, false);
+                   hit_blocks, nullptr, nullptr, cand_status, false);
 }
 
 #ifdef GORGO_PROF

@@ -156,6 +156,8 @@ cudaError_t launch_policy_routes(const TraceView& tr, uint32_t R, bool affinity,
 // Cycle accounting build only: the 64 accumulators (decide warp at 0, cache warp at 16).
 cudaError_t prof_read(unsigned long long* out64, bool reset);
 #endif
+cudaError_t launch_gather(const void* buf, uint64_t n_sectors, uint32_t per_thread, uint32_t blocks,
+                          uint32_t* sink, cudaStream_t st);
 uint32_t window_max();          // largest window the window kernel handles
 uint32_t mask_bytes_for(uint32_t n_replicas);
 uint64_t evict_list_bytes(uint32_t n_replicas);

@@ -160,23 +160,6 @@ template <>
 __device__ __forceinline__ uint64_t mask_load<uint64_t>(const uint64_t* mask, uint32_t id) {
   return __ldcg(reinterpret_cast<const unsigned long long*>(mask) + id);
 }
-template <typename MaskT>
-__device__ __forceinline__ void mask_store(MaskT* mask, uint32_t id, MaskT v) {
-  __stcg(mask + id, v);
-}
-template <>
-__device__ __forceinline__ void mask_store<uint8_t>(uint8_t* mask, uint32_t id, uint8_t v) {
-  __stcg(reinterpret_cast<unsigned char*>(mask) + id, (unsigned char)v);
-}
-template <>
-__device__ __forceinline__ void mask_store<uint16_t>(uint16_t* mask, uint32_t id, uint16_t v) {
-  __stcg(reinterpret_cast<unsigned short*>(mask) + id, (unsigned short)v);
-}
-template <>
-__device__ __forceinline__ void mask_store<uint64_t>(uint64_t* mask, uint32_t id, uint64_t v) {
-  __stcg(reinterpret_cast<unsigned long long*>(mask) + id, (unsigned long long)v);
-}
-
 constexpr int kRegChunks = 2;     // request blocks held in registers: 2 x 32 = 64
 constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
@@ -1856,6 +1839,39 @@ cudaError_t prof_read(unsigned long long* out64, bool reset) {
   return cudaMemcpyToSymbol(g_prof, zero, sizeof(zero));
 }
 #endif
+
+// ------------------------------------------------------------------ gather yardstick
+// Every thread reads `per_thread` 32-byte sectors at pseudo-random positions of a buffer of
+// `n_sectors` sectors (position = splitmix64 finaliser of a counter, so consecutive reads of one
+// thread and the reads of neighbouring threads land on unrelated sectors) and keeps one word of
+// each, eight reads in flight per thread.  What it measures is the rate at which this GPU serves
+// independent 32-byte reads from a footprint of that size: DRAM sectors when the footprint is
+// far larger than L2, L2 sectors when it fits.
+__global__ void __launch_bounds__(256) gather_sectors_kernel(const uint4* buf, uint64_t n_sectors,
+                                                             uint32_t per_thread, uint32_t* sink) {
+  const uint64_t tid = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const uint64_t n_threads = (uint64_t)gridDim.x * blockDim.x;
+  uint32_t acc = 0;
+  for (uint32_t it = 0; it < per_thread; it += 8) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const uint64_t c = ((uint64_t)(it + u) * n_threads + tid) * 0x9E3779B97F4A7C15ULL;
+      const uint64_t sector = mix64(c) % n_sectors;
+      v[u] = __ldcg(buf + sector * 2);                  // first half of the 32-byte sector
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc += v[u].x ^ v[u].w;
+  }
+  if (acc == 0x12345u) *sink = acc;                     // keeps the loads alive
+}
+
+cudaError_t launch_gather(const void* buf, uint64_t n_sectors, uint32_t per_thread, uint32_t blocks,
+                          uint32_t* sink, cudaStream_t st) {
+  gather_sectors_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(buf), n_sectors,
+                                                per_thread, sink);
+  return cudaGetLastError();
+}
 
 uint32_t window_max() { return kWindowMax; }
 

@@ -59,3 +59,26 @@ def gather_results(local: np.ndarray, n_candidates: int, device=None) -> np.ndar
     dist.all_gather(parts, mine)
     out = [parts[r][: hi - lo].cpu().numpy() for r, (lo, hi) in enumerate(sizes)]
     return np.concatenate(out, axis=0)
+
+
+def run_ranks(rank: int, world: int, base_params: np.ndarray, evaluate, steps: int, warmup: int,
+              timer, barrier, device=None):
+    """The rank logic of the benchmark, independent of what evaluates a population: every rank
+    takes a population of the single-GPU size (weak scaling), runs `warmup` untimed and `steps`
+    timed evaluations between two barriers, and the job's time is the slowest rank's.
+    `evaluate(params)` returns this rank's per-candidate results [P, 2]; `timer()` returns a
+    callable that gives the milliseconds since it was created (CUDA events on the launching stream
+    in the benchmark, a wall clock in the CPU test).  Returns (ms_per_step of the job, this rank's
+    results of the last step, candidates evaluated per step by the whole job)."""
+    params = weak_scaling_population(base_params, rank)
+    last = None
+    for _ in range(warmup):
+        last = evaluate(params)
+    barrier()
+    elapsed = timer()
+    for _ in range(steps):
+        last = evaluate(params)
+    ms = elapsed()
+    barrier()
+    ms_job = max_over_ranks(ms, device)
+    return ms_job / max(1, steps), np.asarray(last), int(params.shape[0]) * int(world)

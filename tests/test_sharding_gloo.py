@@ -32,6 +32,49 @@ def _worker(rank, world, port, n_cand, out_dir):
     dist.destroy_process_group()
 
 
+def _bench_worker(rank, world, port, out_dir):
+    """The benchmark's own rank logic (sharding.run_ranks) with the evaluator stubbed: rank r
+    "evaluates" in (r + 1) x 20 ms."""
+    import time
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    base = np.random.default_rng(3).normal(1.0, 0.3, size=(6, 5))
+    calls = []
+
+    def evaluate(params):
+        calls.append(params.copy())
+        time.sleep(0.02 * (rank + 1))
+        return np.stack([params[:, 0], params[:, 1] + rank], axis=1)
+
+    def timer():
+        t0 = time.perf_counter()
+        return lambda: (time.perf_counter() - t0) * 1e3
+
+    ms_per_step, last, per_step = sh.run_ranks(rank, world, base, evaluate, steps=3, warmup=2,
+                                               timer=timer, barrier=dist.barrier)
+    np.savez(os.path.join(out_dir, f"b{rank}.npz"), ms=ms_per_step, last=last, per_step=per_step,
+             n_calls=len(calls), first=calls[0], same=all(np.array_equal(c, calls[0]) for c in calls))
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_run_the_benchmark_rank_logic(tmp_path):
+    world = 2
+    mp.spawn(_bench_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    base = np.random.default_rng(3).normal(1.0, 0.3, size=(6, 5))
+    b0, b1 = np.load(tmp_path / "b0.npz"), np.load(tmp_path / "b1.npz")
+    # weak scaling: every rank evaluates a population of the single-GPU size, warm-up + steps times
+    assert int(b0["n_calls"]) == 5 and int(b1["n_calls"]) == 5 and bool(b0["same"]) and bool(b1["same"])
+    assert int(b0["per_step"]) == 12 and int(b1["per_step"]) == 12
+    assert np.array_equal(b0["first"], base)                   # rank 0 keeps the base draw
+    assert b1["first"].shape == base.shape and not np.array_equal(b1["first"][:, :3], base[:, :3])
+    assert np.array_equal(b1["first"][:, 3:], base[:, 3:])     # normalisers are kept
+    # the job's time is the slowest rank's (40 ms per step), on both ranks
+    assert float(b0["ms"]) == float(b1["ms"]) and 38.0 <= float(b0["ms"]) < 80.0
+    assert np.array_equal(b1["last"][:, 1], b1["first"][:, 1] + 1)
+
+
 def test_shard_bounds_cover_every_candidate_once():
     for n in (1, 7, 8, 256, 1000):
         for world in (1, 2, 3, 8):

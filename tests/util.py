@@ -39,13 +39,16 @@ def small_trace(seed, n_req=300, n_sessions=12, max_blocks=7, structured=True, B
 
 
 def gpu_eval(workload, params=None, scale=None, *, resident=None, max_bytes=None, route=True,
-             hit=True, digest=True, stats=True, sim=None):
-    """Evaluate a population through gorgo_eval_population; returns numpy arrays."""
+             hit=True, digest=True, stats=True, sim=None, debug=None):
+    """Evaluate a population through gorgo_eval_population; returns numpy arrays.  `debug` maps
+    GORGO_DEBUG_* switches to values (set on a simulator created here)."""
     import torch
     from paper_2602_11688_b200 import binding as gb
     own = sim is None
     if own:
         sim = gb.GorgoSim(workload)
+        for what, value in (debug or {}).items():
+            assert gb.gorgo_debug_set(sim.h, what, value) == gb.GORGO_OK
     try:
         params = workload.params if params is None else np.ascontiguousarray(params, np.float64)
         scale = workload.spec.time_scales[0] if scale is None else scale
