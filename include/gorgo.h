@@ -275,6 +275,47 @@ int gorgo_es_run(gorgo_sim_t *sim, const gorgo_es_config_t *cfg, const double *x
                  const double *z, void *workspace, uint64_t workspace_bytes, void *cuda_stream,
                  double *x_best, double *objective_best, double *sigma_final, double *history);
 
+/* The paper's tuner as it runs in the proxy (Section 2.3; Section 4): ONLINE, inside one replay.
+ * The weights in force change every `hop` requests.  Step k = 1, 2, ... of the (1+1)-ES takes
+ * place when window + (k-1)*hop requests have been routed (window 128, hop 32: the 18th step
+ * after 672 samples, as the paper counts) and is scored by the nearest-rank p95 of the TTFTs of
+ * the last `window` requests in trace order.  Step 1 scores the start weights.  Every later step
+ * scores the offspring that was in force during the last hop (the window still holds requests
+ * routed under earlier weights, as a rolling window does), makes it the parent iff its value is
+ * strictly smaller than the parent's, multiplies sigma by `sigma_up` after an accepted step and
+ * by sigma_up^(-1/4) after a rejected one, and puts a new offspring of the parent (Eq. 4, clamped to
+ * [lo, hi]) in force for the next hop.  After `n_draw_steps` steps the weights in force stay.
+ * `n_tuners` independent tuners run side by side, each on its own simulator state, from its own
+ * start weights and draws: x0 HOST [n_tuners*K]; z HOST [n_tuners * n_draw_steps * n_tuned],
+ * z[(p*n_draw_steps + (k-1))*n_tuned + j] perturbs tuned parameter j of tuner p in step k.
+ * The replays, the window values and the final p95s are computed on the device; Eq. 4 and the
+ * accept/reject bookkeeping run on the host between the chunks (C library exp and log, the sum
+ * ln x + sigma*z two rounded operations), so the call synchronises `cuda_stream` once per hop.
+ * Outputs (HOST unless noted): x_final [n_tuners*K] the parents at the end; sigma_final
+ * [n_tuners]; steps_done (may be NULL) the steps taken, min(n_draw_steps, number of full windows);
+ * history, or NULL, [n_tuners * n_draw_steps * (4 + 2*n_tuned)]: per tuner and step the window
+ * value, 1.0 if accepted else 0.0, sigma after the step, the parent's value after the step, the
+ * parent's tuned weights after the step, the tuned weights put in force for the next hop;
+ * p95_ttft_ms / p95_e2e_ms [n_tuners] each, both or neither NULL: p95 over the whole tuned replay;
+ * route DEVICE [n_tuners*N] bytes or NULL.  `workspace` DEVICE, at least
+ * gorgo_workspace_bytes(sim, n_tuners): all tuners stay resident.  Errors: those of gorgo_es_run;
+ * GORGO_ERR_WORKSPACE_TOO_SMALL if the tuners do not all fit. */
+typedef struct {
+  uint32_t n_tuned;        /* number of tuned parameters                                     */
+  uint32_t n_draw_steps;   /* steps for which z holds draws                                  */
+  uint32_t window, hop;    /* rolling window and hop in requests (paper: 128, 32); window <= 2048 */
+  const uint32_t *tuned;   /* [n_tuned] their indices in the K-vector                        */
+  const double *lo;        /* [n_tuned] lower clamp, > 0                                     */
+  const double *hi;        /* [n_tuned] upper clamp, >= lo                                   */
+  double sigma0;           /* initial step size, > 0                                         */
+  double sigma_up;         /* > 1                                                            */
+  double time_scale;       /* as for gorgo_eval_population                                   */
+} gorgo_online_config_t;
+int gorgo_tune_online(gorgo_sim_t *sim, const gorgo_online_config_t *cfg, uint32_t n_tuners,
+                      const double *x0, const double *z, void *workspace, uint64_t workspace_bytes,
+                      void *cuda_stream, double *x_final, double *sigma_final, uint32_t *steps_done,
+                      double *history, double *p95_ttft_ms, double *p95_e2e_ms, uint8_t *route);
+
 /* Measurement aid (no counterpart in the paper): how many candidates (CTAs of the replay kernel)
  * one SM holds at once for this configuration, and the shared memory each takes.  A population
  * larger than SMs x that number is replayed in successive rounds of CTAs. */

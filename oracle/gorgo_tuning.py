@@ -12,6 +12,15 @@ Pure-Python loops over small inputs, fp64, steps in the paper's order and notati
   smaller.  Rechenberg's 1/5 rule with the reading  sigma *= a  after an accepted step and
   sigma *= a**(-1/4)  after a rejected one (the paper names the rule, not its constants).
 
+* ``online_tune``: the same strategy run ONLINE, inside one replay, as the paper's proxy does
+  (Section 4): the weights in force change every `hop` requests.  Step k (k = 1, 2, ...) takes
+  place when 128 + (k-1)*32 requests have been routed (so the 18th step comes after 672 samples,
+  as the paper counts); its value is the p95 TTFT of the last `window` requests.  Step 1 scores
+  the start weights; every later step scores the offspring that was in force during the last hop
+  (the window still holds requests routed under earlier weights: that is what a rolling window
+  does), keeps it iff it is strictly better than the parent's value, adapts sigma and puts a
+  new offspring of the parent in force for the next hop.
+
 Pinned by tests/test_oracle_tuning_pins.py (the paper's own arithmetic 128 + 17*32 = 672 samples
 at the 18th step, sorted and constant inputs, numpy's inverted-CDF percentile per window, the
 stationarity of sigma at one success in five, clamp bounds, a convex toy objective).
@@ -81,3 +90,51 @@ def es_run(objective: Callable[[List[float]], float], x0: Sequence[float], tuned
             sigma = sigma * down
         history.append((f[best], accept, sigma, f_parent, [parent[i] for i in tuned]))
     return parent, f_parent, sigma, history
+
+
+def online_tune(run_chunk: Callable[[List[float], int], Sequence[float]], n_requests: int,
+                x0: Sequence[float], tuned: Sequence[int], lo: Sequence[float], hi: Sequence[float],
+                sigma0: float, sigma_up: float, z: Sequence[Sequence[float]], window: int = 128,
+                hop: int = 32):
+    """Online (1+1)-ES over one replay.  ``run_chunk(weights, count)`` routes the next ``count``
+    requests of the trace with the full parameter vector ``weights`` on one persistent simulator
+    state and returns their TTFTs.  ``z[k-1]`` holds the normal draws of step k (one per tuned
+    parameter); the replay ends with the trace, steps that have no draws left keep the weights
+    in force.  Returns (ttft of every request, schedule, history): schedule[h] = the full
+    weights in force for chunk h (chunk 0 = the first `window` requests, then one per hop),
+    history[k-1] = (window value, accepted, sigma after, parent value after, parent tuned values
+    after, tuned values put in force for the next hop)."""
+    parent = list(x0)
+    live = list(x0)
+    f_parent = None
+    sigma = sigma0
+    down = sigma_up ** -0.25
+    kth = (95 * window + 99) // 100
+    ttft: List[float] = []
+    schedule, history = [], []
+    step = 0
+    while len(ttft) < n_requests:
+        count = min(window if not ttft else hop, n_requests - len(ttft))
+        schedule.append(list(live))
+        ttft.extend(run_chunk(list(live), count))
+        if len(ttft) < window or (len(ttft) - window) % hop != 0:
+            continue                                   # no full window ends here (short last chunk)
+        if step >= len(z):
+            continue                                   # out of draws: keep the weights in force
+        value = sorted(ttft[len(ttft) - window:])[kth - 1]
+        if step == 0:
+            f_parent, accept = value, False            # the start weights themselves
+        else:
+            accept = value < f_parent
+            if accept:
+                parent, f_parent = list(live), value
+                sigma = sigma * sigma_up
+            else:
+                sigma = sigma * down
+        live = list(parent)
+        for idx, v in zip(tuned, mutate([parent[i] for i in tuned], sigma, z[step], lo, hi)):
+            live[idx] = v
+        history.append((value, accept, sigma, f_parent, [parent[i] for i in tuned],
+                        [live[i] for i in tuned]))
+        step += 1
+    return ttft, schedule, history

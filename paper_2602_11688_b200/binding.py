@@ -34,7 +34,7 @@ EXPORTS = [
     "gorgo_eval_population_static", "gorgo_replay_occupancy", "gorgo_strerror",
     "gorgo_window_count", "gorgo_eval_population_windows", "gorgo_es_run",
     "gorgo_last_window_ms", "gorgo_eval_policy", "gorgo_eval_population_scales",
-    "gorgo_sim_set_replica_speeds", "gorgo_debug_set", "gorgo_measure_gather",
+    "gorgo_sim_set_replica_speeds", "gorgo_debug_set", "gorgo_measure_gather", "gorgo_tune_online",
 ]
 GORGO_DEBUG_POLL_LIMIT, GORGO_DEBUG_RING_POLLS, GORGO_DEBUG_PROBE_OFF, GORGO_DEBUG_SCOUT_OFF = 0, 1, 2, 3
 
@@ -52,6 +52,12 @@ class gorgo_es_config_t(C.Structure):
                 ("objective", C.c_uint32), ("tuned", C.c_void_p), ("lo", C.c_void_p),
                 ("hi", C.c_void_p), ("sigma0", C.c_double), ("sigma_up", C.c_double),
                 ("time_scale", C.c_double)]
+
+
+class gorgo_online_config_t(C.Structure):
+    _fields_ = [("n_tuned", C.c_uint32), ("n_draw_steps", C.c_uint32), ("window", C.c_uint32),
+                ("hop", C.c_uint32), ("tuned", C.c_void_p), ("lo", C.c_void_p), ("hi", C.c_void_p),
+                ("sigma0", C.c_double), ("sigma_up", C.c_double), ("time_scale", C.c_double)]
 
 
 class GorgoError(RuntimeError):
@@ -90,6 +96,8 @@ def load():
         "gorgo_state_status": [vp, vp, u64, vp, pu64],
         "gorgo_eval_population_static": [vp, u32, vp, dbl, vp, vp, vp, vp, vp, vp],
         "gorgo_debug_set": [vp, u32, u32],
+        "gorgo_tune_online": [vp, C.POINTER(gorgo_online_config_t), u32, vp, vp, vp, u64, vp, vp, vp,
+                              C.POINTER(C.c_uint32), vp, vp, vp, vp],
         "gorgo_measure_gather": [i32, vp, u64, u64, vp, C.POINTER(C.c_double)],
         "gorgo_replay_occupancy": [vp, C.POINTER(C.c_int32), pu64],
         "gorgo_window_count": [u64, u32, u32, pu64],
@@ -304,6 +312,35 @@ def gorgo_es_run(sim, *, x0, z, tuned, lo, hi, sigma0, sigma_up, n_steps, lam, w
                              workspace.numel(), stream, _np_ptr(x_best), C.byref(fb), C.byref(sg),
                              _np_ptr(hist))
     return rc, x_best, fb.value, sg.value, hist
+
+
+def gorgo_tune_online(sim, *, x0, z, tuned, lo, hi, sigma0, sigma_up, workspace, stream,
+                      time_scale=1.0, window=128, hop=32, route=None):
+    """Online (1+1)-ES inside one replay for ``P = x0.shape[0]`` independent tuners.  ``x0``
+    [P, K], ``z`` [P, n_draw_steps, n_tuned] host arrays; ``route`` a torch CUDA uint8 tensor
+    [P, N] or None.  Returns (status, x_final [P, K], sigma_final [P], steps_done,
+    history [P, n_draw_steps, 4 + 2*n_tuned], p95_ttft [P], p95_e2e [P])."""
+    x0 = np.ascontiguousarray(x0, dtype=np.float64)
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    tuned = np.ascontiguousarray(tuned, dtype=np.uint32)
+    lo = np.ascontiguousarray(lo, dtype=np.float64)
+    hi = np.ascontiguousarray(hi, dtype=np.float64)
+    P, T = x0.shape[0], tuned.shape[0]
+    n_steps = z.shape[1] if z.ndim == 3 else 0
+    assert z.shape == (P, n_steps, T) and lo.shape == (T,) and hi.shape == (T,)
+    cfg = gorgo_online_config_t(int(T), int(n_steps), int(window), int(hop), tuned.ctypes.data,
+                                lo.ctypes.data, hi.ctypes.data, float(sigma0), float(sigma_up),
+                                float(time_scale))
+    x_final = np.zeros_like(x0)
+    sig = np.zeros(P, np.float64)
+    hist = np.zeros((P, n_steps, 4 + 2 * T), np.float64)
+    pt, pe = np.zeros(P, np.float64), np.zeros(P, np.float64)
+    done = C.c_uint32()
+    rc = load().gorgo_tune_online(sim, C.byref(cfg), int(P), _np_ptr(x0), _np_ptr(z),
+                                  _dev_ptr(workspace), workspace.numel(), stream, _np_ptr(x_final),
+                                  _np_ptr(sig), C.byref(done), _np_ptr(hist), _np_ptr(pt), _np_ptr(pe),
+                                  _dev_ptr(route))
+    return rc, x_final, sig, done.value, hist, pt, pe
 
 
 def gorgo_state_bytes(sim):

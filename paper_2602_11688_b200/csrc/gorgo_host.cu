@@ -1,6 +1,7 @@
 // Host shell of libgorgo_b200: the C ABI declared in include/gorgo.h.  Argument checks, trace
 // preparation (validation, dense renumbering of block ids, next-occurrence links), workspace
 // layout, wave scheduling and kernel launches.  No step of the simulation runs on the host.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -709,6 +710,152 @@ int gorgo_es_run(gorgo_sim_t* sim, const gorgo_es_config_t* cfg, const double* x
   std::copy(parent.begin(), parent.end(), x_best);
   *objective_best = f_parent;
   *sigma_final = sigma;
+  return GORGO_OK;
+}
+
+// Online (1+1)-ES inside one replay (paper Section 2.3 and Section 4): P independent tuners, each on
+// its own simulator state, all advanced together: one replay launch per chunk of requests (the
+// first `window`, then `hop` at a time), one launch that reduces the last `window` TTFTs of
+// every tuner to their p95, and the strategy's step on the host (Eq. 4 with the C library's exp
+// and log, like gorgo_es_run).  No step of the simulation runs on the host.
+int gorgo_tune_online(gorgo_sim_t* sim, const gorgo_online_config_t* cfg, uint32_t n_tuners,
+                      const double* x0, const double* z, void* workspace, uint64_t workspace_bytes,
+                      void* cuda_stream, double* x_final, double* sigma_final, uint32_t* steps_done,
+                      double* history, double* p95_ttft_ms, double* p95_e2e_ms, uint8_t* route) {
+  if (!sim || !cfg || !x0 || !workspace || !x_final || !sigma_final || n_tuners == 0)
+    return GORGO_ERR_INVALID_ARG;
+  if (!sim->has_trace) return GORGO_ERR_NO_TRACE;
+  const uint32_t K = sim->m.K, T = cfg->n_tuned, P = n_tuners;
+  const uint64_t N = sim->tr.n_req;
+  if (T == 0 || T > K || !cfg->tuned || !cfg->lo || !cfg->hi || cfg->window == 0 || cfg->hop == 0 ||
+      cfg->window > window_max() || (cfg->n_draw_steps > 0 && !z))
+    return GORGO_ERR_INVALID_ARG;
+  if (!(cfg->sigma0 > 0.0) || !std::isfinite(cfg->sigma0) || !(cfg->sigma_up > 1.0) ||
+      !std::isfinite(cfg->sigma_up) || !finite_nonneg(cfg->time_scale))
+    return GORGO_ERR_NONFINITE_PARAM;
+  if (!all_finite(x0, (uint64_t)P * K) || !all_finite(z, (uint64_t)P * cfg->n_draw_steps * T))
+    return GORGO_ERR_NONFINITE_PARAM;
+  for (uint32_t k = 0; k < T; ++k) {
+    if (cfg->tuned[k] >= K) return GORGO_ERR_INVALID_ARG;
+    if (!(cfg->lo[k] > 0.0) || !(cfg->hi[k] >= cfg->lo[k]) || !std::isfinite(cfg->hi[k]))
+      return GORGO_ERR_INVALID_ARG;
+    for (uint32_t p = 0; p < P; ++p)
+      if (!(x0[(size_t)p * K + cfg->tuned[k]] > 0.0)) return GORGO_ERR_INVALID_ARG;   // ln(x) of Eq. 4
+  }
+  if ((uintptr_t)workspace % kAlign) return GORGO_ERR_INVALID_ARG;
+  const WsLayout w = make_ws(sim, P, true);                 // every tuner's state stays resident
+  if (w.total > workspace_bytes) return GORGO_ERR_WORKSPACE_TOO_SMALL;
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* base = static_cast<unsigned char*>(workspace);
+  double* d_params = reinterpret_cast<double*>(base + w.params);
+  double* d_rtt = reinterpret_cast<double*>(base + w.rtt);
+  int32_t* d_status = reinterpret_cast<int32_t*>(base + w.status);
+  double* d_p95 = reinterpret_cast<double*>(base + w.p95);
+  double* d_ttft = reinterpret_cast<double*>(base + w.ttft);
+  double* d_e2e = reinterpret_cast<double*>(base + w.e2e);
+  if (cudaMemcpyAsync(d_rtt, sim->rtt.data(), sim->rtt.size() * 8, cudaMemcpyHostToDevice, st) !=
+          cudaSuccess ||
+      cudaMemsetAsync(d_status, 0, (size_t)P * 4, st) != cudaSuccess)
+    return GORGO_ERR_CUDA;
+  if (launch_reset(base + w.masks, (uint64_t)P * w.mask_stride,
+                   reinterpret_cast<uint32_t*>(base + w.exp_head), (uint64_t)P * N, base + w.states,
+                   w.st, sim->m, P, st) != cudaSuccess)
+    return GORGO_ERR_CUDA;
+
+  std::vector<double> parent(x0, x0 + (size_t)P * K), live(parent), f_parent(P, 0.0), sigma(P, cfg->sigma0),
+      value(P, 0.0);
+  const double down = std::pow(cfg->sigma_up, -0.25);   // one success in five keeps sigma in place
+  const uint32_t hist_w = 4 + 2 * T;
+  uint64_t done = 0;
+  uint32_t step = 0;
+  while (done < N) {
+    const uint64_t count = std::min<uint64_t>(done == 0 ? cfg->window : cfg->hop, N - done);
+    if (cudaMemcpyAsync(d_params, live.data(), (size_t)P * K * 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+    ReplayArgs a = {};
+    a.m = sim->m; a.tr = sim->tr; a.scale = cfg->time_scale;
+    a.first = (uint32_t)done; a.count = (uint32_t)count; a.check_order = 1;
+    a.poll_limit = sim->poll_limit; a.ring_polls = sim->ring_polls;
+    a.probe_off = sim->probe_off; a.scout_off = sim->scout_off;
+    a.rtt = d_rtt; a.params = d_params;
+    a.masks = base + w.masks; a.mask_stride = w.mask_stride;
+    a.states = base + w.states; a.lay = w.st;
+    a.evict_lists = reinterpret_cast<uint4*>(base + w.lists);
+    a.exp_head = reinterpret_cast<uint32_t*>(base + w.exp_head);
+    a.exp_rec = reinterpret_cast<uint4*>(base + w.exp_rec);
+    a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
+    a.route_log = route ? route : base + w.route_log;
+    a.route_log_stride = N;
+    if (attach_speeds(sim, base, w, st, &a) != GORGO_OK) return GORGO_ERR_CUDA;
+    a.ttft_out = d_ttft + done; a.e2e_out = d_e2e + done; a.out_stride = N;   // request r at [p*N + r]
+    a.status_out = d_status;
+    if (launch_replay(a, P, st) != cudaSuccess) return GORGO_ERR_CUDA;
+    done += count;
+    // a strategy step where a full window ends and draws are left
+    if (done < cfg->window || (done - cfg->window) % cfg->hop != 0 || step >= cfg->n_draw_steps)
+      continue;                                   // (`live` is unchanged: nothing to wait for)
+    WindowArgs wa = {};
+    wa.values = d_ttft + (done - cfg->window); wa.stride = N;
+    wa.window = cfg->window; wa.hop = cfg->hop; wa.n_win = 1;
+    wa.win_p95 = d_p95; wa.win_stride = 1;
+    wa.best = d_p95 + P; wa.best_win = nullptr;
+    if (launch_window(wa, P, st) != cudaSuccess) return GORGO_ERR_CUDA;
+    if (cudaMemcpyAsync(value.data(), d_p95 + P, (size_t)P * 8, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+    for (uint32_t p = 0; p < P; ++p) {
+      double* par = parent.data() + (size_t)p * K;
+      double* lv = live.data() + (size_t)p * K;
+      bool accept = false;
+      if (step == 0) {
+        f_parent[p] = value[p];                             // the start weights themselves
+      } else {
+        accept = value[p] < f_parent[p];
+        if (accept) {
+          std::copy(lv, lv + K, par);
+          f_parent[p] = value[p];
+          sigma[p] *= cfg->sigma_up;
+        } else {
+          sigma[p] *= down;
+        }
+      }
+      std::copy(par, par + K, lv);
+      for (uint32_t k = 0; k < T; ++k) {
+        const double zk = z[((size_t)p * cfg->n_draw_steps + step) * T + k];
+        const double stepv = sigma[p] * zk;
+        double v = std::exp(std::log(par[cfg->tuned[k]]) + stepv);     // Eq. 4
+        if (v < cfg->lo[k]) v = cfg->lo[k];
+        if (v > cfg->hi[k]) v = cfg->hi[k];
+        lv[cfg->tuned[k]] = v;
+      }
+      if (history) {
+        double* h = history + ((size_t)p * cfg->n_draw_steps + step) * hist_w;
+        h[0] = value[p]; h[1] = accept ? 1.0 : 0.0; h[2] = sigma[p]; h[3] = f_parent[p];
+        for (uint32_t k = 0; k < T; ++k) { h[4 + k] = par[cfg->tuned[k]]; h[4 + T + k] = lv[cfg->tuned[k]]; }
+      }
+    }
+    ++step;
+  }
+  if (p95_ttft_ms && p95_e2e_ms) {
+    SelectArgs sa = {};
+    sa.ttft = d_ttft; sa.e2e = d_e2e; sa.stride = N; sa.n = (uint32_t)N;
+    sa.p95_ttft = d_p95; sa.p95_e2e = d_p95 + P;
+    if (launch_select(sa, P, st) != cudaSuccess) return GORGO_ERR_CUDA;
+    if (cudaMemcpyAsync(p95_ttft_ms, d_p95, (size_t)P * 8, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(p95_e2e_ms, d_p95 + P, (size_t)P * 8, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+  }
+  std::vector<int32_t> h_status(P, 0);
+  if (cudaMemcpyAsync(h_status.data(), d_status, (size_t)P * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return GORGO_ERR_CUDA;
+  std::copy(parent.begin(), parent.end(), x_final);
+  std::copy(sigma.begin(), sigma.end(), sigma_final);
+  if (steps_done) *steps_done = step;
+  for (uint32_t p = 0; p < P; ++p)
+    if (h_status[p] != 0) return h_status[p] == -8 ? GORGO_ERR_OUT_OF_ORDER : GORGO_ERR_DEVICE_LIMIT;
   return GORGO_OK;
 }
 

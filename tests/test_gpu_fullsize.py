@@ -54,3 +54,40 @@ def test_sweep_full_size_most_and_least_saturated_scale():
 
 def test_largest_full_size_in_waves():
     check_full("largest", 0.5, n_oracle=4)
+
+
+def test_longctx_full_size_cache_digests_every_65536_requests():
+    """One candidate of the full-size long-context workload routed in batches of 2^16 requests on a
+    persistent state; after every batch the digests of all replica caches equal the oracle's at
+    the same request, so a divergence would be pinned down to one batch."""
+    import torch
+    from oracle import gorgo_oracle as O
+    from paper_2602_11688_b200 import binding as gb
+    w = W.make_workload("longctx")
+    N, R = w.n_requests, w.spec.n_replicas
+    weights = w.params[3]
+    sim = gb.GorgoSim(w)
+    rc, nbytes = gb.gorgo_state_bytes(sim.h)
+    assert rc == gb.GORGO_OK
+    state = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    assert gb.gorgo_sim_reset(sim.h, state, sim.stream) == gb.GORGO_OK
+    oracle = O.Oracle.from_workload(w)
+    step = 1 << 16
+    route = torch.empty(step, dtype=torch.uint8, device="cuda")
+    digest = torch.empty((R, 2), dtype=torch.uint64, device="cuda")
+    checkpoints = 0
+    for first in range(0, N, step):
+        count = min(step, N - first)
+        rc = gb.gorgo_route_batch(sim.h, weights, 0.5, first, count, state, sim.stream, route)
+        assert rc == gb.GORGO_OK
+        assert gb.gorgo_state_digest(sim.h, state, sim.stream, digest) == gb.GORGO_OK
+        torch.cuda.synchronize()
+        ref = oracle.run(weights, 0.5, count=count)
+        assert (route[:count].cpu().numpy() == ref.route).all(), f"routes differ in [{first}, {first + count})"
+        assert digest.cpu().numpy().tolist() == oracle.digest().tolist(), \
+            f"cache digests differ after request {first + count}"
+        checkpoints += 1
+    rc, seen = gb.gorgo_state_status(sim.h, state, sim.stream)
+    assert rc == gb.GORGO_OK and seen == N and checkpoints == -(-N // step)
+    oracle.close()
+    sim.close()

@@ -142,3 +142,74 @@ def test_es_run_rejects_bad_arguments():
         assert gb.gorgo_es_run(sim.h, x0=good, **kw)[0] == gb.GORGO_OK
     finally:
         sim.close()
+
+
+@pytest.mark.parametrize("workload,kw,scale,steps,start,accepts", [
+    ("tiny", dict(n_requests=900, cache_blocks=300), 1.0, 40, [0.5, 1.0, 0.1], False),
+    ("regions", dict(n_requests=1500, cache_blocks=500, population=4), 1.0, 40, [2.0, 1.0, 0.05], True),
+])
+def test_online_tuning_inside_one_replay_matches_oracle(workload, kw, scale, steps, start, accepts):
+    """The paper's online tuner: weights change every 32 requests inside one replay.  Three tuners
+    with their own draws run side by side in the library; each is compared with the oracle's
+    chunked replay: every route, the whole strategy trajectory, final weights and p95s."""
+    import torch
+    from oracle import gorgo_oracle as O
+    from oracle import gorgo_tuning as T
+    from paper_2602_11688_b200 import binding as gb
+    w = W.make_workload(workload, **kw)
+    N, K = w.n_requests, w.n_params
+    P = 3
+    rng = np.random.default_rng(11)
+    x0 = np.tile(np.array(start + [1.0] * (K - 3)), (P, 1))
+    tuned, lo, hi = [0, 2], [0.05, 0.05], [2.0, 0.5]
+    z = rng.normal(size=(P, steps, 2))
+    sim = gb.GorgoSim(w)
+    sim.ensure_workspace(P)
+    route = torch.empty((P, N), dtype=torch.uint8, device="cuda")
+    rc, x_fin, sig, done, hist, pt, pe = gb.gorgo_tune_online(
+        sim.h, x0=x0, z=z, tuned=tuned, lo=lo, hi=hi, sigma0=0.5, sigma_up=1.5,
+        workspace=sim.workspace, stream=sim.stream, time_scale=scale, route=route)
+    assert rc == gb.GORGO_OK, gb.gorgo_strerror(rc)
+    torch.cuda.synchronize()
+    route = route.cpu().numpy()
+    for p in range(P):
+        o = O.Oracle.from_workload(w)
+        routes, e2e = [], []
+
+        def run_chunk(weights, count):
+            r = o.run(np.array(weights), scale, count=count)
+            routes.append(r.route); e2e.extend(r.e2e)
+            return list(r.ttft)
+        ttft, schedule, h = T.online_tune(run_chunk, N, list(x0[p]), tuned, lo, hi, 0.5, 1.5,
+                                          z[p].tolist())
+        assert done == len(h) == min(steps, T.window_count(N))
+        assert (route[p] == np.concatenate(routes)).all()
+        for k, (value, acc, sigma, f_par, par, live) in enumerate(h):
+            assert hist[p, k].tolist() == [value, 1.0 if acc else 0.0, sigma, f_par] + par + live, (p, k)
+        assert [x_fin[p, i] for i in tuned] == h[-1][4] and sig[p] == h[-1][2]
+        assert pt[p] == O.p95(np.array(ttft)) and pe[p] == O.p95(np.array(e2e))
+        o.close()
+    if accepts:                                         # on this case some offspring do get accepted
+        assert any(hist[p, 1:done, 1].sum() > 0 for p in range(P))
+    sim.close()
+
+
+def test_online_tuning_rejects_bad_arguments():
+    from paper_2602_11688_b200 import binding as gb
+    w = W.make_workload("tiny", n_requests=300, cache_blocks=100)
+    sim = gb.GorgoSim(w)
+    sim.ensure_workspace(1)
+    x0 = np.array([[0.5, 1.0, 0.1]])
+    z = np.zeros((1, 4, 2))
+    ok = dict(x0=x0, z=z, tuned=[0, 2], lo=[0.05, 0.05], hi=[2.0, 0.5], sigma0=0.5, sigma_up=1.5,
+              workspace=sim.workspace, stream=sim.stream)
+    assert gb.gorgo_tune_online(sim.h, **ok)[0] == gb.GORGO_OK
+    assert gb.gorgo_tune_online(sim.h, **{**ok, "sigma_up": 1.0})[0] == gb.GORGO_ERR_NONFINITE_PARAM
+    assert gb.gorgo_tune_online(sim.h, **{**ok, "lo": [0.0, 0.05]})[0] == gb.GORGO_ERR_INVALID_ARG
+    assert gb.gorgo_tune_online(sim.h, **{**ok, "tuned": [0, 7]})[0] == gb.GORGO_ERR_INVALID_ARG
+    assert gb.gorgo_tune_online(sim.h, **{**ok, "window": 4096})[0] == gb.GORGO_ERR_INVALID_ARG
+    assert gb.gorgo_tune_online(sim.h, **{**ok, "x0": np.array([[0.5, 1.0, -0.1]])})[0] == gb.GORGO_ERR_INVALID_ARG
+    import torch
+    small = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    assert gb.gorgo_tune_online(sim.h, **{**ok, "workspace": small})[0] == gb.GORGO_ERR_WORKSPACE_TOO_SMALL
+    sim.close()

@@ -112,3 +112,91 @@ def test_es_ties_go_to_the_lowest_index_and_equal_does_not_beat():
     cand = [0.5 * math.exp(0.1), 0.5 * math.exp(-0.1), 0.5 * math.exp(0.1)]
     fs = [obj2([c]) for c in cand]
     assert x2[0] == pytest.approx(cand[fs.index(min(fs))])
+
+
+# ------------------------------------------------------------------ online tuning (one replay)
+def _stub_chunks(values):
+    """run_chunk stand-in: hands out prescribed TTFTs and records (weights, count) per chunk."""
+    it, calls = iter(values), []
+
+    def run_chunk(weights, count):
+        calls.append((list(weights), count))
+        return [next(it) for _ in range(count)]
+    return run_chunk, calls
+
+
+def test_online_steps_follow_the_papers_sample_count():
+    # step k happens after 128 + (k-1)*32 requests: the 18th after 672 samples (convergence figure)
+    n = 700
+    run_chunk, calls = _stub_chunks([1.0] * n)
+    z = [[0.1, -0.1]] * 40
+    ttft, schedule, history = T.online_tune(run_chunk, n, [0.5, 1.0, 0.1], [0, 2], [0.05, 0.05],
+                                            [2.0, 0.5], 0.5, 1.5, z)
+    assert [c for _, c in calls] == [128] + [32] * 17 + [700 - 672]
+    assert len(history) == T.window_count(n) == 18 and len(ttft) == n
+    assert sum(c for _, c in calls[:18]) == 672
+    # weights change only between chunks, and the chunk after step k runs under step k's offspring
+    for k, h in enumerate(history):
+        assert [calls[k + 1][0][i] for i in (0, 2)] == h[5]
+        assert calls[k + 1][0][1] == 1.0                      # the untuned weight stays
+    assert schedule == [c[0] for c in calls]
+    # fewer draws than windows: the last offspring stays in force
+    run_chunk, calls = _stub_chunks([1.0] * n)
+    _, _, history = T.online_tune(run_chunk, n, [0.5, 1.0, 0.1], [0, 2], [0.05, 0.05], [2.0, 0.5],
+                                  0.5, 1.5, z[:3])
+    assert len(history) == 3 and all(c[0] == calls[3][0] for c in calls[3:])
+
+
+def test_online_accept_reject_and_sigma():
+    # window values (constant chunks make the p95 of a window the maximum of its four hops ...
+    # here every chunk is flat, and levels are chosen so that the window value is known):
+    # chunk levels: first window 10; then hops 10, 4, 4, 4, 4, 9 -> window values
+    # 10 (step 1: start weights), 10 (not < 10: rejected), 10, 10, 10 (still holds a 10-hop), ...
+    levels = [10.0] * 128 + [10.0] * 32 + [4.0] * 128 + [9.0] * 32 + [1.0] * 32
+    run_chunk, calls = _stub_chunks(levels)
+    z = [[0.3]] * 20
+    ttft, schedule, hist = T.online_tune(run_chunk, len(levels), [0.5], [0], [0.05], [2.0], 0.5, 1.5, z)
+    values = [h[0] for h in hist]
+    assert values == T.window_p95(levels)                      # each step sees the last 128 TTFTs
+    assert values[:2] == [10.0, 10.0] and values[5] == 4.0
+    accepted = [h[1] for h in hist]
+    assert accepted[0] is False and accepted[1] is False       # step 1 only scores the start weights
+    first_acc = accepted.index(True)
+    assert values[first_acc] < 10.0 and all(v >= 10.0 for v in values[1:first_acc])
+    # sigma: x a after an accepted step, x a^(-1/4) after a rejected one (step 1 changes nothing)
+    sigma = 0.5
+    parent_f = values[0]
+    for k, h in enumerate(hist[1:], start=1):
+        if h[0] < parent_f:
+            sigma *= 1.5; parent_f = h[0]
+        else:
+            sigma *= 1.5 ** -0.25
+        assert h[2] == sigma and h[3] == parent_f and h[1] == (h[0] == parent_f and hist[k - 1][3] != parent_f)
+    # an accepted step makes the offspring in force the new parent; the next offspring mutates it
+    k = first_acc
+    assert hist[k][4] == hist[k - 1][5]
+    assert hist[k][5] == T.mutate(hist[k][4], hist[k][2], z[k], [0.05], [2.0])
+
+
+def test_online_with_clamped_weights_is_the_plain_replay():
+    # lo = hi pins every tuned weight: the schedule never changes and the chunked replay must be
+    # the one-shot replay, request for request
+    from oracle import gorgo_oracle as O
+    from paper_2602_11688_b200 import workloads as W
+    w = W.make_workload("tiny", n_requests=500, cache_blocks=300)
+    x0 = [0.7, 1.0, 0.3]
+    o = O.Oracle.from_workload(w)
+    chunks = []
+
+    def run_chunk(weights, count):
+        r = o.run(np.array(weights), 1.0, count=count)
+        chunks.append(r)
+        return list(r.ttft)
+    rng = np.random.default_rng(0)
+    z = rng.normal(size=(20, 2)).tolist()
+    ttft, schedule, hist = T.online_tune(run_chunk, w.n_requests, x0, [0, 2], [0.7, 0.3], [0.7, 0.3],
+                                         0.5, 1.5, z)
+    assert all(s == x0 for s in schedule) and len(hist) == T.window_count(500)
+    plain, *_ = O.replay(w, np.array(x0), 1.0)
+    assert ttft == list(plain.ttft)
+    assert np.concatenate([c.route for c in chunks]).tolist() == plain.route.tolist()
