@@ -55,6 +55,7 @@ struct Replica {
     std::unordered_map<uint64_t, Key> cache;              // block id -> recency key
     std::map<Key, uint64_t, KeyEvictsBefore> order;       // recency key -> block id
     std::vector<double> free_at;                          // per slot: time it becomes free
+    std::vector<uint64_t> kv;                             // per slot: KV tokens of its newest request
     std::multiset<std::pair<double, uint64_t>> inflight;  // (finish time, input tokens)
     int64_t load = 0;                                     // sum of in-flight input tokens
 };
@@ -92,6 +93,15 @@ struct Oracle {
     // fleet): per-replica prefill time per token and time per output token; empty = the uniform
     // constants.  The cost model does not see them (the proxy has no such signal).
     std::vector<double> rep_prefill_ms, rep_tpot_ms;
+    // Continuous batching "bounded by max concurrency and KV budget" (Section 2.2), and the decode
+    // slow-down of a fuller batch that makes concentrating traffic on one replica cost E2E latency
+    // (Section 5, Appendix D).  Both are this project's statement, off by default:
+    //  * decode_slowdown g >= 0: a request's time per output token is tpot * (1 + g*(b-1)), b = the
+    //    replica's busy slots at its first-token time, itself included;
+    //  * kv_budget > 0: a request needing in+out tokens of KV starts only once the newest requests of
+    //    the other busy slots hold at most kv_budget - need tokens (it runs alone whatever its size).
+    double decode_slowdown = 0.0;
+    uint64_t kv_budget = 0;
 };
 
 }  // namespace
@@ -129,7 +139,7 @@ void* gorgo_oracle_create(const gorgo_oracle_config* cfg, const double* rtt_ms,
     o->off.assign(hash_off, hash_off + n_requests + 1);
     o->ids.assign(hash_ids, hash_ids + hash_off[n_requests]);
     o->rep.resize(o->R);
-    for (auto& rp : o->rep) rp.free_at.assign(o->S, 0.0);
+    for (auto& rp : o->rep) { rp.free_at.assign(o->S, 0.0); rp.kv.assign(o->S, 0); }
     return o;
 }
 
@@ -140,7 +150,7 @@ void gorgo_oracle_reset(void* h) {
     Oracle* o = static_cast<Oracle*>(h);
     for (auto& rp : o->rep) {
         rp.cache.clear(); rp.order.clear(); rp.inflight.clear();
-        rp.free_at.assign(o->S, 0.0); rp.load = 0;
+        rp.free_at.assign(o->S, 0.0); rp.kv.assign(o->S, 0); rp.load = 0;
     }
     o->next = 0;
     std::memset(o->stats, 0, sizeof(o->stats));
@@ -240,15 +250,40 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
         uint32_t slot = 0;
         for (uint32_t s = 1; s < o->S; ++s)
             if (rp.free_at[s] < rp.free_at[slot]) slot = s;
-        const double start = std::max(arrive, rp.free_at[slot]);
+        double start = std::max(arrive, rp.free_at[slot]);
+        const uint32_t out = o->out_tok[r];
+        const uint64_t need = in + out;                    // KV tokens the request holds while it runs
+        if (o->kv_budget > 0) {
+            // admission under the KV budget: wait for other slots to finish until the request fits
+            for (;;) {
+                uint64_t usage = 0;
+                double next_free = 0.0;
+                bool any_busy = false;
+                for (uint32_t s = 0; s < o->S; ++s) {
+                    if (s == slot || !(rp.free_at[s] > start)) continue;
+                    usage += rp.kv[s];
+                    if (!any_busy || rp.free_at[s] < next_free) next_free = rp.free_at[s];
+                    any_busy = true;
+                }
+                if (!any_busy || usage + need <= o->kv_budget) break;
+                start = next_free;
+            }
+        }
         const double prefill =
             (o->rep_prefill_ms.empty() ? o->prefill_ms : o->rep_prefill_ms[best]) * (double)unc[best];
         const double first = start + prefill;
-        const uint32_t out = o->out_tok[r];
-        const double decode = (o->rep_tpot_ms.empty() ? o->tpot_ms : o->rep_tpot_ms[best]) *
-                              (double)(out > 0 ? out - 1 : 0);
+        double tpot = o->rep_tpot_ms.empty() ? o->tpot_ms : o->rep_tpot_ms[best];
+        if (o->decode_slowdown > 0.0) {
+            uint32_t busy = 1;                             // slots busy at the first token, this one included
+            for (uint32_t s = 0; s < o->S; ++s)
+                if (s != slot && rp.free_at[s] > first) ++busy;
+            const double g = 1.0 + o->decode_slowdown * (double)(busy - 1);
+            tpot = tpot * g;
+        }
+        const double decode = tpot * (double)(out > 0 ? out - 1 : 0);
         const double finish = first + decode;
         rp.free_at[slot] = finish;
+        rp.kv[slot] = need;
         rp.inflight.emplace(finish, in);
         rp.load += (int64_t)in;
 
@@ -292,6 +327,16 @@ int gorgo_oracle_set_replica_speeds(void* h, const double* prefill_ms_per_token,
     else o->rep_prefill_ms.clear();
     if (tpot_ms) o->rep_tpot_ms.assign(tpot_ms, tpot_ms + o->R);
     else o->rep_tpot_ms.clear();
+    return 0;
+}
+
+// Decode slow-down per additional busy slot (>= 0, finite) and KV budget in tokens per replica
+// (0 = unlimited).  Returns 0, or -1 for a bad value.
+int gorgo_oracle_set_service_model(void* h, double decode_slowdown, uint64_t kv_budget_tokens) {
+    Oracle* o = static_cast<Oracle*>(h);
+    if (!(decode_slowdown >= 0.0 && std::isfinite(decode_slowdown))) return -1;
+    o->decode_slowdown = decode_slowdown;
+    o->kv_budget = kv_budget_tokens;
     return 0;
 }
 

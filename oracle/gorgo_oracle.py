@@ -59,6 +59,8 @@ def _load():
         lib.gorgo_oracle_set_policy.argtypes = [vp, C.c_uint32, vp]
         lib.gorgo_oracle_set_replica_speeds.restype = C.c_int
         lib.gorgo_oracle_set_replica_speeds.argtypes = [vp, vp, vp]
+        lib.gorgo_oracle_set_service_model.restype = C.c_int
+        lib.gorgo_oracle_set_service_model.argtypes = [vp, C.c_double, C.c_uint64]
         lib.gorgo_oracle_position.restype = u64
         lib.gorgo_oracle_position.argtypes = [vp]
         _lib = lib
@@ -145,6 +147,13 @@ class Oracle:
         if self._lib.gorgo_oracle_set_replica_speeds(self._h, _ptr(a), _ptr(b)) != 0:
             raise ValueError("replica speeds must be finite and >= 0")
 
+    def set_service_model(self, decode_slowdown: float = 0.0, kv_budget_tokens: int = 0):
+        """Decode slow-down per additional busy slot and KV budget per replica in tokens
+        (0 = unlimited); both off by default."""
+        if self._lib.gorgo_oracle_set_service_model(self._h, float(decode_slowdown),
+                                                    int(kv_budget_tokens)) != 0:
+            raise ValueError("decode slow-down must be finite and >= 0")
+
     @property
     def position(self) -> int:
         return int(self._lib.gorgo_oracle_position(self._h))
@@ -194,7 +203,8 @@ class Oracle:
 
 
 def replay(workload, w, scale: float = 1.0, detail: bool = False, queue_in_requests: bool = False,
-           forced_route=None, rep_prefill_ms=None, rep_tpot_ms=None):
+           forced_route=None, rep_prefill_ms=None, rep_tpot_ms=None, decode_slowdown: float = 0.0,
+           kv_budget_tokens: int = 0):
     """Full replay of one candidate from the empty state: (RunResult, p95_ttft, p95_e2e,
     digest[R,2], stats[4])."""
     o = Oracle.from_workload(workload)
@@ -203,6 +213,8 @@ def replay(workload, w, scale: float = 1.0, detail: bool = False, queue_in_reque
             o.set_policy(queue_in_requests, forced_route)
         if rep_prefill_ms is not None or rep_tpot_ms is not None:
             o.set_replica_speeds(rep_prefill_ms, rep_tpot_ms)
+        if decode_slowdown or kv_budget_tokens:
+            o.set_service_model(decode_slowdown, kv_budget_tokens)
         res = o.run(w, scale, detail=detail)
         return res, p95(res.ttft), p95(res.e2e), o.digest(), o.stats()
     finally:
