@@ -171,6 +171,25 @@ int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
 int gorgo_sim_set_replica_speeds(gorgo_sim_t *sim, const double *prefill_ms_per_token,
                                  const double *tpot_ms);
 
+/* Extended service model (the paper's Section 2.2 describes continuous batching as "bounded by
+ * max concurrency and KV budget"; its Section 5 and Appendix D report that concentrating traffic
+ * on one replica lowers TTFT but inflates end-to-end latency).  Both parts are this library's
+ * statement, off by default, and apply to every later replay of this simulator:
+ *   decode_slowdown g >= 0   a request's time per output token is tpot_i * (1 + g*(b-1)), where
+ *                            b counts the replica's slots that are busy at the request's
+ *                            first-token time, its own included (fixed at that time: the request
+ *                            neither speeds up later nor slows the requests already running);
+ *   kv_budget_tokens > 0     a request holds input + output tokens of KV while it runs.  On the
+ *                            slot that frees first it starts at the earliest time T >= arrival,
+ *                            T >= the slot's free time, at which the newest requests of the other
+ *                            slots still busy at T hold at most kv_budget_tokens minus its own
+ *                            need (T moves from one finish time of those slots to the next); once
+ *                            no other slot is busy it starts whatever its size.  0 = no budget.
+ * Only the service model changes (start, first-token and finish times); the score of Eq. 3 does
+ * not see it.  With g = 0 and no budget every result is bit-identical to the plain model.  A
+ * persistent state should keep one setting from reset to its last batch. */
+int gorgo_sim_set_service_model(gorgo_sim_t *sim, double decode_slowdown, uint64_t kv_budget_tokens);
+
 /* Population evaluation with one time scale per candidate (paper Section 3: the time between
  * requests is scaled linearly to move the load; its load sweep replays one trace at several
  * scales).  Candidate p is replayed with time_scales[p]; everything else is

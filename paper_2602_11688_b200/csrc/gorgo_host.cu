@@ -17,6 +17,8 @@ struct gorgo_sim {
   Model m;
   std::vector<double> rtt;
   std::vector<double> rep_prefill, rep_tpot;   // per-replica speeds; empty: the uniform constants
+  double decode_slowdown = 0.0;                // extended service model (0: off)
+  uint64_t kv_budget = 0;
   int device = 0;
   bool has_trace = false;
   TraceView tr = {};
@@ -86,6 +88,7 @@ StateLayout make_layout(const Model& m) {
   l.rep_off = o; o += (uint64_t)m.R * sizeof(RepState);
   const uint64_t rs = (uint64_t)m.R * m.S;
   l.slot_off = o; o += rs * 8;
+  l.slot_kv_off = o; o += rs * 8;
   l.bytes = align_up(o);
   return l;
 }
@@ -130,6 +133,8 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
 int attach_speeds(const gorgo_sim* sim, unsigned char* base, const WsLayout& w, cudaStream_t st,
                   ReplayArgs* a) {
   const uint32_t R = sim->m.R;
+  a->decode_slowdown = sim->decode_slowdown;
+  a->kv_budget = sim->kv_budget;
   double* d = reinterpret_cast<double*>(base + w.speeds);
   if (!sim->rep_prefill.empty()) {
     if (cudaMemcpyAsync(d, sim->rep_prefill.data(), R * 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
@@ -385,6 +390,13 @@ int gorgo_sim_set_replica_speeds(gorgo_sim_t* sim, const double* prefill_ms_per_
   else sim->rep_prefill.clear();
   if (tpot_ms) sim->rep_tpot.assign(tpot_ms, tpot_ms + R);
   else sim->rep_tpot.clear();
+  return GORGO_OK;
+}
+
+int gorgo_sim_set_service_model(gorgo_sim_t* sim, double decode_slowdown, uint64_t kv_budget_tokens) {
+  if (!sim || !finite_nonneg(decode_slowdown)) return GORGO_ERR_INVALID_ARG;
+  sim->decode_slowdown = decode_slowdown;
+  sim->kv_budget = kv_budget_tokens;
   return GORGO_OK;
 }
 

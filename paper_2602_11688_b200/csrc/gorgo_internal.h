@@ -66,6 +66,7 @@ struct Model {
 struct StateLayout {
   uint64_t rep_off;        // RepState[R]
   uint64_t slot_off;       // double[R*S]: time each slot frees (finish of its newest request)
+  uint64_t slot_kv_off;    // uint64[R*S]: KV tokens held by each slot's newest request
   uint64_t bytes;          // size of the block (multiple of 256)
 };
 
@@ -104,6 +105,10 @@ struct ReplayArgs {
   // [R] each) or null for the uniform constants of the model
   const double* rep_prefill_ms;
   const double* rep_tpot_ms;
+  // extended service model (0 = off): decode slow-down per additional busy slot, KV budget of a
+  // replica in tokens
+  double decode_slowdown;
+  unsigned long long kv_budget;
   // outputs, candidate p at + p*out_stride, request r at + (r-first); any may be null
   uint8_t* route_out;
   uint16_t* hit_out;

@@ -378,6 +378,7 @@ struct Ctx {
   uint32_t* lru_next;
   uint8_t* route_log;
   double* free_at;             // [R*S] time each slot frees (shared or global memory)
+  unsigned long long* slot_kv; // [R*S] KV tokens of each slot's newest request (global memory)
   volatile uint32_t* route;    // chosen replica of the current request
   volatile int32_t* status;    // first device-side limit hit by any warp
   // staging of the coming requests by the probe warp (kStageDepth stages + one of the cache warp)
@@ -640,14 +641,48 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
         PROF_LAP(3);
         const double bv = __longlong_as_double((long long)bk);   // the slot's free time
         const double arrive = __dadd_rn(t, sm.rtt[(size_t)rec.origin * R + istar]);
-        const double start = (bv > arrive) ? bv : arrive;
-        // (per-replica speeds, if any, only in the build that also carries the baseline switches)
+        double start = (bv > arrive) ? bv : arrive;
+        // (per-replica speeds and the extended service model only in the build that also carries
+        // the baseline switches)
+        const unsigned long long need_kv = (unsigned long long)in_tok + rec.out_tok;
+        if (kBaseline && a.kv_budget > 0) {
+          // admission under the KV budget: wait for other slots to finish until the request fits
+          const unsigned long long* kv = cx.slot_kv + (size_t)istar * S;
+          #pragma unroll 1
+          for (uint32_t round = 0; round <= S; ++round) {
+            unsigned long long usage = 0;
+            uint64_t nf = ~0ull;                       // earliest finish among the other busy slots
+            #pragma unroll 1
+            for (uint32_t s2 = lane; s2 < S; s2 += 32) {
+              const double f = fa[s2];
+              if (s2 != bs && f > start) {
+                usage += kv[s2];
+                nf = min(nf, (uint64_t)__double_as_longlong(f));
+              }
+            }
+            usage = warp_sum_u64(usage);
+            uint32_t none = kNone;
+            warp_argmin_key(nf, none);
+            if (nf == ~0ull || usage + need_kv <= a.kv_budget) break;
+            start = __longlong_as_double((long long)nf);
+          }
+        }
         const double pre_ms = (kBaseline && a.rep_prefill_ms) ? a.rep_prefill_ms[istar] : a.m.prefill_ms;
-        const double tok_ms = (kBaseline && a.rep_tpot_ms) ? a.rep_tpot_ms[istar] : a.m.tpot_ms;
+        double tok_ms = (kBaseline && a.rep_tpot_ms) ? a.rep_tpot_ms[istar] : a.m.tpot_ms;
         const double first = __dadd_rn(start, __dmul_rn(pre_ms, (double)unc));
+        if (kBaseline && a.decode_slowdown > 0.0) {
+          // a fuller batch decodes slower: busy slots at the first token, this one included
+          uint32_t busy = 0;
+          #pragma unroll 1
+          for (uint32_t s2 = lane; s2 < S; s2 += 32) busy += (s2 != bs && fa[s2] > first) ? 1u : 0u;
+          busy = __reduce_add_sync(kFull, busy);
+          const double g = __dadd_rn(1.0, __dmul_rn(a.decode_slowdown, (double)busy));
+          tok_ms = __dmul_rn(tok_ms, g);
+        }
         const uint32_t dec_tok = rec.out_tok > 0 ? rec.out_tok - 1 : 0;
         const double finish = __dadd_rn(first, __dmul_rn(tok_ms, (double)dec_tok));
         if (lane == 0) {
+          if (kBaseline && a.kv_budget > 0) cx.slot_kv[(size_t)istar * S + bs] = need_kv;
           free_at[(size_t)istar * S + bs] = finish;
           const size_t o = (size_t)p * a.out_stride + (s - a.first);
           if (a.route_out) a.route_out[o] = (uint8_t)istar;
@@ -1439,6 +1474,7 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
                              : a.evict_lists + (size_t)p * R * kListCap;
   }
   cx.mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
+  cx.slot_kv = reinterpret_cast<unsigned long long*>(st + a.lay.slot_kv_off);
   cx.exp_head = a.exp_head + (size_t)p * N;
   cx.exp_rec = a.exp_rec + (size_t)p * N;
   cx.lru_next = a.lru_next + (size_t)p * N;
@@ -1526,7 +1562,8 @@ __global__ void reset_states_kernel(unsigned char* states, StateLayout lay, uint
   }
   double* slot = reinterpret_cast<double*>(st + lay.slot_off);
   const uint32_t RS = R * S;
-  for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) slot[x] = 0.0;   // free from time 0
+  unsigned long long* kv = reinterpret_cast<unsigned long long*>(st + lay.slot_kv_off);
+  for (uint32_t x = threadIdx.x; x < RS; x += blockDim.x) { slot[x] = 0.0; kv[x] = 0; }   // free from time 0
 }
 
 // ------------------------------------------------------------------------------ select
@@ -1754,7 +1791,8 @@ cudaError_t launch_replay_tb(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
 
 template <typename MaskT>
 cudaError_t launch_replay_t(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st) {
-  if (a.queue_in_requests || a.forced_route || a.rep_prefill_ms || a.rep_tpot_ms)
+  if (a.queue_in_requests || a.forced_route || a.rep_prefill_ms || a.rep_tpot_ms ||
+      a.decode_slowdown > 0.0 || a.kv_budget > 0)
     return launch_replay_tb<MaskT, true>(a, n_cand, st);
   return launch_replay_tb<MaskT, false>(a, n_cand, st);
 }
