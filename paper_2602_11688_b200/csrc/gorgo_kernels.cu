@@ -1682,6 +1682,55 @@ __global__ void __launch_bounds__(kWindowThreads) window_p95_kernel(const Window
   }
 }
 
+// The same for windows of up to 256 values, without shared memory and without sorting: only the
+// largest W - k + 1 values matter for the k-th smallest (about 5 % of the window).  Every lane
+// holds its NR keys (values lane, lane+32, ...) in registers, sorted descending; the warp then
+// takes the maximum over the lanes' current tops W - k + 1 times (two reductions on the halves of
+// the 64-bit keys), each time popping it from the lowest lane that holds it.
+template <int NR>
+__global__ void __launch_bounds__(kWindowThreads) window_p95_select_kernel(const WindowArgs a) {
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+  const uint32_t warps = kWindowThreads / 32;
+  const uint32_t p = blockIdx.x;
+  const double* v = a.values + (size_t)p * a.stride;
+  double* out = a.win_p95 + (size_t)p * a.win_stride;
+  const uint32_t W = a.window;
+  const uint32_t takes = W - (uint32_t)((95ull * W + 99ull) / 100ull) + 1u;   // the answer is the takes-th largest
+  for (uint32_t j = blockIdx.y * warps + warp; j < a.n_win; j += gridDim.y * warps) {
+    const double* wv = v + (size_t)j * a.hop;
+    uint64_t k[NR];
+#pragma unroll
+    for (int i = 0; i < NR; ++i) {
+      const uint32_t idx = lane + 32u * i;
+      k[i] = idx < W ? key_of(wv[idx]) : 0ull;          // (0 is below the key of every double)
+    }
+    // sort the lane's keys descending (odd-even transposition over NR registers)
+#pragma unroll
+    for (int round = 0; round < NR; ++round) {
+#pragma unroll
+      for (int i = round & 1; i + 1 < NR; i += 2) {
+        const uint64_t hi = k[i] > k[i + 1] ? k[i] : k[i + 1];
+        const uint64_t lo = k[i] > k[i + 1] ? k[i + 1] : k[i];
+        k[i] = hi; k[i + 1] = lo;
+      }
+    }
+    uint64_t best = 0;
+    for (uint32_t t = 0; t < takes; ++t) {
+      const uint32_t hi = (uint32_t)(k[0] >> 32), lo = (uint32_t)k[0];
+      const uint32_t mh = __reduce_max_sync(kFull, hi);
+      const uint32_t ml = __reduce_max_sync(kFull, hi == mh ? lo : 0u);
+      best = ((uint64_t)mh << 32) | ml;
+      const unsigned owners = __ballot_sync(kFull, k[0] == best);
+      if (lane == (uint32_t)__ffs((int)owners) - 1u) {   // pop it from one lane
+#pragma unroll
+        for (int i = 0; i + 1 < NR; ++i) k[i] = k[i + 1];
+        k[NR - 1] = 0ull;
+      }
+    }
+    if (lane == 0) out[j] = value_of(best);
+  }
+}
+
 // Smallest window value of every candidate and the first window that attains it.
 __global__ void __launch_bounds__(256) window_best_kernel(const WindowArgs a) {
   const uint32_t p = blockIdx.x;
@@ -1926,7 +1975,12 @@ cudaError_t launch_window(const WindowArgs& a, uint32_t n_cand, cudaStream_t st)
     }
     const uint32_t groups_needed = (a.n_win + warps - 1) / warps;
     const uint32_t groups = groups_needed < 1024u ? groups_needed : 1024u;
-    window_p95_kernel<<<dim3(n_cand, groups), kWindowThreads, smem, st>>>(a, wpad);
+    const dim3 grid(n_cand, groups);
+    if (wpad <= 32) window_p95_select_kernel<1><<<grid, kWindowThreads, 0, st>>>(a);
+    else if (wpad == 64) window_p95_select_kernel<2><<<grid, kWindowThreads, 0, st>>>(a);
+    else if (wpad == 128) window_p95_select_kernel<4><<<grid, kWindowThreads, 0, st>>>(a);
+    else if (wpad == 256) window_p95_select_kernel<8><<<grid, kWindowThreads, 0, st>>>(a);
+    else window_p95_kernel<<<grid, kWindowThreads, smem, st>>>(a, wpad);
   }
   window_best_kernel<<<n_cand, 256, 0, st>>>(a);
   return cudaGetLastError();
