@@ -160,7 +160,7 @@ template <>
 __device__ __forceinline__ uint64_t mask_load<uint64_t>(const uint64_t* mask, uint32_t id) {
   return __ldcg(reinterpret_cast<const unsigned long long*>(mask) + id);
 }
-constexpr int kRegChunks = 2;     // request blocks held in registers: 2 x 32 = 64
+constexpr int kRegChunks = 3;     // request blocks held in registers: 3 x 32 = 96
 constexpr uint32_t kListCap = 256;     // pre-validated eviction victims kept per replica
 constexpr uint32_t kScouts = 2;        // scout warps per candidate (replicas split between them)
 constexpr int kScoutBatches = 1;       // touches examined per lane and scout round
@@ -189,7 +189,7 @@ struct Smem {
   volatile uint32_t* progress;    // [kCommitWarps] requests each commit warp has passed
   volatile uint32_t* abort_flag;  // a bounded wait ran out: the other waits stop too
   volatile uint32_t* jobs;        // requests handed to the commit warps
-  uint32_t* job;                  // [kJobRing] replica | stage << 8 | blocks << 16
+  uint2* job;                     // [kJobRing] (replica | stage << 8 | blocks << 16, offset of the request's ids)
   // hand-over between the route, service and expiry warps
   volatile uint32_t* routed;      // requests routed so far
   volatile uint32_t* serviced;    // [kServices] requests each service warp has passed (serviced and filed, or not its own)
@@ -1024,7 +1024,7 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
   // does a commit since its staged read share a block with request idx?  (prev: the latest earlier
   // request that shares a block with it)
   auto shares = [&](uint32_t prev, uint32_t idx) { return prev != kNone && prev + kWindow >= idx; };
-  uint32_t n = 0;                  // blocks of the current request
+  uint32_t n = 0, off_cur = 0;     // blocks of the current request, offset of its ids
 
   PROF_BEGIN();
   for (uint32_t r = a.first; r < end; ++r) {
@@ -1041,7 +1041,7 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
       } else {
         q_cur = fetch_ahead(req, r, end);
       }
-      n = q_cur.nblk;
+      n = q_cur.nblk; off_cur = q_cur.off;
       const bool sh = shares(q_cur.prev_share, r);
       uint32_t done_to = sh ? r : 0u;                         // requests < done_to must be committed
       if (!sh) {
@@ -1091,7 +1091,7 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
     PROF_LAP(1);
     const uint32_t istar = *cx.route;
     if (lane == 0) {
-      sm.job[r % kJobRing] = istar | (slot << 8) | (n << 16);
+      sm.job[r % kJobRing] = make_uint2(istar | (slot << 8) | (n << 16), off_cur);
       smem_order();
       *sm.jobs = r + 1;                                   // the commit warps may take request r
     }
@@ -1113,7 +1113,7 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
         }
         if (okk) {
           slot = ss;
-          n = meta.y & 0xFFFFu;
+          n = meta.y & 0xFFFFu; off_cur = meta.w;
           hand_over(slot, n);
           posted = true;
           PROF_ADD(14, 1);
@@ -1163,7 +1163,8 @@ __device__ __forceinline__ void commit_warp(const ReplayArgs& a, const Ctx<MaskT
     }
     smem_order();
     PROF_LAP(0);
-    const uint32_t job = sm.job[r % kJobRing];
+    const uint2 job2 = sm.job[r % kJobRing];
+    const uint32_t job = job2.x;
     const uint32_t istar = job & 0xFFu;
     if (istar % kCommitWarps != which) {                    // another warp's replica
       if (lane == 0) sm.progress[which] = r + 1;
@@ -1348,7 +1349,7 @@ __device__ __forceinline__ void commit_warp(const ReplayArgs& a, const Ctx<MaskT
         uint32_t id;
         MaskT mv;
         if (c < kStageBlocks) { id = sid[k]; mv = smk[k]; }
-        else { id = ids[req[r].off + k]; mv = mask_load<MaskT>(mask, id); }
+        else { id = ids[job2.y + k]; mv = 0; }     // beyond the stage: set the bit without looking
         if (!(mv & bit)) mask_set_bit<MaskT>(mask, id, bit);
       }
     }
@@ -1446,8 +1447,8 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
   sm.jobs = unext + 9;
   sm.serviced = unext + 10;                                // [kServices] (<= 2)
   sm.route_ring = unext + 12;                              // [kRouteRing]
-  sm.job = sm.route_ring + kRouteRing;                     // [kJobRing]
-  cx.evhit = sm.job + kJobRing;                            // [kHitRing]
+  sm.job = reinterpret_cast<uint2*>(sm.route_ring + kRouteRing);   // [kJobRing] (8-byte aligned: 4R + 12 + kRouteRing words after an aligned start)
+  cx.evhit = reinterpret_cast<uint32_t*>(sm.job + kJobRing);       // [kHitRing]
   sm.act = const_cast<uint32_t*>(cx.evhit) + kHitRing;
   sm.ring_head = sm.act + R;
   sm.ring_tail = sm.ring_head + R;
@@ -1509,7 +1510,7 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
   }
   if (threadIdx.x < kCommitWarps) sm.progress[threadIdx.x] = a.first;
   if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
-  if (threadIdx.x < kJobRing) sm.job[threadIdx.x] = 0;
+  if (threadIdx.x < kJobRing) sm.job[threadIdx.x] = make_uint2(0u, 0u);
   if (threadIdx.x < kHitRing) cx.evhit[threadIdx.x] = kNone;
   __syncthreads();
 
@@ -1807,7 +1808,7 @@ size_t replay_smem_bytes(ReplayArgs& a) {
   a.slots_in_smem = rs * 8 <= 40 * 1024 ? 1u : 0u;
   a.lists_in_smem = list_bytes <= 64 * 1024 ? 1u : 0u;
   size_t smem = (2 * (size_t)a.m.G * a.m.R + a.m.K + (2 + kExpRing) * (size_t)a.m.R) * sizeof(double) +
-                (9 * (size_t)a.m.R + 12 + kRouteRing + kJobRing + kHitRing) * sizeof(uint32_t) + 16 +
+                (9 * (size_t)a.m.R + 12 + kRouteRing + 2 * kJobRing + kHitRing) * sizeof(uint32_t) + 16 +
                 (kStageDepth + 2) * (sizeof(unsigned long long) + sizeof(uint4)) + 16 +
                 (kStageDepth + 1 + (kStageDepth + 2) * ((size_t)a.m.R + kStageBlocks)) * sizeof(uint32_t) +
                 8 + (kStageDepth + 2) * (size_t)a.m.R * sizeof(double) +
