@@ -171,6 +171,20 @@ int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
 int gorgo_sim_set_replica_speeds(gorgo_sim_t *sim, const double *prefill_ms_per_token,
                                  const double *tpot_ms);
 
+/* Time-varying network (paper Section 2.2: the proxy's network signal is an exponentially
+ * weighted moving average of an RTT probe sent every 30 s; its Section 4 shows the probes of one
+ * run).  `samples_ms` HOST [n_epochs][G][R]: the probe result of every epoch of `epoch_ms`
+ * milliseconds of (scaled) trace time, finite and >= 0.  A request that arrives at scaled time t
+ * belongs to epoch e = the largest k <= n_epochs-1 with k*epoch_ms <= t.  The score of Eq. 3 uses
+ * the proxy's signal of that epoch, ewma_0 = sample_0, ewma_e = ewma_{e-1} + alpha*(sample_e -
+ * ewma_{e-1}) (0 < alpha <= 1, three rounded operations, computed by this call); the delay the
+ * request experiences on its way to the engine is the epoch's probe itself.  A constant series
+ * gives bit-identical results to the static matrix of the configuration.  n_epochs = 0 restores
+ * the static matrix.  The series is copied; it applies to every later replay of this simulator
+ * (gorgo_workspace_bytes and gorgo_state_bytes grow by 16*n_epochs*G*R bytes: call them again). */
+int gorgo_sim_set_rtt_series(gorgo_sim_t *sim, uint32_t n_epochs, double epoch_ms, double alpha,
+                             const double *samples_ms);
+
 /* Extended service model (the paper's Section 2.2 describes continuous batching as "bounded by
  * max concurrency and KV budget"; its Section 5 and Appendix D report that concentrating traffic
  * on one replica lowers TTFT but inflates end-to-end latency).  Both parts are this library's

@@ -102,7 +102,21 @@ struct Oracle {
     //    the other busy slots hold at most kv_budget - need tokens (it runs alone whatever its size).
     double decode_slowdown = 0.0;
     uint64_t kv_budget = 0;
+    // Time-varying network (paper Section 2.2: the proxy's RTT signal is an exponentially weighted
+    // moving average of a probe sent every 30 s).  rtt_raw[e][g][i] is the probe result of epoch e,
+    // which is also the delay a request dispatched in that epoch experiences; rtt_ewma[e][g][i] is
+    // what the proxy believes during epoch e and puts into the score.  Empty = the static matrix.
+    std::vector<double> rtt_raw, rtt_ewma;
+    uint32_t n_epochs = 0;
+    double epoch_ms = 0.0;
 };
+
+// Epoch of (scaled) time t: the largest k in [0, n_epochs-1] with k * epoch_ms <= t.
+uint32_t epoch_of(const Oracle* o, double t) {
+    uint32_t k = 0;
+    while (k + 1 < o->n_epochs && (double)(k + 1) * o->epoch_ms <= t) ++k;
+    return k;
+}
 
 }  // namespace
 
@@ -182,6 +196,14 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
         const uint64_t n = o->off[r + 1] - o->off[r];
         const uint64_t* id = o->ids.data() + o->off[r];
         const uint64_t in = o->in_tok[r];
+        // the proxy's RTT signal and the delay of the network at this time
+        const double* rtt_signal = o->rtt.data() + (size_t)g * R;
+        const double* rtt_delay = rtt_signal;
+        if (o->n_epochs > 0) {
+            const size_t e = epoch_of(o, t);
+            rtt_signal = o->rtt_ewma.data() + (e * o->G + g) * R;
+            rtt_delay = o->rtt_raw.data() + (e * o->G + g) * R;
+        }
 
         for (uint32_t i = 0; i < R; ++i) {
             Replica& rp = o->rep[i];
@@ -198,7 +220,7 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
             double q = o->queue_in_requests ? (double)rp.inflight.size() : (double)rp.load;
             if (o->K != 3) q = q * w[3 + i];               // per-replica queue-load normaliser
             // Eq. 3 with explicit weights: three products, two sums, in this order
-            const double a = w[0] * o->rtt[(size_t)g * R + i];
+            const double a = w[0] * rtt_signal[i];
             const double b = w[1] * (double)unc[i];
             const double c = w[2] * q;
             cost[i] = (a + b) + c;
@@ -246,7 +268,7 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
         }
 
         // ---- service commit on the chosen replica ----
-        const double arrive = t + o->rtt[(size_t)g * R + best];
+        const double arrive = t + rtt_delay[best];
         uint32_t slot = 0;
         for (uint32_t s = 1; s < o->S; ++s)
             if (rp.free_at[s] < rp.free_at[slot]) slot = s;
@@ -337,6 +359,32 @@ int gorgo_oracle_set_service_model(void* h, double decode_slowdown, uint64_t kv_
     if (!(decode_slowdown >= 0.0 && std::isfinite(decode_slowdown))) return -1;
     o->decode_slowdown = decode_slowdown;
     o->kv_budget = kv_budget_tokens;
+    return 0;
+}
+
+// Probe results per epoch, samples[e][g][i] >= 0, one epoch every epoch_ms > 0 of (scaled) time,
+// smoothing factor 0 < alpha <= 1.  The proxy's signal is ewma_0 = s_0,
+// ewma_e = ewma_{e-1} + alpha * (s_e - ewma_{e-1}) (three rounded operations).  n_epochs = 0
+// restores the static matrix.  Returns 0, or -1 for a bad argument.
+int gorgo_oracle_set_rtt_series(void* h, uint32_t n_epochs, double epoch_ms, double alpha,
+                                const double* samples) {
+    Oracle* o = static_cast<Oracle*>(h);
+    if (n_epochs == 0) { o->n_epochs = 0; o->rtt_raw.clear(); o->rtt_ewma.clear(); return 0; }
+    if (!samples || !(epoch_ms > 0.0) || !std::isfinite(epoch_ms) || !(alpha > 0.0 && alpha <= 1.0)) return -1;
+    const size_t gr = (size_t)o->G * o->R;
+    for (size_t x = 0; x < n_epochs * gr; ++x)
+        if (!(samples[x] >= 0.0 && std::isfinite(samples[x]))) return -1;
+    o->rtt_raw.assign(samples, samples + n_epochs * gr);
+    o->rtt_ewma.assign(samples, samples + n_epochs * gr);
+    for (uint32_t e = 1; e < n_epochs; ++e)
+        for (size_t x = 0; x < gr; ++x) {
+            const double prev = o->rtt_ewma[(e - 1) * gr + x];
+            const double diff = samples[e * gr + x] - prev;
+            const double step = alpha * diff;
+            o->rtt_ewma[e * gr + x] = prev + step;
+        }
+    o->n_epochs = n_epochs;
+    o->epoch_ms = epoch_ms;
     return 0;
 }
 

@@ -59,6 +59,8 @@ def _load():
         lib.gorgo_oracle_set_policy.argtypes = [vp, C.c_uint32, vp]
         lib.gorgo_oracle_set_replica_speeds.restype = C.c_int
         lib.gorgo_oracle_set_replica_speeds.argtypes = [vp, vp, vp]
+        lib.gorgo_oracle_set_rtt_series.restype = C.c_int
+        lib.gorgo_oracle_set_rtt_series.argtypes = [vp, C.c_uint32, C.c_double, C.c_double, vp]
         lib.gorgo_oracle_set_service_model.restype = C.c_int
         lib.gorgo_oracle_set_service_model.argtypes = [vp, C.c_double, C.c_uint64]
         lib.gorgo_oracle_position.restype = u64
@@ -147,6 +149,18 @@ class Oracle:
         if self._lib.gorgo_oracle_set_replica_speeds(self._h, _ptr(a), _ptr(b)) != 0:
             raise ValueError("replica speeds must be finite and >= 0")
 
+    def set_rtt_series(self, samples=None, epoch_ms: float = 30_000.0, alpha: float = 0.3):
+        """Time-varying network: samples[e, g, i] = RTT probe of epoch e (also the delay of requests
+        dispatched in it); the score uses their EWMA.  None restores the static matrix."""
+        if samples is None:
+            self._lib.gorgo_oracle_set_rtt_series(self._h, 0, 0.0, 0.0, None)
+            return
+        s = np.ascontiguousarray(samples, dtype=np.float64)
+        assert s.ndim == 3 and s.shape[2] == self.R
+        if self._lib.gorgo_oracle_set_rtt_series(self._h, s.shape[0], float(epoch_ms), float(alpha),
+                                                 _ptr(s)) != 0:
+            raise ValueError("bad RTT series")
+
     def set_service_model(self, decode_slowdown: float = 0.0, kv_budget_tokens: int = 0):
         """Decode slow-down per additional busy slot and KV budget per replica in tokens
         (0 = unlimited); both off by default."""
@@ -204,7 +218,7 @@ class Oracle:
 
 def replay(workload, w, scale: float = 1.0, detail: bool = False, queue_in_requests: bool = False,
            forced_route=None, rep_prefill_ms=None, rep_tpot_ms=None, decode_slowdown: float = 0.0,
-           kv_budget_tokens: int = 0):
+           kv_budget_tokens: int = 0, rtt_series=None, epoch_ms: float = 30_000.0, alpha: float = 0.3):
     """Full replay of one candidate from the empty state: (RunResult, p95_ttft, p95_e2e,
     digest[R,2], stats[4])."""
     o = Oracle.from_workload(workload)
@@ -215,6 +229,8 @@ def replay(workload, w, scale: float = 1.0, detail: bool = False, queue_in_reque
             o.set_replica_speeds(rep_prefill_ms, rep_tpot_ms)
         if decode_slowdown or kv_budget_tokens:
             o.set_service_model(decode_slowdown, kv_budget_tokens)
+        if rtt_series is not None:
+            o.set_rtt_series(rtt_series, epoch_ms, alpha)
         res = o.run(w, scale, detail=detail)
         return res, p95(res.ttft), p95(res.e2e), o.digest(), o.stats()
     finally:

@@ -19,6 +19,9 @@ struct gorgo_sim {
   std::vector<double> rep_prefill, rep_tpot;   // per-replica speeds; empty: the uniform constants
   double decode_slowdown = 0.0;                // extended service model (0: off)
   uint64_t kv_budget = 0;
+  std::vector<double> rtt_raw, rtt_ewma;       // time-varying network, [n_epochs][G][R] each; empty: static
+  uint32_t n_epochs = 0;
+  double epoch_ms = 0.0;
   int device = 0;
   bool has_trace = false;
   TraceView tr = {};
@@ -95,7 +98,7 @@ StateLayout make_layout(const Model& m) {
 
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
-  uint64_t params, scales, rtt, speeds, status, p95, forced, draws, masks, states, lists, exp_head, exp_rec, lru_next,
+  uint64_t params, scales, rtt, speeds, status, p95, forced, draws, series, masks, states, lists, exp_head, exp_rec, lru_next,
       route_log, ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
@@ -112,6 +115,7 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.scales = o; o = align_up(o + res * 8);       // one time scale per candidate (optional)
   w.rtt = o; o = align_up(o + (uint64_t)m.G * m.R * 8);
   w.speeds = o; o = align_up(o + (uint64_t)m.R * 16);   // per-replica speeds (optional)
+  w.series = o; o = align_up(o + (uint64_t)s->n_epochs * m.G * m.R * 16);   // RTT series (optional)
   w.status = o; o = align_up(o + res * 4);
   w.p95 = o; o = align_up(o + res * 16);
   w.forced = o; o = align_up(o + N);          // baseline policies: one route per request
@@ -135,6 +139,15 @@ int attach_speeds(const gorgo_sim* sim, unsigned char* base, const WsLayout& w, 
   const uint32_t R = sim->m.R;
   a->decode_slowdown = sim->decode_slowdown;
   a->kv_budget = sim->kv_budget;
+  if (sim->n_epochs > 0) {
+    const size_t n = sim->rtt_raw.size();
+    double* ds = reinterpret_cast<double*>(base + w.series);
+    if (cudaMemcpyAsync(ds, sim->rtt_ewma.data(), n * 8, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ds + n, sim->rtt_raw.data(), n * 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return GORGO_ERR_CUDA;
+    a->rtt_ewma = ds; a->rtt_raw = ds + n;
+    a->n_epochs = sim->n_epochs; a->epoch_ms = sim->epoch_ms;
+  }
   double* d = reinterpret_cast<double*>(base + w.speeds);
   if (!sim->rep_prefill.empty()) {
     if (cudaMemcpyAsync(d, sim->rep_prefill.data(), R * 8, cudaMemcpyHostToDevice, st) != cudaSuccess)
@@ -390,6 +403,34 @@ int gorgo_sim_set_replica_speeds(gorgo_sim_t* sim, const double* prefill_ms_per_
   else sim->rep_prefill.clear();
   if (tpot_ms) sim->rep_tpot.assign(tpot_ms, tpot_ms + R);
   else sim->rep_tpot.clear();
+  return GORGO_OK;
+}
+
+int gorgo_sim_set_rtt_series(gorgo_sim_t* sim, uint32_t n_epochs, double epoch_ms, double alpha,
+                             const double* samples_ms) {
+  if (!sim) return GORGO_ERR_INVALID_ARG;
+  if (n_epochs == 0) {
+    sim->n_epochs = 0; sim->rtt_raw.clear(); sim->rtt_ewma.clear();
+    return GORGO_OK;
+  }
+  if (!samples_ms || !(epoch_ms > 0.0) || !std::isfinite(epoch_ms) || !(alpha > 0.0 && alpha <= 1.0) ||
+      n_epochs > (1u << 20))
+    return GORGO_ERR_INVALID_ARG;
+  const size_t gr = (size_t)sim->m.G * sim->m.R;
+  for (size_t x = 0; x < (size_t)n_epochs * gr; ++x)
+    if (!finite_nonneg(samples_ms[x])) return GORGO_ERR_INVALID_ARG;
+  sim->rtt_raw.assign(samples_ms, samples_ms + (size_t)n_epochs * gr);
+  sim->rtt_ewma.assign(samples_ms, samples_ms + (size_t)n_epochs * gr);
+  // the proxy's signal: ewma_e = ewma_{e-1} + alpha * (probe_e - ewma_{e-1}), three rounded operations
+  for (uint32_t e = 1; e < n_epochs; ++e)
+    for (size_t x = 0; x < gr; ++x) {
+      const double prev = sim->rtt_ewma[(e - 1) * gr + x];
+      const double diff = samples_ms[e * gr + x] - prev;
+      const double step = alpha * diff;
+      sim->rtt_ewma[e * gr + x] = prev + step;
+    }
+  sim->n_epochs = n_epochs;
+  sim->epoch_ms = epoch_ms;
   return GORGO_OK;
 }
 

@@ -105,6 +105,12 @@ struct ReplayArgs {
   // [R] each) or null for the uniform constants of the model
   const double* rep_prefill_ms;
   const double* rep_tpot_ms;
+  // time-varying network: per epoch the proxy's RTT signal (EWMA of the probes) and the probes
+  // themselves (the delay a request experiences), [n_epochs][G][R] each, device; null = static
+  const double* rtt_ewma;
+  const double* rtt_raw;
+  uint32_t n_epochs;
+  double epoch_ms;
   // extended service model (0 = off): decode slow-down per additional busy slot, KV budget of a
   // replica in tokens
   double decode_slowdown;

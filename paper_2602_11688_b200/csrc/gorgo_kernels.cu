@@ -412,6 +412,18 @@ __device__ __forceinline__ uint32_t wait_counter(volatile uint32_t* counter, uin
   return v;
 }
 
+// Epoch of the (scaled) time t under a time-varying network: the largest k in [0, n_epochs-1]
+// with k * epoch_ms <= t (a quotient as first guess, then the defining comparison).
+__device__ __forceinline__ uint32_t epoch_of(const ReplayArgs& a, double t) {
+  const double q = t / a.epoch_ms;
+  uint32_t k = q >= (double)(a.n_epochs - 1) ? a.n_epochs - 1 : (uint32_t)q;
+  #pragma unroll 1
+  while (k + 1 < a.n_epochs && __dmul_rn((double)(k + 1), a.epoch_ms) <= t) ++k;
+  #pragma unroll 1
+  while (k > 0 && __dmul_rn((double)k, a.epoch_ms) > t) --k;
+  return k;
+}
+
 // Route warp: the serial chain of a replay.  Per request it adds the queue term to the staged
 // part of the score of Eq. 3, takes the lowest-index argmin and posts the route.  Lane i (and
 // i+32) keeps replica i's in-flight signal in registers: tokens (or requests) dispatched there,
@@ -640,7 +652,10 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
         bs = warp_argmin_key(bk, bs);
         PROF_LAP(3);
         const double bv = __longlong_as_double((long long)bk);   // the slot's free time
-        const double arrive = __dadd_rn(t, sm.rtt[(size_t)rec.origin * R + istar]);
+        double delay = sm.rtt[(size_t)rec.origin * R + istar];
+        if (kBaseline && a.rtt_raw)        // time-varying network: the probe of the request's epoch
+          delay = a.rtt_raw[((size_t)epoch_of(a, t) * a.m.G + rec.origin) * R + istar];
+        const double arrive = __dadd_rn(t, delay);
         double start = (bv > arrive) ? bv : arrive;
         // (per-replica speeds and the extended service model only in the build that also carries
         // the baseline switches)
@@ -827,13 +842,13 @@ __device__ __forceinline__ void expiry_warp(const ReplayArgs& a, const Smem& sm,
 }
 
 // What a warp needs to know of a request ahead of time.
-struct Ahead { uint32_t off, nblk, prev_share, in_tok, origin; };
+struct Ahead { uint32_t off, nblk, prev_share, in_tok, origin; double ts; };
 __device__ __forceinline__ Ahead fetch_ahead(const ReqRec* req, uint32_t q, uint32_t end) {
-  Ahead h = {0u, 0u, kNone, 0u, 0u};
+  Ahead h = {0u, 0u, kNone, 0u, 0u, 0.0};
   if (q < end) {
     const ReqRec x = req[q];
     h.off = x.off; h.nblk = x.nblk; h.prev_share = x.prev_share; h.in_tok = x.in_tok;
-    h.origin = x.origin;
+    h.origin = x.origin; h.ts = x.ts_ms;
   }
   return h;
 }
@@ -889,12 +904,16 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
 // Stage the prefix hits of a request and the part of its score (Eq. 3) that depends on them:
 // ab_i = (w_net * RTT[g][i]) + (w_prefill * uncached_i), same operations and order as the score.
 // st_hits packs (prefix hit, blocks present << 16) of a replica into one word.
-template <typename MaskT>
+template <typename MaskT, bool kBaseline>
 __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<MaskT>& cx,
                                              const Ahead& q, uint32_t slot, uint32_t h0,
                                              uint32_t h1, uint32_t p0, uint32_t p1,
-                                             unsigned long long where, uint32_t lane) {
+                                             unsigned long long where, uint32_t lane, double scale) {
   const uint32_t R = a.m.R;
+  // (time-varying network, extended build only: the proxy's signal of the request's epoch)
+  const double* ewma_row = nullptr;
+  if (kBaseline && a.rtt_ewma)
+    ewma_row = a.rtt_ewma + ((size_t)epoch_of(a, __dmul_rn(scale, q.ts)) * a.m.G + q.origin) * R;
   if (lane == 0) {
     cx.st_where[slot] = where;
     cx.st_meta[slot] = make_uint4(q.in_tok, q.nblk | (q.origin << 16), q.prev_share, q.off);
@@ -909,7 +928,8 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
       const unsigned long long hb = (unsigned long long)h * a.m.B;
       const uint32_t unc = q.in_tok - (uint32_t)(hb < q.in_tok ? hb : q.in_tok);
       cx.st_hits[slot * R + i] = h | (pr << 16);
-      cx.st_ab[slot * R + i] = __dadd_rn(wrtt_row[i], __dmul_rn(w_pre, (double)unc));
+      const double net = (kBaseline && ewma_row) ? __dmul_rn(cx.sm.w[0], ewma_row[i]) : wrtt_row[i];
+      cx.st_ab[slot * R + i] = __dadd_rn(net, __dmul_rn(w_pre, (double)unc));
     }
   }
 }
@@ -919,9 +939,10 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
 // them and publishes the prefix hits.  Its reads may predate the commits of the last kWindow
 // requests; the cache warp knows which of those commits can have touched request q and then
 // repeats the work itself, so this warp is an accelerator only and may stop at any time.
-template <typename MaskT>
-__device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>& cx,
+template <typename MaskT, bool kBaseline>
+__device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
                                            uint32_t lane, uint32_t which) {
+  const double scale = a.scales ? a.scales[p] : a.scale;
   const Smem& sm = cx.sm;
   const ReqRec* req = a.tr.req;
   const uint32_t* ids = a.tr.ids;
@@ -971,7 +992,7 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
       uint32_t h0, h1, p0, p1;
       unsigned long long where;
       probe_staged<MaskT>(smk, mask, ids, q_b, R, lane, h0, h1, p0, p1, where);
-      stage_scores<MaskT>(a, cx, q_b, slot, h0, h1, p0, p1, where, lane);
+      stage_scores<MaskT, kBaseline>(a, cx, q_b, slot, h0, h1, p0, p1, where, lane, scale);
       smem_order();
       __syncwarp();
       if (lane == 0) cx.st_ready[slot] = qb + 1;
@@ -991,9 +1012,10 @@ __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>
 // (`st_where`).  If neither can be the case the staged hits go out the moment the previous route
 // is known; otherwise the gate waits for the commits in question and looks at what they report
 // (`evhit`), and if need be reads and probes the mask words again itself.
-template <typename MaskT>
+template <typename MaskT, bool kBaseline>
 __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
                                           uint32_t lane) {
+  const double scale = a.scales ? a.scales[p] : a.scale;
   const Smem& sm = cx.sm;
   const uint32_t R = a.m.R;
   const ReqRec* req = a.tr.req;
@@ -1038,6 +1060,7 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
         const uint4 meta = cx.st_meta[ss];
         q_cur.in_tok = meta.x; q_cur.nblk = meta.y & 0xFFFFu; q_cur.origin = meta.y >> 16;
         q_cur.prev_share = meta.z; q_cur.off = meta.w;
+        q_cur.ts = (kBaseline && a.rtt_ewma) ? a.tr.ts[r] : 0.0;
       } else {
         q_cur = fetch_ahead(req, r, end);
       }
@@ -1080,7 +1103,7 @@ __device__ __forceinline__ void gate_warp(const ReplayArgs& a, const Ctx<MaskT>&
         __syncwarp();
         unsigned long long where = 0;
         probe_staged<MaskT>(smk, mask, ids, q_cur, R, lane, h0, h1, p0, p1, where);
-        stage_scores<MaskT>(a, cx, q_cur, slot, h0, h1, p0, p1, where, lane);
+        stage_scores<MaskT, kBaseline>(a, cx, q_cur, slot, h0, h1, p0, p1, where, lane, scale);
         __syncwarp();
       }
       hand_over(slot, n);
@@ -1518,9 +1541,9 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
   uint32_t which;
   role_of(warp, role, which);
   if (role == kRoleRoute) route_warp<MaskT, kBaseline>(a, cx, p, lane);
-  else if (role == kRoleGate) gate_warp<MaskT>(a, cx, p, lane);
+  else if (role == kRoleGate) gate_warp<MaskT, kBaseline>(a, cx, p, lane);
   else if (role == kRoleCommit) commit_warp<MaskT>(a, cx, p, lane, which);
-  else if (role == kRoleProbe) probe_warp<MaskT>(a, cx, lane, which);
+  else if (role == kRoleProbe) probe_warp<MaskT, kBaseline>(a, cx, p, lane, which);
   else if (role == kRoleService) service_warp<MaskT, kBaseline>(a, cx, p, lane, which);
   else if (role == kRoleExpiry)
     expiry_warp<kBaseline>(a, sm, cx.exp_head, cx.exp_rec, sm.abort_flag, cx.status, p, lane);
@@ -1842,7 +1865,7 @@ cudaError_t launch_replay_tb(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
 template <typename MaskT>
 cudaError_t launch_replay_t(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st) {
   if (a.queue_in_requests || a.forced_route || a.rep_prefill_ms || a.rep_tpot_ms ||
-      a.decode_slowdown > 0.0 || a.kv_budget > 0)
+      a.decode_slowdown > 0.0 || a.kv_budget > 0 || a.rtt_ewma)
     return launch_replay_tb<MaskT, true>(a, n_cand, st);
   return launch_replay_tb<MaskT, false>(a, n_cand, st);
 }
