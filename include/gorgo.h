@@ -171,6 +171,16 @@ int gorgo_state_status(gorgo_sim_t *sim, void *state_workspace, uint64_t state_b
 int gorgo_sim_set_replica_speeds(gorgo_sim_t *sim, const double *prefill_ms_per_token,
                                  const double *tpot_ms);
 
+/* Proxy index that drifts from the replica's cache (paper Section 7 names it as a limitation: the
+ * proxy's prefix index is built from the requests it dispatched and does not observe what the
+ * replica evicts).  With `enable` nonzero the score of Eq. 3 takes its prefix hits from the
+ * proxy's index of a replica -- every block of every request dispatched to it so far, never
+ * forgotten -- while the prefill time, the reported hit length, the cache contents and their
+ * digests follow the replica's real LRU cache.  As long as nothing is evicted both are the same.
+ * Applies to every later replay of this simulator; a persistent state should keep one setting
+ * from reset to its last batch. */
+int gorgo_sim_set_proxy_index(gorgo_sim_t *sim, int enable);
+
 /* Time-varying network (paper Section 2.2: the proxy's network signal is an exponentially
  * weighted moving average of an RTT probe sent every 30 s; its Section 4 shows the probes of one
  * run).  `samples_ms` HOST [n_epochs][G][R]: the probe result of every epoch of `epoch_ms`

@@ -56,6 +56,7 @@ struct Replica {
     std::map<Key, uint64_t, KeyEvictsBefore> order;       // recency key -> block id
     std::vector<double> free_at;                          // per slot: time it becomes free
     std::vector<uint64_t> kv;                             // per slot: KV tokens of its newest request
+    std::set<uint64_t> index;                             // the proxy's index: blocks ever dispatched here
     std::multiset<std::pair<double, uint64_t>> inflight;  // (finish time, input tokens)
     int64_t load = 0;                                     // sum of in-flight input tokens
 };
@@ -109,6 +110,12 @@ struct Oracle {
     std::vector<double> rtt_raw, rtt_ewma;
     uint32_t n_epochs = 0;
     double epoch_ms = 0.0;
+    // Proxy index that drifts from the replica's cache (paper Section 7: the proxy's prefix index is
+    // built from the requests it dispatched and does not observe what the replica evicts).  When
+    // on, the score of Eq. 3 takes the prefix hit from the index -- every block ever dispatched to
+    // the replica, never forgotten -- while prefill time, the reported hit and the cache itself
+    // follow the replica's real LRU cache.
+    bool proxy_index = false;
 };
 
 // Epoch of (scaled) time t: the largest k in [0, n_epochs-1] with k * epoch_ms <= t.
@@ -163,7 +170,7 @@ void gorgo_oracle_destroy(void* h) { delete static_cast<Oracle*>(h); }
 void gorgo_oracle_reset(void* h) {
     Oracle* o = static_cast<Oracle*>(h);
     for (auto& rp : o->rep) {
-        rp.cache.clear(); rp.order.clear(); rp.inflight.clear();
+        rp.cache.clear(); rp.order.clear(); rp.inflight.clear(); rp.index.clear();
         rp.free_at.assign(o->S, 0.0); rp.kv.assign(o->S, 0); rp.load = 0;
     }
     o->next = 0;
@@ -217,11 +224,17 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
             while (hh < n && rp.cache.count(id[hh])) ++hh;
             hits[i] = hh;
             unc[i] = in - std::min<uint64_t>(hh * o->B, in);
+            uint64_t unc_score = unc[i];                   // what the proxy believes is uncached
+            if (o->proxy_index) {
+                uint64_t hb = 0;
+                while (hb < n && rp.index.count(id[hb])) ++hb;
+                unc_score = in - std::min<uint64_t>(hb * o->B, in);
+            }
             double q = o->queue_in_requests ? (double)rp.inflight.size() : (double)rp.load;
             if (o->K != 3) q = q * w[3 + i];               // per-replica queue-load normaliser
             // Eq. 3 with explicit weights: three products, two sums, in this order
             const double a = w[0] * rtt_signal[i];
-            const double b = w[1] * (double)unc[i];
+            const double b = w[1] * (double)unc_score;
             const double c = w[2] * q;
             cost[i] = (a + b) + c;
             if (hit_all) hit_all[done * R + i] = (uint16_t)hh;
@@ -266,6 +279,8 @@ uint64_t gorgo_oracle_run(void* h, const double* w, double scale, uint64_t count
                 rp.order.emplace(key, id[k]);
             }
         }
+
+        if (o->proxy_index) rp.index.insert(id, id + n);   // the proxy learns what it dispatched
 
         // ---- service commit on the chosen replica ----
         const double arrive = t + rtt_delay[best];
@@ -361,6 +376,10 @@ int gorgo_oracle_set_service_model(void* h, double decode_slowdown, uint64_t kv_
     o->kv_budget = kv_budget_tokens;
     return 0;
 }
+
+// Proxy index separate from the replica's cache (see the Oracle struct); takes effect from the
+// empty state.
+void gorgo_oracle_set_proxy_index(void* h, uint32_t on) { static_cast<Oracle*>(h)->proxy_index = on != 0; }
 
 // Probe results per epoch, samples[e][g][i] >= 0, one epoch every epoch_ms > 0 of (scaled) time,
 // smoothing factor 0 < alpha <= 1.  The proxy's signal is ewma_0 = s_0,

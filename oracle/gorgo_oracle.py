@@ -59,6 +59,8 @@ def _load():
         lib.gorgo_oracle_set_policy.argtypes = [vp, C.c_uint32, vp]
         lib.gorgo_oracle_set_replica_speeds.restype = C.c_int
         lib.gorgo_oracle_set_replica_speeds.argtypes = [vp, vp, vp]
+        lib.gorgo_oracle_set_proxy_index.restype = None
+        lib.gorgo_oracle_set_proxy_index.argtypes = [vp, C.c_uint32]
         lib.gorgo_oracle_set_rtt_series.restype = C.c_int
         lib.gorgo_oracle_set_rtt_series.argtypes = [vp, C.c_uint32, C.c_double, C.c_double, vp]
         lib.gorgo_oracle_set_service_model.restype = C.c_int
@@ -149,6 +151,11 @@ class Oracle:
         if self._lib.gorgo_oracle_set_replica_speeds(self._h, _ptr(a), _ptr(b)) != 0:
             raise ValueError("replica speeds must be finite and >= 0")
 
+    def set_proxy_index(self, on: bool = True):
+        """Score with the proxy's own index (every block ever dispatched to a replica) instead of
+        the replica's real cache; set it on the empty state."""
+        self._lib.gorgo_oracle_set_proxy_index(self._h, int(bool(on)))
+
     def set_rtt_series(self, samples=None, epoch_ms: float = 30_000.0, alpha: float = 0.3):
         """Time-varying network: samples[e, g, i] = RTT probe of epoch e (also the delay of requests
         dispatched in it); the score uses their EWMA.  None restores the static matrix."""
@@ -218,7 +225,8 @@ class Oracle:
 
 def replay(workload, w, scale: float = 1.0, detail: bool = False, queue_in_requests: bool = False,
            forced_route=None, rep_prefill_ms=None, rep_tpot_ms=None, decode_slowdown: float = 0.0,
-           kv_budget_tokens: int = 0, rtt_series=None, epoch_ms: float = 30_000.0, alpha: float = 0.3):
+           kv_budget_tokens: int = 0, rtt_series=None, epoch_ms: float = 30_000.0, alpha: float = 0.3,
+           proxy_index: bool = False):
     """Full replay of one candidate from the empty state: (RunResult, p95_ttft, p95_e2e,
     digest[R,2], stats[4])."""
     o = Oracle.from_workload(workload)
@@ -231,6 +239,8 @@ def replay(workload, w, scale: float = 1.0, detail: bool = False, queue_in_reque
             o.set_service_model(decode_slowdown, kv_budget_tokens)
         if rtt_series is not None:
             o.set_rtt_series(rtt_series, epoch_ms, alpha)
+        if proxy_index:
+            o.set_proxy_index(True)
         res = o.run(w, scale, detail=detail)
         return res, p95(res.ttft), p95(res.e2e), o.digest(), o.stats()
     finally:

@@ -35,7 +35,7 @@ EXPORTS = [
     "gorgo_window_count", "gorgo_eval_population_windows", "gorgo_es_run",
     "gorgo_last_window_ms", "gorgo_eval_policy", "gorgo_eval_population_scales",
     "gorgo_sim_set_replica_speeds", "gorgo_debug_set", "gorgo_measure_gather", "gorgo_tune_online",
-    "gorgo_sim_set_service_model", "gorgo_sim_set_rtt_series",
+    "gorgo_sim_set_service_model", "gorgo_sim_set_rtt_series", "gorgo_sim_set_proxy_index",
 ]
 GORGO_DEBUG_POLL_LIMIT, GORGO_DEBUG_RING_POLLS, GORGO_DEBUG_PROBE_OFF, GORGO_DEBUG_SCOUT_OFF = 0, 1, 2, 3
 
@@ -99,6 +99,7 @@ def load():
         "gorgo_debug_set": [vp, u32, u32],
         "gorgo_sim_set_service_model": [vp, dbl, u64],
         "gorgo_sim_set_rtt_series": [vp, u32, dbl, dbl, vp],
+        "gorgo_sim_set_proxy_index": [vp, i32],
         "gorgo_tune_online": [vp, C.POINTER(gorgo_online_config_t), u32, vp, vp, vp, u64, vp, vp, vp,
                               C.POINTER(C.c_uint32), vp, vp, vp, vp],
         "gorgo_measure_gather": [i32, vp, u64, u64, vp, C.POINTER(C.c_double)],
@@ -241,6 +242,12 @@ def gorgo_sim_set_replica_speeds(sim, prefill_ms_per_token=None, tpot_ms=None) -
     a = None if prefill_ms_per_token is None else np.ascontiguousarray(prefill_ms_per_token, np.float64)
     b = None if tpot_ms is None else np.ascontiguousarray(tpot_ms, np.float64)
     return load().gorgo_sim_set_replica_speeds(sim, _np_ptr(a), _np_ptr(b))
+
+
+def gorgo_sim_set_proxy_index(sim, enable: bool = True) -> int:
+    """Score with the proxy's own index (blocks ever dispatched to a replica) instead of the
+    replica's cache."""
+    return load().gorgo_sim_set_proxy_index(sim, int(bool(enable)))
 
 
 def gorgo_sim_set_rtt_series(sim, samples=None, epoch_ms: float = 30_000.0, alpha: float = 0.3) -> int:

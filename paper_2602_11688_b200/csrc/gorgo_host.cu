@@ -19,6 +19,7 @@ struct gorgo_sim {
   std::vector<double> rep_prefill, rep_tpot;   // per-replica speeds; empty: the uniform constants
   double decode_slowdown = 0.0;                // extended service model (0: off)
   uint64_t kv_budget = 0;
+  uint32_t proxy_index = 0;                    // score with the proxy's own index instead of the cache
   std::vector<double> rtt_raw, rtt_ewma;       // time-varying network, [n_epochs][G][R] each; empty: static
   uint32_t n_epochs = 0;
   double epoch_ms = 0.0;
@@ -139,6 +140,7 @@ int attach_speeds(const gorgo_sim* sim, unsigned char* base, const WsLayout& w, 
   const uint32_t R = sim->m.R;
   a->decode_slowdown = sim->decode_slowdown;
   a->kv_budget = sim->kv_budget;
+  a->proxy_index = sim->proxy_index;
   if (sim->n_epochs > 0) {
     const size_t n = sim->rtt_raw.size();
     double* ds = reinterpret_cast<double*>(base + w.series);
@@ -406,6 +408,12 @@ int gorgo_sim_set_replica_speeds(gorgo_sim_t* sim, const double* prefill_ms_per_
   return GORGO_OK;
 }
 
+int gorgo_sim_set_proxy_index(gorgo_sim_t* sim, int enable) {
+  if (!sim) return GORGO_ERR_INVALID_ARG;
+  sim->proxy_index = enable ? 1u : 0u;
+  return GORGO_OK;
+}
+
 int gorgo_sim_set_rtt_series(gorgo_sim_t* sim, uint32_t n_epochs, double epoch_ms, double alpha,
                              const double* samples_ms) {
   if (!sim) return GORGO_ERR_INVALID_ARG;
@@ -444,7 +452,8 @@ int gorgo_sim_set_service_model(gorgo_sim_t* sim, double decode_slowdown, uint64
 int gorgo_trace_bytes(uint64_t n_requests, uint64_t n_block_ids, uint64_t* bytes_out) {
   if (!bytes_out) return GORGO_ERR_INVALID_ARG;
   *bytes_out = align_up(n_requests * sizeof(ReqRec)) + align_up(n_block_ids * 4) +
-               align_up(n_block_ids * 8) + align_up(n_block_ids * 8) + align_up(n_requests * 8) +
+               align_up(n_block_ids * 8) + align_up(n_block_ids * 8) + align_up(n_block_ids * 8) +
+               align_up(n_requests * 8) +
                align_up((n_requests + 1) * 4) + kAlign;
   return GORGO_OK;
 }
@@ -509,14 +518,24 @@ int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_m
   }
   const uint64_t D = raw.size();
 
-  // next occurrence of the same block, and the request it belongs to
-  std::vector<uint2> occ(T);
+  // next and previous occurrence of the same block, and the request each belongs to
+  std::vector<uint2> occ(T), occ_before(T);
   {
     std::vector<uint32_t> last_g(D, kNone), last_r(D, kNone);
     for (uint64_t r = N; r-- > 0;) {
       for (uint64_t g = hash_off[r + 1]; g-- > hash_off[r];) {
         const uint32_t d = ids[g];
         occ[g] = make_uint2(last_g[d], last_r[d]);
+        last_g[d] = (uint32_t)g;
+        last_r[d] = (uint32_t)r;
+      }
+    }
+    std::fill(last_g.begin(), last_g.end(), kNone);
+    std::fill(last_r.begin(), last_r.end(), kNone);
+    for (uint64_t r = 0; r < N; ++r) {
+      for (uint64_t g = hash_off[r]; g < hash_off[r + 1]; ++g) {
+        const uint32_t d = ids[g];
+        occ_before[g] = make_uint2(last_g[d], last_r[d]);
         last_g[d] = (uint32_t)g;
         last_r[d] = (uint32_t)r;
       }
@@ -553,6 +572,7 @@ int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_m
   unsigned char* d_ids = base + o; o += align_up(T * 4);
   unsigned char* d_occ = base + o; o += align_up(T * 8);
   unsigned char* d_raw = base + o; o += align_up(D * 8);
+  unsigned char* d_prev = base + o; o += align_up(T * 8);
   unsigned char* d_ts = base + o; o += align_up(N * 8);
   unsigned char* d_grid = base + o; o += align_up((N + 1) * 4);
   bool ok = cudaMemcpyAsync(d_req, req.data(), N * sizeof(ReqRec), cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -563,12 +583,14 @@ int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_m
     ok = ok && cudaMemcpyAsync(d_ids, ids.data(), T * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(d_occ, occ.data(), T * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(d_raw, raw.data(), D * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(d_prev, occ_before.data(), T * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
   }
   ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
   if (!ok) { cudaGetLastError(); sim->has_trace = false; return GORGO_ERR_CUDA; }
   sim->tr.req = reinterpret_cast<const ReqRec*>(d_req);
   sim->tr.ids = reinterpret_cast<const uint32_t*>(d_ids);
   sim->tr.occ_next = reinterpret_cast<const uint2*>(d_occ);
+  sim->tr.occ_prev = reinterpret_cast<const uint2*>(d_prev);
   sim->tr.raw_id = reinterpret_cast<const uint64_t*>(d_raw);
   sim->tr.ts = reinterpret_cast<const double*>(d_ts);
   sim->tr.grid = reinterpret_cast<const uint32_t*>(d_grid);

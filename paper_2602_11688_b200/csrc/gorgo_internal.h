@@ -44,6 +44,7 @@ struct TraceView {
   const uint32_t* ids;     // [T] dense block ids, request after request
   const uint2* occ_next;   // [T] (.x = flat index of the next occurrence of the same block or
                            //      kNone, .y = request of that occurrence)
+  const uint2* occ_prev;   // [T] the same for the previous occurrence
   const uint64_t* raw_id;  // [D] caller's 64-bit id of each dense id
   const double* ts;        // [N] arrival times (unscaled), the same values as in `req`
   // time grid over the unscaled arrival times: grid[b] = first request with ts >= b * grid_dt,
@@ -105,6 +106,9 @@ struct ReplayArgs {
   // [R] each) or null for the uniform constants of the model
   const double* rep_prefill_ms;
   const double* rep_tpot_ms;
+  // 1: the score takes prefix hits from the proxy's own index (blocks ever dispatched to a
+  // replica) instead of the replica's cache
+  uint32_t proxy_index;
   // time-varying network: per epoch the proxy's RTT signal (EWMA of the probes) and the probes
   // themselves (the delay a request experiences), [n_epochs][G][R] each, device; null = static
   const double* rtt_ewma;

@@ -868,19 +868,17 @@ __device__ __forceinline__ MaskT warp_or_mask(MaskT m) {
 // and lane+32): h = leading blocks whose mask has the replica's bit (the prefix hit), p = all
 // blocks of the request whose mask has it (what a commit there does not have to insert).  The
 // first kStageBlocks words come from `smk`; longer prompts read the rest from memory.
-template <typename MaskT>
-__device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask,
-                                             const uint32_t* ids, const Ahead& q, uint32_t R,
-                                             uint32_t lane, uint32_t& h0, uint32_t& h1,
-                                             uint32_t& p0, uint32_t& p1, unsigned long long& where) {
+template <typename MaskT, typename LoadWord>
+__device__ __forceinline__ void probe_words(LoadWord load_word, uint32_t n, uint32_t R,
+                                            uint32_t lane, uint32_t& h0, uint32_t& h1,
+                                            uint32_t& p0, uint32_t& p1, unsigned long long& where) {
   h0 = 0; h1 = 0; p0 = 0; p1 = 0; where = 0;
-  const uint32_t n = q.nblk;
   MaskT alive = (R >= sizeof(MaskT) * 8) ? (MaskT)~(MaskT)0 : (MaskT)((((MaskT)1) << (R & 63)) - 1);
   #pragma unroll 1
   for (uint32_t c = 0; c < n; c += 32) {
     const uint32_t k = c + lane;
     MaskT m = 0;
-    if (k < n) m = (c < kStageBlocks) ? smk[k] : mask_load<MaskT>(mask, ids[q.off + k]);
+    if (k < n) m = load_word(c, k);
     MaskT it = warp_or_mask<MaskT>(m);      // replicas that hold any block of this chunk
     where |= (unsigned long long)it;
     MaskT still = 0;
@@ -901,6 +899,38 @@ __device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask
   }
 }
 
+// The same from staged mask words: the first kStageBlocks words come from `smk`; longer prompts
+// read the rest from memory.
+template <typename MaskT>
+__device__ __forceinline__ void probe_staged(const MaskT* smk, const MaskT* mask,
+                                             const uint32_t* ids, const Ahead& q, uint32_t R,
+                                             uint32_t lane, uint32_t& h0, uint32_t& h1,
+                                             uint32_t& p0, uint32_t& p1, unsigned long long& where) {
+  probe_words<MaskT>([&](uint32_t c, uint32_t k) -> MaskT {
+    return (c < kStageBlocks) ? smk[k] : mask_load<MaskT>(mask, ids[q.off + k]);
+  }, q.nblk, R, lane, h0, h1, p0, p1, where);
+}
+
+// Prefix hits of a request in the PROXY'S INDEX (extended build): bit i of a block's word says that
+// an earlier request containing the block was routed to replica i, whatever the replica has
+// evicted since.  The word is gathered by walking the block's earlier occurrences.
+template <typename MaskT>
+__device__ __forceinline__ void probe_index(const TraceView& tr, const uint8_t* route_log, const Ahead& q,
+                                            uint32_t R, uint32_t lane, uint32_t& h0, uint32_t& h1) {
+  uint32_t p0, p1;
+  unsigned long long where;
+  probe_words<MaskT>([&](uint32_t, uint32_t k) -> MaskT {
+    unsigned long long w = 0;
+    uint2 pv = tr.occ_prev[q.off + k];
+    #pragma unroll 1
+    for (uint32_t guard = 0; pv.x != kNone && guard < tr.n_req; ++guard) {
+      w |= 1ull << ((uint32_t)__ldcg(route_log + pv.y) & 63u);
+      pv = tr.occ_prev[pv.x];
+    }
+    return (MaskT)w;
+  }, q.nblk, R, lane, h0, h1, p0, p1, where);
+}
+
 // Stage the prefix hits of a request and the part of its score (Eq. 3) that depends on them:
 // ab_i = (w_net * RTT[g][i]) + (w_prefill * uncached_i), same operations and order as the score.
 // st_hits packs (prefix hit, blocks present << 16) of a replica into one word.
@@ -910,6 +940,9 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
                                              uint32_t h1, uint32_t p0, uint32_t p1,
                                              unsigned long long where, uint32_t lane, double scale) {
   const uint32_t R = a.m.R;
+  // (proxy index, extended build only: the score takes its hits from the index)
+  uint32_t s0 = h0, s1 = h1;
+  if (kBaseline && a.proxy_index) probe_index<MaskT>(a.tr, cx.route_log, q, R, lane, s0, s1);
   // (time-varying network, extended build only: the proxy's signal of the request's epoch)
   const double* ewma_row = nullptr;
   if (kBaseline && a.rtt_ewma)
@@ -925,7 +958,7 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
     const uint32_t i = lane + 32u * half;
     if (i < R) {
       const uint32_t h = half ? h1 : h0, pr = half ? p1 : p0;
-      const unsigned long long hb = (unsigned long long)h * a.m.B;
+      const unsigned long long hb = (unsigned long long)(half ? s1 : s0) * a.m.B;
       const uint32_t unc = q.in_tok - (uint32_t)(hb < q.in_tok ? hb : q.in_tok);
       cx.st_hits[slot * R + i] = h | (pr << 16);
       const double net = (kBaseline && ewma_row) ? __dmul_rn(cx.sm.w[0], ewma_row[i]) : wrtt_row[i];
@@ -1865,7 +1898,7 @@ cudaError_t launch_replay_tb(ReplayArgs a, uint32_t n_cand, cudaStream_t st) {
 template <typename MaskT>
 cudaError_t launch_replay_t(const ReplayArgs& a, uint32_t n_cand, cudaStream_t st) {
   if (a.queue_in_requests || a.forced_route || a.rep_prefill_ms || a.rep_tpot_ms ||
-      a.decode_slowdown > 0.0 || a.kv_budget > 0 || a.rtt_ewma)
+      a.decode_slowdown > 0.0 || a.kv_budget > 0 || a.rtt_ewma || a.proxy_index)
     return launch_replay_tb<MaskT, true>(a, n_cand, st);
   return launch_replay_tb<MaskT, false>(a, n_cand, st);
 }
