@@ -92,6 +92,33 @@ int gorgo_trace_upload(gorgo_sim_t *sim, uint64_t n_requests, const double *ts_m
                        const uint64_t *hash_ids, void *dev_trace_buf, uint64_t dev_trace_bytes,
                        void *cuda_stream);
 
+/* Online boundary (Section 2.3: the proxy routes requests as they arrive): a trace that grows.
+ * gorgo_trace_begin lays `dev_trace_buf` (DEVICE, >= gorgo_trace_bytes(max_requests,
+ * max_block_ids) bytes, 256-byte aligned) out for up to `max_requests` requests with up to
+ * `max_block_ids` block ids in total and forgets any earlier trace of the handle.
+ * gorgo_trace_append adds `n_requests` >= 1 requests after the ones already there; the arguments
+ * are those of gorgo_trace_upload for the new requests alone (`hash_off` starts at 0; `ts_ms`
+ * continues non-decreasing from the last request so far).  The copies are enqueued on
+ * `cuda_stream`, ordered after earlier batches on the same stream; the call returns when the
+ * host arrays may be reused.  Returns GORGO_ERR_WORKSPACE_TOO_SMALL when a capacity would be
+ * exceeded and GORGO_ERR_BAD_TRACE for a violated precondition; in both cases the trace is as
+ * it was before the call.  GORGO_ERR_NO_TRACE without a preceding gorgo_trace_begin (a trace
+ * given to gorgo_trace_upload cannot grow).
+ *   Once the first batch is in, every call that takes a trace works on the requests appended so
+ * far.  Workspace and state sizes (gorgo_workspace_bytes, gorgo_state_bytes) are computed for
+ * the capacities, so a persistent state set up by gorgo_sim_reset stays valid while the trace
+ * grows: gorgo_route_batch may route requests that were not known when the state was reset or
+ * when earlier batches ran.  Routing appended requests batch by batch gives bit for bit what
+ * routing the whole trace at once gives (a request still in flight at the end of the known
+ * trace is kept in the state and leaves the queue signal of Eq. 2 at the first appended request
+ * that arrives at or after its finish time); use one time scale from reset on. */
+int gorgo_trace_begin(gorgo_sim_t *sim, uint64_t max_requests, uint64_t max_block_ids,
+                      void *dev_trace_buf, uint64_t dev_trace_bytes);
+int gorgo_trace_append(gorgo_sim_t *sim, uint64_t n_requests, const double *ts_ms,
+                       const uint32_t *input_tokens, const uint32_t *output_tokens,
+                       const uint16_t *origin, const uint64_t *hash_off, const uint64_t *hash_ids,
+                       void *cuda_stream);
+
 /* Facts about the uploaded trace: requests, block ids in total, distinct block ids. */
 int gorgo_trace_info(const gorgo_sim_t *sim, uint64_t *n_requests, uint64_t *n_block_ids,
                      uint64_t *n_distinct);

@@ -36,6 +36,7 @@ EXPORTS = [
     "gorgo_last_window_ms", "gorgo_eval_policy", "gorgo_eval_population_scales",
     "gorgo_sim_set_replica_speeds", "gorgo_debug_set", "gorgo_measure_gather", "gorgo_tune_online",
     "gorgo_sim_set_service_model", "gorgo_sim_set_rtt_series", "gorgo_sim_set_proxy_index",
+    "gorgo_trace_begin", "gorgo_trace_append",
 ]
 GORGO_DEBUG_POLL_LIMIT, GORGO_DEBUG_RING_POLLS, GORGO_DEBUG_PROBE_OFF, GORGO_DEBUG_SCOUT_OFF = 0, 1, 2, 3
 
@@ -100,6 +101,8 @@ def load():
         "gorgo_sim_set_service_model": [vp, dbl, u64],
         "gorgo_sim_set_rtt_series": [vp, u32, dbl, dbl, vp],
         "gorgo_sim_set_proxy_index": [vp, i32],
+        "gorgo_trace_begin": [vp, u64, u64, vp, u64],
+        "gorgo_trace_append": [vp, u64, vp, vp, vp, vp, vp, vp, vp],
         "gorgo_tune_online": [vp, C.POINTER(gorgo_online_config_t), u32, vp, vp, vp, u64, vp, vp, vp,
                               C.POINTER(C.c_uint32), vp, vp, vp, vp],
         "gorgo_measure_gather": [i32, vp, u64, u64, vp, C.POINTER(C.c_double)],
@@ -174,6 +177,24 @@ def gorgo_trace_upload(sim, ts_ms, input_tokens, output_tokens, origin, hash_off
     return load().gorgo_trace_upload(sim, ts.shape[0], _np_ptr(ts), _np_ptr(it), _np_ptr(ot),
                                      _np_ptr(org), _np_ptr(off), _np_ptr(ids),
                                      _dev_ptr(dev_trace_buf), dev_trace_buf.numel(), stream)
+
+
+def gorgo_trace_begin(sim, max_requests: int, max_block_ids: int, dev_trace_buf) -> int:
+    return load().gorgo_trace_begin(sim, int(max_requests), int(max_block_ids),
+                                    _dev_ptr(dev_trace_buf), dev_trace_buf.numel())
+
+
+def gorgo_trace_append(sim, ts_ms, input_tokens, output_tokens, origin, hash_off, hash_ids,
+                       stream: int = 0) -> int:
+    """Appends requests (``hash_off`` starts at 0 for the first new one)."""
+    ts = np.ascontiguousarray(ts_ms, dtype=np.float64)
+    it = np.ascontiguousarray(input_tokens, dtype=np.uint32)
+    ot = np.ascontiguousarray(output_tokens, dtype=np.uint32)
+    org = None if origin is None else np.ascontiguousarray(origin, dtype=np.uint16)
+    off = np.ascontiguousarray(hash_off, dtype=np.uint64)
+    ids = np.ascontiguousarray(hash_ids, dtype=np.uint64)
+    return load().gorgo_trace_append(sim, ts.shape[0], _np_ptr(ts), _np_ptr(it), _np_ptr(ot),
+                                     _np_ptr(org), _np_ptr(off), _np_ptr(ids), stream)
 
 
 def gorgo_trace_info(sim):

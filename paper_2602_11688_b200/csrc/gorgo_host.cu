@@ -6,6 +6,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <memory>
 #include <vector>
 
 #include "../../include/gorgo.h"
@@ -13,8 +14,62 @@
 
 using namespace gorgo;
 
+// 64-bit id -> dense number, open addressing, grows by doubling.
+struct IdMap {
+  std::vector<uint64_t> keys;
+  std::vector<uint32_t> vals;  // 0 = empty, else dense + 1
+  uint64_t mask = 0, used = 0;
+  static uint64_t hash(uint64_t z) {
+    z ^= z >> 33; z *= 0xff51afd7ed558ccdULL; z ^= z >> 33; z *= 0xc4ceb9fe1a85ec53ULL;
+    return z ^ (z >> 33);
+  }
+  explicit IdMap(uint64_t cap_pow2) : keys(cap_pow2), vals(cap_pow2, 0), mask(cap_pow2 - 1) {}
+  void grow() {
+    IdMap bigger((mask + 1) * 2);
+    for (uint64_t i = 0; i <= mask; ++i)
+      if (vals[i]) bigger.put(keys[i], vals[i]);
+    keys.swap(bigger.keys); vals.swap(bigger.vals); mask = bigger.mask;
+  }
+  void put(uint64_t k, uint32_t v) {
+    uint64_t i = hash(k) & mask;
+    while (vals[i]) i = (i + 1) & mask;
+    keys[i] = k; vals[i] = v; ++used;
+  }
+  // returns dense number, assigning `next` if the id is new
+  uint32_t get_or_add(uint64_t k, uint32_t& next) {
+    uint64_t i = hash(k) & mask;
+    while (vals[i]) {
+      if (keys[i] == k) return vals[i] - 1;
+      i = (i + 1) & mask;
+    }
+    if ((used + 1) * 2 > mask + 1) { grow(); return get_or_add(k, next); }
+    keys[i] = k; vals[i] = next + 1; ++used;
+    return next++;
+  }
+};
+
+// Host side of a trace that is still growing (gorgo_trace_begin / gorgo_trace_append): what the
+// next batch needs to know about the requests before it, and where the device regions lie.
+struct TraceBuilder {
+  IdMap map{1ull << 16};
+  std::vector<uint32_t> seen_in;          // per dense id: request (+1) that last contained it
+  std::vector<uint32_t> last_g, last_r;   // per dense id: flat position and request of its last occurrence
+  std::vector<uint64_t> raw_new;          // caller's ids of the dense ids added by the current batch
+  std::vector<double> ts;                 // arrival times so far
+  uint64_t cap_req = 0, cap_ids = 0;      // capacities the device regions were laid out for
+  uint64_t N = 0, T = 0;
+  uint32_t D = 0;
+  double grid_dt = 0.0;
+  uint32_t grid_n = 0;
+  uint64_t grid_cursor = 0;               // first request not yet behind the last grid edge
+  unsigned char *d_req = nullptr, *d_ids = nullptr, *d_occ = nullptr, *d_raw = nullptr,
+                *d_prev = nullptr, *d_ts = nullptr, *d_grid = nullptr;
+};
+
 struct gorgo_sim {
   Model m;
+  std::unique_ptr<TraceBuilder> tb;       // set while the trace can still grow
+  uint64_t cap_req = 0, cap_ids = 0;      // appendable trace: sizes the workspaces are laid out for (else 0)
   std::vector<double> rtt;
   std::vector<double> rep_prefill, rep_tpot;   // per-replica speeds; empty: the uniform constants
   double decode_slowdown = 0.0;                // extended service model (0: off)
@@ -52,40 +107,6 @@ struct DeviceGuard {
   ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
 };
 
-// 64-bit id -> dense number, open addressing, grows by doubling.
-struct IdMap {
-  std::vector<uint64_t> keys;
-  std::vector<uint32_t> vals;  // 0 = empty, else dense + 1
-  uint64_t mask = 0, used = 0;
-  static uint64_t hash(uint64_t z) {
-    z ^= z >> 33; z *= 0xff51afd7ed558ccdULL; z ^= z >> 33; z *= 0xc4ceb9fe1a85ec53ULL;
-    return z ^ (z >> 33);
-  }
-  explicit IdMap(uint64_t cap_pow2) : keys(cap_pow2), vals(cap_pow2, 0), mask(cap_pow2 - 1) {}
-  void grow() {
-    IdMap bigger((mask + 1) * 2);
-    for (uint64_t i = 0; i <= mask; ++i)
-      if (vals[i]) bigger.put(keys[i], vals[i]);
-    keys.swap(bigger.keys); vals.swap(bigger.vals); mask = bigger.mask;
-  }
-  void put(uint64_t k, uint32_t v) {
-    uint64_t i = hash(k) & mask;
-    while (vals[i]) i = (i + 1) & mask;
-    keys[i] = k; vals[i] = v; ++used;
-  }
-  // returns dense number, assigning `next` if the id is new
-  uint32_t get_or_add(uint64_t k, uint32_t& next) {
-    uint64_t i = hash(k) & mask;
-    while (vals[i]) {
-      if (keys[i] == k) return vals[i] - 1;
-      i = (i + 1) & mask;
-    }
-    if ((used + 1) * 2 > mask + 1) { grow(); return get_or_add(k, next); }
-    keys[i] = k; vals[i] = next + 1; ++used;
-    return next++;
-  }
-};
-
 StateLayout make_layout(const Model& m) {
   StateLayout l;
   uint64_t o = sizeof(CandHeader);
@@ -100,7 +121,7 @@ StateLayout make_layout(const Model& m) {
 // Byte offsets of the regions of a workspace for `res` resident candidates.
 struct WsLayout {
   uint64_t params, scales, rtt, speeds, status, p95, forced, draws, series, masks, states, lists, exp_head, exp_rec, lru_next,
-      route_log, ttft, e2e, total;
+      route_log, finish, ttft, e2e, total;
   uint64_t mask_stride;
   StateLayout st;
 };
@@ -108,9 +129,12 @@ struct WsLayout {
 WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   WsLayout w;
   const Model& m = s->m;
-  const uint64_t N = s->tr.n_req;
+  // an appendable trace lays everything out for its capacities, so that a persistent state stays
+  // valid while the trace grows
+  const uint64_t N = s->cap_req ? s->cap_req : s->tr.n_req;
+  const uint64_t D = s->cap_req ? s->cap_ids : s->tr.n_distinct;
   w.st = make_layout(m);
-  w.mask_stride = align_up((uint64_t)s->tr.n_distinct * mask_bytes_for(m.R));
+  w.mask_stride = align_up(D * mask_bytes_for(m.R));
   uint64_t o = 0;
   w.params = o; o = align_up(o + res * m.K * 8);
   w.scales = o; o = align_up(o + res * 8);       // one time scale per candidate (optional)
@@ -128,6 +152,7 @@ WsLayout make_ws(const gorgo_sim* s, uint64_t res, bool with_latency) {
   w.exp_rec = o; o = align_up(o + res * N * 16);
   w.lru_next = o; o = align_up(o + res * N * 4);
   w.route_log = o; o = align_up(o + res * N);
+  w.finish = o; if (!with_latency) o = align_up(o + res * N * 8);   // persistent state only
   w.ttft = o; if (with_latency) o = align_up(o + res * N * 8);
   w.e2e = o; if (with_latency) o = align_up(o + res * N * 8);
   w.total = o;
@@ -458,147 +483,228 @@ int gorgo_trace_bytes(uint64_t n_requests, uint64_t n_block_ids, uint64_t* bytes
   return GORGO_OK;
 }
 
+// Appends `n_new` requests to the trace under construction in `sim->tb`.  With `atomic` a trace
+// that fails a check is left as it was; without it the caller discards the builder on failure.
+static int trace_append_impl(gorgo_sim_t* sim, uint64_t n_new, const double* ts_ms,
+                             const uint32_t* input_tokens, const uint32_t* output_tokens,
+                             const uint16_t* origin, const uint64_t* hash_off,
+                             const uint64_t* hash_ids, cudaStream_t st, bool atomic) {
+  TraceBuilder& tb = *sim->tb;
+  const Model& m = sim->m;
+  if (n_new < 1 || hash_off[0] != 0) return GORGO_ERR_BAD_TRACE;
+  for (uint64_t k = 0; k < n_new; ++k)
+    if (hash_off[k + 1] < hash_off[k]) return GORGO_ERR_BAD_TRACE;
+  const uint64_t Tn = hash_off[n_new];
+  const uint64_t N0 = tb.N, T0 = tb.T, N = N0 + n_new, T = T0 + Tn;
+  if (N > tb.cap_req || T > tb.cap_ids) return GORGO_ERR_WORKSPACE_TOO_SMALL;
+  if (Tn > 0 && !hash_ids) return GORGO_ERR_INVALID_ARG;
+  const uint64_t nmax = m.C < 65535 ? m.C : 65535;
+
+  std::vector<ReqRec> req(n_new);
+  double prev_t = N0 ? tb.ts.back() : 0.0;
+  for (uint64_t k = 0; k < n_new; ++k) {
+    const double t = ts_ms[k];
+    if (!finite_nonneg(t) || t < prev_t) return GORGO_ERR_BAD_TRACE;
+    prev_t = t;
+    const uint64_t n = hash_off[k + 1] - hash_off[k];
+    const uint64_t want = ((uint64_t)input_tokens[k] + m.B - 1) / m.B;
+    if (n != want || n > nmax) return GORGO_ERR_BAD_TRACE;
+    const uint16_t g = origin ? origin[k] : (uint16_t)0;
+    if (g >= m.G) return GORGO_ERR_BAD_TRACE;
+    ReqRec& q = req[k];
+    q.ts_ms = t; q.off = (uint32_t)(T0 + hash_off[k]); q.in_tok = input_tokens[k];
+    q.out_tok = output_tokens[k]; q.nblk = (uint16_t)n; q.origin = g; q.prev_share = kNone; q.pad = 0;
+  }
+  if (atomic) {   // an id twice in one request: found before anything is changed
+    std::vector<uint64_t> tmp;
+    for (uint64_t k = 0; k < n_new; ++k) {
+      tmp.assign(hash_ids + hash_off[k], hash_ids + hash_off[k + 1]);
+      std::sort(tmp.begin(), tmp.end());
+      if (std::adjacent_find(tmp.begin(), tmp.end()) != tmp.end()) return GORGO_ERR_BAD_TRACE;
+    }
+  }
+
+  // dense renumbering in order of first appearance; per block the previous occurrence, and the
+  // next one where that lies in this batch (an earlier batch's entry is patched on the device)
+  std::vector<uint32_t> ids(Tn);
+  std::vector<uint2> occ(Tn, make_uint2(kNone, kNone)), occ_before(Tn);
+  const uint32_t D0 = tb.D;
+  bool patch_old = false;
+  for (uint64_t k = 0; k < n_new; ++k) {
+    const uint32_t r = (uint32_t)(N0 + k);
+    uint32_t latest = 0;  // latest earlier request (+1) that contains one of this one's blocks
+    for (uint64_t gl = hash_off[k]; gl < hash_off[k + 1]; ++gl) {
+      const uint32_t before = tb.D;
+      const uint32_t d = tb.map.get_or_add(hash_ids[gl], tb.D);
+      if (tb.D != before) {
+        tb.raw_new.push_back(hash_ids[gl]);
+        tb.seen_in.push_back(0); tb.last_g.push_back(kNone); tb.last_r.push_back(kNone);
+      }
+      if (tb.seen_in[d] == r + 1) return GORGO_ERR_BAD_TRACE;   // (not reached when `atomic`)
+      if (tb.seen_in[d] > latest) latest = tb.seen_in[d];
+      tb.seen_in[d] = r + 1;
+      ids[gl] = d;
+      const uint32_t g = (uint32_t)(T0 + gl);
+      const uint32_t pg = tb.last_g[d];
+      occ_before[gl] = make_uint2(pg, tb.last_r[d]);
+      if (pg != kNone) {
+        if (pg >= T0) occ[pg - T0] = make_uint2(g, r);
+        else patch_old = true;
+      }
+      tb.last_g[d] = g; tb.last_r[d] = r;
+    }
+    req[k].prev_share = latest ? latest - 1 : kNone;
+  }
+  tb.ts.insert(tb.ts.end(), ts_ms, ts_ms + n_new);
+
+  // time grid over the arrivals: grid[b] = first request with ts >= b * dt (the last request if
+  // there is none), b = 0..n_grid; none while all requests arrive at one instant.  The first
+  // build takes about one request per bucket; later batches add buckets of the same width.
+  // Entries written earlier stay valid: the replay only needs a lower bound of the request it
+  // searches for.
+  std::vector<uint32_t> grid;
+  uint32_t grid_from = 0;
+  {
+    const double span = tb.ts.back();
+    const double buckets = tb.grid_n ? std::floor(span / tb.grid_dt) : 0.0;
+    if (tb.grid_n == 0 || buckets > (double)tb.cap_req) {
+      const double dt = span / (double)N;
+      tb.grid_n = 0; tb.grid_dt = 0.0;
+      if (dt > 0.0 && std::isfinite(dt) && dt >= span * 0x1p-40) {
+        tb.grid_n = (uint32_t)N; tb.grid_dt = dt;
+        grid.resize((size_t)N + 1);
+        uint64_t r = 0;
+        for (uint32_t b = 0; b <= tb.grid_n; ++b) {
+          const double edge = (double)b * dt;
+          while (r < N && tb.ts[r] < edge) ++r;
+          grid[b] = (uint32_t)(r < N ? r : N - 1);
+        }
+        tb.grid_cursor = r;
+      }
+    } else if ((uint32_t)buckets > tb.grid_n) {
+      grid_from = tb.grid_n + 1;
+      const uint32_t upto = (uint32_t)buckets;
+      grid.resize(upto - tb.grid_n);
+      uint64_t r = tb.grid_cursor;
+      for (uint32_t b = grid_from; b <= upto; ++b) {
+        const double edge = (double)b * tb.grid_dt;
+        while (r < N && tb.ts[r] < edge) ++r;
+        grid[b - grid_from] = (uint32_t)(r < N ? r : N - 1);
+      }
+      tb.grid_cursor = r;
+      tb.grid_n = upto;
+    }
+  }
+
+  DeviceGuard guard(sim->device);
+  if (!guard.ok) return GORGO_ERR_CUDA;
+  const uint64_t Dn = tb.D - D0;
+  bool ok = cudaMemcpyAsync(tb.d_req + N0 * sizeof(ReqRec), req.data(), n_new * sizeof(ReqRec),
+                            cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(tb.d_ts + N0 * 8, ts_ms, n_new * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!grid.empty())
+    ok = ok && cudaMemcpyAsync(tb.d_grid + (size_t)grid_from * 4, grid.data(), grid.size() * 4,
+                               cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (Tn > 0) {
+    ok = ok && cudaMemcpyAsync(tb.d_ids + T0 * 4, ids.data(), Tn * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(tb.d_occ + T0 * 8, occ.data(), Tn * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(tb.d_prev + T0 * 8, occ_before.data(), Tn * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (Dn > 0)
+      ok = ok && cudaMemcpyAsync(tb.d_raw + (size_t)D0 * 8, tb.raw_new.data(), Dn * 8,
+                                 cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  tb.raw_new.clear();
+  tb.N = N; tb.T = T;
+  if (!ok) { cudaGetLastError(); sim->has_trace = false; return GORGO_ERR_CUDA; }
+  sim->tr.req = reinterpret_cast<const ReqRec*>(tb.d_req);
+  sim->tr.ids = reinterpret_cast<const uint32_t*>(tb.d_ids);
+  sim->tr.occ_next = reinterpret_cast<const uint2*>(tb.d_occ);
+  sim->tr.occ_prev = reinterpret_cast<const uint2*>(tb.d_prev);
+  sim->tr.raw_id = reinterpret_cast<const uint64_t*>(tb.d_raw);
+  sim->tr.ts = reinterpret_cast<const double*>(tb.d_ts);
+  sim->tr.grid = reinterpret_cast<const uint32_t*>(tb.d_grid);
+  sim->tr.grid_dt = tb.grid_dt;
+  sim->tr.grid_n = tb.grid_n;
+  sim->tr.n_req = (uint32_t)N; sim->tr.n_ids = (uint32_t)T; sim->tr.n_distinct = tb.D;
+  // earlier batches' last occurrences now have a successor
+  if (patch_old && launch_link_occurrences(sim->tr, (uint32_t)N0, (uint32_t)n_new, (uint32_t)T0,
+                                           reinterpret_cast<uint2*>(tb.d_occ), st) != cudaSuccess) {
+    sim->has_trace = false;
+    return GORGO_ERR_CUDA;
+  }
+  sim->has_trace = true;
+  return GORGO_OK;
+}
+
+static int trace_begin_impl(gorgo_sim_t* sim, uint64_t max_requests, uint64_t max_block_ids,
+                            void* dev_trace_buf, uint64_t dev_trace_bytes) {
+  if (!sim || !dev_trace_buf) return GORGO_ERR_INVALID_ARG;
+  if ((uintptr_t)dev_trace_buf % kAlign) return GORGO_ERR_INVALID_ARG;
+  if (max_requests < 1 || max_requests >= 0xFFFFFFFFull || max_block_ids >= 0xFFFFFFFFull)
+    return GORGO_ERR_BAD_TRACE;
+  uint64_t need = 0;
+  gorgo_trace_bytes(max_requests, max_block_ids, &need);
+  if (dev_trace_bytes < need) return GORGO_ERR_WORKSPACE_TOO_SMALL;
+  sim->has_trace = false;
+  sim->tr = TraceView{};
+  sim->cap_req = sim->cap_ids = 0;
+  sim->tb.reset(new TraceBuilder());
+  TraceBuilder& tb = *sim->tb;
+  tb.cap_req = max_requests; tb.cap_ids = max_block_ids;
+  const uint64_t N = max_requests, T = max_block_ids;
+  unsigned char* base = static_cast<unsigned char*>(dev_trace_buf);
+  uint64_t o = 0;
+  tb.d_req = base + o; o += align_up(N * sizeof(ReqRec));
+  tb.d_ids = base + o; o += align_up(T * 4);
+  tb.d_occ = base + o; o += align_up(T * 8);
+  tb.d_raw = base + o; o += align_up(T * 8);
+  tb.d_prev = base + o; o += align_up(T * 8);
+  tb.d_ts = base + o; o += align_up(N * 8);
+  tb.d_grid = base + o; o += align_up((N + 1) * 4);
+  return GORGO_OK;
+}
+
 int gorgo_trace_upload(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_ms,
                        const uint32_t* input_tokens, const uint32_t* output_tokens,
                        const uint16_t* origin, const uint64_t* hash_off, const uint64_t* hash_ids,
                        void* dev_trace_buf, uint64_t dev_trace_bytes, void* cuda_stream) {
   if (!sim || !ts_ms || !input_tokens || !output_tokens || !hash_off || !dev_trace_buf)
     return GORGO_ERR_INVALID_ARG;
-  if ((uintptr_t)dev_trace_buf % kAlign) return GORGO_ERR_INVALID_ARG;
-  const Model& m = sim->m;
-  const uint64_t N = n_requests;
-  if (N < 1 || N >= 0xFFFFFFFFull) return GORGO_ERR_BAD_TRACE;
+  if (n_requests < 1 || n_requests >= 0xFFFFFFFFull) return GORGO_ERR_BAD_TRACE;
   if (hash_off[0] != 0) return GORGO_ERR_BAD_TRACE;
-  for (uint64_t r = 0; r < N; ++r)
+  for (uint64_t r = 0; r < n_requests; ++r)
     if (hash_off[r + 1] < hash_off[r]) return GORGO_ERR_BAD_TRACE;
-  const uint64_t T = hash_off[N];
-  if (T >= 0xFFFFFFFFull) return GORGO_ERR_BAD_TRACE;
-  if (T > 0 && !hash_ids) return GORGO_ERR_INVALID_ARG;
-  uint64_t need = 0;
-  gorgo_trace_bytes(N, T, &need);
-  if (dev_trace_bytes < need) return GORGO_ERR_WORKSPACE_TOO_SMALL;
-  const uint64_t nmax = m.C < 65535 ? m.C : 65535;
-
-  std::vector<ReqRec> req(N);
-  double prev_t = 0.0;
-  for (uint64_t r = 0; r < N; ++r) {
-    const double t = ts_ms[r];
-    if (!finite_nonneg(t) || t < prev_t) return GORGO_ERR_BAD_TRACE;
-    prev_t = t;
-    const uint64_t n = hash_off[r + 1] - hash_off[r];
-    const uint64_t want = ((uint64_t)input_tokens[r] + m.B - 1) / m.B;
-    if (n != want || n > nmax) return GORGO_ERR_BAD_TRACE;
-    const uint16_t g = origin ? origin[r] : (uint16_t)0;
-    if (g >= m.G) return GORGO_ERR_BAD_TRACE;
-    ReqRec& q = req[r];
-    q.ts_ms = t; q.off = (uint32_t)hash_off[r]; q.in_tok = input_tokens[r];
-    q.out_tok = output_tokens[r]; q.nblk = (uint16_t)n; q.origin = g; q.prev_share = kNone; q.pad = 0;
-  }
-
-  // dense renumbering in order of first appearance; an id twice in one request is an error
-  std::vector<uint32_t> ids(T);
-  std::vector<uint64_t> raw;
-  {
-    IdMap map(1ull << 16);
-    std::vector<uint32_t> seen_in;  // request (+1) that last contained the dense id
-    uint32_t next = 0;
-    for (uint64_t r = 0; r < N; ++r) {
-      uint32_t latest = 0;  // latest earlier request (+1) that contains one of this one's blocks
-      for (uint64_t g = hash_off[r]; g < hash_off[r + 1]; ++g) {
-        const uint32_t before = next;
-        const uint32_t d = map.get_or_add(hash_ids[g], next);
-        if (next != before) { raw.push_back(hash_ids[g]); seen_in.push_back(0); }
-        if (seen_in[d] == (uint32_t)r + 1) return GORGO_ERR_BAD_TRACE;
-        if (seen_in[d] > latest) latest = seen_in[d];
-        seen_in[d] = (uint32_t)r + 1;
-        ids[g] = d;
-      }
-      req[r].prev_share = latest ? latest - 1 : kNone;
+  // a fixed trace is an appendable one of exactly its own size, built in one batch
+  int rc = trace_begin_impl(sim, n_requests, hash_off[n_requests], dev_trace_buf, dev_trace_bytes);
+  if (rc == GORGO_OK) {
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    rc = trace_append_impl(sim, n_requests, ts_ms, input_tokens, output_tokens, origin, hash_off,
+                           hash_ids, st, false);
+    if (rc == GORGO_OK) {
+      DeviceGuard guard(sim->device);
+      if (!guard.ok || cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); rc = GORGO_ERR_CUDA; }
     }
   }
-  const uint64_t D = raw.size();
+  sim->tb.reset();           // nothing can be appended to an uploaded trace
+  if (rc != GORGO_OK) sim->has_trace = false;
+  return rc;
+}
 
-  // next and previous occurrence of the same block, and the request each belongs to
-  std::vector<uint2> occ(T), occ_before(T);
-  {
-    std::vector<uint32_t> last_g(D, kNone), last_r(D, kNone);
-    for (uint64_t r = N; r-- > 0;) {
-      for (uint64_t g = hash_off[r + 1]; g-- > hash_off[r];) {
-        const uint32_t d = ids[g];
-        occ[g] = make_uint2(last_g[d], last_r[d]);
-        last_g[d] = (uint32_t)g;
-        last_r[d] = (uint32_t)r;
-      }
-    }
-    std::fill(last_g.begin(), last_g.end(), kNone);
-    std::fill(last_r.begin(), last_r.end(), kNone);
-    for (uint64_t r = 0; r < N; ++r) {
-      for (uint64_t g = hash_off[r]; g < hash_off[r + 1]; ++g) {
-        const uint32_t d = ids[g];
-        occ_before[g] = make_uint2(last_g[d], last_r[d]);
-        last_g[d] = (uint32_t)g;
-        last_r[d] = (uint32_t)r;
-      }
-    }
-  }
+int gorgo_trace_begin(gorgo_sim_t* sim, uint64_t max_requests, uint64_t max_block_ids,
+                      void* dev_trace_buf, uint64_t dev_trace_bytes) {
+  const int rc = trace_begin_impl(sim, max_requests, max_block_ids, dev_trace_buf, dev_trace_bytes);
+  if (rc == GORGO_OK) { sim->cap_req = max_requests; sim->cap_ids = max_block_ids; }
+  return rc;
+}
 
-  // time grid over the arrivals: grid[b] = first request with ts >= b * dt, b = 0..n_grid, with
-  // about one request per bucket; none when all requests arrive at one instant
-  uint32_t n_grid = 0;
-  double grid_dt = 0.0;
-  std::vector<uint32_t> grid;
-  {
-    const double span = ts_ms[N - 1];
-    const double dt = span / (double)N;
-    if (dt > 0.0 && std::isfinite(dt) && dt >= span * 0x1p-40) {
-      n_grid = (uint32_t)N;
-      grid_dt = dt;
-      grid.resize((size_t)n_grid + 1);
-      uint64_t r = 0;
-      for (uint32_t b = 0; b <= n_grid; ++b) {
-        const double edge = (double)b * dt;
-        while (r < N && ts_ms[r] < edge) ++r;
-        grid[b] = (uint32_t)(r < N ? r : N - 1);
-      }
-    }
-  }
-
-  DeviceGuard guard(sim->device);
-  if (!guard.ok) return GORGO_ERR_CUDA;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  unsigned char* base = static_cast<unsigned char*>(dev_trace_buf);
-  uint64_t o = 0;
-  unsigned char* d_req = base + o; o += align_up(N * sizeof(ReqRec));
-  unsigned char* d_ids = base + o; o += align_up(T * 4);
-  unsigned char* d_occ = base + o; o += align_up(T * 8);
-  unsigned char* d_raw = base + o; o += align_up(D * 8);
-  unsigned char* d_prev = base + o; o += align_up(T * 8);
-  unsigned char* d_ts = base + o; o += align_up(N * 8);
-  unsigned char* d_grid = base + o; o += align_up((N + 1) * 4);
-  bool ok = cudaMemcpyAsync(d_req, req.data(), N * sizeof(ReqRec), cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(d_ts, ts_ms, N * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (n_grid > 0)
-    ok = ok && cudaMemcpyAsync(d_grid, grid.data(), ((size_t)n_grid + 1) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (T > 0) {
-    ok = ok && cudaMemcpyAsync(d_ids, ids.data(), T * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(d_occ, occ.data(), T * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(d_raw, raw.data(), D * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(d_prev, occ_before.data(), T * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  }
-  ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
-  if (!ok) { cudaGetLastError(); sim->has_trace = false; return GORGO_ERR_CUDA; }
-  sim->tr.req = reinterpret_cast<const ReqRec*>(d_req);
-  sim->tr.ids = reinterpret_cast<const uint32_t*>(d_ids);
-  sim->tr.occ_next = reinterpret_cast<const uint2*>(d_occ);
-  sim->tr.occ_prev = reinterpret_cast<const uint2*>(d_prev);
-  sim->tr.raw_id = reinterpret_cast<const uint64_t*>(d_raw);
-  sim->tr.ts = reinterpret_cast<const double*>(d_ts);
-  sim->tr.grid = reinterpret_cast<const uint32_t*>(d_grid);
-  sim->tr.grid_dt = grid_dt;
-  sim->tr.grid_n = n_grid;
-  sim->tr.n_req = (uint32_t)N; sim->tr.n_ids = (uint32_t)T; sim->tr.n_distinct = (uint32_t)D;
-  sim->has_trace = true;
-  return GORGO_OK;
+int gorgo_trace_append(gorgo_sim_t* sim, uint64_t n_requests, const double* ts_ms,
+                       const uint32_t* input_tokens, const uint32_t* output_tokens,
+                       const uint16_t* origin, const uint64_t* hash_off, const uint64_t* hash_ids,
+                       void* cuda_stream) {
+  if (!sim || !ts_ms || !input_tokens || !output_tokens || !hash_off) return GORGO_ERR_INVALID_ARG;
+  if (!sim->tb) return GORGO_ERR_NO_TRACE;
+  return trace_append_impl(sim, n_requests, ts_ms, input_tokens, output_tokens, origin, hash_off,
+                           hash_ids, static_cast<cudaStream_t>(cuda_stream), true);
 }
 
 int gorgo_trace_info(const gorgo_sim_t* sim, uint64_t* n_requests, uint64_t* n_block_ids,
@@ -959,7 +1065,7 @@ int gorgo_sim_reset(gorgo_sim_t* sim, void* state_workspace, uint64_t state_byte
   if (!guard.ok) return GORGO_ERR_CUDA;
   unsigned char* base = static_cast<unsigned char*>(state_workspace);
   if (launch_reset(base + w.masks, w.mask_stride, reinterpret_cast<uint32_t*>(base + w.exp_head),
-                   sim->tr.n_req, base + w.states, w.st, sim->m, 1,
+                   sim->cap_req ? sim->cap_req : sim->tr.n_req, base + w.states, w.st, sim->m, 1,
                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
     return GORGO_ERR_CUDA;
   return GORGO_OK;
@@ -1001,6 +1107,7 @@ int gorgo_route_batch(gorgo_sim_t* sim, const double* params, double time_scale,
   a.exp_rec = reinterpret_cast<uint4*>(base + w.exp_rec);
   a.lru_next = reinterpret_cast<uint32_t*>(base + w.lru_next);
   a.route_log = base + w.route_log; a.route_log_stride = N;
+  a.finish_log = reinterpret_cast<double*>(base + w.finish);
   if (attach_speeds(sim, base, w, st, &a) != GORGO_OK) return GORGO_ERR_CUDA;
   a.route_out = route; a.hit_out = hit_blocks; a.ttft_out = ttft_ms; a.e2e_out = e2e_ms;
   a.out_stride = count;

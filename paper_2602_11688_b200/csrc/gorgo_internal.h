@@ -35,7 +35,10 @@ static_assert(sizeof(RepState) == 32, "RepState layout");
 struct __align__(32) CandHeader {
   uint32_t processed;  // requests replayed so far
   int32_t status;      // 0, or a gorgo_status recorded by a kernel
-  uint32_t pad[6];
+  uint32_t overflow;   // persistent state: 1 + the newest request that completes after the end of
+                       // the trace known so far (0: none); such requests are chained through
+                       // their completion records until an appended request takes them
+  uint32_t pad[5];
 };
 
 // Device-resident trace (pointers into the caller's trace buffer).
@@ -106,6 +109,8 @@ struct ReplayArgs {
   // [R] each) or null for the uniform constants of the model
   const double* rep_prefill_ms;
   const double* rep_tpot_ms;
+  // persistent state only: finish time of every request that completes after the trace's end
+  double* finish_log;
   // 1: the score takes prefix hits from the proxy's own index (blocks ever dispatched to a
   // replica) instead of the replica's cache
   uint32_t proxy_index;
@@ -171,6 +176,10 @@ cudaError_t launch_policy_routes(const TraceView& tr, uint32_t R, bool affinity,
 // Cycle accounting build only: the 64 accumulators (decide warp at 0, cache warp at 16).
 cudaError_t prof_read(unsigned long long* out64, bool reset);
 #endif
+// After requests [first_new, first_new + n_new) were appended: every block of theirs whose previous
+// occurrence lies before flat position `ids_before` becomes that occurrence's successor.
+cudaError_t launch_link_occurrences(const TraceView& tr, uint32_t first_new, uint32_t n_new,
+                                    uint32_t ids_before, uint2* occ_next, cudaStream_t st);
 cudaError_t launch_gather(const void* buf, uint64_t n_sectors, uint32_t per_thread, uint32_t blocks,
                           uint32_t* sink, cudaStream_t st);
 uint32_t window_max();          // largest window the window kernel handles

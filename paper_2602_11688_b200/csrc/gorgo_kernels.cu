@@ -373,6 +373,8 @@ template <typename MaskT>
 struct Ctx {
   Smem sm;
   MaskT* mask;
+  CandHeader* hdr;
+  double* finish_log;
   uint32_t* exp_head;
   uint4* exp_rec;
   uint32_t* lru_next;
@@ -580,6 +582,9 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
   uint32_t routed_seen = a.first, published = a.first;
   uint32_t idle = 0;
   bool failed = false;
+  // persistent state: requests that complete after the last known arrival are chained here
+  // (1 + request, 0: none) until the trace has grown past their finish time
+  uint32_t overflow = cx.finish_log ? cx.hdr->overflow : 0u;
 
   PROF_BEGIN();
   while (true) {
@@ -709,6 +714,13 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
         j1 = s; f1 = finish; tok1 = in_tok; rep1 = istar;
         ins1 = s + 1 < N && t_last >= finish;
         lo1 = s + 1;
+        if (!ins1 && cx.finish_log) {
+          if (lane == 0) {
+            cx.finish_log[s] = finish;
+            cx.exp_rec[s] = make_uint4(overflow - 1u, in_tok, istar, 0u);
+          }
+          overflow = s + 1;
+        }
         if (ins1 && use_grid && lane == 0) {
           const double bf = __dmul_rn(finish, to_bucket);
           uint32_t b = 0;
@@ -730,6 +742,7 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
     PROF_LAP(5);
   }
   PROF_END(16);
+  if (cx.finish_log && lane == 0) cx.hdr->overflow = overflow;
   status = __reduce_min_sync(kFull, status);
   if (lane == 0 && status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
 }
@@ -1532,6 +1545,8 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
   }
   cx.mask = reinterpret_cast<MaskT*>(a.masks + (size_t)p * a.mask_stride);
   cx.slot_kv = reinterpret_cast<unsigned long long*>(st + a.lay.slot_kv_off);
+  cx.hdr = hdr;
+  cx.finish_log = a.finish_log ? a.finish_log + (size_t)p * N : nullptr;
   cx.exp_head = a.exp_head + (size_t)p * N;
   cx.exp_rec = a.exp_rec + (size_t)p * N;
   cx.lru_next = a.lru_next + (size_t)p * N;
@@ -1563,6 +1578,31 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
     *cx.status = 0; *cx.probe_gone = 0; *sm.abort_flag = 0;
     *sm.routed = a.first; *sm.exp_ready = a.first; *sm.jobs = a.first;
     sm.serviced[0] = a.first; if (kServices > 1) sm.serviced[1] = a.first;
+  }
+  if (cx.finish_log && threadIdx.x == 32) {
+    // the trace may have grown since the last batch: requests that were to complete after its
+    // old end are filed under the first request, not yet replayed, that arrives at or after
+    // their finish time; the rest stay chained
+    const double scale = a.scales ? a.scales[p] : a.scale;
+    const double t_last = __dmul_rn(scale, a.tr.ts[N - 1]);
+    uint32_t e = hdr->overflow - 1u, keep = kNone;
+    #pragma unroll 1
+    for (uint32_t guard = 0; e != kNone && guard < N; ++guard) {
+      uint4 rec = cx.exp_rec[e];
+      const uint32_t nxt = rec.x;
+      const double f = cx.finish_log[e];
+      if (e + 1 < N && t_last >= f) {
+        const uint32_t x = first_arrival_at_or_after(a.tr.ts, scale, f, max(e + 1u, a.first), N - 1);
+        rec.x = cx.exp_head[x];
+        cx.exp_head[x] = e;
+      } else {
+        rec.x = keep;
+        keep = e;
+      }
+      cx.exp_rec[e] = rec;
+      e = nxt;
+    }
+    hdr->overflow = keep + 1u;
   }
   if (threadIdx.x < kCommitWarps) sm.progress[threadIdx.x] = a.first;
   if (threadIdx.x < kStageDepth) cx.st_ready[threadIdx.x] = 0;
@@ -1601,6 +1641,20 @@ __global__ void __launch_bounds__(kReplayThreads, kReplayMinCtas) replay_kernel(
 }
 
 // ------------------------------------------------------------------------------- reset
+// One warp per appended request: a block whose previous occurrence belongs to an earlier batch
+// becomes that occurrence's successor.
+__global__ void link_occurrences_kernel(TraceView tr, uint32_t first_new, uint32_t n_new,
+                                        uint32_t ids_before, uint2* occ_next) {
+  const uint32_t k = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+  if (k >= n_new) return;
+  const uint32_t r = first_new + k;
+  const ReqRec q = tr.req[r];
+  for (uint32_t c = threadIdx.x % 32; c < q.nblk; c += 32) {
+    const uint2 pv = tr.occ_prev[q.off + c];
+    if (pv.x != kNone && pv.x < ids_before) occ_next[pv.x] = make_uint2(q.off + c, r);
+  }
+}
+
 __global__ void reset_states_kernel(unsigned char* states, StateLayout lay, uint32_t R, uint32_t S,
                                     uint32_t n_cand) {
   const uint32_t p = blockIdx.x;
@@ -1952,6 +2006,12 @@ cudaError_t launch_reset(unsigned char* masks, uint64_t mask_bytes_total, uint32
   e = cudaMemsetAsync(exp_head, 0xFF, exp_head_count * sizeof(uint32_t), st);   // kNone: empty lists
   if (e != cudaSuccess) return e;
   reset_states_kernel<<<n_cand, 128, 0, st>>>(states, lay, m.R, m.S, n_cand);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_link_occurrences(const TraceView& tr, uint32_t first_new, uint32_t n_new,
+                                    uint32_t ids_before, uint2* occ_next, cudaStream_t st) {
+  link_occurrences_kernel<<<(n_new + 7) / 8, 256, 0, st>>>(tr, first_new, n_new, ids_before, occ_next);
   return cudaGetLastError();
 }
 
