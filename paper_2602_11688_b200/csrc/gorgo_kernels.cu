@@ -336,6 +336,9 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
         tail += __popc(lv);
       }
       cp -= 32 * kScoutBatches;
+      // every lane's entries are stored before lane 0 publishes the new tail (the lanes that
+      // listed nothing must not run ahead of the ones that did)
+      __syncwarp();
       __threadfence_block();
       if (lane == 0) {
         sm.scan_cr[i] = cr;

@@ -225,6 +225,51 @@ def test_route_batch_continues_a_persistent_state():
     sim.close()
 
 
+@pytest.mark.parametrize("R", [3, 17, 64])
+def test_many_small_batches_on_tiny_caches_repeatedly(R):
+    # Every batch starts with full caches, so its first commits evict while the scout warps have
+    # only just begun to list victims: the commit warps then take each victim the moment it is
+    # published.  Routes and the cache digest after every batch must equal the oracle's in every
+    # repetition (a hand-over that is not ordered shows up as a rare mismatch).
+    import torch
+    from paper_2602_11688_b200 import binding as gb
+    from tests.util import small_trace
+    rng = np.random.default_rng(R)
+    reqs = small_trace(R + 5, n_req=260, structured=False, rate_ms=12.0)
+    K = 3 + R if R > 32 else 3
+    par = np.concatenate([rng.normal(1.0, 0.3, size=3), rng.lognormal(0, 0.3, size=K - 3)])
+    w = W.handmade(rng.uniform(5, 60, size=R), reqs, slots=2, cache_blocks=9, params=[par])
+    N = w.n_requests
+    ends = list(range(20, N, 20)) + [N]
+    o = O.Oracle.from_workload(w)
+    want_route, want_digest, first = [], [], 0
+    for e in ends:
+        want_route.append(o.run(par, 0.8, e - first).route)
+        want_digest.append(o.digest().tolist())
+        first = e
+    o.close()
+    want_route = np.concatenate(want_route)
+    sim = gb.GorgoSim(w)
+    rc, nbytes = gb.gorgo_state_bytes(sim.h)
+    state = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    for rep in range(25):
+        assert gb.gorgo_sim_reset(sim.h, state, sim.stream) == gb.GORGO_OK
+        route = torch.empty(N, dtype=torch.uint8, device="cuda")
+        digests, first = [], 0
+        for e in ends:
+            assert gb.gorgo_route_batch(sim.h, par, 0.8, first, e - first, state, sim.stream,
+                                        route[first:]) == gb.GORGO_OK
+            dg = torch.empty((R, 2), dtype=torch.uint64, device="cuda")
+            assert gb.gorgo_state_digest(sim.h, state, sim.stream, dg) == gb.GORGO_OK
+            digests.append(dg)
+            first = e
+        torch.cuda.synchronize()
+        assert route.cpu().numpy().tolist() == want_route.tolist(), rep
+        for b, dg in enumerate(digests):
+            assert dg.cpu().numpy().tolist() == want_digest[b], (rep, ends[b])
+    sim.close()
+
+
 def test_abi_rejects_bad_input():
     import torch
     from paper_2602_11688_b200 import binding as gb
