@@ -95,12 +95,13 @@ class ClockSampler:
         return out
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the replay kernel per
-# candidate x request, from the ncu captures summarised under profiles/ (taken on reduced cases
-# of the workload, which hold a few GB on the device; the per-request figure barely moves with
-# the trace length, see there).  Reported only while the kernel source is the one that was
-# captured (first 16 hex digits of its sha256); scaled to a full launch by the units it processes.
-NCU_TRAFFIC = {"longctx": {"bytes_per_candidate_request": None, "kernel_sha256_16": None}}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one replay-kernel launch per
+# candidate x request, from the single-pass ncu capture of the full-size workload summarised under
+# profiles/ (the per-request figure grows with the footprint, so a reduced case is not scaled up).
+# Reported only while the kernel source is the one that was captured (first 16 hex digits of its
+# sha256) and only for the unreduced workload.
+NCU_TRAFFIC = {"longctx": {"bytes_per_candidate_request": (122_645_897_472 + 44_458_263_296) / (256 * 500_000),
+                           "kernel_sha256_16": "cae79d007fb1877a"}}
 
 
 def kernel_sha16():
@@ -226,6 +227,9 @@ def main():
     ap.add_argument("--cache-blocks", type=int, default=None)
     ap.add_argument("--ref-requests", type=int, default=None,
                     help="requests per candidate in one reference / cpu-baseline sample")
+    ap.add_argument("--all-scales", action="store_true",
+                    help="evaluate the population at every time scale of the workload as ONE "
+                         "population (candidates x scales) instead of the first scale only")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-yardsticks", action="store_true",
                     help="skip the random-sector and L2 gather measurements")
@@ -274,6 +278,12 @@ def main():
 
     base_params = w.params
     w.params = sharding.weak_scaling_population(base_params, rank)
+    cand_scales = None
+    if args.all_scales:
+        all_scales = np.asarray(w.spec.time_scales, dtype=np.float64)
+        P0 = w.params.shape[0]
+        cand_scales = np.repeat(all_scales, P0)
+        w.params = np.tile(w.params, (len(all_scales), 1))
     P, N, R, K = w.params.shape[0], w.n_requests, w.spec.n_replicas, w.n_params
 
     sim = gb.GorgoSim(w, device=local)
@@ -291,13 +301,34 @@ def main():
     h_p95_e = torch.empty(P, dtype=torch.float64).pin_memory()
 
     def step_device(with_stats=False):
-        rc = gb.gorgo_eval_population(sim.h, P, d_params, scale, sim.workspace, stream, p95_t,
-                                      p95_e, None, None, None, stats if with_stats else None,
-                                      status)
+        if cand_scales is not None and not with_stats:
+            rc = gb.gorgo_eval_population_scales(sim.h, P, d_params, cand_scales, sim.workspace,
+                                                 stream, p95_t, p95_e, None, None, None, status)
+        elif cand_scales is not None:
+            # counters of the byte model: one evaluation per scale (the call with per-candidate
+            # scales has no counter output)
+            P0 = P // len(all_scales)
+            rc = gb.GORGO_OK
+            for k, sc in enumerate(all_scales):
+                sl = slice(k * P0, (k + 1) * P0)
+                rc = rc or gb.gorgo_eval_population(sim.h, P0, d_params[sl], float(sc), sim.workspace,
+                                                    stream, p95_t[sl], p95_e[sl], None, None, None,
+                                                    stats[sl], status[sl])
+        else:
+            rc = gb.gorgo_eval_population(sim.h, P, d_params, scale, sim.workspace, stream, p95_t,
+                                          p95_e, None, None, None, stats if with_stats else None,
+                                          status)
         if rc != gb.GORGO_OK:
             raise gb.GorgoError(rc, "gorgo_eval_population")
 
     def step_host():
+        if cand_scales is not None:       # (no host-buffer call with per-candidate scales: copies here)
+            d_params.copy_(h_params, non_blocking=True)
+            step_device()
+            h_p95_t.copy_(p95_t, non_blocking=True)
+            h_p95_e.copy_(p95_e, non_blocking=True)
+            torch.cuda.current_stream(dev).synchronize()
+            return
         rc = gb.gorgo_eval_population_host(sim.h, P, h_params, scale, sim.workspace, stream,
                                            h_p95_t, h_p95_e)
         if rc != gb.GORGO_OK:
@@ -369,7 +400,7 @@ def main():
     #      its kernels timed by the library's own events on the launching stream
     win_ms, win_launches = None, 0
     rc, n_win = gb.gorgo_window_count(N, 128, 32)
-    if n_win > 0:
+    if n_win > 0 and cand_scales is None:
         best_w = torch.empty(P, dtype=torch.float64, device=dev)
         gb.gorgo_set_profiling(sim.h, True)
         rc = gb.gorgo_eval_population_windows(sim.h, P, d_params, scale, sim.workspace, stream, 128,
@@ -398,6 +429,7 @@ def main():
                 yard["l2_peak"] = {"value": gbs, "unit": "GB/s", "footprint_bytes": small}
 
     if rank == 0:
+        rc, ctas_per_sm, smem_cta = gb.gorgo_replay_occupancy(sim.h)
         peak, peak_kind = measured_peak_gbs()
         launch_ms = replay["ms"] / max(1, replay["launches"])
         bytes_per_launch = alg_bytes / waves
@@ -430,7 +462,9 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {**workload_config(w, scale), "resident_candidates": resident, "waves": waves,
+            "config": {**workload_config(w, "all of %s" % list(map(float, all_scales)) if args.all_scales else scale),
+                       "resident_candidates": resident, "waves": waves,
+                       "replay_ctas_per_sm": int(ctas_per_sm), "replay_smem_bytes_per_cta": int(smem_cta),
                        "l2": l2_note},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(P * K * 8),
                     "d2h_bytes_per_step": int(P * 20), "ms_per_step": e2e_ms,
@@ -447,7 +481,7 @@ def main():
                 "achieved": win_bytes / (win_ms * 1e-3) / 1e9, "unit": "GB/s",
                 "frac_of_hbm_peak": win_bytes / (win_ms * 1e-3) / 1e9 / peak,
                 "share_of_step": win_ms / ms_per_step}
-        if not args.no_cpu_baseline and world == 1:
+        if not args.no_cpu_baseline and world == 1 and cand_scales is None:
             cores = max(1, min(os.cpu_count() or 1, 8))
             n_cand = oracle_candidates(w, cores)
             n_req = min(N, args.ref_requests)

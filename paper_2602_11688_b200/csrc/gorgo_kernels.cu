@@ -585,9 +585,6 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
   uint32_t routed_seen = a.first, published = a.first;
   uint32_t idle = 0;
   bool failed = false;
-  // persistent state: requests that complete after the last known arrival are chained here
-  // (1 + request, 0: none) until the trace has grown past their finish time
-  uint32_t overflow = cx.finish_log ? cx.hdr->overflow : 0u;
 
   PROF_BEGIN();
   while (true) {
@@ -717,12 +714,11 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
         j1 = s; f1 = finish; tok1 = in_tok; rep1 = istar;
         ins1 = s + 1 < N && t_last >= finish;
         lo1 = s + 1;
-        if (!ins1 && cx.finish_log) {
-          if (lane == 0) {
-            cx.finish_log[s] = finish;
-            cx.exp_rec[s] = make_uint4(overflow - 1u, in_tok, istar, 0u);
-          }
-          overflow = s + 1;
+        if (!ins1 && cx.finish_log && lane == 0) {
+          // completes after the last known arrival: chained in the state (read by the next launch)
+          cx.finish_log[s] = finish;
+          const uint32_t before = atomicExch(&cx.hdr->overflow, s + 1u);
+          cx.exp_rec[s] = make_uint4(before - 1u, in_tok, istar, 0u);
         }
         if (ins1 && use_grid && lane == 0) {
           const double bf = __dmul_rn(finish, to_bucket);
@@ -745,7 +741,6 @@ __device__ __forceinline__ void service_warp(const ReplayArgs& a, const Ctx<Mask
     PROF_LAP(5);
   }
   PROF_END(16);
-  if (cx.finish_log && lane == 0) cx.hdr->overflow = overflow;
   status = __reduce_min_sync(kFull, status);
   if (lane == 0 && status != 0) atomicMin(const_cast<int32_t*>(cx.status), status);
 }
@@ -1469,8 +1464,8 @@ __device__ __forceinline__ void role_of(uint32_t warp, Role& role, uint32_t& whi
   const uint32_t sched = warp & 3u, k = warp >> 2;
   which = k;
   if (sched == 0) role = k == 0 ? kRoleRoute : k == 1 ? kRoleExpiry : kRoleScout;
-  else if (sched == 1) { role = k == 0 ? kRoleGate : (k - 1 < kServices ? kRoleService : kRoleScout); which = k - 1; }
-  else if (sched == 2) role = k < kProbes ? kRoleProbe : (kServices == 2 && k == 2 ? kRoleScout : kRoleNone);
+  else if (sched == 1) { role = k == 0 ? kRoleGate : k == 1 ? kRoleService : kRoleScout; which = 0; }
+  else if (sched == 2) { role = k < kProbes ? kRoleProbe : (kServices == 2 && k == 2 ? kRoleService : kRoleNone); if (role == kRoleService) which = 1; }
   else role = k < kCommitWarps ? kRoleCommit : kRoleNone;
   if (role == kRoleScout) which = sched == 0 ? 0 : 1;      // scout 0 and scout 1
 }

@@ -17,27 +17,29 @@ import json
 import numpy as np
 
 ROLES = {
-    "route": (0, ["wait for completion sums / ring room", "completion sums, queue term of the score",
-                  "wait for the prefix hits", "score and order key", "argmin over replicas",
-                  "hit of the chosen replica, route stores, barrier", None, None,
-                  "gate's hand-over stamp -> route warp past the barrier"]),
+    "route": (0, ["load update of the previous route, wait for the completion sums",
+                  "completion sums, queue term of the score", "wait for the prefix hits (barrier)",
+                  "staged part of the score, order key", "argmin over replicas",
+                  "hit of the chosen replica, route stores, barrier arrive"]),
     "service": (16, ["retire: list entry, window vote, grid value", "fence and publish",
-                     "issue list exchange and window loads", "slot argmin",
+                     "next pipeline stage: list exchange, window loads", "slot argmin",
                      "times, outputs, grid load", "idle round"]),
-    "gate": (32, ["hand-over at the request's own turn (rest)", "wait for the route",
-                  "job, early hand-over of the next request", "own turn: wait for the staged read",
-                  "own turn: wait for commits", "early: route read, job post", "early: staged?", "early: shares/conflict",
-                  "route warp's stamp -> gate warp past the barrier", None,
-                  "#not early: shares a block with a recent request", "#probes redone here",
-                  "#not early: not staged yet", "#not early: recent route to a holder of its blocks",
+    "gate": (32, ["own turn: probe here if needed, hand over", "wait for the route (barrier)",
+                  "job post, early hand-over of the next request",
+                  "own turn: staged? recent route to a holder?", "own turn: wait for commits",
+                  None, None, None, None, None, None,
+                  "#probes done by this warp", "#next request not staged yet at hand-over time",
+                  "#next request not handed over early (shared block or recent route to a holder)",
                   "#hits handed over early"]),
-    "commit (all warps)": (48, ["wait for the next routed request", "need and eviction",
-                                "mask bits of the inserted blocks", "recency list, progress",
-                                "requests of other warps' replicas", None,
-                                None, None, "#evictions: clean case", "#evictions: an entry was void or touched again",
-                                "#evictions: ring held too few entries", "#evictions: more than 96 victims or ring not in use",
-                                "#requests that evict", "#evictions finished by own walk", "#polls for ring entries",
-                                "#blocks evicted"]),
+    "commit (all three warps)": (48, ["wait for the next routed request", "need and eviction",
+                                      "mask bits of the inserted blocks", "recency list, progress",
+                                      "requests of other warps' replicas", None, None, None,
+                                      "#evictions: clean case (victims taken from the ring as listed)",
+                                      "#evictions: an entry was void or touched again",
+                                      "#evictions: ring held too few entries",
+                                      "#evictions: more than 96 victims or ring not in use",
+                                      "#requests that evict", "#evictions finished by own walk",
+                                      "#polls for ring entries", "#blocks evicted"]),
 }
 
 
