@@ -100,8 +100,8 @@ class ClockSampler:
 # profiles/ (the per-request figure grows with the footprint, so a reduced case is not scaled up).
 # Reported only while the kernel source is the one that was captured (first 16 hex digits of its
 # sha256) and only for the unreduced workload.
-NCU_TRAFFIC = {"longctx": {"bytes_per_candidate_request": (122_645_897_472 + 44_458_263_296) / (256 * 500_000),
-                           "kernel_sha256_16": "cae79d007fb1877a"}}
+NCU_TRAFFIC = {"longctx": {"bytes_per_candidate_request": (120_785_143_040 + 44_431_718_144) / (256 * 500_000),
+                           "kernel_sha256_16": "31f37f777b3f47f3"}}
 
 
 def kernel_sha16():

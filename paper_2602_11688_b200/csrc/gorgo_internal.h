@@ -173,7 +173,7 @@ cudaError_t launch_window(const WindowArgs& a, uint32_t n_cand, cudaStream_t st)
 cudaError_t launch_policy_routes(const TraceView& tr, uint32_t R, bool affinity,
                                  const uint32_t* draws, uint8_t* route, cudaStream_t st);
 #ifdef GORGO_PROF
-// Cycle accounting build only: the 64 accumulators (decide warp at 0, cache warp at 16).
+// Cycle accounting build only: the 64 accumulators (route warp at 0, service at 16, gate at 32, commit warps at 48).
 cudaError_t prof_read(unsigned long long* out64, bool reset);
 #endif
 // After requests [first_new, first_new + n_new) were appended: every block of theirs whose previous

@@ -12,18 +12,25 @@
 //    block's latest touch on replica i iff no later occurrence of the block (static
 //    `occ_next` links computed at upload) belongs to a request routed to i.  Live touches at
 //    the cursor are the LRU victims; stale ones are skipped for good;
-//  * in-flight accounting through per-slot FIFO chains (finish times on one slot never
-//    decrease), with the earliest finish per replica cached so the common case is one compare.
+//  * completions as per-request lists: a routed request stops counting in the queue signal at
+//    the first later request that arrives at or after its finish time; the service warp finds
+//    that request (time grid over the arrivals, then a 32-wide window) and pushes the completion
+//    onto its list, the expiry warp sums every request's list ahead of the route warp.
 // Requests are strictly ordered inside a candidate and every step depends on the one before, so
-// a replay is bound by the latency of that chain, not by bandwidth.  One CTA of five warps
+// a replay is bound by the latency of that chain, not by bandwidth.  One CTA of twelve warps
 // replays one candidate and the warps split the chain:
-//   decide  queue signal, score (Eq. 3), argmin, service model, outputs;
-//   cache   validates the staged prefix hits, sizes and performs the eviction, recency list;
-//   probe   runs up to three requests ahead: reads block ids and mask words, probes them and
-//           stages hits and the hit-dependent part of the score in shared memory;
-//   scout   (two warps) validate touches ahead of every replica's eviction cursor and keep a
-//           ring of ready victims per replica.
-// A staged read may predate the commits of the last three requests; the cache warp knows which
+//   route    queue signal, score (Eq. 3), argmin; reads no global memory;
+//   gate     decides whether the staged prefix hits of the next request may be used, else
+//            waits for the commits concerned and probes itself; posts the commit jobs;
+//   probe    (two warps) run up to kWindow requests ahead: read block ids and mask words,
+//            probe them and stage hits and the hit-dependent part of the score;
+//   commit   (three warps, replicas split) size and perform the eviction, set the mask bits,
+//            keep the recency lists;
+//   scout    (two warps) validate touches ahead of every replica's eviction cursor and keep a
+//            ring of ready victims per replica;
+//   service  slots, start / first-token / finish times, outputs, completion filing;
+//   expiry   completion sums per request.
+// A staged read may predate the commits of the last kWindow requests; the gate warp knows which
 // of those commits can have touched the request (shared block, or evicted block that occurs in
 // it) and then repeats the read itself, so results never depend on the timing of the warps.
 #include "gorgo_internal.h"
@@ -34,9 +41,9 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
-// Cycle accounting of the two serial warps (built only with -DGORGO_PROF; the normal library
+// Cycle accounting of the warps (built only with -DGORGO_PROF; the normal library
 // carries none of it).  Every lap adds the SM clock ticks since the previous lap of the same
-// warp to one of 32 per-role accumulators; the totals of all candidates end up in g_prof.
+// warp to one of 16 per-role accumulators; the totals of all candidates end up in g_prof.
 #ifdef GORGO_PROF
 __device__ unsigned long long g_prof[64];
 #define PROF_BEGIN() unsigned long long pf[16] = {}; long long pf_t = clock64()
@@ -196,12 +203,12 @@ struct Smem {
   volatile uint32_t* exp_ready;   // requests whose completion sums are published
   uint32_t* route_ring;           // [kRouteRing] chosen replica | prefix hit there << 8
   long long* exp_sum;             // [kExpRing][R] tokens (or requests) that completed by the request's arrival
-  // eviction rings, one per replica: filled by the scout warp, drained by the replay warp.
+  // eviction rings, one per replica: filled by the scout warp, drained by the commit warp.
   // entry = (block id, request of the block's next occurrence after the entry was made or kNone,
   //          position of the touch in its request, request of the touch), in eviction order
   uint4* lst;                     // [R][kListCap]
   volatile uint32_t* act;         // replay -> scout: the replica's cache is close to full
-  volatile uint32_t* ring_head;   // entries consumed (replay warp)
+  volatile uint32_t* ring_head;   // entries consumed (commit warp)
   volatile uint32_t* ring_tail;   // entries produced (scout warp)
   volatile uint32_t* scan_cr;     // scout's own cursor into the recency order (set at activation)
   volatile int32_t* scan_cp;
@@ -245,7 +252,7 @@ __device__ __forceinline__ uint32_t wait_serviced(const Smem& sm, uint32_t want,
 
 // Scout warp: for every replica whose cache is close to full it walks the recency order ahead
 // of the eviction cursor and appends to the replica's ring the touches that are still the latest
-// touch of their block (the coming eviction victims, in order).  The replay warp evicts from the
+// touch of their block (the coming eviction victims, in order).  The commit warp evicts from the
 // ring instead of validating touches on its critical path; entries that went stale after they
 // were appended are recognised there by their next-occurrence field.
 template <typename MaskT>
@@ -359,7 +366,7 @@ __device__ __forceinline__ void scout_warp(const ReplayArgs& a, const Smem& sm, 
 // would also wait for the warp's global loads in flight, which the pipelines below avoid.
 __device__ __forceinline__ void smem_order() { asm volatile("" ::: "memory"); }
 
-// Named CTA barriers pairing the decide warp and the cache warp (32 + 32 threads each).  The
+// Named CTA barriers pairing the route warp and the gate warp (32 + 32 threads each).  The
 // barrier itself orders the arriving warp's earlier memory accesses before the waiting warp's
 // later ones.
 __device__ __forceinline__ void bar_arrive(int id) {
@@ -368,8 +375,8 @@ __device__ __forceinline__ void bar_arrive(int id) {
 __device__ __forceinline__ void bar_wait(int id) {
   asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory");
 }
-constexpr int kBarHits = 1;    // cache warp -> decide warp: prefix hits of the request are posted
-constexpr int kBarRoute = 2;   // decide warp -> cache warp: the chosen replica is posted
+constexpr int kBarHits = 1;    // gate warp -> route warp: prefix hits of the request are posted
+constexpr int kBarRoute = 2;   // route warp -> gate warp: the chosen replica is posted
 
 // Everything the warps of one candidate share.
 template <typename MaskT>
@@ -386,10 +393,10 @@ struct Ctx {
   unsigned long long* slot_kv; // [R*S] KV tokens of each slot's newest request (global memory)
   volatile uint32_t* route;    // chosen replica of the current request
   volatile int32_t* status;    // first device-side limit hit by any warp
-  // staging of the coming requests by the probe warp (kStageDepth stages + one of the cache warp)
+  // staging of the coming requests by the probe warp (kStageDepth stages + two of the gate warp)
   volatile uint32_t* st_ready; // [kStageDepth] request (+1) whose data the stage holds
   volatile uint32_t* probe_gone;  // the probe warp has stopped
-  // (stages kStageDepth and kStageDepth+1 belong to the cache warp, used alternately)
+  // (stages kStageDepth and kStageDepth+1 belong to the gate warp, used alternately)
   uint32_t* st_hits;           // [kStageDepth+2][R] prefix hit | blocks present << 16
   double* st_ab;               // [kStageDepth+2][R] (w_net*RTT + w_prefill*uncached) per replica
   uint4* st_meta;              // [kStageDepth+2] (input tokens, blocks | origin << 16, latest earlier request sharing a block, offset of its ids)
@@ -517,7 +524,7 @@ __device__ __forceinline__ void route_warp(const ReplayArgs& a, const Ctx<MaskT>
       smem_order();
       *sm.routed = r + 1;
     }
-    bar_arrive(kBarRoute);                                // the cache warp may commit request r
+    bar_arrive(kBarRoute);                                // the gate warp posts the commit of request r
     PROF_LAP(5);
     const long long add = by_requests ? 1ll : (long long)in_tok;
     if (istar == i0) ld0 += add;
@@ -978,10 +985,10 @@ __device__ __forceinline__ void stage_scores(const ReplayArgs& a, const Ctx<Mask
   }
 }
 
-// Probe warp: runs up to kWindow requests ahead of the cache warp.  For request q it reads the
+// Probe warp: runs up to kWindow requests ahead of the commit warps.  For request q it reads the
 // block ids and the mask words (first kStageBlocks blocks), stages them in shared memory, probes
 // them and publishes the prefix hits.  Its reads may predate the commits of the last kWindow
-// requests; the cache warp knows which of those commits can have touched request q and then
+// requests; the gate warp knows which of those commits can have touched request q and then
 // repeats the work itself, so this warp is an accelerator only and may stop at any time.
 template <typename MaskT, bool kBaseline>
 __device__ __forceinline__ void probe_warp(const ReplayArgs& a, const Ctx<MaskT>& cx, uint32_t p,
